@@ -1,0 +1,258 @@
+/*
+ * spm.h — C ABI of the offloaded sparse-MoE decode step with prediction-guided,
+ * window-budgeted expert prefetch (SpecPrefetch), for one NVIDIA B200 (sm_100a).
+ *
+ * One decode step pushes nb hidden rows through L MoE layers. Per layer l:
+ *   1. native router (frozen):  x = RMSNorm(h);  z = W_r x;  p = softmax(z);
+ *      T = Top_K(z);  w_e = p_e / sum_{j in T} p_j            [Section 3.1, first equation]
+ *   2. batch demand T_batch = union of the tokens' Top-K sets  [Section 3.1, second equation];
+ *      experts of T_batch without a cache slot are copied on demand from the pinned
+ *      host store ("any required expert that is not available is loaded on demand",
+ *      Section 3.3, last paragraph)
+ *   3. adapter (l <= L-2):  z^ = Bup (A x);  pi^ = softmax(z^);  s_e = sum over tokens of pi^_e
+ *      [Section 3.2, equations 1, 3, 4]; the experts of layer l+1 are ranked by s
+ *   4. budgeted selection  P = Top_{M_max}({ s_e : e not available, not in transfer }),
+ *      issued asynchronously in descending priority, |P| <= M_max   [Section 3.3]
+ *   5. routed (+ shared) SwiGLU experts read in place from their slots:
+ *      h += sum_k w_k W_down( silu(W_gate x) * (W_up x) )
+ * The prediction only moves transfers earlier; routing and outputs never depend on it
+ * (Section 3.1, last paragraph).
+ *
+ * Conventions
+ *   - every function returns an int status (SPM_OK or a negative SPM_ERR_*); nothing throws
+ *     or aborts; results come back through out-pointers; spm_last_error() gives a message.
+ *   - "dev" pointers are CUDA device pointers, "host" pointers ordinary host memory,
+ *     "pinned" page-locked host memory. The library never frees or reallocates caller memory.
+ *   - the caller owns all weights, the pinned expert store, the device arena and both CUDA
+ *     streams (passed as cudaStream_t cast to void*); the library owns its context, the slot
+ *     tables, its CUDA events and a small host-mapped mailbox.
+ *   - one context per host thread. GPU work is enqueued on the caller's streams; a call
+ *     returns as soon as the host has what it needs (calls that hand expert ids to the host
+ *     wait, with a deadline, for the routing kernel only).
+ *   - layers, experts, slots are 0-based. Adapter `l` scores layer l+1 and exists for l <= L-2.
+ *   - all matrices are row-major. dtype applies to every weight matrix (router, adapter,
+ *     experts); activations, logits, scores and routing weights are fp32.
+ */
+#ifndef SPM_H
+#define SPM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes ---------------------------------------------------- */
+#define SPM_OK                 0
+#define SPM_ERR_INVALID_ARG   (-1)  /* null pointer, index out of range                       */
+#define SPM_ERR_CONFIG        (-2)  /* unsupported shape, slots < top_k at batch 1, ...        */
+#define SPM_ERR_CUDA          (-3)  /* a CUDA runtime call failed (message has the detail)    */
+#define SPM_ERR_TIMEOUT       (-4)  /* routing kernel did not report within the deadline      */
+#define SPM_ERR_NOT_RESIDENT  (-5)  /* an expert handed to the FFN has no loaded slot         */
+#define SPM_ERR_STATE         (-6)  /* call made in the wrong order (e.g. no hint trace set)  */
+
+#define SPM_DTYPE_FP32 0
+#define SPM_DTYPE_BF16 1
+
+/* prefetch policies */
+#define SPM_POLICY_ADAPTER    0   /* rank next-layer experts with the low-rank adapter (the method)    */
+#define SPM_POLICY_ON_DEMAND  1   /* no prediction, no prefetch (the paper's OFF arm, Table 4)          */
+#define SPM_POLICY_HINT_TRACE 2   /* perfect knowledge: ranking = recorded true next-layer experts      */
+#define SPM_POLICY_PRED0      3   /* predict and select, issue no transfer (the paper's PRED0, Table 4) */
+
+/* cache event kinds (spm_event.kind) */
+#define SPM_EV_HIT            1   /* needed expert already has a slot                                   */
+#define SPM_EV_HIT_PREFETCHED 2   /* ... and this is the first use of a prefetched expert               */
+#define SPM_EV_MISS           3   /* loaded on demand into `slot`                                        */
+#define SPM_EV_EVICT          4   /* `expert` removed from `slot`                                        */
+#define SPM_EV_EVICT_WASTED   5   /* ... it had been prefetched and was never used                       */
+#define SPM_EV_PREFETCH       6   /* prefetch of `expert` into `slot` issued                             */
+#define SPM_EV_TOUCH_PRED     7   /* resident expert protected because the prediction ranks it high      */
+#define SPM_EV_WAVE           8   /* demand exceeds the slots: a new wave starts (`expert` = wave index) */
+#define SPM_EV_PLAN           9   /* PRED0: selected but not issued (`slot` = -1)                        */
+#define SPM_EV_DROPPED        10  /* fault injection: prefetch request lost (`slot` = -1)                */
+
+#define SPM_MAX_BATCH   64
+#define SPM_MAX_TOPK    16        /* top_k + n_shared <= SPM_MAX_TOPK */
+#define SPM_MAX_EXPERTS 1024
+
+typedef struct spm_ctx spm_ctx;   /* GPU decode context           */
+typedef struct spm_sim spm_sim;   /* host-only slot-table policy  */
+
+typedef struct {
+    int32_t n_layers;      /* L                                             */
+    int32_t hidden;        /* D                                             */
+    int32_t n_experts;     /* n routed experts per layer                    */
+    int32_t inter;         /* I, SwiGLU intermediate size                   */
+    int32_t top_k;         /* K                                             */
+    int32_t n_shared;      /* always-resident shared experts per layer      */
+    int32_t adapter_rank;  /* r                                             */
+    int32_t dtype;         /* SPM_DTYPE_*                                   */
+    int32_t renormalize;   /* 1: w_e = p_e / sum over the Top-K             */
+    int32_t max_batch;     /* largest nb any call will pass (<= SPM_MAX_BATCH) */
+    float   rms_eps;
+} spm_model_cfg;
+
+typedef struct {
+    const void* rms_gamma;       /* dev   fp32 [L][D]                                            */
+    const void* router_w;        /* dev   [L][n][D]                                              */
+    const void* adapter_a;       /* dev   [L-1][r][D]   (may be NULL when L == 1)                */
+    const void* adapter_b;       /* dev   [L-1][n][r]                                            */
+    const void* shared_experts;  /* dev   [L][n_shared] packed blobs (NULL when n_shared == 0)   */
+    const void* host_experts;    /* pinned [L][n] packed blobs: the offloaded expert store       */
+    void*       arena;           /* dev, 256-byte aligned: slot pools + workspace                */
+    size_t      arena_bytes;     /* >= spm_query_arena()                                         */
+    void*       compute_stream;  /* cudaStream_t                                                 */
+    void*       copy_stream;     /* cudaStream_t, different from compute_stream                  */
+} spm_buffers;
+
+typedef struct { int32_t step, layer, kind, expert, slot; } spm_event;
+
+typedef struct {
+    uint64_t steps, tokens;
+    uint64_t hits, hits_prefetched, misses, evictions, wasted;
+    uint64_t prefetch_issued, touches, waves, planned, dropped;
+    uint64_t late_arrivals;      /* needed expert whose prefetch copy was still in flight (timing only) */
+    uint64_t h2d_bytes;          /* expert bytes copied host -> HBM                                      */
+    uint64_t ffn_launches;       /* expert-FFN kernel launches timed below                               */
+    uint64_t kernel_launches;    /* all kernels this context launched                                    */
+    double   ffn_us;             /* summed device time of those launches (needs spm_set_timing(ctx, 1))  */
+    double   stall_us;           /* summed gap "routing kernel done -> expert FFN may start" per layer    */
+    double   ready_sum;          /* sum over (step, layer >= 1, token) of |T ∩ has-slot| / K at demand   */
+    uint64_t ready_count;        /*   ... and the number of terms (ReadyRecall = ready_sum / ready_count) */
+    double   recall_sum;         /* sum over (step, layer >= 1, token) of |T ∩ Top_M(s)| / K, M = budget  */
+    uint64_t recall_count;       /*   ExpertRecall@M = recall_sum / recall_count  (Section 4.1)          */
+} spm_stats;
+
+/* ---- packed expert layout ------------------------------------------------
+ * One expert = one contiguous blob of 3*I*D elements, identical in the host store, in a
+ * cache slot and in shared_experts, so one transfer is one copy:
+ *     blob[j][0][0..D) = W_gate[j][:]      j = 0..I-1
+ *     blob[j][1][0..D) = W_up[j][:]
+ *     blob[j][2][0..D) = W_down[:][j]      (column j of W_down[D][I])
+ * Writes 3*I*D*sizeof(element) to *bytes.                                               */
+int spm_expert_blob_bytes(const spm_model_cfg* cfg, size_t* bytes);
+
+/* Bytes of device arena needed for `slots_per_layer` routed slots per layer plus workspace. */
+int spm_query_arena(const spm_model_cfg* cfg, int slots_per_layer, size_t* bytes);
+
+/* Create a context. budget = M_max >= 0, or -1 to derive it from the profiled overlap window
+ * (spm_profile_window is then run once here: max(1, floor(W / t_xfer)); Section 3.3, first
+ * paragraphs). Slot tables start empty (cold cache). Fails with SPM_ERR_CONFIG when
+ * max_batch == 1 and slots_per_layer < top_k, or when the shape is not supported by the
+ * kernels (hidden must be a multiple of 256 (bf16) / 128 (fp32) and <= 8192). */
+int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget,
+             const spm_buffers* buffers, spm_ctx** out);
+int spm_destroy(spm_ctx* ctx);
+const char* spm_last_error(const spm_ctx* ctx);   /* ctx may be NULL: last error of spm_init */
+
+/* Native router of `layer` (Section 3.1, first equation): RMSNorm, gate GEMV, softmax, Top-K,
+ * renormalise.   h dev [nb][D] -> x_norm dev [nb][D], w dev [nb][K] (rank order),
+ * logits dev [nb][n] (may be NULL), ids HOST [nb][K] (rank order: ties to the lower id).
+ * Returns after the ids have reached the host (bounded wait, SPM_ERR_TIMEOUT). */
+int spm_router_topk(spm_ctx* ctx, int layer, const float* h, int nb,
+                    float* x_norm, int32_t* ids, float* w, float* logits);
+
+/* Adapter of `layer` (Section 3.2): priorities of the experts of layer+1.
+ * x_norm dev [nb][D] -> scores HOST [n] (s_e summed over the nb tokens in token order),
+ * order HOST [n] (expert ids by (s descending, id ascending)). layer <= L-2. */
+int spm_adapter_predict(spm_ctx* ctx, int layer, const float* x_norm, int nb,
+                        float* scores, int32_t* order);
+
+/* Selection of Section 3.3 for pool `target_layer`: walk `order` (host, n_ranked ids in
+ * descending priority), skip experts that have a slot (available or in transfer), keep at
+ * most `budget` (budget < 0: the context's M_max). Host logic only; nothing is issued.
+ * protect_all = 0: the resident experts ranked above the last selected one are remembered for
+ * the next spm_prefetch_async on this layer (predicted-use touch); 1: every resident expert in
+ * `order` (use when `order` lists exactly the experts that will be needed).
+ * out_ids host [>= min(budget, slots)], descending priority. */
+int spm_budget_select(spm_ctx* ctx, int target_layer, const int32_t* order, int n_ranked,
+                      int budget, int protect_all, int32_t* out_ids, int* out_count);
+
+/* Issue host->HBM copies of experts `ids` (host, descending priority) of `target_layer` on the
+ * copy stream into least-recently-used slots of that layer's pool; one CUDA event per slot.
+ * Experts that already have a slot are skipped. Stops when no unprotected slot is left.
+ * *out_issued (may be NULL) = number of copies enqueued. Asynchronous. */
+int spm_prefetch_async(spm_ctx* ctx, int target_layer, const int32_t* ids, int count,
+                       int* out_issued);
+
+/* Routed + shared SwiGLU experts of `layer` for nb tokens, slot-indexed (no gather):
+ * resolves the batch demand against the slot table, loads misses on demand, makes the compute
+ * stream wait for exactly the slots it reads, and enqueues h_inout += sum_k w_k FFN_{ids_k}(x).
+ * x_norm dev [nb][D], ids HOST [nb][K], w dev [nb][K], h_inout dev [nb][D]. Asynchronous.
+ * When more distinct experts are needed than there are slots the work is split in waves. */
+int spm_moe_ffn(spm_ctx* ctx, int layer, const float* x_norm, const int32_t* ids,
+                const float* w, int nb, float* h_inout);
+
+/* One decode step through all L layers under the context's policy: h_in dev [nb][D] ->
+ * h_out dev [nb][D] (may alias h_in). Equivalent to, per layer: spm_router_topk,
+ * spm_adapter_predict, spm_moe_ffn, spm_budget_select + spm_prefetch_async for layer+1,
+ * with router and adapter fused in one kernel. The last layer's work is left in flight. */
+int spm_decode_step(spm_ctx* ctx, const float* h_in, int nb, float* h_out);
+
+/* Same, with HOST buffers (pinned for speed): copies h_in to the device, runs the step, copies
+ * h_out back and waits for it. */
+int spm_decode_step_host(spm_ctx* ctx, const float* h_in_host, int nb, float* h_out_host);
+
+/* ---- control, profiling, accounting ------------------------------------ */
+int spm_set_policy(spm_ctx* ctx, int policy);
+int spm_set_budget(spm_ctx* ctx, int budget);             /* M_max >= 0 */
+int spm_get_budget(spm_ctx* ctx, int* budget);
+int spm_set_plain_lru(spm_ctx* ctx, int on);              /* 1: no predicted-use touch */
+int spm_set_timing(spm_ctx* ctx, int on);                 /* record CUDA events around FFN / stalls */
+int spm_set_ffn_ctas(spm_ctx* ctx, int ctas);             /* CTAs per token of the GEMV FFN (0 = default) */
+/* Perfect-knowledge ranking for SPM_POLICY_HINT_TRACE: for step s (counted from the last
+ * spm_cache_reset) and layer l, hint[(s*L + l)*stride .. +count[s*L+l]) are the experts that
+ * layer truly needs, in priority order. Copied. */
+int spm_set_hint_trace(spm_ctx* ctx, const int32_t* hint, const int32_t* count,
+                       int n_steps, int stride);
+/* Fault injection on the host: every prefetch request with (step + expert) % modulo == 0 is
+ * lost before it reaches the GPU (0 switches it off). The demand path must then load it. */
+int spm_set_drop_modulo(spm_ctx* ctx, int modulo);
+/* Host deadline of the routing-kernel handshake, in milliseconds (default 5000). */
+int spm_set_deadline_ms(spm_ctx* ctx, int ms);
+
+/* Profile the overlap window (Section 3.3): window_us = median device time of the expert FFN
+ * of one layer with K resident experts, t_xfer_us = median time of one expert copy from the
+ * pinned store, *budget_raw = floor(window / t_xfer). Uses and then empties the cache. */
+int spm_profile_window(spm_ctx* ctx, double* window_us, double* t_xfer_us, int* budget_raw);
+
+int spm_cache_reset(spm_ctx* ctx);                         /* cold cache, step counter, stats, events */
+int spm_get_stats(spm_ctx* ctx, spm_stats* out);           /* waits for timed work to finish */
+/* Per-layer sums since the last reset: stall_us[L], ffn_us[L], and the number of steps in them. */
+int spm_get_layer_times(spm_ctx* ctx, double* stall_us, double* ffn_us, uint64_t* steps);
+int spm_get_events(spm_ctx* ctx, spm_event* out, size_t capacity, size_t* count);
+int spm_get_slot_table(spm_ctx* ctx, int layer, int32_t* slot_expert /* host [slots] */);
+int spm_synchronize(spm_ctx* ctx);                         /* both streams idle */
+
+/* Pinned host memory for the expert store (thin wrappers over cudaHostAlloc / cudaFreeHost). */
+int spm_host_alloc(size_t bytes, void** out);
+int spm_host_free(void* p);
+
+/* ---- host-only slot-table policy (no GPU needed) ------------------------
+ * The same slot table the context uses, exposed so the cache policy can be driven and checked
+ * on a machine without a GPU. Arrays are host memory.                                        */
+int spm_sim_create(int n_layers, int n_experts, int slots, int plain_lru, spm_sim** out);
+int spm_sim_destroy(spm_sim* sim);
+/* Demand of `layer`: need[count] expert ids (any order, duplicates allowed). Outputs, one entry
+ * per distinct expert in processing order: expert, slot, wave index, missed flag. */
+int spm_sim_demand(spm_sim* sim, int layer, const int32_t* need, int count,
+                   int32_t* out_expert, int32_t* out_slot, int32_t* out_wave,
+                   int32_t* out_missed, int* out_count, int* out_waves);
+int spm_sim_plan(spm_sim* sim, int layer, const int32_t* order, int n_ranked, int budget,
+                 int protect_all, int32_t* out_ids, int* out_count,
+                 int32_t* out_protect, int* out_n_protect);
+int spm_sim_prefetch(spm_sim* sim, int layer, const int32_t* ids, int count,
+                     const int32_t* protect, int n_protect, int drop_modulo,
+                     int32_t* out_slots /* [count], -1 = not issued */, int* out_issued);
+int spm_sim_plan_only(spm_sim* sim, int layer, const int32_t* ids, int count);
+int spm_sim_end_step(spm_sim* sim);
+int spm_sim_events(spm_sim* sim, spm_event* out, size_t capacity, size_t* count);
+int spm_sim_stats(spm_sim* sim, spm_stats* out);
+int spm_sim_slot_table(spm_sim* sim, int layer, int32_t* slot_expert /* [slots] */);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPM_H */

@@ -1,0 +1,246 @@
+// Fused native router + prediction adapter for one layer and nb tokens.
+//
+// Router (Section 3.1): x = RMSNorm(h); z = W_r x; p = softmax(z); T = Top_K(z) with ties to the
+// lower id; w_e = p_e / sum_{j in T} p_j.
+// Adapter (Section 3.2): u = A x; z^ = Bup u; pi^ = softmax(z^); s_e = sum over tokens of pi^_e
+// in token order; the experts of the next layer are ranked by (s descending, id ascending).
+//
+// Grid (C, nb): the C CTAs of a token split the n + r weight rows (one warp per row, 16-byte
+// read-only loads, shuffle reduction). The last CTA of a token to finish (atomic ticket) does
+// that token's softmax / Top-K / adapter tail; the last token-tail to finish does the batch
+// aggregation and ranking, copies ids / order / scores into the host-mapped mailbox, fences at
+// system scope and publishes the launch's sequence number, which the host polls.
+// Every reduction has a fixed order, so results are bitwise reproducible.
+#pragma once
+
+#include "ptx.cuh"
+#include "../../include/spm.h"
+
+namespace spm {
+
+constexpr int kRouterWarps = 8;
+constexpr int kRouterThreads = kRouterWarps * 32;
+
+// Host-mapped pinned mailbox (the device writes, the host polls `seq`).
+struct Mailbox {
+    volatile uint32_t seq;
+    uint32_t pad[3];
+    int32_t ids[SPM_MAX_BATCH * SPM_MAX_TOPK];   // [nb][K]
+    int32_t order[SPM_MAX_EXPERTS];              // [n]
+    float scores[SPM_MAX_EXPERTS];               // [n]
+};
+
+struct RouterArgs {
+    const float* h;          // [nb][D] hidden rows (do_router) ...
+    const float* x_in;       // ... or already-normalised rows (adapter only)
+    const float* gamma;      // [D]
+    const void* router_w;    // [n][D]
+    const void* adapter_a;   // [r][D]
+    const void* adapter_b;   // [n][r]
+    float* x_norm;           // out [nb][D]
+    float* logits;           // workspace [nb][n]
+    float* logits_out;       // optional copy for the caller
+    float* u;                // workspace [nb][r]
+    float* pihat;            // workspace [nb][n]
+    int32_t* ids;            // out [nb][K]
+    float* w;                // out [nb][K]
+    float* scores;           // out [n]
+    int32_t* order;          // out [n]
+    unsigned* counters;      // [1 + nb], zero between launches
+    Mailbox* mailbox;        // device view of the host-mapped mailbox
+    uint32_t seq;
+    int D, n, K, r, nb, renorm, do_router, do_adapter;
+    float eps;
+};
+
+__device__ __forceinline__ float block_reduce(float v, float* scratch, bool is_max) {
+    // fixed-shape tree: shuffle inside warps, then warp 0 over the 8 warp results
+    const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float t = __shfl_xor_sync(0xffffffffu, v, o);
+        v = is_max ? fmaxf(v, t) : v + t;
+    }
+    __syncthreads();
+    if (lane == 0) scratch[wi] = v;
+    __syncthreads();
+    float r = scratch[0];
+#pragma unroll
+    for (int i = 1; i < kRouterWarps; ++i) r = is_max ? fmaxf(r, scratch[i]) : r + scratch[i];
+    return r;
+}
+
+// softmax of v[0..n) in shared memory, in place
+__device__ __forceinline__ void block_softmax(float* v, int n, float* scratch) {
+    float m = -INFINITY;
+    for (int e = threadIdx.x; e < n; e += kRouterThreads) m = fmaxf(m, v[e]);
+    m = block_reduce(m, scratch, true);
+    float s = 0.f;
+    for (int e = threadIdx.x; e < n; e += kRouterThreads) {
+        const float t = expf(v[e] - m);
+        v[e] = t;
+        s += t;
+    }
+    s = block_reduce(s, scratch, false);
+    for (int e = threadIdx.x; e < n; e += kRouterThreads) v[e] = v[e] / s;
+    __syncthreads();
+}
+
+// position of element e in the ordering (value descending, index ascending)
+__device__ __forceinline__ int rank_of(const float* v, int n, int e) {
+    const float ve = v[e];
+    int c = 0;
+    for (int j = 0; j < n; ++j) c += (v[j] > ve) || (v[j] == ve && j < e);
+    return c;
+}
+
+template <typename WT>
+__global__ void __launch_bounds__(kRouterThreads)
+router_adapter_kernel(const __grid_constant__ RouterArgs a) {
+    constexpr int VEC = 16 / int(sizeof(WT));
+    extern __shared__ __align__(16) float sm[];
+    float* xs = sm;                 // [D]
+    float* zs = xs + a.D;           // [n] logits -> probabilities
+    float* ps = zs + a.n;           // [n] adapter logits -> probabilities / scores
+    float* scratch = ps + a.n;      // [8] + small tails
+    float* psel = scratch + kRouterWarps;           // [K]
+    int* isel = reinterpret_cast<int*>(psel + SPM_MAX_TOPK);   // [K]
+    float* us = reinterpret_cast<float*>(isel + SPM_MAX_TOPK); // [r]
+    __shared__ int s_last;
+
+    const int tok = blockIdx.y, C = gridDim.x;
+    const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
+    const int D = a.D, n = a.n;
+
+    // ---- router input ---------------------------------------------------
+    if (a.do_router) {
+        const float* ht = a.h + size_t(tok) * D;
+        float ss = 0.f;
+        for (int i = threadIdx.x; i < D; i += kRouterThreads) {
+            const float v = ht[i];
+            xs[i] = v;
+            ss = fmaf(v, v, ss);
+        }
+        ss = block_reduce(ss, scratch, false);
+        const float inv = 1.0f / sqrtf(ss / float(D) + a.eps);
+        for (int i = threadIdx.x; i < D; i += kRouterThreads) {
+            const float v = xs[i] * a.gamma[i] * inv;
+            xs[i] = v;
+            if (blockIdx.x == 0 && a.x_norm) a.x_norm[size_t(tok) * D + i] = v;
+        }
+    } else {
+        const float* xt = a.x_in + size_t(tok) * D;
+        for (int i = threadIdx.x; i < D; i += kRouterThreads) xs[i] = xt[i];
+    }
+    __syncthreads();
+
+    // ---- weight rows: router rows then adapter-A rows, one warp per row ----
+    const int n_r = a.do_router ? n : 0;
+    const int rows = n_r + (a.do_adapter ? a.r : 0);
+    for (int row = blockIdx.x * kRouterWarps + wi; row < rows; row += C * kRouterWarps) {
+        const WT* wrow = row < n_r ? static_cast<const WT*>(a.router_w) + size_t(row) * D
+                                   : static_cast<const WT*>(a.adapter_a) + size_t(row - n_r) * D;
+        float acc = 0.f;
+        for (int i = lane * VEC; i < D; i += 32 * VEC) {
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(wrow + i));
+            float f[VEC];
+            unpack16(v, f);
+#pragma unroll
+            for (int q = 0; q < VEC; ++q) acc = fmaf(f[q], xs[i + q], acc);
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) {
+            if (row < n_r) a.logits[size_t(tok) * n + row] = acc;
+            else a.u[size_t(tok) * a.r + (row - n_r)] = acc;
+        }
+    }
+
+    // ---- ticket: the last CTA of this token runs the tail ------------------
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(&a.counters[1 + tok], 1u) == unsigned(C - 1);
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+
+    if (a.do_router) {
+        for (int e = threadIdx.x; e < n; e += kRouterThreads) {
+            const float z = __ldcg(a.logits + size_t(tok) * n + e);
+            zs[e] = z;
+            ps[e] = z;
+            if (a.logits_out) a.logits_out[size_t(tok) * n + e] = z;
+        }
+        __syncthreads();
+        block_softmax(ps, n, scratch);          // ps = p, zs = z (ranking is taken on the logits)
+        for (int e = threadIdx.x; e < n; e += kRouterThreads) {
+            const int rk = rank_of(zs, n, e);
+            if (rk < a.K) { isel[rk] = e; psel[rk] = ps[e]; }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            float tot = 0.f;
+            for (int k = 0; k < a.K; ++k) tot += psel[k];
+            for (int k = 0; k < a.K; ++k) {
+                a.ids[size_t(tok) * a.K + k] = isel[k];
+                a.w[size_t(tok) * a.K + k] = a.renorm ? psel[k] / tot : psel[k];
+            }
+        }
+    }
+    if (a.do_adapter) {
+        __syncthreads();
+        for (int q = threadIdx.x; q < a.r; q += kRouterThreads) us[q] = __ldcg(a.u + size_t(tok) * a.r + q);
+        __syncthreads();
+        const WT* B = static_cast<const WT*>(a.adapter_b);
+        for (int e = threadIdx.x; e < n; e += kRouterThreads) {
+            float acc = 0.f;
+            for (int q = 0; q < a.r; ++q) {
+                float bw;
+                if (sizeof(WT) == 2) bw = __uint_as_float(uint32_t(reinterpret_cast<const uint16_t*>(B)[size_t(e) * a.r + q]) << 16);
+                else bw = reinterpret_cast<const float*>(B)[size_t(e) * a.r + q];
+                acc = fmaf(bw, us[q], acc);
+            }
+            ps[e] = acc;
+        }
+        __syncthreads();
+        block_softmax(ps, n, scratch);
+        for (int e = threadIdx.x; e < n; e += kRouterThreads) a.pihat[size_t(tok) * n + e] = ps[e];
+    }
+
+    // ---- ticket over tokens: the last tail aggregates and publishes ---------
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(&a.counters[0], 1u) == unsigned(a.nb - 1);
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+
+    Mailbox* mb = a.mailbox;
+    if (a.do_adapter) {
+        for (int e = threadIdx.x; e < n; e += kRouterThreads) {
+            float s = 0.f;
+            for (int t = 0; t < a.nb; ++t) s += __ldcg(a.pihat + size_t(t) * n + e);
+            ps[e] = s;
+        }
+        __syncthreads();
+        for (int e = threadIdx.x; e < n; e += kRouterThreads) {
+            const int rk = rank_of(ps, n, e);
+            a.order[rk] = e;
+            a.scores[e] = ps[e];
+            mb->order[rk] = e;
+            mb->scores[e] = ps[e];
+        }
+    }
+    if (a.do_router) {
+        for (int i = threadIdx.x; i < a.nb * a.K; i += kRouterThreads) mb->ids[i] = __ldcg(a.ids + i);
+    }
+    for (int i = threadIdx.x; i <= a.nb; i += kRouterThreads) a.counters[i] = 0u;
+    __threadfence_system();
+    __syncthreads();
+    if (threadIdx.x == 0) mb->seq = a.seq;
+}
+
+inline size_t router_smem_bytes(int D, int n, int r) {
+    return sizeof(float) * (size_t(D) + 2 * size_t(n) + kRouterWarps + 2 * SPM_MAX_TOPK + size_t(r));
+}
+
+}  // namespace spm

@@ -1,0 +1,1001 @@
+// C ABI of the offloaded-MoE decode step (see include/spm.h): context, slot pools, copy-stream
+// scheduling with CUDA events, kernel launches. All arithmetic of the path runs in the kernels
+// of ffn_gemv.cuh / router_adapter.cuh; this file is host control only.
+#include <algorithm>
+#include <atomic>
+#include <chrono>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include <cuda_runtime.h>
+#include <immintrin.h>
+
+#include "../../include/spm.h"
+#include "ffn_gemv.cuh"
+#include "router_adapter.cuh"
+#include "slot_table.h"
+
+using namespace spm;
+
+namespace {
+
+thread_local std::string g_init_error;
+
+struct bf16_t { uint16_t v; };
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Timing {            // CUDA events of one step, per layer
+    std::vector<cudaEvent_t> k1_done, ffn_start, ffn_end;
+    std::vector<uint8_t> used;
+};
+
+}  // namespace
+
+struct spm_ctx {
+    spm_model_cfg cfg{};
+    int S = 0, budget = 0, policy = SPM_POLICY_ADAPTER;
+    spm_buffers buf{};
+    cudaStream_t compute = nullptr, copy = nullptr;
+    SlotTable* table = nullptr;
+    size_t elem = 2, blob = 0, row_bytes = 0;
+    int nseg = 0, depth = 2, num_sms = 148, ffn_ctas = 0;
+    // arena carve-up
+    unsigned char* pools = nullptr;
+    float *ws_x = nullptr, *ws_logits = nullptr, *ws_u = nullptr, *ws_pihat = nullptr, *ws_w = nullptr;
+    float *ws_scores = nullptr, *ws_partial = nullptr, *ws_h = nullptr;
+    int32_t *ws_ids = nullptr, *ws_order = nullptr;
+    unsigned* ws_counters = nullptr;
+    int* ws_status = nullptr;
+    // mailbox
+    Mailbox* mb_host = nullptr;
+    Mailbox* mb_dev = nullptr;
+    uint32_t seq = 0;
+    int deadline_ms = 5000;
+    // per-slot copy events
+    std::vector<cudaEvent_t> slot_ev;
+    std::vector<uint8_t> slot_pending;
+    std::vector<cudaEvent_t> pool_free;       // recorded after the last FFN that read pool l
+    std::vector<uint8_t> pool_free_valid;
+    cudaEvent_t wave_done = nullptr;
+    // timing
+    bool timing = false;
+    Timing tim[2];
+    int tim_cur = 0;
+    std::vector<double> layer_stall_us, layer_ffn_us;
+    uint64_t timed_steps = 0;
+    // policy inputs
+    std::vector<int32_t> hint, hint_count;
+    int hint_steps = 0, hint_stride = 0;
+    int drop_modulo = 0;
+    std::vector<std::vector<int32_t>> pending_protect;
+    std::vector<uint8_t> has_plan;
+    std::vector<int32_t> prev_order;          // ranking produced at the previous layer of this step
+    bool prev_order_valid = false;
+    // scratch
+    std::vector<Placement> placements;
+    std::vector<int32_t> need, sel, protect, slots_tmp;
+    std::vector<int16_t> wave_slot;
+    uint64_t extra_late = 0, h2d_bytes = 0, ffn_launches = 0, kernel_launches = 0, tokens = 0;
+    double ready_sum = 0, recall_sum = 0;
+    uint64_t ready_count = 0, recall_count = 0;
+    std::string err;
+};
+
+namespace {
+
+int fail(spm_ctx* c, int code, const char* fmt, ...) {
+    char b[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(b, sizeof b, fmt, ap);
+    va_end(ap);
+    if (c) c->err = b; else g_init_error = b;
+    return code;
+}
+
+#define CU(c, call)                                                                        \
+    do {                                                                                   \
+        cudaError_t e_ = (call);                                                           \
+        if (e_ != cudaSuccess)                                                             \
+            return fail((c), SPM_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); \
+    } while (0)
+
+int check_cfg(const spm_model_cfg* m, int S, spm_ctx* c) {
+    if (!m) return fail(c, SPM_ERR_INVALID_ARG, "cfg is null");
+    if (m->dtype != SPM_DTYPE_FP32 && m->dtype != SPM_DTYPE_BF16) return fail(c, SPM_ERR_CONFIG, "unknown dtype %d", m->dtype);
+    const int seg = m->dtype == SPM_DTYPE_BF16 ? 256 : 128;
+    if (m->n_layers < 1 || m->hidden < seg || m->hidden % seg || m->hidden / seg > 8)
+        return fail(c, SPM_ERR_CONFIG, "hidden %d unsupported: need a multiple of %d, at most %d", m->hidden, seg, 8 * seg);
+    if (m->n_experts < 1 || m->n_experts > SPM_MAX_EXPERTS) return fail(c, SPM_ERR_CONFIG, "n_experts %d out of range", m->n_experts);
+    if (m->top_k < 1 || m->top_k > m->n_experts || m->n_shared < 0 || m->top_k + m->n_shared > SPM_MAX_TOPK)
+        return fail(c, SPM_ERR_CONFIG, "top_k %d + n_shared %d unsupported (max %d)", m->top_k, m->n_shared, SPM_MAX_TOPK);
+    if (m->inter < 1) return fail(c, SPM_ERR_CONFIG, "inter %d", m->inter);
+    if (m->adapter_rank < 1 || m->adapter_rank > 256) return fail(c, SPM_ERR_CONFIG, "adapter_rank %d out of range", m->adapter_rank);
+    if (m->max_batch < 1 || m->max_batch > SPM_MAX_BATCH) return fail(c, SPM_ERR_CONFIG, "max_batch %d out of range", m->max_batch);
+    if (S < 1 || S > 32767) return fail(c, SPM_ERR_CONFIG, "slots_per_layer %d out of range", S);
+    if (m->max_batch == 1 && S < m->top_k) return fail(c, SPM_ERR_CONFIG, "slots_per_layer %d < top_k %d at batch 1", S, m->top_k);
+    return SPM_OK;
+}
+
+size_t blob_bytes_of(const spm_model_cfg* m) {
+    return size_t(3) * m->inter * m->hidden * (m->dtype == SPM_DTYPE_BF16 ? 2 : 4);
+}
+
+constexpr int kMaxCtasBatch1 = 296;
+
+int ffn_grid_for(const spm_ctx* c, int nb) {
+    if (nb == 1) return c->ffn_ctas > 0 ? std::min(c->ffn_ctas, kMaxCtasBatch1) : c->num_sms;
+    return std::max(1, kMaxCtasBatch1 / nb);
+}
+
+struct Carve {
+    size_t off = 0;
+    size_t take(size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; }
+};
+
+struct Layout {
+    size_t pools, x, logits, u, pihat, w, scores, partial, h, ids, order, counters, status, total;
+};
+
+Layout layout_of(const spm_model_cfg* m, int S) {
+    Layout l{};
+    Carve c;
+    const size_t nb = m->max_batch, D = m->hidden, n = m->n_experts;
+    l.pools = c.take(size_t(m->n_layers) * S * blob_bytes_of(m));
+    l.x = c.take(nb * D * 4);
+    l.logits = c.take(nb * n * 4);
+    l.u = c.take(nb * m->adapter_rank * 4);
+    l.pihat = c.take(nb * n * 4);
+    l.w = c.take(nb * SPM_MAX_TOPK * 4);
+    l.scores = c.take(n * 4);
+    l.partial = c.take((kMaxCtasBatch1 + nb) * D * 4);
+    l.h = c.take(nb * D * 4);
+    l.ids = c.take(nb * SPM_MAX_TOPK * 4);
+    l.order = c.take(n * 4);
+    l.counters = c.take((nb + 1) * 4);
+    l.status = c.take(4);
+    l.total = c.off;
+    return l;
+}
+
+// ---- kernel dispatch -------------------------------------------------------
+template <typename WT, int NSEG, int MAXNB>
+cudaError_t launch_gemv_t(const FfnArgs<MAXNB>& a, int G, int nb, int depth, size_t smem, cudaStream_t st) {
+    static bool attr_set = false;
+    auto kern = ffn_gemv_kernel<WT, NSEG, MAXNB>;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    kern<<<dim3(G, nb), kFfnThreads, smem, st>>>(a, depth);
+    return cudaGetLastError();
+}
+
+template <typename WT, int MAXNB>
+cudaError_t launch_gemv_seg(int nseg, const FfnArgs<MAXNB>& a, int G, int nb, int depth, size_t smem, cudaStream_t st) {
+    switch (nseg) {
+        case 1: return launch_gemv_t<WT, 1, MAXNB>(a, G, nb, depth, smem, st);
+        case 2: return launch_gemv_t<WT, 2, MAXNB>(a, G, nb, depth, smem, st);
+        case 3: return launch_gemv_t<WT, 3, MAXNB>(a, G, nb, depth, smem, st);
+        case 4: return launch_gemv_t<WT, 4, MAXNB>(a, G, nb, depth, smem, st);
+        case 5: return launch_gemv_t<WT, 5, MAXNB>(a, G, nb, depth, smem, st);
+        case 6: return launch_gemv_t<WT, 6, MAXNB>(a, G, nb, depth, smem, st);
+        case 7: return launch_gemv_t<WT, 7, MAXNB>(a, G, nb, depth, smem, st);
+        case 8: return launch_gemv_t<WT, 8, MAXNB>(a, G, nb, depth, smem, st);
+    }
+    return cudaErrorInvalidValue;
+}
+
+template <int MAXNB>
+cudaError_t launch_gemv(const spm_ctx* c, const FfnArgs<MAXNB>& a, int G, int nb) {
+    const size_t smem = ffn_gemv_smem(c->row_bytes, c->depth);
+    if (c->cfg.dtype == SPM_DTYPE_BF16) return launch_gemv_seg<bf16_t, MAXNB>(c->nseg, a, G, nb, c->depth, smem, c->compute);
+    return launch_gemv_seg<float, MAXNB>(c->nseg, a, G, nb, c->depth, smem, c->compute);
+}
+
+int launch_router(spm_ctx* c, int layer, const float* h, const float* x_in, int nb, float* x_norm,
+                  float* logits_out, bool do_router, bool do_adapter) {
+    const spm_model_cfg& m = c->cfg;
+    RouterArgs a{};
+    const size_t D = m.hidden, n = m.n_experts, r = m.adapter_rank;
+    a.h = h;
+    a.x_in = x_in;
+    a.gamma = static_cast<const float*>(c->buf.rms_gamma) + size_t(layer) * D;
+    a.router_w = static_cast<const unsigned char*>(c->buf.router_w) + size_t(layer) * n * D * c->elem;
+    if (do_adapter) {
+        a.adapter_a = static_cast<const unsigned char*>(c->buf.adapter_a) + size_t(layer) * r * D * c->elem;
+        a.adapter_b = static_cast<const unsigned char*>(c->buf.adapter_b) + size_t(layer) * n * r * c->elem;
+    }
+    a.x_norm = x_norm;
+    a.logits = c->ws_logits;
+    a.logits_out = logits_out;
+    a.u = c->ws_u;
+    a.pihat = c->ws_pihat;
+    a.ids = c->ws_ids;
+    a.w = c->ws_w;
+    a.scores = c->ws_scores;
+    a.order = c->ws_order;
+    a.counters = c->ws_counters;
+    a.mailbox = c->mb_dev;
+    a.seq = ++c->seq;
+    a.D = m.hidden; a.n = m.n_experts; a.K = m.top_k; a.r = m.adapter_rank; a.nb = nb;
+    a.renorm = m.renormalize; a.do_router = do_router; a.do_adapter = do_adapter;
+    a.eps = m.rms_eps;
+    const int rows = (do_router ? m.n_experts : 0) + (do_adapter ? m.adapter_rank : 0);
+    int C = (rows + kRouterWarps - 1) / kRouterWarps;
+    C = std::max(1, std::min(C, 32));
+    const size_t smem = router_smem_bytes(m.hidden, m.n_experts, m.adapter_rank);
+    if (m.dtype == SPM_DTYPE_BF16)
+        router_adapter_kernel<bf16_t><<<dim3(C, nb), kRouterThreads, smem, c->compute>>>(a);
+    else
+        router_adapter_kernel<float><<<dim3(C, nb), kRouterThreads, smem, c->compute>>>(a);
+    CU(c, cudaGetLastError());
+    c->kernel_launches++;
+    return SPM_OK;
+}
+
+// Wait (bounded) until the routing kernel of the current sequence number has published.
+int wait_mailbox(spm_ctx* c) {
+    const uint32_t want = c->seq;
+    const auto t0 = std::chrono::steady_clock::now();
+    uint64_t spins = 0;
+    while (c->mb_host->seq != want) {
+        _mm_pause();
+        if ((++spins & 0x3fff) == 0) {
+            cudaError_t q = cudaStreamQuery(c->compute);
+            if (q != cudaSuccess && q != cudaErrorNotReady)
+                return fail(c, SPM_ERR_CUDA, "compute stream failed while waiting for the router: %s", cudaGetErrorString(q));
+            auto ms = std::chrono::duration_cast<std::chrono::milliseconds>(std::chrono::steady_clock::now() - t0).count();
+            if (ms > c->deadline_ms)
+                return fail(c, SPM_ERR_TIMEOUT, "routing kernel did not report within %d ms", c->deadline_ms);
+        }
+    }
+    std::atomic_thread_fence(std::memory_order_acquire);
+    return SPM_OK;
+}
+
+unsigned char* slot_ptr(spm_ctx* c, int layer, int slot) {
+    return c->pools + (size_t(layer) * c->S + slot) * c->blob;
+}
+const unsigned char* host_blob(spm_ctx* c, int layer, int e) {
+    return static_cast<const unsigned char*>(c->buf.host_experts) + (size_t(layer) * c->cfg.n_experts + e) * c->blob;
+}
+
+// Enqueue one expert transfer on the copy stream and arm the slot's event.
+int issue_copy(spm_ctx* c, int layer, int e, int slot) {
+    const size_t k = size_t(layer) * c->S + slot;
+    CU(c, cudaMemcpyAsync(slot_ptr(c, layer, slot), host_blob(c, layer, e), c->blob, cudaMemcpyHostToDevice, c->copy));
+    CU(c, cudaEventRecord(c->slot_ev[k], c->copy));
+    c->slot_pending[k] = 1;
+    c->h2d_bytes += c->blob;
+    return SPM_OK;
+}
+
+// The copy stream may overwrite pool `layer` only after the last kernel that read it.
+int order_copy_after_readers(spm_ctx* c, int layer) {
+    if (c->pool_free_valid[layer]) CU(c, cudaStreamWaitEvent(c->copy, c->pool_free[layer], 0));
+    return SPM_OK;
+}
+
+void harvest(spm_ctx* c, Timing& t) {
+    const int L = c->cfg.n_layers;
+    bool any = false;
+    for (int l = 0; l < L; ++l) {
+        if (!t.used[l]) continue;
+        float a = 0, b = 0;
+        cudaEventSynchronize(t.ffn_end[l]);
+        if (cudaEventElapsedTime(&a, t.k1_done[l], t.ffn_start[l]) == cudaSuccess) c->layer_stall_us[l] += a * 1e3;
+        if (cudaEventElapsedTime(&b, t.ffn_start[l], t.ffn_end[l]) == cudaSuccess) c->layer_ffn_us[l] += b * 1e3;
+        t.used[l] = 0;
+        any = true;
+    }
+    if (any) c->timed_steps++;
+}
+
+// Demand resolution, on-demand copies, stream waits and FFN launches of one layer.
+// `t` (may be null) receives the timing events of this layer.
+int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, const float* w, int nb,
+            float* h_inout, Timing* t) {
+    const spm_model_cfg& m = c->cfg;
+    const int K = m.top_k;
+    SlotTable& tb = *c->table;
+
+    c->need.clear();
+    for (int i = 0; i < nb * K; ++i) {
+        if (ids[i] < 0 || ids[i] >= m.n_experts) return fail(c, SPM_ERR_INVALID_ARG, "expert id %d out of range", ids[i]);
+        c->need.push_back(ids[i]);
+    }
+    if (layer >= 1) {   // logical ReadyRecall: needed experts that already have a slot
+        for (int tk = 0; tk < nb; ++tk) {
+            int have = 0;
+            for (int k = 0; k < K; ++k) have += tb.slot_of(layer, ids[tk * K + k]) >= 0;
+            c->ready_sum += double(have) / K;
+            c->ready_count++;
+        }
+    }
+    int n_waves = 1;
+    tb.demand(layer, c->need.data(), int(c->need.size()), c->placements, &n_waves);
+
+    const int G = ffn_grid_for(c, nb);
+    std::vector<int16_t>& slot_of_expert = c->wave_slot;   // experts computed in the current wave
+    for (int wave = 0; wave < n_waves; ++wave) {
+        slot_of_expert.assign(m.n_experts, -1);
+        bool any_copy = false;
+        for (size_t i = 0; i < c->placements.size(); ++i) {
+            const Placement& p = c->placements[i];
+            if (p.wave != wave) continue;
+            slot_of_expert[p.expert] = int16_t(p.slot);
+            if (p.missed) {
+                if (!any_copy) {
+                    if (int rc = order_copy_after_readers(c, layer)) return rc;
+                    if (wave > 0) CU(c, cudaStreamWaitEvent(c->copy, c->wave_done, 0));
+                    any_copy = true;
+                }
+                if (int rc = issue_copy(c, layer, p.expert, p.slot)) return rc;
+            }
+        }
+        for (size_t i = 0; i < c->placements.size(); ++i) {
+            const Placement& p = c->placements[i];
+            if (p.wave != wave) continue;
+            const size_t k = size_t(layer) * c->S + p.slot;
+            if (!c->slot_pending[k]) continue;
+            cudaError_t q = cudaEventQuery(c->slot_ev[k]);
+            if (q == cudaErrorNotReady) {
+                if (!p.missed) c->extra_late++;
+                CU(c, cudaStreamWaitEvent(c->compute, c->slot_ev[k], 0));
+            } else if (q != cudaSuccess) {
+                return fail(c, SPM_ERR_CUDA, "copy event query: %s", cudaGetErrorString(q));
+            }
+            c->slot_pending[k] = 0;
+        }
+
+        const bool first = wave == 0, last = wave == n_waves - 1;
+        auto fill = [&](auto& a) {
+            a.pool = slot_ptr(c, layer, 0);
+            a.shared = m.n_shared ? static_cast<const unsigned char*>(c->buf.shared_experts) + size_t(layer) * m.n_shared * c->blob : nullptr;
+            a.x = x_norm;
+            a.w = w;
+            a.partial = c->ws_partial;
+            a.status = c->ws_status;
+            a.blob_bytes = c->blob;
+            a.I = m.inter; a.K = K; a.n_slots = c->S; a.n_shared = m.n_shared;
+            for (int tk = 0; tk < nb; ++tk) {
+                int cnt = 0;
+                for (int k = 0; k < K; ++k) {
+                    const int s = slot_of_expert[ids[tk * K + k]];
+                    if (s < 0) continue;
+                    a.code[tk * SPM_MAX_TOPK + cnt] = short(s);
+                    a.kidx[tk * SPM_MAX_TOPK + cnt] = (unsigned char)k;
+                    ++cnt;
+                }
+                if (first)
+                    for (int s = 0; s < m.n_shared; ++s) {
+                        a.code[tk * SPM_MAX_TOPK + cnt] = short(-1 - s);
+                        a.kidx[tk * SPM_MAX_TOPK + cnt] = 255;
+                        ++cnt;
+                    }
+                a.count[tk] = (unsigned char)cnt;
+            }
+        };
+        if (t && first) CU(c, cudaEventRecord(t->ffn_start[layer], c->compute));
+        if (nb == 1) {
+            FfnArgs<1> a{};
+            fill(a);
+            CU(c, launch_gemv<1>(c, a, G, nb));
+        } else {
+            FfnArgs<SPM_MAX_BATCH> a{};
+            fill(a);
+            CU(c, launch_gemv<SPM_MAX_BATCH>(c, a, G, nb));
+        }
+        if (t && last) CU(c, cudaEventRecord(t->ffn_end[layer], c->compute));
+        ffn_reduce_kernel<<<dim3((m.hidden + 127) / 128, nb), 128, 0, c->compute>>>(c->ws_partial, h_inout, h_inout, G, m.hidden);
+        CU(c, cudaGetLastError());
+        c->kernel_launches += 2;
+        c->ffn_launches++;
+        if (!last) CU(c, cudaEventRecord(c->wave_done, c->compute));
+    }
+    CU(c, cudaEventRecord(c->pool_free[layer], c->compute));
+    c->pool_free_valid[layer] = 1;
+    if (t) t->used[layer] = 1;
+    return SPM_OK;
+}
+
+int do_prefetch(spm_ctx* c, int target, const int32_t* ids, int count, const int32_t* protect, int n_protect,
+                int* out_issued) {
+    SlotTable& tb = *c->table;
+    c->slots_tmp.assign(size_t(std::max(count, 1)), -1);
+    const int issued = tb.prefetch(target, ids, count, protect, n_protect, c->drop_modulo, c->slots_tmp.data());
+    if (issued > 0) {
+        if (int rc = order_copy_after_readers(c, target)) return rc;
+        for (int i = 0; i < count; ++i)
+            if (c->slots_tmp[i] >= 0)
+                if (int rc = issue_copy(c, target, ids[i], c->slots_tmp[i])) return rc;
+    }
+    if (out_issued) *out_issued = issued;
+    return SPM_OK;
+}
+
+int check_layer(spm_ctx* c, int layer, int nb) {
+    if (!c) return SPM_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, SPM_ERR_INVALID_ARG, "layer %d out of range", layer);
+    if (nb < 1 || nb > c->cfg.max_batch) return fail(c, SPM_ERR_INVALID_ARG, "nb %d out of range (max_batch %d)", nb, c->cfg.max_batch);
+    return SPM_OK;
+}
+
+int check_status(spm_ctx* c) {
+    int st = 0;
+    CU(c, cudaMemcpy(&st, c->ws_status, sizeof st, cudaMemcpyDeviceToHost));
+    if (st & kStatusCopyTimeout) return fail(c, SPM_ERR_TIMEOUT, "expert FFN kernel gave up waiting for a weight copy");
+    if (st & kStatusBadSlot) return fail(c, SPM_ERR_NOT_RESIDENT, "expert FFN kernel received a slot number outside the pool");
+    return SPM_OK;
+}
+
+}  // namespace
+
+// ============================================================================
+extern "C" {
+
+int spm_expert_blob_bytes(const spm_model_cfg* cfg, size_t* bytes) {
+    if (!cfg || !bytes) return SPM_ERR_INVALID_ARG;
+    *bytes = blob_bytes_of(cfg);
+    return SPM_OK;
+}
+
+int spm_query_arena(const spm_model_cfg* cfg, int slots_per_layer, size_t* bytes) {
+    if (!bytes) return SPM_ERR_INVALID_ARG;
+    if (int rc = check_cfg(cfg, slots_per_layer, nullptr)) return rc;
+    *bytes = layout_of(cfg, slots_per_layer).total;
+    return SPM_OK;
+}
+
+const char* spm_last_error(const spm_ctx* ctx) { return ctx ? ctx->err.c_str() : g_init_error.c_str(); }
+
+int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const spm_buffers* b, spm_ctx** out) {
+    if (!out || !b) return fail(nullptr, SPM_ERR_INVALID_ARG, "null argument");
+    *out = nullptr;
+    if (int rc = check_cfg(cfg, slots_per_layer, nullptr)) return rc;
+    if (budget < -1) return fail(nullptr, SPM_ERR_INVALID_ARG, "budget %d", budget);
+    if (!b->rms_gamma || !b->router_w || !b->host_experts || !b->arena) return fail(nullptr, SPM_ERR_INVALID_ARG, "a required buffer is null");
+    if (cfg->n_layers > 1 && (!b->adapter_a || !b->adapter_b)) return fail(nullptr, SPM_ERR_INVALID_ARG, "adapter buffers are null");
+    if (cfg->n_shared > 0 && !b->shared_experts) return fail(nullptr, SPM_ERR_INVALID_ARG, "shared_experts is null");
+    if (b->compute_stream == b->copy_stream) return fail(nullptr, SPM_ERR_INVALID_ARG, "compute and copy stream must differ");
+    if (reinterpret_cast<uintptr_t>(b->arena) % 256) return fail(nullptr, SPM_ERR_INVALID_ARG, "arena must be 256-byte aligned");
+    const Layout lay = layout_of(cfg, slots_per_layer);
+    if (b->arena_bytes < lay.total) return fail(nullptr, SPM_ERR_INVALID_ARG, "arena too small: %zu < %zu", b->arena_bytes, lay.total);
+
+    int dev_count = 0;
+    cudaError_t e = cudaGetDeviceCount(&dev_count);
+    if (e != cudaSuccess || dev_count == 0)
+        return fail(nullptr, SPM_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(e));
+
+    spm_ctx* c = new spm_ctx();
+    c->cfg = *cfg;
+    c->S = slots_per_layer;
+    c->buf = *b;
+    c->compute = static_cast<cudaStream_t>(b->compute_stream);
+    c->copy = static_cast<cudaStream_t>(b->copy_stream);
+    c->elem = cfg->dtype == SPM_DTYPE_BF16 ? 2 : 4;
+    c->blob = blob_bytes_of(cfg);
+    c->row_bytes = size_t(3) * cfg->hidden * c->elem;
+    c->nseg = cfg->hidden / (cfg->dtype == SPM_DTYPE_BF16 ? 256 : 128);
+    c->depth = int(std::min<size_t>(4, (232448 - 1024) / (size_t(kFfnWarps) * c->row_bytes)));
+    auto bail = [&](int rc) { g_init_error = c->err; spm_destroy(c); return rc; };
+    if (c->depth < 1) { c->err = "hidden too large for the shared-memory ring"; return bail(SPM_ERR_CONFIG); }
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceProp prop{};
+    if (cudaGetDeviceProperties(&prop, dev) == cudaSuccess) c->num_sms = prop.multiProcessorCount;
+    if (prop.major != 10) { c->err = "this library is built for sm_100a (B200) only"; return bail(SPM_ERR_CONFIG); }
+
+    unsigned char* base = static_cast<unsigned char*>(b->arena);
+    c->pools = base + lay.pools;
+    c->ws_x = reinterpret_cast<float*>(base + lay.x);
+    c->ws_logits = reinterpret_cast<float*>(base + lay.logits);
+    c->ws_u = reinterpret_cast<float*>(base + lay.u);
+    c->ws_pihat = reinterpret_cast<float*>(base + lay.pihat);
+    c->ws_w = reinterpret_cast<float*>(base + lay.w);
+    c->ws_scores = reinterpret_cast<float*>(base + lay.scores);
+    c->ws_partial = reinterpret_cast<float*>(base + lay.partial);
+    c->ws_h = reinterpret_cast<float*>(base + lay.h);
+    c->ws_ids = reinterpret_cast<int32_t*>(base + lay.ids);
+    c->ws_order = reinterpret_cast<int32_t*>(base + lay.order);
+    c->ws_counters = reinterpret_cast<unsigned*>(base + lay.counters);
+    c->ws_status = reinterpret_cast<int*>(base + lay.status);
+
+    const int L = cfg->n_layers;
+    c->table = new SlotTable(L, cfg->n_experts, c->S, false);
+    c->pending_protect.resize(L);
+    c->has_plan.assign(L, 0);
+    c->layer_stall_us.assign(L, 0.0);
+    c->layer_ffn_us.assign(L, 0.0);
+    c->slot_pending.assign(size_t(L) * c->S, 0);
+    c->pool_free_valid.assign(L, 0);
+
+    auto cu = [&](cudaError_t err, const char* what) {
+        if (err == cudaSuccess) return true;
+        c->err = std::string(what) + " failed: " + cudaGetErrorString(err);
+        return false;
+    };
+    if (!cu(cudaMemsetAsync(base + lay.counters, 0, lay.total - lay.counters, c->compute), "cudaMemsetAsync")) return bail(SPM_ERR_CUDA);
+    if (!cu(cudaHostAlloc(reinterpret_cast<void**>(&c->mb_host), sizeof(Mailbox), cudaHostAllocMapped), "cudaHostAlloc(mailbox)")) return bail(SPM_ERR_CUDA);
+    memset(c->mb_host, 0, sizeof(Mailbox));
+    if (!cu(cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->mb_dev), c->mb_host, 0), "cudaHostGetDevicePointer")) return bail(SPM_ERR_CUDA);
+    c->slot_ev.resize(size_t(L) * c->S);
+    for (auto& ev : c->slot_ev) if (!cu(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming), "cudaEventCreate")) return bail(SPM_ERR_CUDA);
+    c->pool_free.resize(L);
+    for (auto& ev : c->pool_free) if (!cu(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming), "cudaEventCreate")) return bail(SPM_ERR_CUDA);
+    if (!cu(cudaEventCreateWithFlags(&c->wave_done, cudaEventDisableTiming), "cudaEventCreate")) return bail(SPM_ERR_CUDA);
+    for (auto& t : c->tim) {
+        t.k1_done.resize(L); t.ffn_start.resize(L); t.ffn_end.resize(L); t.used.assign(L, 0);
+        for (int l = 0; l < L; ++l)
+            if (!cu(cudaEventCreate(&t.k1_done[l]), "cudaEventCreate") || !cu(cudaEventCreate(&t.ffn_start[l]), "cudaEventCreate") ||
+                !cu(cudaEventCreate(&t.ffn_end[l]), "cudaEventCreate")) return bail(SPM_ERR_CUDA);
+    }
+    if (!cu(cudaStreamSynchronize(c->compute), "cudaStreamSynchronize")) return bail(SPM_ERR_CUDA);
+
+    c->budget = budget < 0 ? 1 : budget;
+    if (budget < 0) {
+        double W = 0, tx = 0;
+        int raw = 0;
+        int rc = spm_profile_window(c, &W, &tx, &raw);
+        if (rc) return bail(rc);
+        c->budget = std::max(1, raw);
+    }
+    *out = c;
+    return SPM_OK;
+}
+
+int spm_destroy(spm_ctx* c) {
+    if (!c) return SPM_OK;
+    if (c->compute) cudaStreamSynchronize(c->compute);
+    if (c->copy) cudaStreamSynchronize(c->copy);
+    for (auto ev : c->slot_ev) if (ev) cudaEventDestroy(ev);
+    for (auto ev : c->pool_free) if (ev) cudaEventDestroy(ev);
+    if (c->wave_done) cudaEventDestroy(c->wave_done);
+    for (auto& t : c->tim) {
+        for (auto ev : t.k1_done) if (ev) cudaEventDestroy(ev);
+        for (auto ev : t.ffn_start) if (ev) cudaEventDestroy(ev);
+        for (auto ev : t.ffn_end) if (ev) cudaEventDestroy(ev);
+    }
+    if (c->mb_host) cudaFreeHost(c->mb_host);
+    delete c->table;
+    delete c;
+    return SPM_OK;
+}
+
+int spm_router_topk(spm_ctx* c, int layer, const float* h, int nb, float* x_norm, int32_t* ids, float* w,
+                    float* logits) {
+    if (int rc = check_layer(c, layer, nb)) return rc;
+    if (!h || !x_norm || !ids || !w) return fail(c, SPM_ERR_INVALID_ARG, "null argument");
+    if (int rc = launch_router(c, layer, h, nullptr, nb, x_norm, logits, true, false)) return rc;
+    CU(c, cudaMemcpyAsync(w, c->ws_w, size_t(nb) * c->cfg.top_k * 4, cudaMemcpyDeviceToDevice, c->compute));
+    if (int rc = wait_mailbox(c)) return rc;
+    memcpy(ids, c->mb_host->ids, size_t(nb) * c->cfg.top_k * 4);
+    return SPM_OK;
+}
+
+int spm_adapter_predict(spm_ctx* c, int layer, const float* x_norm, int nb, float* scores, int32_t* order) {
+    if (int rc = check_layer(c, layer, nb)) return rc;
+    if (layer > c->cfg.n_layers - 2) return fail(c, SPM_ERR_INVALID_ARG, "layer %d has no adapter (L-1 adapters)", layer);
+    if (!x_norm || !scores || !order) return fail(c, SPM_ERR_INVALID_ARG, "null argument");
+    if (int rc = launch_router(c, layer, nullptr, x_norm, nb, nullptr, nullptr, false, true)) return rc;
+    if (int rc = wait_mailbox(c)) return rc;
+    memcpy(scores, c->mb_host->scores, size_t(c->cfg.n_experts) * 4);
+    memcpy(order, c->mb_host->order, size_t(c->cfg.n_experts) * 4);
+    return SPM_OK;
+}
+
+int spm_budget_select(spm_ctx* c, int target, const int32_t* order, int n_ranked, int budget, int protect_all,
+                      int32_t* out_ids, int* out_count) {
+    if (int rc = check_layer(c, target, 1)) return rc;
+    if (!order || !out_ids || !out_count || n_ranked < 0 || n_ranked > c->cfg.n_experts)
+        return fail(c, SPM_ERR_INVALID_ARG, "bad ranking argument");
+    for (int i = 0; i < n_ranked; ++i)
+        if (order[i] < 0 || order[i] >= c->cfg.n_experts) return fail(c, SPM_ERR_INVALID_ARG, "expert id %d out of range", order[i]);
+    const int bud = budget < 0 ? c->budget : budget;
+    c->table->plan(target, order, n_ranked, bud, protect_all != 0, c->sel, c->pending_protect[target]);
+    c->has_plan[target] = 1;
+    std::copy(c->sel.begin(), c->sel.end(), out_ids);
+    *out_count = int(c->sel.size());
+    return SPM_OK;
+}
+
+int spm_prefetch_async(spm_ctx* c, int target, const int32_t* ids, int count, int* out_issued) {
+    if (int rc = check_layer(c, target, 1)) return rc;
+    if (count < 0 || (count > 0 && !ids)) return fail(c, SPM_ERR_INVALID_ARG, "bad id list");
+    for (int i = 0; i < count; ++i)
+        if (ids[i] < 0 || ids[i] >= c->cfg.n_experts) return fail(c, SPM_ERR_INVALID_ARG, "expert id %d out of range", ids[i]);
+    const std::vector<int32_t> none;
+    const std::vector<int32_t>& prot = c->has_plan[target] ? c->pending_protect[target] : none;
+    int rc = do_prefetch(c, target, ids, count, prot.data(), int(prot.size()), out_issued);
+    c->has_plan[target] = 0;
+    return rc;
+}
+
+int spm_moe_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, const float* w, int nb, float* h_inout) {
+    if (int rc = check_layer(c, layer, nb)) return rc;
+    if (!x_norm || !ids || !w || !h_inout) return fail(c, SPM_ERR_INVALID_ARG, "null argument");
+    return run_ffn(c, layer, x_norm, ids, w, nb, h_inout, nullptr);
+}
+
+int spm_decode_step(spm_ctx* c, const float* h_in, int nb, float* h_out) {
+    if (int rc = check_layer(c, 0, nb)) return rc;
+    if (!h_in || !h_out) return fail(c, SPM_ERR_INVALID_ARG, "null argument");
+    const spm_model_cfg& m = c->cfg;
+    const int L = m.n_layers, K = m.top_k, n = m.n_experts;
+    SlotTable& tb = *c->table;
+    if (c->policy == SPM_POLICY_HINT_TRACE && tb.step() >= c->hint_steps)
+        return fail(c, SPM_ERR_STATE, "no hint trace for step %d", tb.step());
+    if (h_out != h_in)
+        CU(c, cudaMemcpyAsync(h_out, h_in, size_t(nb) * m.hidden * 4, cudaMemcpyDeviceToDevice, c->compute));
+    Timing* t = nullptr;
+    if (c->timing) {
+        c->tim_cur ^= 1;
+        t = &c->tim[c->tim_cur];
+        harvest(c, *t);
+    }
+    const bool predict = c->policy == SPM_POLICY_ADAPTER || c->policy == SPM_POLICY_PRED0;
+    c->prev_order_valid = false;
+    std::vector<int32_t> ids(size_t(nb) * K);
+    for (int l = 0; l < L; ++l) {
+        const bool has_adapter = l <= L - 2;
+        if (int rc = launch_router(c, l, h_out, nullptr, nb, c->ws_x, nullptr, true, predict && has_adapter)) return rc;
+        if (t) CU(c, cudaEventRecord(t->k1_done[l], c->compute));
+        if (int rc = wait_mailbox(c)) return rc;
+        memcpy(ids.data(), c->mb_host->ids, ids.size() * 4);
+
+        if (c->prev_order_valid) {   // ExpertRecall@M of the previous layer's prediction, M = budget
+            const int M = std::min(c->budget, n);
+            for (int tk = 0; tk < nb; ++tk) {
+                int hit = 0;
+                for (int k = 0; k < K; ++k)
+                    for (int q = 0; q < M; ++q) hit += c->prev_order[q] == ids[tk * K + k];
+                c->recall_sum += double(hit) / K;
+                c->recall_count++;
+            }
+        }
+        if (int rc = run_ffn(c, l, c->ws_x, ids.data(), c->ws_w, nb, h_out, t)) return rc;
+
+        c->prev_order_valid = false;
+        if (has_adapter && c->policy != SPM_POLICY_ON_DEMAND) {
+            const int32_t* ranking;
+            int n_ranked;
+            bool protect_all = false;
+            if (c->policy == SPM_POLICY_HINT_TRACE) {
+                const size_t cell = size_t(tb.step()) * L + (l + 1);
+                ranking = c->hint.data() + cell * c->hint_stride;
+                n_ranked = c->hint_count[cell];
+                protect_all = true;
+            } else {
+                c->prev_order.assign(c->mb_host->order, c->mb_host->order + n);
+                c->prev_order_valid = true;
+                ranking = c->prev_order.data();
+                n_ranked = n;
+            }
+            tb.plan(l + 1, ranking, n_ranked, c->budget, protect_all, c->sel, c->protect);
+            if (c->policy == SPM_POLICY_PRED0) {
+                tb.plan_only(l + 1, c->sel.data(), int(c->sel.size()));
+            } else {
+                if (int rc = do_prefetch(c, l + 1, c->sel.data(), int(c->sel.size()), c->protect.data(),
+                                         int(c->protect.size()), nullptr)) return rc;
+            }
+        }
+    }
+    tb.end_step();
+    tb.stats().steps++;
+    c->tokens += nb;
+    return SPM_OK;
+}
+
+int spm_decode_step_host(spm_ctx* c, const float* h_in_host, int nb, float* h_out_host) {
+    if (int rc = check_layer(c, 0, nb)) return rc;
+    if (!h_in_host || !h_out_host) return fail(c, SPM_ERR_INVALID_ARG, "null argument");
+    const size_t bytes = size_t(nb) * c->cfg.hidden * 4;
+    CU(c, cudaMemcpyAsync(c->ws_h, h_in_host, bytes, cudaMemcpyHostToDevice, c->compute));
+    if (int rc = spm_decode_step(c, c->ws_h, nb, c->ws_h)) return rc;
+    CU(c, cudaMemcpyAsync(h_out_host, c->ws_h, bytes, cudaMemcpyDeviceToHost, c->compute));
+    CU(c, cudaStreamSynchronize(c->compute));
+    return SPM_OK;
+}
+
+// ---- control --------------------------------------------------------------
+int spm_set_policy(spm_ctx* c, int policy) {
+    if (!c) return SPM_ERR_INVALID_ARG;
+    if (policy < SPM_POLICY_ADAPTER || policy > SPM_POLICY_PRED0) return fail(c, SPM_ERR_INVALID_ARG, "policy %d", policy);
+    if (policy != SPM_POLICY_ON_DEMAND && c->cfg.n_layers > 1 && (!c->buf.adapter_a || !c->buf.adapter_b) && policy != SPM_POLICY_HINT_TRACE)
+        return fail(c, SPM_ERR_STATE, "no adapter weights");
+    c->policy = policy;
+    return SPM_OK;
+}
+int spm_set_budget(spm_ctx* c, int budget) {
+    if (!c) return SPM_ERR_INVALID_ARG;
+    if (budget < 0) return fail(c, SPM_ERR_INVALID_ARG, "budget %d", budget);
+    c->budget = budget;
+    return SPM_OK;
+}
+int spm_get_budget(spm_ctx* c, int* budget) {
+    if (!c || !budget) return SPM_ERR_INVALID_ARG;
+    *budget = c->budget;
+    return SPM_OK;
+}
+int spm_set_plain_lru(spm_ctx* c, int on) {
+    if (!c) return SPM_ERR_INVALID_ARG;
+    c->table->set_plain_lru(on != 0);
+    return SPM_OK;
+}
+int spm_set_timing(spm_ctx* c, int on) {
+    if (!c) return SPM_ERR_INVALID_ARG;
+    c->timing = on != 0;
+    return SPM_OK;
+}
+int spm_set_ffn_ctas(spm_ctx* c, int ctas) {
+    if (!c) return SPM_ERR_INVALID_ARG;
+    if (ctas < 0 || ctas > kMaxCtasBatch1) return fail(c, SPM_ERR_INVALID_ARG, "ctas %d (max %d)", ctas, kMaxCtasBatch1);
+    c->ffn_ctas = ctas;
+    return SPM_OK;
+}
+int spm_set_hint_trace(spm_ctx* c, const int32_t* hint, const int32_t* count, int n_steps, int stride) {
+    if (!c) return SPM_ERR_INVALID_ARG;
+    if (!hint || !count || n_steps < 0 || stride < 1) return fail(c, SPM_ERR_INVALID_ARG, "bad hint trace");
+    const size_t cells = size_t(n_steps) * c->cfg.n_layers;
+    for (size_t i = 0; i < cells; ++i) {
+        if (count[i] < 0 || count[i] > stride) return fail(c, SPM_ERR_INVALID_ARG, "hint count out of range");
+        for (int q = 0; q < count[i]; ++q)
+            if (hint[i * stride + q] < 0 || hint[i * stride + q] >= c->cfg.n_experts)
+                return fail(c, SPM_ERR_INVALID_ARG, "hint expert id out of range");
+    }
+    c->hint.assign(hint, hint + cells * stride);
+    c->hint_count.assign(count, count + cells);
+    c->hint_steps = n_steps;
+    c->hint_stride = stride;
+    return SPM_OK;
+}
+int spm_set_drop_modulo(spm_ctx* c, int modulo) {
+    if (!c || modulo < 0) return SPM_ERR_INVALID_ARG;
+    c->drop_modulo = modulo;
+    return SPM_OK;
+}
+int spm_set_deadline_ms(spm_ctx* c, int ms) {
+    if (!c || ms < 1) return SPM_ERR_INVALID_ARG;
+    c->deadline_ms = ms;
+    return SPM_OK;
+}
+
+int spm_synchronize(spm_ctx* c) {
+    if (!c) return SPM_ERR_INVALID_ARG;
+    CU(c, cudaStreamSynchronize(c->copy));
+    CU(c, cudaStreamSynchronize(c->compute));
+    return check_status(c);
+}
+
+int spm_cache_reset(spm_ctx* c) {
+    if (!c) return SPM_ERR_INVALID_ARG;
+    CU(c, cudaStreamSynchronize(c->copy));
+    CU(c, cudaStreamSynchronize(c->compute));
+    for (auto& t : c->tim) std::fill(t.used.begin(), t.used.end(), 0);
+    c->table->reset();
+    std::fill(c->slot_pending.begin(), c->slot_pending.end(), 0);
+    std::fill(c->has_plan.begin(), c->has_plan.end(), 0);
+    std::fill(c->layer_stall_us.begin(), c->layer_stall_us.end(), 0.0);
+    std::fill(c->layer_ffn_us.begin(), c->layer_ffn_us.end(), 0.0);
+    c->timed_steps = 0;
+    c->extra_late = c->h2d_bytes = c->ffn_launches = c->kernel_launches = c->tokens = 0;
+    c->ready_sum = c->recall_sum = 0;
+    c->ready_count = c->recall_count = 0;
+    c->prev_order_valid = false;
+    return SPM_OK;
+}
+
+int spm_profile_window(spm_ctx* c, double* window_us, double* t_xfer_us, int* budget_raw) {
+    if (!c || !window_us || !t_xfer_us || !budget_raw) return SPM_ERR_INVALID_ARG;
+    if (int rc = spm_cache_reset(c)) return rc;
+    const spm_model_cfg& m = c->cfg;
+    const int K = std::min(m.top_k, c->S);
+    const int pools = std::min(m.n_layers, 4);
+    cudaEvent_t e0, e1;
+    CU(c, cudaEventCreate(&e0));
+    CU(c, cudaEventCreate(&e1));
+    // expert transfer: one blob from the pinned store into a slot, timed on the copy stream
+    std::vector<float> tx;
+    for (int it = 0; it < 11; ++it) {
+        const int layer = it % pools, e = it % m.n_experts;
+        CU(c, cudaEventRecord(e0, c->copy));
+        CU(c, cudaMemcpyAsync(slot_ptr(c, layer, it % K), host_blob(c, layer, e), c->blob, cudaMemcpyHostToDevice, c->copy));
+        CU(c, cudaEventRecord(e1, c->copy));
+        CU(c, cudaEventSynchronize(e1));
+        float ms = 0;
+        CU(c, cudaEventElapsedTime(&ms, e0, e1));
+        if (it >= 2) tx.push_back(ms * 1e3f);
+    }
+    // make the first K slots of a few pools valid experts, then time the FFN over them,
+    // cycling through the pools so that the weights come from HBM, not from L2
+    for (int layer = 0; layer < pools; ++layer)
+        for (int s = 0; s < K; ++s)
+            CU(c, cudaMemcpyAsync(slot_ptr(c, layer, s), host_blob(c, layer, s % m.n_experts), c->blob, cudaMemcpyHostToDevice, c->copy));
+    CU(c, cudaStreamSynchronize(c->copy));
+    std::vector<float> wv(K, 1.0f / K);
+    CU(c, cudaMemcpyAsync(c->ws_w, wv.data(), size_t(K) * 4, cudaMemcpyHostToDevice, c->compute));
+    CU(c, cudaMemsetAsync(c->ws_x, 0, size_t(m.hidden) * 4, c->compute));
+    std::vector<float> wt;
+    const int G = ffn_grid_for(c, 1);
+    for (int it = 0; it < 14; ++it) {
+        const int layer = it % pools;
+        FfnArgs<1> a{};
+        a.pool = slot_ptr(c, layer, 0);
+        a.shared = m.n_shared ? static_cast<const unsigned char*>(c->buf.shared_experts) + size_t(layer) * m.n_shared * c->blob : nullptr;
+        a.x = c->ws_x; a.w = c->ws_w; a.partial = c->ws_partial; a.status = c->ws_status;
+        a.blob_bytes = c->blob; a.I = m.inter; a.K = m.top_k; a.n_slots = c->S; a.n_shared = m.n_shared;
+        int cnt = 0;
+        for (int k = 0; k < K; ++k) { a.code[cnt] = short(k); a.kidx[cnt] = (unsigned char)k; ++cnt; }
+        for (int s = 0; s < m.n_shared; ++s) { a.code[cnt] = short(-1 - s); a.kidx[cnt] = 255; ++cnt; }
+        a.count[0] = (unsigned char)cnt;
+        CU(c, cudaEventRecord(e0, c->compute));
+        CU(c, launch_gemv<1>(c, a, G, 1));
+        CU(c, cudaEventRecord(e1, c->compute));
+        CU(c, cudaEventSynchronize(e1));
+        float ms = 0;
+        CU(c, cudaEventElapsedTime(&ms, e0, e1));
+        if (it >= 5) wt.push_back(ms * 1e3f);
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    std::sort(tx.begin(), tx.end());
+    std::sort(wt.begin(), wt.end());
+    *t_xfer_us = tx[tx.size() / 2];
+    *window_us = wt[wt.size() / 2];
+    *budget_raw = int(*window_us / *t_xfer_us);
+    if (int rc = check_status(c)) return rc;
+    return spm_cache_reset(c);
+}
+
+int spm_get_stats(spm_ctx* c, spm_stats* out) {
+    if (!c || !out) return SPM_ERR_INVALID_ARG;
+    CU(c, cudaStreamSynchronize(c->copy));
+    CU(c, cudaStreamSynchronize(c->compute));
+    for (auto& t : c->tim) harvest(c, t);
+    *out = c->table->stats();
+    out->tokens = c->tokens;
+    out->late_arrivals = c->extra_late;
+    out->h2d_bytes = c->h2d_bytes;
+    out->ffn_launches = c->ffn_launches;
+    out->kernel_launches = c->kernel_launches;
+    out->ffn_us = 0;
+    out->stall_us = 0;
+    for (int l = 0; l < c->cfg.n_layers; ++l) { out->ffn_us += c->layer_ffn_us[l]; out->stall_us += c->layer_stall_us[l]; }
+    out->ready_sum = c->ready_sum; out->ready_count = c->ready_count;
+    out->recall_sum = c->recall_sum; out->recall_count = c->recall_count;
+    return check_status(c);
+}
+
+int spm_get_layer_times(spm_ctx* c, double* stall_us, double* ffn_us, uint64_t* steps) {
+    if (!c || !stall_us || !ffn_us || !steps) return SPM_ERR_INVALID_ARG;
+    CU(c, cudaStreamSynchronize(c->compute));
+    for (auto& t : c->tim) harvest(c, t);
+    for (int l = 0; l < c->cfg.n_layers; ++l) { stall_us[l] = c->layer_stall_us[l]; ffn_us[l] = c->layer_ffn_us[l]; }
+    *steps = c->timed_steps;
+    return SPM_OK;
+}
+
+int spm_get_events(spm_ctx* c, spm_event* out, size_t capacity, size_t* count) {
+    if (!c || !count) return SPM_ERR_INVALID_ARG;
+    const auto& ev = c->table->events();
+    *count = ev.size();
+    if (out) memcpy(out, ev.data(), std::min(capacity, ev.size()) * sizeof(spm_event));
+    return SPM_OK;
+}
+
+int spm_get_slot_table(spm_ctx* c, int layer, int32_t* slot_expert) {
+    if (int rc = check_layer(c, layer, 1)) return rc;
+    if (!slot_expert) return SPM_ERR_INVALID_ARG;
+    for (int s = 0; s < c->S; ++s) slot_expert[s] = c->table->expert_in(layer, s);
+    return SPM_OK;
+}
+
+int spm_host_alloc(size_t bytes, void** out) {
+    if (!out || bytes == 0) return SPM_ERR_INVALID_ARG;
+    cudaError_t e = cudaHostAlloc(out, bytes, cudaHostAllocDefault);
+    if (e != cudaSuccess) { g_init_error = std::string("cudaHostAlloc failed: ") + cudaGetErrorString(e); *out = nullptr; return SPM_ERR_CUDA; }
+    return SPM_OK;
+}
+int spm_host_free(void* p) {
+    if (!p) return SPM_OK;
+    return cudaFreeHost(p) == cudaSuccess ? SPM_OK : SPM_ERR_CUDA;
+}
+
+// ---- host-only simulator ----------------------------------------------------
+}  // extern "C"
+
+struct spm_sim {
+    SlotTable table;
+    std::vector<Placement> placements;
+    std::vector<int32_t> sel, protect;
+    spm_sim(int L, int n, int S, bool plain) : table(L, n, S, plain) {}
+};
+
+extern "C" {
+
+int spm_sim_create(int n_layers, int n_experts, int slots, int plain_lru, spm_sim** out) {
+    if (!out || n_layers < 1 || n_experts < 1 || n_experts > SPM_MAX_EXPERTS || slots < 1) return SPM_ERR_INVALID_ARG;
+    *out = new spm_sim(n_layers, n_experts, slots, plain_lru != 0);
+    return SPM_OK;
+}
+int spm_sim_destroy(spm_sim* s) { delete s; return SPM_OK; }
+
+static bool sim_ids_ok(spm_sim* s, int layer, const int32_t* ids, int count) {
+    if (!s || layer < 0 || layer >= s->table.layers() || count < 0 || (count > 0 && !ids)) return false;
+    for (int i = 0; i < count; ++i) if (ids[i] < 0 || ids[i] >= s->table.experts()) return false;
+    return true;
+}
+
+int spm_sim_demand(spm_sim* s, int layer, const int32_t* need, int count, int32_t* out_expert, int32_t* out_slot,
+                   int32_t* out_wave, int32_t* out_missed, int* out_count, int* out_waves) {
+    if (!sim_ids_ok(s, layer, need, count) || !out_expert || !out_slot || !out_wave || !out_missed || !out_count) return SPM_ERR_INVALID_ARG;
+    int waves = 1;
+    s->table.demand(layer, need, count, s->placements, &waves);
+    for (size_t i = 0; i < s->placements.size(); ++i) {
+        out_expert[i] = s->placements[i].expert; out_slot[i] = s->placements[i].slot;
+        out_wave[i] = s->placements[i].wave; out_missed[i] = s->placements[i].missed;
+    }
+    *out_count = int(s->placements.size());
+    if (out_waves) *out_waves = waves;
+    return SPM_OK;
+}
+
+int spm_sim_plan(spm_sim* s, int layer, const int32_t* order, int n_ranked, int budget, int protect_all,
+                 int32_t* out_ids, int* out_count, int32_t* out_protect, int* out_n_protect) {
+    if (!sim_ids_ok(s, layer, order, n_ranked) || budget < 0 || !out_ids || !out_count || !out_protect || !out_n_protect) return SPM_ERR_INVALID_ARG;
+    s->table.plan(layer, order, n_ranked, budget, protect_all != 0, s->sel, s->protect);
+    std::copy(s->sel.begin(), s->sel.end(), out_ids);
+    std::copy(s->protect.begin(), s->protect.end(), out_protect);
+    *out_count = int(s->sel.size());
+    *out_n_protect = int(s->protect.size());
+    return SPM_OK;
+}
+
+int spm_sim_prefetch(spm_sim* s, int layer, const int32_t* ids, int count, const int32_t* protect, int n_protect,
+                     int drop_modulo, int32_t* out_slots, int* out_issued) {
+    if (!sim_ids_ok(s, layer, ids, count) || !sim_ids_ok(s, layer, protect, n_protect) || !out_slots || drop_modulo < 0) return SPM_ERR_INVALID_ARG;
+    int issued = s->table.prefetch(layer, ids, count, protect, n_protect, drop_modulo, out_slots);
+    if (out_issued) *out_issued = issued;
+    return SPM_OK;
+}
+
+int spm_sim_plan_only(spm_sim* s, int layer, const int32_t* ids, int count) {
+    if (!sim_ids_ok(s, layer, ids, count)) return SPM_ERR_INVALID_ARG;
+    s->table.plan_only(layer, ids, count);
+    return SPM_OK;
+}
+
+int spm_sim_end_step(spm_sim* s) {
+    if (!s) return SPM_ERR_INVALID_ARG;
+    s->table.end_step();
+    s->table.stats().steps++;
+    return SPM_OK;
+}
+
+int spm_sim_events(spm_sim* s, spm_event* out, size_t capacity, size_t* count) {
+    if (!s || !count) return SPM_ERR_INVALID_ARG;
+    const auto& ev = s->table.events();
+    *count = ev.size();
+    if (out) memcpy(out, ev.data(), std::min(capacity, ev.size()) * sizeof(spm_event));
+    return SPM_OK;
+}
+
+int spm_sim_stats(spm_sim* s, spm_stats* out) {
+    if (!s || !out) return SPM_ERR_INVALID_ARG;
+    *out = s->table.stats();
+    return SPM_OK;
+}
+
+int spm_sim_slot_table(spm_sim* s, int layer, int32_t* slot_expert) {
+    if (!s || !slot_expert || layer < 0 || layer >= s->table.layers()) return SPM_ERR_INVALID_ARG;
+    for (int i = 0; i < s->table.slots(); ++i) slot_expert[i] = s->table.expert_in(layer, i);
+    return SPM_OK;
+}
+
+}  // extern "C"

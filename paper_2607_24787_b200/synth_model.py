@@ -1,0 +1,55 @@
+"""Builds an OffloadedMoE from the counter-based synthetic generator (module `synth`): weights
+are generated on the GPU layer by layer, packed, and copied down into the pinned expert store."""
+from __future__ import annotations
+
+import torch
+
+import synth
+
+from .model import OffloadedMoE, PinnedStore, pack_experts
+
+
+def fill_store(cfg: synth.ModelCfg, store: PinnedStore, device, chunk: int = 32):
+    """Generate and pack every routed expert of every layer into the pinned host store."""
+    blob = cfg.expert_bytes
+    for l in range(cfg.n_layers):
+        for e0 in range(0, cfg.n_experts, chunk):
+            es = range(e0, min(e0 + chunk, cfg.n_experts))
+            g, u, d = synth.expert_matrices(cfg, l, es, device=device)
+            packed = pack_experts(g, u, d).view(torch.uint8).reshape(-1)
+            off = (l * cfg.n_experts + e0) * blob
+            store.tensor[off:off + packed.numel()].copy_(packed)
+            del g, u, d, packed
+    torch.cuda.synchronize(device)
+
+
+def build_from_synth(cfg: synth.ModelCfg, slots=None, budget=None, max_batch=None, device="cuda:0",
+                     store: PinnedStore | None = None) -> OffloadedMoE:
+    """Random-init model of the configuration's shape, experts offloaded to pinned host memory."""
+    dev = torch.device(device)
+    L = cfg.n_layers
+    gamma = torch.ones(L, cfg.hidden, dtype=torch.float32, device=dev)
+    router = torch.stack([synth.router_w(cfg, l, dev) for l in range(L)]).contiguous()
+    if L > 1:
+        a = torch.stack([synth.adapter_a(cfg, l, dev) for l in range(L - 1)]).contiguous()
+        b = torch.stack([synth.adapter_b(cfg, l, dev) for l in range(L - 1)]).contiguous()
+    else:
+        a = b = None
+    shared = None
+    if cfg.n_shared:
+        per_layer = []
+        for l in range(L):
+            g, u, d = synth.expert_matrices(cfg, l, range(cfg.n_experts, cfg.n_experts + cfg.n_shared), dev)
+            per_layer.append(pack_experts(g, u, d))
+        shared = torch.stack(per_layer).contiguous()
+    if store is None:
+        store = PinnedStore(L * cfg.n_experts * cfg.expert_bytes)
+        fill_store(cfg, store, dev)
+    return OffloadedMoE(n_layers=L, hidden=cfg.hidden, n_experts=cfg.n_experts, inter=cfg.inter,
+                        top_k=cfg.top_k, n_shared=cfg.n_shared, adapter_rank=cfg.adapter_rank,
+                        dtype=cfg.dtype, renormalize=cfg.renormalize, rms_eps=cfg.rms_eps,
+                        max_batch=cfg.batch if max_batch is None else max_batch,
+                        slots=cfg.slots if slots is None else slots,
+                        budget=cfg.budget if budget is None else budget,
+                        gamma=gamma, router_w=router, adapter_a=a, adapter_b=b, shared_blobs=shared,
+                        store=store, device=device)

@@ -1,0 +1,111 @@
+"""CPU-only checks of the C-ABI library: it builds for sm_100a, loads without a GPU, exports every
+symbol include/spm.h declares, and its host-side slot table matches the policy oracle bit for bit."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import ref_policy as P
+from paper_2607_24787_b200 import binding as B
+from paper_2607_24787_b200.build import build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def lib():
+    build()
+    return B.load()
+
+
+def test_header_symbols_exported(lib):
+    hdr = open(os.path.join(ROOT, "include", "spm.h")).read()
+    declared = sorted(set(re.findall(r"\b(spm_[a-z0-9_]+)\s*\(", hdr)))
+    assert declared == B.EXPORTS, set(declared) ^ set(B.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_query_and_config_errors():
+    cfg = B.make_cfg(48, 2048, 128, 768, 8, 0, 16, B.DTYPE_BF16)
+    assert B.spm_expert_blob_bytes(cfg) == 9437184
+    assert B.spm_query_arena(cfg, 16) > 48 * 16 * 9437184
+    with pytest.raises(B.SpmError) as e:
+        B.spm_query_arena(cfg, 4)                       # slots < top_k at batch 1
+    assert e.value.code == -2
+    with pytest.raises(B.SpmError):
+        B.spm_query_arena(B.make_cfg(2, 1000, 16, 128, 2, 0, 8, B.DTYPE_BF16), 4)   # hidden not a multiple of 256
+    with pytest.raises(B.SpmError):
+        B.spm_query_arena(B.make_cfg(2, 256, 16, 128, 2, 15, 8, B.DTYPE_FP32), 4)   # top_k + shared too large
+
+
+def test_init_fails_loudly_without_gpu():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("has a GPU")
+    cfg = B.make_cfg(2, 256, 16, 128, 2, 0, 8, B.DTYPE_FP32)
+    buf = B.Buffers(256, 256, 256, 256, None, 256, 256, 1 << 40, 1, 2)
+    with pytest.raises(B.SpmError) as e:
+        B.spm_init(cfg, 4, 2, buf)
+    assert e.value.code == -3
+
+
+def drive(policy_obj, trace, ranks, L, budget, mode, drop=0):
+    """Feed one recorded trace to either the oracle SlotPolicy or the library's Sim."""
+    for t, per_layer in enumerate(trace):
+        for l in range(L):
+            policy_obj.demand(l, per_layer[l])
+            if l <= L - 2 and mode != "on_demand":
+                if mode == "hint":
+                    sel, prot = policy_obj.plan(l + 1, per_layer[l + 1], budget, True)
+                else:
+                    sel, prot = policy_obj.plan(l + 1, ranks[t][l], budget, False)
+                if mode == "pred0":
+                    policy_obj.plan_only(l + 1, sel)
+                elif isinstance(policy_obj, P.SlotPolicy):
+                    dropped = {e for e in sel if drop and (policy_obj.step + e) % drop == 0}
+                    policy_obj.prefetch(l + 1, sel, prot, dropped)
+                else:
+                    policy_obj.prefetch(l + 1, sel, prot, drop)
+        if isinstance(policy_obj, P.SlotPolicy):
+            policy_obj.step += 1
+        else:
+            policy_obj.end_step()
+
+
+@pytest.mark.parametrize("mode,S,budget,nb,plain,drop", [
+    ("adapter", 4, 2, 1, False, 0), ("adapter", 8, 3, 1, True, 0), ("hint", 6, 2, 1, False, 0),
+    ("pred0", 4, 2, 1, False, 0), ("on_demand", 5, 0, 1, False, 0), ("adapter", 5, 2, 7, False, 0),
+    ("adapter", 3, 4, 9, False, 3), ("hint", 16, 8, 4, False, 0), ("adapter", 16, 1, 1, False, 2),
+])
+def test_slot_table_matches_policy_oracle(mode, S, budget, nb, plain, drop):
+    L, n, K, steps = 3, 24, 3, 80
+    rng = np.random.default_rng(hash((mode, S, budget, nb)) % (1 << 31))
+    trace, ranks = [], []
+    for _ in range(steps):
+        trace.append([sorted({int(e) for _ in range(nb) for e in rng.permutation(n)[:K]}) for _ in range(L)])
+        ranks.append([[int(e) for e in rng.permutation(n)] for _ in range(L)])
+    ref = P.SlotPolicy(L, n, S, plain)
+    sim = B.Sim(L, n, S, plain)
+    drive(ref, trace, ranks, L, budget, mode, drop)
+    drive(sim, trace, ranks, L, budget, mode, drop)
+    assert sim.events() == ref.events
+    st = sim.stats()
+    for k in ("hits", "hits_prefetched", "misses", "evictions", "wasted", "prefetch_issued", "touches",
+              "waves", "planned"):
+        assert st[k] == getattr(ref.stats, k), k
+    for l in range(L):
+        assert sim.slot_table(l) == ref.pools[l].slot_expert
+    sim.close()
+
+
+def test_sim_rejects_bad_arguments():
+    sim = B.Sim(2, 8, 3)
+    with pytest.raises(B.SpmError):
+        sim.demand(5, [1])
+    with pytest.raises(B.SpmError):
+        sim.demand(0, [99])
+    with pytest.raises(B.SpmError):
+        sim.plan(1, [0, 1, 8], 2)
+    sim.close()

@@ -1,0 +1,276 @@
+"""GPU parity: every spm_* entry point against the CPU oracle on the same seeded inputs.
+
+Tolerances (max|a-b| / max|b| per output vector): 1e-5 for fp32 weights; the target for bf16
+weights with fp32 accumulation is 2e-2, and because this path keeps activations in fp32 the test
+holds it to 1e-4. Integer results (expert ids, rankings, prefetch sets, cache events) are bit-exact
+given identical logits / scores; end to end they are bit-exact except at flagged near-ties.
+"""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from helpers import SynthWeights, f64, make_ref
+from oracle import ref_decode, ref_math as M, ref_policy as P
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"fp32": 1e-5, "bf16": 1e-4}
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2607_24787_b200.build import build
+    build()
+
+
+def gpu_model(cfg, **kw):
+    from paper_2607_24787_b200.synth_model import build_from_synth
+    return build_from_synth(cfg, **kw)
+
+
+def dev(a):
+    t = torch.as_tensor(np.ascontiguousarray(a), dtype=torch.float32).cuda()
+    torch.cuda.synchronize()
+    return t
+
+
+def host(t, m):
+    m.synchronize()
+    return t.detach().cpu().numpy().astype(np.float64)
+
+
+SHAPES = {
+    "tiny": synth.get_config("tiny"),
+    # bf16, several 256-wide segments, row count (K+shared)*I not a multiple of the CTA count
+    "ds_small": synth.get_config("dsvl2", n_layers=3, n_experts=16, inter=224, slots=8, budget=2),
+    "qw_small": synth.get_config("qwen3", n_layers=2, n_experts=24, inter=96, slots=10, budget=3),
+    "odd": synth.get_config("tiny", hidden=384, inter=50, n_experts=11, top_k=3, adapter_rank=5, slots=5, seed=7),
+}
+
+
+@pytest.fixture(scope="module", params=list(SHAPES))
+def setup(request, lib):
+    cfg = SHAPES[request.param]
+    m = gpu_model(cfg)
+    wts = SynthWeights(cfg)
+    tok = synth.zipf_tokens(cfg, steps=24)
+    H = synth.embedding_rows(cfg, tok[:, 0]).numpy()
+    yield cfg, m, wts, H
+    m.close()
+
+
+# ---------------------------------------------------------------- per-call parity (P1)
+def test_router_topk(setup):
+    cfg, m, wts, H = setup
+    for layer in range(cfg.n_layers):
+        h = H[3 * layer:3 * layer + 1]
+        x, ids, w, logits = m.router_topk(layer, dev(h), want_logits=True)
+        xr = M.rmsnorm(h[0], wts.gamma(layer), cfg.rms_eps)
+        zr = M.router_logits(wts.router(layer), xr)
+        ids_r, w_r = M.route(zr, cfg.top_k, bool(cfg.renormalize))
+        assert M.rel_linf(host(x, m)[0], xr) < TOL[cfg.dtype]
+        z = host(logits, m)[0]
+        assert M.rel_linf(z, zr) < TOL[cfg.dtype]
+        # bit-exact given identical logits: the oracle's Top-K of the GPU's own logits
+        assert list(ids[0]) == list(M.top_k(z.astype(np.float32), cfg.top_k))
+        if not M.near_tie(zr, cfg.top_k):
+            assert list(ids[0]) == list(ids_r)
+            assert M.rel_linf(host(w, m)[0], w_r) < TOL[cfg.dtype]
+        assert abs(host(w, m)[0].sum() - 1.0) < 1e-6
+
+
+def test_adapter_predict(setup):
+    cfg, m, wts, H = setup
+    for layer in range(cfg.n_layers - 1):
+        x = np.stack([M.rmsnorm(H[i], wts.gamma(layer), cfg.rms_eps) for i in range(2)]).astype(np.float32)
+        if m.max_batch < 2:
+            x = x[:1]
+        scores, order = m.adapter_predict(layer, dev(x))
+        A, Bup = wts.adapter(layer)
+        s_r = M.adapter_scores(A, Bup, x)
+        assert M.rel_linf(scores, s_r) < TOL[cfg.dtype]
+        assert list(order) == list(M.rank_desc(scores))               # ranking of its own scores: bit-exact
+        assert abs(scores.sum() - x.shape[0]) < 1e-5
+    with pytest.raises(Exception):
+        m.adapter_predict(cfg.n_layers - 1, dev(H[:1]))               # only L-1 adapters exist
+
+
+def test_moe_ffn_resident_and_offloaded(setup):
+    cfg, m, wts, H = setup
+    m.cache_reset()
+    for it in range(6):
+        layer = it % cfg.n_layers
+        h = H[it:it + 1]
+        x = M.rmsnorm(h[0], wts.gamma(layer), cfg.rms_eps)
+        ids_r, w_r = M.route(M.router_logits(wts.router(layer), x), cfg.top_k, bool(cfg.renormalize))
+        y = M.moe_ffn(x, ids_r, w_r, lambda e: wts.expert(layer, e), wts.shared(layer))
+        hd = dev(h)
+        m.moe_ffn(layer, dev(x[None]), ids_r[None].astype(np.int32), dev(w_r[None]), hd)
+        got = host(hd, m)[0]
+        assert M.rel_linf(got - h[0], y) < TOL[cfg.dtype], (layer, it)
+        assert M.rel_linf(got, h[0] + y) < TOL[cfg.dtype]
+    st = m.stats()
+    assert st["misses"] + st["hits"] == 6 * cfg.top_k and st["h2d_bytes"] == st["misses"] * cfg.expert_bytes
+
+
+def test_budget_select_and_prefetch_match_policy_oracle(setup):
+    cfg, m, wts, H = setup
+    m.cache_reset()
+    rng = np.random.default_rng(3)
+    ref = P.SlotPolicy(cfg.n_layers, cfg.n_experts, cfg.slots)
+    hd = dev(H[:1])
+    for it in range(12):
+        layer = 1 + it % (cfg.n_layers - 1)
+        ranking = [int(e) for e in rng.permutation(cfg.n_experts)]
+        sel_r, prot_r = ref.plan(layer, ranking, 2)
+        issued_r = ref.prefetch(layer, sel_r, prot_r)
+        sel = m.budget_select(layer, ranking, budget=2)
+        assert list(sel) == sel_r
+        assert m.prefetch_async(layer, sel) == len(issued_r)
+        need = sorted(int(e) for e in rng.permutation(cfg.n_experts)[:cfg.top_k])
+        ref.demand(layer, need)
+        x = dev(H[it:it + 1])
+        m.moe_ffn(layer, x, np.array([need], np.int32), dev(np.full((1, cfg.top_k), 1.0 / cfg.top_k)), hd)
+        assert list(m.slot_table(layer)) == ref.pools[layer].slot_expert
+    m.synchronize()
+    assert m.events() == ref.events
+
+
+# ---------------------------------------------------------------- whole decode step (P2, P3)
+def run_gpu(m, H, steps, nb=1):
+    outs = []
+    for s in range(steps):
+        out = m.decode_step(dev(H[s * nb:(s + 1) * nb]))
+        outs.append(host(out, m))
+    return np.stack(outs)
+
+
+def run_ref(cfg, wts, H, steps, nb=1, hint=None, **kw):
+    ref = make_ref(cfg, weights=wts, **kw)
+    outs, recs = [], []
+    for s in range(steps):
+        h, r = ref.step(H[s * nb:(s + 1) * nb], hint=None if hint is None else hint[s])
+        outs.append(h); recs.append(r)
+    return ref, np.stack(outs), recs
+
+
+def fragile(recs, K, budget):
+    """Steps/layers whose decisions sit on a near-tie in the oracle (logits or priorities)."""
+    flags = set()
+    for s, step in enumerate(recs):
+        for l, r in enumerate(step):
+            if any(M.near_tie(r.logits[t], K) for t in range(r.logits.shape[0])):
+                flags.add((s, l))
+            if r.scores is not None:
+                srt = np.sort(r.scores)[::-1]
+                if np.any((srt[:-1] - srt[1:]) / srt[:-1] < 1e-5):
+                    flags.add((s, l))
+    return flags
+
+
+@pytest.mark.parametrize("policy", ["adapter", "on_demand", "pred0", "hint_trace"])
+def test_decode_step_free_running(setup, policy):
+    cfg, m, wts, H = setup
+    steps = 24 if cfg.n_experts * cfg.inter * cfg.hidden < 3e6 else 8
+    budget = cfg.budget if cfg.budget >= 0 else 2
+    _, base_out, base_recs = run_ref(cfg, wts, H, steps, slots=cfg.n_experts, policy=P.ON_DEMAND, budget=budget)
+    hint = ref_decode.true_demand_trace(base_recs)
+    ref, out_r, recs = run_ref(cfg, wts, H, steps, policy=policy, budget=budget, hint=hint)
+    m.cache_reset()
+    m.set_policy(policy)
+    m.set_budget(budget)
+    if policy == "hint_trace":
+        m.set_hint_trace(hint)
+    out = run_gpu(m, H, steps)
+    for s in range(steps):
+        assert M.rel_linf(out[s], out_r[s]) < 4 * TOL[cfg.dtype], s      # error accumulates over L layers
+    ev = m.events()
+    if ev != ref.table.events:
+        # only acceptable when the oracle itself sits on a near-tie somewhere before the divergence
+        first = next(i for i, (a, b) in enumerate(zip(ev, ref.table.events)) if a != b)
+        s_bad, l_bad = ref.table.events[first][0], ref.table.events[first][1]
+        fl = fragile(recs, cfg.top_k, budget)
+        assert any(fs < s_bad or (fs == s_bad and fl_ <= l_bad) for fs, fl_ in fl), (first, ev[first], ref.table.events[first])
+        pytest.xfail("near-tie in the oracle's own decisions")
+    st = m.stats()
+    for k in ("hits", "hits_prefetched", "misses", "evictions", "wasted", "prefetch_issued", "touches", "planned"):
+        assert st[k] == getattr(ref.table.stats, k), k
+    if policy in ("adapter", "pred0"):
+        rr = np.mean([M.expert_recall_at_m(recs[s][l + 1].ids, recs[s][l].scores, min(budget, cfg.n_experts), cfg.top_k)
+                      for s in range(steps) for l in range(cfg.n_layers - 1)])
+        assert abs(st["recall_sum"] / st["recall_count"] - rr) < 1e-9
+    rdy = np.mean([recs[s][l].ready for s in range(steps) for l in range(1, cfg.n_layers)])
+    assert abs(st["ready_sum"] / st["ready_count"] - rdy) < 1e-9
+
+
+def test_router_preserving_bitwise_on_gpu(setup):
+    cfg, m, wts, H = setup
+    steps = 10
+    outs = {}
+    _, _, base_recs = run_ref(cfg, wts, H, steps, slots=cfg.n_experts, policy=P.ON_DEMAND, budget=1)
+    hint = ref_decode.true_demand_trace(base_recs)
+    for name, policy, budget, drop, plain in (("od", "on_demand", 0, 0, 0), ("ad", "adapter", 2, 0, 0),
+                                              ("ad4", "adapter", 4, 0, 1), ("drop", "adapter", 3, 2, 0),
+                                              ("hint", "hint_trace", cfg.top_k, 0, 0), ("p0", "pred0", 2, 0, 0)):
+        m.cache_reset()
+        m.set_policy(policy); m.set_budget(budget); m.set_drop_modulo(drop); m.set_plain_lru(plain)
+        if policy == "hint_trace":
+            m.set_hint_trace(hint)
+        outs[name] = run_gpu(m, H, steps)
+    m.set_drop_modulo(0); m.set_plain_lru(0)
+    for name in outs:
+        assert np.array_equal(outs[name], outs["od"]), name       # outputs never depend on the policy
+    # and a fully-resident context gives the same bits
+    full = gpu_model(cfg, slots=cfg.n_experts, budget=0)
+    full.set_policy("on_demand")
+    assert np.array_equal(run_gpu(full, H, steps), outs["od"])
+    full.close()
+
+
+def test_decode_step_host_matches_device(setup):
+    cfg, m, wts, H = setup
+    m.cache_reset(); m.set_policy("adapter"); m.set_budget(2)
+    a = run_gpu(m, H, 4)
+    m.cache_reset()
+    hin = torch.from_numpy(H[:4].copy()).pin_memory()
+    hout = torch.empty(1, cfg.hidden).pin_memory()
+    for s in range(4):
+        m.decode_step_host(hin[s:s + 1], hout)
+        assert np.array_equal(hout.numpy().astype(np.float64), a[s])
+
+
+# ---------------------------------------------------------------- batched decode, waves
+@pytest.mark.parametrize("slots,nb", [(3, 6), (16, 5)])
+def test_batched_decode_with_waves(lib, slots, nb):
+    cfg = synth.get_config("tiny", batch=nb, slots=slots)
+    m = gpu_model(cfg)
+    wts = SynthWeights(cfg)
+    steps = 5
+    tok = synth.zipf_tokens(cfg, steps=steps)
+    H = synth.embedding_rows(cfg, tok.reshape(-1)).numpy()
+    ref, out_r, recs = run_ref(cfg, wts, H, steps, nb=nb, slots=slots, budget=2)
+    out = run_gpu(m, H, steps, nb=nb)
+    for s in range(steps):
+        for t in range(nb):
+            assert M.rel_linf(out[s][t], out_r[s][t]) < 4e-5
+    assert m.events() == ref.table.events
+    if slots == 3:
+        assert m.stats()["waves"] > 0
+    m.close()
+
+
+def test_argument_errors(setup):
+    cfg, m, wts, H = setup
+    from paper_2607_24787_b200 import binding as B
+    with pytest.raises(B.SpmError):
+        m.moe_ffn(cfg.n_layers, dev(H[:1]), np.zeros((1, cfg.top_k), np.int32), dev(np.ones((1, cfg.top_k))), dev(H[:1]))
+    with pytest.raises(B.SpmError):
+        m.moe_ffn(0, dev(H[:1]), np.full((1, cfg.top_k), cfg.n_experts, np.int32), dev(np.ones((1, cfg.top_k))), dev(H[:1]))
+    with pytest.raises(B.SpmError):
+        m.set_budget(-3)
+    m.set_policy("hint_trace"); m.cache_reset()
+    B.spm_set_hint_trace(m.ctx, [])
+    with pytest.raises(B.SpmError):
+        m.decode_step(dev(H[:1]))                                  # no hint for step 0
+    m.set_policy("adapter")
