@@ -117,7 +117,9 @@ typedef struct {
     uint64_t h2d_bytes;          /* expert bytes copied host -> HBM                                      */
     uint64_t ffn_launches;       /* expert-FFN kernel launches timed below                               */
     uint64_t kernel_launches;    /* all kernels this context launched                                    */
-    double   ffn_us;             /* summed device time of those launches (needs spm_set_timing(ctx, 1))  */
+    double   ffn_us;             /* summed CUDA-event time around those launches (needs spm_set_timing(ctx, 1)) */
+    double   ffn_window_us;      /* same launches, first CTA start to last CTA end read from %globaltimer
+                                    inside the kernel: excludes launch latency (profiling aid)            */
     double   stall_us;           /* summed gap "routing kernel done -> expert FFN may start" per layer    */
     double   ready_sum;          /* sum over (step, layer >= 1, token) of |T ∩ has-slot| / K at demand   */
     uint64_t ready_count;        /*   ... and the number of terms (ReadyRecall = ready_sum / ready_count) */
@@ -219,6 +221,7 @@ int spm_set_deadline_ms(spm_ctx* ctx, int ms);
 int spm_profile_window(spm_ctx* ctx, double* window_us, double* t_xfer_us, int* budget_raw);
 
 int spm_cache_reset(spm_ctx* ctx);                         /* cold cache, step counter, stats, events */
+int spm_reset_stats(spm_ctx* ctx);                         /* counters, timings and event log only; cache kept */
 int spm_get_stats(spm_ctx* ctx, spm_stats* out);           /* waits for timed work to finish */
 /* Per-layer sums since the last reset: stall_us[L], ffn_us[L], and the number of steps in them. */
 int spm_get_layer_times(spm_ctx* ctx, double* stall_us, double* ffn_us, uint64_t* steps);

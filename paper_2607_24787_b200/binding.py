@@ -51,7 +51,7 @@ class Stats(C.Structure):
     _fields_ = ([(k, C.c_uint64) for k in ("steps", "tokens", "hits", "hits_prefetched", "misses", "evictions",
                                            "wasted", "prefetch_issued", "touches", "waves", "planned", "dropped",
                                            "late_arrivals", "h2d_bytes", "ffn_launches", "kernel_launches")]
-                + [("ffn_us", C.c_double), ("stall_us", C.c_double), ("ready_sum", C.c_double),
+                + [("ffn_us", C.c_double), ("ffn_window_us", C.c_double), ("stall_us", C.c_double), ("ready_sum", C.c_double),
                    ("ready_count", C.c_uint64), ("recall_sum", C.c_double), ("recall_count", C.c_uint64)])
 
     def as_dict(self):
@@ -83,6 +83,7 @@ _SIG = {
     "spm_set_deadline_ms": [_P, C.c_int],
     "spm_profile_window": [_P, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int)],
     "spm_cache_reset": [_P],
+    "spm_reset_stats": [_P],
     "spm_get_stats": [_P, C.POINTER(Stats)],
     "spm_get_layer_times": [_P, _P, _P, C.POINTER(C.c_uint64)],
     "spm_get_events": [_P, _P, C.c_size_t, C.POINTER(C.c_size_t)],
@@ -268,6 +269,10 @@ def spm_profile_window(ctx):
 
 def spm_cache_reset(ctx):
     _check(load().spm_cache_reset(ctx), ctx)
+
+
+def spm_reset_stats(ctx):
+    _check(load().spm_reset_stats(ctx), ctx)
 
 
 def spm_get_stats(ctx) -> dict:

@@ -11,7 +11,8 @@
 // Work decomposition: the (expert, j) rows of a token are split evenly over gridDim.x CTAs; in
 // a CTA each warp owns a private ring of row buffers in shared memory that lane 0 keeps full
 // with 1-D bulk async copies (cp.async.bulk + mbarrier byte counting, no multicast), so about
-// 190 KB per SM are in flight without costing registers. Per-warp partial y vectors live in
+// 170-220 KB per SM are in flight without costing registers. The host picks the number of warps
+// per CTA so that rows divide evenly: the kernel ends when its busiest warp does. Per-warp partial y vectors live in
 // registers, are summed across warps in a fixed order through shared memory, and each CTA
 // writes one partial row; ffn_reduce_kernel adds the partials in CTA order (deterministic, so
 // outputs are bitwise reproducible for a given launch geometry).
@@ -22,8 +23,8 @@
 
 namespace spm {
 
-constexpr int kFfnWarps = 8;
-constexpr int kFfnThreads = kFfnWarps * 32;
+constexpr int kFfnMaxWarps = 9;                    // 9 * 32 threads * 216 registers fit one SM
+constexpr int kFfnMaxThreads = kFfnMaxWarps * 32;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s: give up, set status, return
 
 // kernel status bits (device int, read by the host)
@@ -38,6 +39,7 @@ struct FfnArgs {
     const float* w;                 // [nb][K] routing weights
     float* partial;                 // [nb][gridDim.x][D]
     int* status;
+    unsigned long long* clock;      // optional {earliest CTA start, latest CTA end} in ns (globaltimer)
     unsigned long long blob_bytes;
     int I, K, n_slots, n_shared;
     unsigned char count[MAXNB];                     // expert entries of token t in this launch
@@ -46,14 +48,20 @@ struct FfnArgs {
 };
 
 template <typename WT, int NSEG, int MAXNB>
-__global__ void __launch_bounds__(kFfnThreads, 1)
+__global__ void __launch_bounds__(kFfnMaxThreads, 1)
 ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
     constexpr int VEC = 16 / int(sizeof(WT));
     constexpr int D = NSEG * 32 * VEC;
     constexpr uint32_t ROWB = 3u * D * sizeof(WT);
 
     extern __shared__ __align__(128) unsigned char smem[];
+#ifdef SPM_FFN_TIMESTAMPS
+    const unsigned long long ts_start = global_timer_ns();
+    unsigned long long ts_first = 0, ts_loop = 0;
+#endif
     const int wi = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nw = blockDim.x >> 5;      // warps per CTA, chosen by the host to balance rows per warp
+    if (a.clock && threadIdx.x == 0) atomicMin(a.clock, global_timer_ns());
     const int tok = blockIdx.y;
     const int G = gridDim.x, c = blockIdx.x;
     const int I = a.I;
@@ -61,10 +69,10 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
     const int r_begin = int((long long)R * c / G);
     const int r_end = int((long long)R * (c + 1) / G);
     const int span = r_end - r_begin - wi;
-    const int my_n = span > 0 ? (span + kFfnWarps - 1) / kFfnWarps : 0;
+    const int my_n = span > 0 ? (span + nw - 1) / nw : 0;
 
     unsigned char* ring = smem + size_t(wi) * depth * ROWB;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + size_t(kFfnWarps) * depth * ROWB);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + size_t(nw) * depth * ROWB);
     const uint32_t bar0 = smem_u32(bars + wi * depth);
     const uint32_t ring0 = smem_u32(ring);
 
@@ -78,7 +86,7 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
     bool ok = true;
 
     auto issue = [&](int i) {
-        const int r = r_begin + wi + i * kFfnWarps;
+        const int r = r_begin + wi + i * nw;
         const int ent = r / I;
         const int j = r - ent * I;
         const int code = a.code[tok * SPM_MAX_TOPK + ent];
@@ -136,7 +144,10 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
                 break;
             }
             done = i + 1;
-            const int r = r_begin + wi + i * kFfnWarps;
+#ifdef SPM_FFN_TIMESTAMPS
+            if (i == 0) ts_first = global_timer_ns();
+#endif
+            const int r = r_begin + wi + i * nw;
             const int ent = r / I;
             if (ent != cur_ent) {
                 cur_ent = ent;
@@ -183,6 +194,9 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
             if (!mbar_wait_bounded(bar0 + 8u * (i % depth), (i / depth) & 1, kWaitLimitNs)) break;
     }
 
+#ifdef SPM_FFN_TIMESTAMPS
+    ts_loop = global_timer_ns();
+#endif
     // sum the warps' partial y in warp order, one partial row per CTA
     __syncthreads();
     float* red = reinterpret_cast<float*>(smem);
@@ -194,35 +208,81 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
                 make_float4(ya[s][v], ya[s][v + 1], ya[s][v + 2], ya[s][v + 3]);
     __syncthreads();
     float* out = a.partial + (size_t(tok) * G + c) * D;
-    for (int d = threadIdx.x; d < D; d += kFfnThreads) {
+    for (int d = threadIdx.x; d < D; d += blockDim.x) {
         float acc = red[d];
-#pragma unroll
-        for (int w2 = 1; w2 < kFfnWarps; ++w2) acc += red[w2 * D + d];
+        for (int w2 = 1; w2 < nw; ++w2) acc += red[w2 * D + d];
         out[d] = acc;
     }
-}
-
-// h_out[t][d] = h_in[t][d] + sum over CTAs (in CTA order) of partial[t][c][d]
-__global__ void ffn_reduce_kernel(const float* __restrict__ partial, const float* h_in, float* h_out,
-                                  int G, int D) {
-    const int tok = blockIdx.y;
-    const int d = blockIdx.x * blockDim.x + threadIdx.x;
-    if (d >= D) return;
-    const float* p = partial + size_t(tok) * G * D + d;
-    float acc = 0.f;
-    int c = 0;
-    for (; c + 4 <= G; c += 4) {
-        const float p0 = p[size_t(c) * D], p1 = p[size_t(c + 1) * D];
-        const float p2 = p[size_t(c + 2) * D], p3 = p[size_t(c + 3) * D];
-        acc += p0; acc += p1; acc += p2; acc += p3;
+    if (a.clock) {
+        __syncthreads();
+        if (threadIdx.x == 0) atomicMax(a.clock + 1, global_timer_ns());
     }
-    for (; c < G; ++c) acc += p[size_t(c) * D];
-    h_out[size_t(tok) * D + d] = h_in[size_t(tok) * D + d] + acc;
+#ifdef SPM_FFN_TIMESTAMPS
+    // profiling aid: per-warp phase times, appended behind the partial rows
+    if (lane == 0) {
+        unsigned long long* ts = reinterpret_cast<unsigned long long*>(a.partial + size_t(gridDim.y) * G * D) + (size_t(c) * nw + wi) * 4;
+        ts[0] = ts_start; ts[1] = ts_first; ts[2] = ts_loop; ts[3] = global_timer_ns();
+    }
+#endif
 }
 
-// Shared-memory bytes of the GEMV kernel for a row of `row_bytes` and ring depth `depth`.
-inline size_t ffn_gemv_smem(size_t row_bytes, int depth) {
-    return size_t(kFfnWarps) * depth * row_bytes + size_t(kFfnWarps) * depth * 8;
+// h_out[t][d] = h_in[t][d] + sum over CTAs (in CTA order) of partial[t][c][d].
+// A block owns kReduceCols columns; its kReduceGroups thread groups each sum a contiguous run of
+// partial rows (all loads of a thread are independent, so they are in flight together), and the
+// group sums are combined in group order: the summation order is fixed by (G, launch geometry).
+constexpr int kReduceCols = 32;
+constexpr int kReduceGroups = 8;
+constexpr int kReduceMaxRows = 40;     // rows per group: kReduceGroups * kReduceMaxRows >= max G
+
+__global__ void __launch_bounds__(kReduceCols * kReduceGroups)
+ffn_reduce_kernel(const float* __restrict__ partial, const float* h_in, float* h_out, int G, int D) {
+    __shared__ float part[kReduceGroups][kReduceCols];
+    const int tok = blockIdx.y;
+    const int col = threadIdx.x % kReduceCols, grp = threadIdx.x / kReduceCols;
+    const int d = blockIdx.x * kReduceCols + col;
+    const int per = (G + kReduceGroups - 1) / kReduceGroups;
+    const int c0 = grp * per, c1 = min(G, c0 + per);
+    const float* p = partial + size_t(tok) * G * D + d;
+    float v[kReduceMaxRows];
+#pragma unroll
+    for (int i = 0; i < kReduceMaxRows; ++i) v[i] = (d < D && c0 + i < c1) ? __ldcg(p + size_t(c0 + i) * D) : 0.f;
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < kReduceMaxRows; ++i) acc += v[i];
+    part[grp][col] = acc;
+    __syncthreads();
+    if (grp == 0 && d < D) {
+        float tot = part[0][col];
+#pragma unroll
+        for (int g = 1; g < kReduceGroups; ++g) tot += part[g][col];
+        h_out[size_t(tok) * D + d] = h_in[size_t(tok) * D + d] + tot;
+    }
+}
+
+constexpr size_t kFfnSmemLimit = 232448;   // 227 KB per CTA
+
+// Shared-memory bytes of the GEMV kernel: `warps` private rings of `depth` rows + their barriers.
+inline size_t ffn_gemv_smem(size_t row_bytes, int warps, int depth) {
+    return size_t(warps) * depth * row_bytes + size_t(warps) * depth * 8;
+}
+
+// Launch shape for `rows_per_cta` rows of `row_bytes`: the warp count that leaves the fewest rows
+// on the busiest warp (the kernel ends when that warp does), then the most bytes in flight.
+inline void ffn_gemv_shape(size_t row_bytes, int rows_per_cta, int* warps, int* depth) {
+    int best_w = 0, best_d = 0, best_cost = 1 << 30;
+    size_t best_flight = 0;
+    for (int w = 4; w <= kFfnMaxWarps; ++w) {
+        int d = int((kFfnSmemLimit - 1024) / (size_t(w) * row_bytes));
+        if (d > 4) d = 4;
+        if (d < 2 && !(w == 4 && d == 1)) continue;      // want double buffering; 4 warps x 1 is the last resort
+        const int cost = (rows_per_cta + w - 1) / w;
+        const size_t flight = size_t(w) * d * row_bytes;
+        if (cost < best_cost || (cost == best_cost && flight > best_flight)) {
+            best_w = w; best_d = d; best_cost = cost; best_flight = flight;
+        }
+    }
+    *warps = best_w;
+    *depth = best_d;
 }
 
 }  // namespace spm

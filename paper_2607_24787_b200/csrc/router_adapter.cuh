@@ -5,11 +5,13 @@
 // Adapter (Section 3.2): u = A x; z^ = Bup u; pi^ = softmax(z^); s_e = sum over tokens of pi^_e
 // in token order; the experts of the next layer are ranked by (s descending, id ascending).
 //
-// Grid (C, nb): the C CTAs of a token split the n + r weight rows (one warp per row, 16-byte
-// read-only loads, shuffle reduction). The last CTA of a token to finish (atomic ticket) does
-// that token's softmax / Top-K / adapter tail; the last token-tail to finish does the batch
-// aggregation and ranking, copies ids / order / scores into the host-mapped mailbox, fences at
-// system scope and publishes the launch's sequence number, which the host polls.
+// One thread-block cluster per token: its CTAs split the n + r weight rows (one warp per row,
+// 16-byte read-only loads all issued before the first use, shuffle reduction) and store the dot
+// products into the leader CTA's shared memory over DSMEM; after one cluster barrier the leader
+// does the token's softmax / Top-K / adapter tail. With several tokens the last leader to
+// finish (atomic ticket) does the batch aggregation. The publishing CTA ranks the priorities,
+// copies ids / order / scores into the host-mapped mailbox, fences at system scope and writes
+// the launch's sequence number, which the host polls.
 // Every reduction has a fixed order, so results are bitwise reproducible.
 #pragma once
 
@@ -94,23 +96,64 @@ __device__ __forceinline__ int rank_of(const float* v, int n, int e) {
     return c;
 }
 
+constexpr int kRouterCluster = 8;   // CTAs per token, one thread-block cluster
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// store one float into the shared memory of CTA `rank` of this cluster (same offset as `local`)
+__device__ __forceinline__ void dsmem_store(float* local, uint32_t rank, float v) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local)), "r"(rank));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+template <typename WT>
+__device__ __forceinline__ float load_weight(const WT* p, size_t i) {
+    if (sizeof(WT) == 2) return __uint_as_float(uint32_t(reinterpret_cast<const uint16_t*>(p)[i]) << 16);
+    return reinterpret_cast<const float*>(p)[i];
+}
+
+// Grid (kRouterCluster, nb), cluster (kRouterCluster, 1, 1): the CTAs of a cluster split the n + r
+// weight rows of one token and deliver their dot products straight into the leader CTA's shared
+// memory; after one cluster barrier the leader alone runs the softmax / Top-K / adapter tail.
 template <typename WT>
 __global__ void __launch_bounds__(kRouterThreads)
 router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     constexpr int VEC = 16 / int(sizeof(WT));
+    constexpr int MAXIT = 8;        // hidden <= MAXIT * 32 * VEC
     extern __shared__ __align__(16) float sm[];
     float* xs = sm;                 // [D]
-    float* zs = xs + a.D;           // [n] logits -> probabilities
-    float* ps = zs + a.n;           // [n] adapter logits -> probabilities / scores
-    float* scratch = ps + a.n;      // [8] + small tails
-    float* psel = scratch + kRouterWarps;           // [K]
-    int* isel = reinterpret_cast<int*>(psel + SPM_MAX_TOPK);   // [K]
-    float* us = reinterpret_cast<float*>(isel + SPM_MAX_TOPK); // [r]
+    float* zs = xs + a.D;           // [n] logits (leader: filled by the whole cluster)
+    float* ps = zs + a.n;           // [n] probabilities / adapter logits / scores
+    float* us = ps + a.n;           // [r] adapter hidden (leader: filled by the whole cluster)
+    float* scratch = us + a.r;      // [8]
+    float* psel = scratch + kRouterWarps;                       // [K]
+    int* isel = reinterpret_cast<int*>(psel + SPM_MAX_TOPK);    // [K]
+    float* bs = reinterpret_cast<float*>(isel + SPM_MAX_TOPK);  // [n * r] adapter up-projection (leader)
     __shared__ int s_last;
 
-    const int tok = blockIdx.y, C = gridDim.x;
+    const int tok = blockIdx.y;
+    const uint32_t cr = cluster_ctarank();
+    const bool leader = cr == 0;
     const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
     const int D = a.D, n = a.n;
+
+    // every CTA of the cluster must be running before anyone writes into the leader's shared
+    // memory: arrive now, wait just before the first remote store
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+
+    // leader: start fetching the small adapter up-projection now, it is needed only in the tail
+    if (leader && a.do_adapter) {
+        const WT* B = static_cast<const WT*>(a.adapter_b);
+        for (int i = threadIdx.x; i < n * a.r; i += kRouterThreads) bs[i] = load_weight(B, i);
+    }
 
     // ---- router input ---------------------------------------------------
     if (a.do_router) {
@@ -126,7 +169,7 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
         for (int i = threadIdx.x; i < D; i += kRouterThreads) {
             const float v = xs[i] * a.gamma[i] * inv;
             xs[i] = v;
-            if (blockIdx.x == 0 && a.x_norm) a.x_norm[size_t(tok) * D + i] = v;
+            if (leader && a.x_norm) a.x_norm[size_t(tok) * D + i] = v;
         }
     } else {
         const float* xt = a.x_in + size_t(tok) * D;
@@ -137,37 +180,39 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     // ---- weight rows: router rows then adapter-A rows, one warp per row ----
     const int n_r = a.do_router ? n : 0;
     const int rows = n_r + (a.do_adapter ? a.r : 0);
-    for (int row = blockIdx.x * kRouterWarps + wi; row < rows; row += C * kRouterWarps) {
+    asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+    for (int row = int(cr) * kRouterWarps + wi; row < rows; row += kRouterCluster * kRouterWarps) {
         const WT* wrow = row < n_r ? static_cast<const WT*>(a.router_w) + size_t(row) * D
                                    : static_cast<const WT*>(a.adapter_a) + size_t(row - n_r) * D;
-        float acc = 0.f;
-        for (int i = lane * VEC; i < D; i += 32 * VEC) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(wrow + i));
-            float f[VEC];
-            unpack16(v, f);
+        uint4 v[MAXIT];
 #pragma unroll
-            for (int q = 0; q < VEC; ++q) acc = fmaf(f[q], xs[i + q], acc);
+        for (int it = 0; it < MAXIT; ++it) {
+            const int i = (it * 32 + lane) * VEC;
+            if (i < D) v[it] = __ldg(reinterpret_cast<const uint4*>(wrow + i));
+        }
+        float acc = 0.f;
+#pragma unroll
+        for (int it = 0; it < MAXIT; ++it) {
+            const int i = (it * 32 + lane) * VEC;
+            if (i < D) {
+                float f[VEC];
+                unpack16(v[it], f);
+#pragma unroll
+                for (int q = 0; q < VEC; ++q) acc = fmaf(f[q], xs[i + q], acc);
+            }
         }
         acc = warp_sum(acc);
-        if (lane == 0) {
-            if (row < n_r) a.logits[size_t(tok) * n + row] = acc;
-            else a.u[size_t(tok) * a.r + (row - n_r)] = acc;
-        }
+        if (lane == 0) dsmem_store(row < n_r ? zs + row : us + (row - n_r), 0, acc);
     }
+    cluster_sync_all();
+    if (!leader) return;
 
-    // ---- ticket: the last CTA of this token runs the tail ------------------
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) s_last = atomicAdd(&a.counters[1 + tok], 1u) == unsigned(C - 1);
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-
+    // ---- tail (leader CTA of the token) -------------------------------------
     if (a.do_router) {
         for (int e = threadIdx.x; e < n; e += kRouterThreads) {
-            const float z = __ldcg(a.logits + size_t(tok) * n + e);
-            zs[e] = z;
+            const float z = zs[e];
             ps[e] = z;
+            a.logits[size_t(tok) * n + e] = z;
             if (a.logits_out) a.logits_out[size_t(tok) * n + e] = z;
         }
         __syncthreads();
@@ -188,40 +233,38 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     }
     if (a.do_adapter) {
         __syncthreads();
-        for (int q = threadIdx.x; q < a.r; q += kRouterThreads) us[q] = __ldcg(a.u + size_t(tok) * a.r + q);
-        __syncthreads();
-        const WT* B = static_cast<const WT*>(a.adapter_b);
         for (int e = threadIdx.x; e < n; e += kRouterThreads) {
             float acc = 0.f;
-            for (int q = 0; q < a.r; ++q) {
-                float bw;
-                if (sizeof(WT) == 2) bw = __uint_as_float(uint32_t(reinterpret_cast<const uint16_t*>(B)[size_t(e) * a.r + q]) << 16);
-                else bw = reinterpret_cast<const float*>(B)[size_t(e) * a.r + q];
-                acc = fmaf(bw, us[q], acc);
-            }
+            for (int q = 0; q < a.r; ++q) acc = fmaf(bs[e * a.r + q], us[q], acc);
             ps[e] = acc;
         }
         __syncthreads();
         block_softmax(ps, n, scratch);
-        for (int e = threadIdx.x; e < n; e += kRouterThreads) a.pihat[size_t(tok) * n + e] = ps[e];
+        if (a.nb > 1)
+            for (int e = threadIdx.x; e < n; e += kRouterThreads) a.pihat[size_t(tok) * n + e] = ps[e];
     }
 
-    // ---- ticket over tokens: the last tail aggregates and publishes ---------
-    __threadfence();
+    // ---- several tokens: the last leader to finish aggregates ----------------
+    if (a.nb > 1) {
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) s_last = atomicAdd(&a.counters[0], 1u) == unsigned(a.nb - 1);
+        __syncthreads();
+        if (!s_last) return;
+        __threadfence();
+        if (a.do_adapter) {
+            for (int e = threadIdx.x; e < n; e += kRouterThreads) {
+                float s = 0.f;
+                for (int t = 0; t < a.nb; ++t) s += __ldcg(a.pihat + size_t(t) * n + e);
+                ps[e] = s;
+            }
+        }
+        if (threadIdx.x == 0) a.counters[0] = 0u;
+    }
     __syncthreads();
-    if (threadIdx.x == 0) s_last = atomicAdd(&a.counters[0], 1u) == unsigned(a.nb - 1);
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
 
     Mailbox* mb = a.mailbox;
     if (a.do_adapter) {
-        for (int e = threadIdx.x; e < n; e += kRouterThreads) {
-            float s = 0.f;
-            for (int t = 0; t < a.nb; ++t) s += __ldcg(a.pihat + size_t(t) * n + e);
-            ps[e] = s;
-        }
-        __syncthreads();
         for (int e = threadIdx.x; e < n; e += kRouterThreads) {
             const int rk = rank_of(ps, n, e);
             a.order[rk] = e;
@@ -231,16 +274,19 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
         }
     }
     if (a.do_router) {
-        for (int i = threadIdx.x; i < a.nb * a.K; i += kRouterThreads) mb->ids[i] = __ldcg(a.ids + i);
+        if (a.nb > 1) {
+            for (int i = threadIdx.x; i < a.nb * a.K; i += kRouterThreads) mb->ids[i] = __ldcg(a.ids + i);
+        } else if (threadIdx.x < a.K) {
+            mb->ids[threadIdx.x] = isel[threadIdx.x];
+        }
     }
-    for (int i = threadIdx.x; i <= a.nb; i += kRouterThreads) a.counters[i] = 0u;
     __threadfence_system();
     __syncthreads();
     if (threadIdx.x == 0) mb->seq = a.seq;
 }
 
 inline size_t router_smem_bytes(int D, int n, int r) {
-    return sizeof(float) * (size_t(D) + 2 * size_t(n) + kRouterWarps + 2 * SPM_MAX_TOPK + size_t(r));
+    return sizeof(float) * (size_t(D) + 2 * size_t(n) + size_t(r) + kRouterWarps + 2 * SPM_MAX_TOPK + size_t(n) * r);
 }
 
 }  // namespace spm

@@ -42,6 +42,11 @@ public:
         stats_ = spm_stats{};
     }
 
+    void reset_accounting() {
+        events_.clear();
+        stats_ = spm_stats{};
+    }
+
     int layers() const { return L_; }
     int experts() const { return n_; }
     int slots() const { return S_; }

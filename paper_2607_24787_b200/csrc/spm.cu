@@ -50,6 +50,9 @@ struct spm_ctx {
     int32_t *ws_ids = nullptr, *ws_order = nullptr;
     unsigned* ws_counters = nullptr;
     int* ws_status = nullptr;
+    unsigned long long* ws_clock = nullptr;
+    int clock_used = 0;
+    double window_us = 0;
     // mailbox
     Mailbox* mb_host = nullptr;
     Mailbox* mb_dev = nullptr;
@@ -67,6 +70,11 @@ struct spm_ctx {
     int tim_cur = 0;
     std::vector<double> layer_stall_us, layer_ffn_us;
     uint64_t timed_steps = 0;
+    // spm_moe_ffn called on its own: ring of event pairs around the FFN kernel
+    std::vector<cudaEvent_t> ring_start, ring_end;
+    std::vector<uint8_t> ring_used;
+    size_t ring_pos = 0;
+    double ring_us = 0;
     // policy inputs
     std::vector<int32_t> hint, hint_count;
     int hint_steps = 0, hint_stride = 0;
@@ -114,7 +122,8 @@ int check_cfg(const spm_model_cfg* m, int S, spm_ctx* c) {
     if (m->top_k < 1 || m->top_k > m->n_experts || m->n_shared < 0 || m->top_k + m->n_shared > SPM_MAX_TOPK)
         return fail(c, SPM_ERR_CONFIG, "top_k %d + n_shared %d unsupported (max %d)", m->top_k, m->n_shared, SPM_MAX_TOPK);
     if (m->inter < 1) return fail(c, SPM_ERR_CONFIG, "inter %d", m->inter);
-    if (m->adapter_rank < 1 || m->adapter_rank > 256) return fail(c, SPM_ERR_CONFIG, "adapter_rank %d out of range", m->adapter_rank);
+    if (m->adapter_rank < 1 || m->adapter_rank > 256 || m->n_experts * m->adapter_rank > 32768)
+        return fail(c, SPM_ERR_CONFIG, "adapter_rank %d out of range (n_experts * rank <= 32768)", m->adapter_rank);
     if (m->max_batch < 1 || m->max_batch > SPM_MAX_BATCH) return fail(c, SPM_ERR_CONFIG, "max_batch %d out of range", m->max_batch);
     if (S < 1 || S > 32767) return fail(c, SPM_ERR_CONFIG, "slots_per_layer %d out of range", S);
     if (m->max_batch == 1 && S < m->top_k) return fail(c, SPM_ERR_CONFIG, "slots_per_layer %d < top_k %d at batch 1", S, m->top_k);
@@ -126,6 +135,8 @@ size_t blob_bytes_of(const spm_model_cfg* m) {
 }
 
 constexpr int kMaxCtasBatch1 = 296;
+constexpr int kClockSlots = 4096;     // in-kernel {start, end} pairs between two harvests
+static_assert(kMaxCtasBatch1 <= kReduceGroups * kReduceMaxRows, "reduce kernel covers every grid size");
 
 int ffn_grid_for(const spm_ctx* c, int nb) {
     if (nb == 1) return c->ffn_ctas > 0 ? std::min(c->ffn_ctas, kMaxCtasBatch1) : c->num_sms;
@@ -138,7 +149,7 @@ struct Carve {
 };
 
 struct Layout {
-    size_t pools, x, logits, u, pihat, w, scores, partial, h, ids, order, counters, status, total;
+    size_t pools, x, logits, u, pihat, w, scores, partial, h, ids, order, clock, counters, status, total;
 };
 
 Layout layout_of(const spm_model_cfg* m, int S) {
@@ -156,6 +167,7 @@ Layout layout_of(const spm_model_cfg* m, int S) {
     l.h = c.take(nb * D * 4);
     l.ids = c.take(nb * SPM_MAX_TOPK * 4);
     l.order = c.take(n * 4);
+    l.clock = c.take(size_t(kClockSlots) * 16);
     l.counters = c.take((nb + 1) * 4);
     l.status = c.take(4);
     l.total = c.off;
@@ -164,38 +176,43 @@ Layout layout_of(const spm_model_cfg* m, int S) {
 
 // ---- kernel dispatch -------------------------------------------------------
 template <typename WT, int NSEG, int MAXNB>
-cudaError_t launch_gemv_t(const FfnArgs<MAXNB>& a, int G, int nb, int depth, size_t smem, cudaStream_t st) {
+cudaError_t launch_gemv_t(const FfnArgs<MAXNB>& a, int G, int nb, int warps, int depth, size_t smem, cudaStream_t st) {
     static bool attr_set = false;
     auto kern = ffn_gemv_kernel<WT, NSEG, MAXNB>;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kFfnSmemLimit));
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    kern<<<dim3(G, nb), kFfnThreads, smem, st>>>(a, depth);
+    kern<<<dim3(G, nb), warps * 32, smem, st>>>(a, depth);
     return cudaGetLastError();
 }
 
 template <typename WT, int MAXNB>
-cudaError_t launch_gemv_seg(int nseg, const FfnArgs<MAXNB>& a, int G, int nb, int depth, size_t smem, cudaStream_t st) {
+cudaError_t launch_gemv_seg(int nseg, const FfnArgs<MAXNB>& a, int G, int nb, int warps, int depth, size_t smem, cudaStream_t st) {
     switch (nseg) {
-        case 1: return launch_gemv_t<WT, 1, MAXNB>(a, G, nb, depth, smem, st);
-        case 2: return launch_gemv_t<WT, 2, MAXNB>(a, G, nb, depth, smem, st);
-        case 3: return launch_gemv_t<WT, 3, MAXNB>(a, G, nb, depth, smem, st);
-        case 4: return launch_gemv_t<WT, 4, MAXNB>(a, G, nb, depth, smem, st);
-        case 5: return launch_gemv_t<WT, 5, MAXNB>(a, G, nb, depth, smem, st);
-        case 6: return launch_gemv_t<WT, 6, MAXNB>(a, G, nb, depth, smem, st);
-        case 7: return launch_gemv_t<WT, 7, MAXNB>(a, G, nb, depth, smem, st);
-        case 8: return launch_gemv_t<WT, 8, MAXNB>(a, G, nb, depth, smem, st);
+        case 1: return launch_gemv_t<WT, 1, MAXNB>(a, G, nb, warps, depth, smem, st);
+        case 2: return launch_gemv_t<WT, 2, MAXNB>(a, G, nb, warps, depth, smem, st);
+        case 3: return launch_gemv_t<WT, 3, MAXNB>(a, G, nb, warps, depth, smem, st);
+        case 4: return launch_gemv_t<WT, 4, MAXNB>(a, G, nb, warps, depth, smem, st);
+        case 5: return launch_gemv_t<WT, 5, MAXNB>(a, G, nb, warps, depth, smem, st);
+        case 6: return launch_gemv_t<WT, 6, MAXNB>(a, G, nb, warps, depth, smem, st);
+        case 7: return launch_gemv_t<WT, 7, MAXNB>(a, G, nb, warps, depth, smem, st);
+        case 8: return launch_gemv_t<WT, 8, MAXNB>(a, G, nb, warps, depth, smem, st);
     }
     return cudaErrorInvalidValue;
 }
 
 template <int MAXNB>
 cudaError_t launch_gemv(const spm_ctx* c, const FfnArgs<MAXNB>& a, int G, int nb) {
-    const size_t smem = ffn_gemv_smem(c->row_bytes, c->depth);
-    if (c->cfg.dtype == SPM_DTYPE_BF16) return launch_gemv_seg<bf16_t, MAXNB>(c->nseg, a, G, nb, c->depth, smem, c->compute);
-    return launch_gemv_seg<float, MAXNB>(c->nseg, a, G, nb, c->depth, smem, c->compute);
+    int max_cnt = 1;
+    for (int t = 0; t < nb; ++t) max_cnt = std::max(max_cnt, int(a.count[t]));
+    const int rows_per_cta = (max_cnt * c->cfg.inter + G - 1) / G;
+    int warps = 8, depth = 2;
+    ffn_gemv_shape(c->row_bytes, rows_per_cta, &warps, &depth);
+    const size_t smem = ffn_gemv_smem(c->row_bytes, warps, depth);
+    if (c->cfg.dtype == SPM_DTYPE_BF16) return launch_gemv_seg<bf16_t, MAXNB>(c->nseg, a, G, nb, warps, depth, smem, c->compute);
+    return launch_gemv_seg<float, MAXNB>(c->nseg, a, G, nb, warps, depth, smem, c->compute);
 }
 
 int launch_router(spm_ctx* c, int layer, const float* h, const float* x_in, int nb, float* x_norm,
@@ -226,14 +243,26 @@ int launch_router(spm_ctx* c, int layer, const float* h, const float* x_in, int 
     a.D = m.hidden; a.n = m.n_experts; a.K = m.top_k; a.r = m.adapter_rank; a.nb = nb;
     a.renorm = m.renormalize; a.do_router = do_router; a.do_adapter = do_adapter;
     a.eps = m.rms_eps;
-    const int rows = (do_router ? m.n_experts : 0) + (do_adapter ? m.adapter_rank : 0);
-    int C = (rows + kRouterWarps - 1) / kRouterWarps;
-    C = std::max(1, std::min(C, 32));
     const size_t smem = router_smem_bytes(m.hidden, m.n_experts, m.adapter_rank);
-    if (m.dtype == SPM_DTYPE_BF16)
-        router_adapter_kernel<bf16_t><<<dim3(C, nb), kRouterThreads, smem, c->compute>>>(a);
-    else
-        router_adapter_kernel<float><<<dim3(C, nb), kRouterThreads, smem, c->compute>>>(a);
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(kRouterCluster, nb);
+    lc.blockDim = dim3(kRouterThreads);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = c->compute;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = kRouterCluster;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    lc.attrs = at;
+    lc.numAttrs = 1;
+    if (m.dtype == SPM_DTYPE_BF16) {
+        if (smem > 48 * 1024) CU(c, cudaFuncSetAttribute(router_adapter_kernel<bf16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+        CU(c, cudaLaunchKernelEx(&lc, router_adapter_kernel<bf16_t>, a));
+    } else {
+        if (smem > 48 * 1024) CU(c, cudaFuncSetAttribute(router_adapter_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+        CU(c, cudaLaunchKernelEx(&lc, router_adapter_kernel<float>, a));
+    }
     CU(c, cudaGetLastError());
     c->kernel_launches++;
     return SPM_OK;
@@ -297,10 +326,41 @@ void harvest(spm_ctx* c, Timing& t) {
     if (any) c->timed_steps++;
 }
 
+// Read back the in-kernel {first start, last end} pairs written so far and re-arm the slots.
+int harvest_clock(spm_ctx* c) {
+    if (c->clock_used == 0) return SPM_OK;
+    std::vector<unsigned long long> h(size_t(c->clock_used) * 2);
+    CU(c, cudaStreamSynchronize(c->compute));
+    CU(c, cudaMemcpy(h.data(), c->ws_clock, h.size() * 8, cudaMemcpyDeviceToHost));
+    for (int i = 0; i < c->clock_used; ++i)
+        if (h[2 * i + 1] > h[2 * i]) c->window_us += double(h[2 * i + 1] - h[2 * i]) * 1e-3;
+    for (int i = 0; i < c->clock_used; ++i) { h[2 * i] = ~0ull; h[2 * i + 1] = 0; }
+    CU(c, cudaMemcpy(c->ws_clock, h.data(), h.size() * 8, cudaMemcpyHostToDevice));
+    c->clock_used = 0;
+    return SPM_OK;
+}
+
+int arm_clock(spm_ctx* c) {   // whole ring to {max, 0}
+    std::vector<unsigned long long> h(size_t(kClockSlots) * 2);
+    for (int i = 0; i < kClockSlots; ++i) { h[2 * i] = ~0ull; h[2 * i + 1] = 0; }
+    CU(c, cudaMemcpy(c->ws_clock, h.data(), h.size() * 8, cudaMemcpyHostToDevice));
+    c->clock_used = 0;
+    return SPM_OK;
+}
+
+void harvest_ring(spm_ctx* c, size_t i) {
+    if (!c->ring_used[i]) return;
+    float ms = 0;
+    cudaEventSynchronize(c->ring_end[i]);
+    if (cudaEventElapsedTime(&ms, c->ring_start[i], c->ring_end[i]) == cudaSuccess) c->ring_us += ms * 1e3;
+    c->ring_used[i] = 0;
+}
+
 // Demand resolution, on-demand copies, stream waits and FFN launches of one layer.
-// `t` (may be null) receives the timing events of this layer.
+// `t` (may be null) receives the timing events of this layer; `ring` >= 0 selects an event pair
+// of the stand-alone timing ring instead.
 int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, const float* w, int nb,
-            float* h_inout, Timing* t) {
+            float* h_inout, Timing* t, int ring = -1) {
     const spm_model_cfg& m = c->cfg;
     const int K = m.top_k;
     SlotTable& tb = *c->table;
@@ -355,6 +415,11 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
         }
 
         const bool first = wave == 0, last = wave == n_waves - 1;
+        unsigned long long* clock_slot = nullptr;
+        if (c->timing) {
+            if (c->clock_used == kClockSlots) if (int rc = harvest_clock(c)) return rc;
+            clock_slot = c->ws_clock + 2 * size_t(c->clock_used++);
+        }
         auto fill = [&](auto& a) {
             a.pool = slot_ptr(c, layer, 0);
             a.shared = m.n_shared ? static_cast<const unsigned char*>(c->buf.shared_experts) + size_t(layer) * m.n_shared * c->blob : nullptr;
@@ -362,6 +427,7 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
             a.w = w;
             a.partial = c->ws_partial;
             a.status = c->ws_status;
+            a.clock = clock_slot;
             a.blob_bytes = c->blob;
             a.I = m.inter; a.K = K; a.n_slots = c->S; a.n_shared = m.n_shared;
             for (int tk = 0; tk < nb; ++tk) {
@@ -383,6 +449,7 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
             }
         };
         if (t && first) CU(c, cudaEventRecord(t->ffn_start[layer], c->compute));
+        if (ring >= 0 && first) CU(c, cudaEventRecord(c->ring_start[ring], c->compute));
         if (nb == 1) {
             FfnArgs<1> a{};
             fill(a);
@@ -393,7 +460,9 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
             CU(c, launch_gemv<SPM_MAX_BATCH>(c, a, G, nb));
         }
         if (t && last) CU(c, cudaEventRecord(t->ffn_end[layer], c->compute));
-        ffn_reduce_kernel<<<dim3((m.hidden + 127) / 128, nb), 128, 0, c->compute>>>(c->ws_partial, h_inout, h_inout, G, m.hidden);
+        if (ring >= 0 && last) { CU(c, cudaEventRecord(c->ring_end[ring], c->compute)); c->ring_used[ring] = 1; }
+        ffn_reduce_kernel<<<dim3((m.hidden + kReduceCols - 1) / kReduceCols, nb), kReduceCols * kReduceGroups, 0, c->compute>>>(
+            c->ws_partial, h_inout, h_inout, G, m.hidden);
         CU(c, cudaGetLastError());
         c->kernel_launches += 2;
         c->ffn_launches++;
@@ -483,7 +552,7 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
     c->blob = blob_bytes_of(cfg);
     c->row_bytes = size_t(3) * cfg->hidden * c->elem;
     c->nseg = cfg->hidden / (cfg->dtype == SPM_DTYPE_BF16 ? 256 : 128);
-    c->depth = int(std::min<size_t>(4, (232448 - 1024) / (size_t(kFfnWarps) * c->row_bytes)));
+    c->depth = int((kFfnSmemLimit - 1024) / (4 * c->row_bytes));   // ring depth with the fewest warps
     auto bail = [&](int rc) { g_init_error = c->err; spm_destroy(c); return rc; };
     if (c->depth < 1) { c->err = "hidden too large for the shared-memory ring"; return bail(SPM_ERR_CONFIG); }
     int dev = 0;
@@ -504,6 +573,7 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
     c->ws_h = reinterpret_cast<float*>(base + lay.h);
     c->ws_ids = reinterpret_cast<int32_t*>(base + lay.ids);
     c->ws_order = reinterpret_cast<int32_t*>(base + lay.order);
+    c->ws_clock = reinterpret_cast<unsigned long long*>(base + lay.clock);
     c->ws_counters = reinterpret_cast<unsigned*>(base + lay.counters);
     c->ws_status = reinterpret_cast<int*>(base + lay.status);
 
@@ -536,8 +606,12 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
             if (!cu(cudaEventCreate(&t.k1_done[l]), "cudaEventCreate") || !cu(cudaEventCreate(&t.ffn_start[l]), "cudaEventCreate") ||
                 !cu(cudaEventCreate(&t.ffn_end[l]), "cudaEventCreate")) return bail(SPM_ERR_CUDA);
     }
+    c->ring_start.resize(64); c->ring_end.resize(64); c->ring_used.assign(64, 0);
+    for (size_t i = 0; i < 64; ++i)
+        if (!cu(cudaEventCreate(&c->ring_start[i]), "cudaEventCreate") || !cu(cudaEventCreate(&c->ring_end[i]), "cudaEventCreate")) return bail(SPM_ERR_CUDA);
     if (!cu(cudaStreamSynchronize(c->compute), "cudaStreamSynchronize")) return bail(SPM_ERR_CUDA);
 
+    if (arm_clock(c) != SPM_OK) return bail(SPM_ERR_CUDA);
     c->budget = budget < 0 ? 1 : budget;
     if (budget < 0) {
         double W = 0, tx = 0;
@@ -562,6 +636,8 @@ int spm_destroy(spm_ctx* c) {
         for (auto ev : t.ffn_start) if (ev) cudaEventDestroy(ev);
         for (auto ev : t.ffn_end) if (ev) cudaEventDestroy(ev);
     }
+    for (auto ev : c->ring_start) if (ev) cudaEventDestroy(ev);
+    for (auto ev : c->ring_end) if (ev) cudaEventDestroy(ev);
     if (c->mb_host) cudaFreeHost(c->mb_host);
     delete c->table;
     delete c;
@@ -620,7 +696,12 @@ int spm_prefetch_async(spm_ctx* c, int target, const int32_t* ids, int count, in
 int spm_moe_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, const float* w, int nb, float* h_inout) {
     if (int rc = check_layer(c, layer, nb)) return rc;
     if (!x_norm || !ids || !w || !h_inout) return fail(c, SPM_ERR_INVALID_ARG, "null argument");
-    return run_ffn(c, layer, x_norm, ids, w, nb, h_inout, nullptr);
+    int ring = -1;
+    if (c->timing) {
+        ring = int(c->ring_pos++ % c->ring_start.size());
+        harvest_ring(c, size_t(ring));
+    }
+    return run_ffn(c, layer, x_norm, ids, w, nb, h_inout, nullptr, ring);
 }
 
 int spm_decode_step(spm_ctx* c, const float* h_in, int nb, float* h_out) {
@@ -773,12 +854,35 @@ int spm_synchronize(spm_ctx* c) {
     return check_status(c);
 }
 
+int spm_reset_stats(spm_ctx* c) {
+    if (!c) return SPM_ERR_INVALID_ARG;
+    CU(c, cudaStreamSynchronize(c->copy));
+    CU(c, cudaStreamSynchronize(c->compute));
+    for (auto& t : c->tim) std::fill(t.used.begin(), t.used.end(), 0);
+    c->table->reset_accounting();
+    std::fill(c->ring_used.begin(), c->ring_used.end(), 0);
+    c->ring_us = 0;
+    if (int rc = arm_clock(c)) return rc;
+    c->window_us = 0;
+    std::fill(c->layer_stall_us.begin(), c->layer_stall_us.end(), 0.0);
+    std::fill(c->layer_ffn_us.begin(), c->layer_ffn_us.end(), 0.0);
+    c->timed_steps = 0;
+    c->extra_late = c->h2d_bytes = c->ffn_launches = c->kernel_launches = c->tokens = 0;
+    c->ready_sum = c->recall_sum = 0;
+    c->ready_count = c->recall_count = 0;
+    return SPM_OK;
+}
+
 int spm_cache_reset(spm_ctx* c) {
     if (!c) return SPM_ERR_INVALID_ARG;
     CU(c, cudaStreamSynchronize(c->copy));
     CU(c, cudaStreamSynchronize(c->compute));
     for (auto& t : c->tim) std::fill(t.used.begin(), t.used.end(), 0);
     c->table->reset();
+    std::fill(c->ring_used.begin(), c->ring_used.end(), 0);
+    c->ring_us = 0;
+    if (int rc = arm_clock(c)) return rc;
+    c->window_us = 0;
     std::fill(c->slot_pending.begin(), c->slot_pending.end(), 0);
     std::fill(c->has_plan.begin(), c->has_plan.end(), 0);
     std::fill(c->layer_stall_us.begin(), c->layer_stall_us.end(), 0.0);
@@ -858,13 +962,16 @@ int spm_get_stats(spm_ctx* c, spm_stats* out) {
     CU(c, cudaStreamSynchronize(c->copy));
     CU(c, cudaStreamSynchronize(c->compute));
     for (auto& t : c->tim) harvest(c, t);
+    for (size_t i = 0; i < c->ring_used.size(); ++i) harvest_ring(c, i);
     *out = c->table->stats();
     out->tokens = c->tokens;
     out->late_arrivals = c->extra_late;
     out->h2d_bytes = c->h2d_bytes;
     out->ffn_launches = c->ffn_launches;
     out->kernel_launches = c->kernel_launches;
-    out->ffn_us = 0;
+    if (int rc = harvest_clock(c)) return rc;
+    out->ffn_window_us = c->window_us;
+    out->ffn_us = c->ring_us;
     out->stall_us = 0;
     for (int l = 0; l < c->cfg.n_layers; ++l) { out->ffn_us += c->layer_ffn_us[l]; out->stall_us += c->layer_stall_us[l]; }
     out->ready_sum = c->ready_sum; out->ready_count = c->ready_count;

@@ -138,6 +138,7 @@ class OffloadedMoE:
     def set_drop_modulo(self, m): B.spm_set_drop_modulo(self.ctx, m)
     def profile_window(self): return B.spm_profile_window(self.ctx)
     def cache_reset(self): B.spm_cache_reset(self.ctx)
+    def reset_stats(self): B.spm_reset_stats(self.ctx)
     def stats(self): return B.spm_get_stats(self.ctx)
     def layer_times(self): return B.spm_get_layer_times(self.ctx, self.L)
     def events(self): return B.spm_get_events(self.ctx)
