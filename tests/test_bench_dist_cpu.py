@@ -1,0 +1,59 @@
+"""The benchmark's multi-rank logic on CPU: 2 gloo ranks, independent token streams per rank,
+max-over-ranks time and summed tokens (no collective on the data path)."""
+import os
+import socket
+import subprocess
+import sys
+import textwrap
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+WORKER = textwrap.dedent("""
+    import json, sys
+    sys.path.insert(0, %r)
+    import bench, synth
+    rank, local, world = bench.dist_setup("gloo")
+    cfg = synth.get_config("tiny")
+    tok, H = bench.hidden_rows(cfg, 16, stream=rank)
+    bench.barrier(world)
+    t, n = bench.aggregate(10.0 + 5.0 * rank, 16 * cfg.batch, world)
+    print(json.dumps({"rank": rank, "world": world, "t": t, "n": n, "tok": tok[:, 0].tolist(), "shape": list(H.shape)}))
+""") % ROOT
+
+
+def test_two_gloo_ranks_shard_by_sequence():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    procs = []
+    for r in range(2):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, "-c", WORKER], env=env, stdout=subprocess.PIPE,
+                                      stderr=subprocess.PIPE, text=True))
+    outs = []
+    for p in procs:
+        out, err = p.communicate(timeout=180)
+        assert p.returncode == 0, err[-2000:]
+        outs.append(__import__("json").loads(out.strip().splitlines()[-1]))
+    outs.sort(key=lambda o: o["rank"])
+    assert [o["world"] for o in outs] == [2, 2]
+    assert all(o["t"] == 15.0 for o in outs)            # max over ranks
+    assert all(o["n"] == 32 for o in outs)              # tokens of all ranks
+    assert outs[0]["tok"] != outs[1]["tok"]             # every rank decodes its own sequence
+    assert outs[0]["shape"] == [16, 1, 256]
+
+
+def test_reference_arm_prints_contract_line():
+    """`--impl reference` (the CPU oracle) runs without a GPU and prints one JSON line."""
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--config", "tiny",
+                          "--steps", "4", "--warmup", "3"], capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = __import__("json").loads(out.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["value"] > 0 and line["unit"] == "tokens/s"
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+    # under torchrun only rank 0 prints; the others exit 0 without work
+    env = dict(os.environ, RANK="1", LOCAL_RANK="1", WORLD_SIZE="2")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--config", "tiny"],
+                         capture_output=True, text=True, timeout=120, env=env)
+    assert out.returncode == 0 and out.stdout.strip() == ""
