@@ -229,6 +229,43 @@ int spm_get_events(spm_ctx* ctx, spm_event* out, size_t capacity, size_t* count)
 int spm_get_slot_table(spm_ctx* ctx, int layer, int32_t* slot_expert /* host [slots] */);
 int spm_synchronize(spm_ctx* ctx);                         /* both streams idle */
 
+/* Expert FFN for callers that may not allocate (the paper has no counterpart: this is a deployment
+ * convenience of this library, not part of the method).
+ *
+ * Some callers cannot call cudaMalloc or anything that allocates: a serving loop that has frozen
+ * its memory map, a process whose device memory is owned entirely by another allocator, code that
+ * must not wait on the driver's allocation lock. They cannot create an spm_ctx either (that
+ * creates CUDA events and pinned memory). For them this call computes, for ONE token,
+ *     h_inout += sum_{i < count} w[i] * FFN_{which[i]}(x_norm)          (SwiGLU experts, as spm_moe_ffn)
+ * reading packed expert blobs in place and using no memory but its arguments and a fixed scratch
+ * array of SPM_NOALLOC_SCRATCH_BYTES that is part of the library image (every GPU that loads the
+ * library holds that array until the process exits). It calls no cudaMalloc, cudaFree, event or
+ * stream creation, nor any other allocating routine.
+ *
+ *   cfg       only dtype, hidden and inter are read. hidden: a multiple of 256 (bf16) / 128 (fp32),
+ *             at most SPM_NOALLOC_MAX_HIDDEN (bf16) / 1024 (fp32); larger sizes are rejected with
+ *             SPM_ERR_CONFIG and a message in spm_last_error(NULL), because the scratch array holds
+ *             SPM_NOALLOC_MAX_CTAS partial rows of SPM_NOALLOC_MAX_HIDDEN floats and no more.
+ *   blobs     dev: n_blobs packed expert blobs back to back (layout of spm_expert_blob_bytes), 16-byte aligned
+ *   which     HOST [count]: index into `blobs` of each expert to apply, count <= SPM_MAX_TOPK
+ *   w         dev fp32 [count] weights;  x_norm dev fp32 [hidden];  h_inout dev fp32 [hidden]
+ *   stream    cudaStream_t; the work is enqueued there and the call returns, unless
+ *   wait_and_check != 0: then the call also waits for the stream and returns SPM_ERR_TIMEOUT /
+ *             SPM_ERR_NOT_RESIDENT if the kernel recorded a failure.
+ *
+ * The first call on a device looks up the scratch array's device address and sets a kernel attribute
+ * for that device (the device must be current); make that first call before starting any stream
+ * capture. All calls on a device share the one array and it keeps the previous call's contents: the
+ * call clears the part that must start at zero itself, but two calls whose GPU work overlaps (two
+ * streams, two threads) race on it and give wrong results -- keep them on one stream or otherwise
+ * serialised. */
+#define SPM_NOALLOC_MAX_CTAS      148
+#define SPM_NOALLOC_MAX_HIDDEN    2048
+#define SPM_NOALLOC_SCRATCH_BYTES (256 + SPM_NOALLOC_MAX_CTAS * SPM_NOALLOC_MAX_HIDDEN * 4)   /* 1,212,672 B */
+int spm_ffn_noalloc(const spm_model_cfg* cfg, const void* blobs, int n_blobs, const int32_t* which,
+                    const float* w, int count, const float* x_norm, float* h_inout, void* stream,
+                    int wait_and_check);
+
 /* Pinned host memory for the expert store (thin wrappers over cudaHostAlloc / cudaFreeHost). */
 int spm_host_alloc(size_t bytes, void** out);
 int spm_host_free(void* p);

@@ -89,6 +89,7 @@ _SIG = {
     "spm_get_events": [_P, _P, C.c_size_t, C.POINTER(C.c_size_t)],
     "spm_get_slot_table": [_P, C.c_int, _P],
     "spm_synchronize": [_P],
+    "spm_ffn_noalloc": [C.POINTER(ModelCfg), _P, C.c_int, _P, _P, C.c_int, _P, _P, _P, C.c_int],
     "spm_host_alloc": [C.c_size_t, C.POINTER(_P)],
     "spm_host_free": [_P],
     "spm_sim_create": [C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(_P)],
@@ -309,6 +310,15 @@ def spm_get_slot_table(ctx, layer, slots) -> np.ndarray:
 
 def spm_synchronize(ctx):
     _check(load().spm_synchronize(ctx), ctx)
+
+
+def spm_ffn_noalloc(cfg: ModelCfg, blobs, n_blobs, which, w, x_norm, h_inout, stream=None, wait_and_check=False):
+    """Expert FFN of one token for callers that may not allocate (see include/spm.h): no context,
+    no arena; the partial rows go to a fixed array inside the library. `which` is a host list of
+    blob indices, everything else is device memory; `stream` a raw cudaStream_t (None = default)."""
+    which = np.ascontiguousarray(which, np.int32)
+    _check(load().spm_ffn_noalloc(C.byref(cfg), _ptr(blobs), n_blobs, _ptr(which), _ptr(w), len(which),
+                                  _ptr(x_norm), _ptr(h_inout), stream, int(wait_and_check)))
 
 
 def spm_host_alloc(nbytes: int) -> int:

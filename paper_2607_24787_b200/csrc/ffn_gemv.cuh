@@ -234,7 +234,7 @@ constexpr int kReduceCols = 32;
 constexpr int kReduceGroups = 8;
 constexpr int kReduceMaxRows = 40;     // rows per group: kReduceGroups * kReduceMaxRows >= max G
 
-__global__ void __launch_bounds__(kReduceCols * kReduceGroups)
+static __global__ void __launch_bounds__(kReduceCols * kReduceGroups)
 ffn_reduce_kernel(const float* __restrict__ partial, const float* h_in, float* h_out, int G, int D) {
     __shared__ float part[kReduceGroups][kReduceCols];
     const int tok = blockIdx.y;

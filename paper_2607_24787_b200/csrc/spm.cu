@@ -506,6 +506,11 @@ int check_status(spm_ctx* c) {
 
 }  // namespace
 
+namespace spm {
+// lets other translation units of the library leave a message for spm_last_error(NULL)
+void set_thread_error(const std::string& msg) { g_init_error = msg; }
+}  // namespace spm
+
 // ============================================================================
 extern "C" {
 
