@@ -204,6 +204,11 @@ int spm_get_budget(spm_ctx* ctx, int* budget);
 int spm_set_plain_lru(spm_ctx* ctx, int on);              /* 1: no predicted-use touch */
 int spm_set_timing(spm_ctx* ctx, int on);                 /* record CUDA events around FFN / stalls */
 int spm_set_ffn_ctas(spm_ctx* ctx, int ctas);             /* CTAs per token of the GEMV FFN (0 = default) */
+/* Expert FFN used when nb > 1. 0 (default): the grouped tensor-core kernel (tcgen05, bf16
+ * activations, fp32 accumulation) whenever the shape allows it (bf16 weights, no shared experts,
+ * inter and hidden multiples of 128), else the GEMV kernel once per token. 1: always the GEMV
+ * kernel per token (fp32 activations). */
+int spm_set_batched_path(spm_ctx* ctx, int mode);
 /* Perfect-knowledge ranking for SPM_POLICY_HINT_TRACE: for step s (counted from the last
  * spm_cache_reset) and layer l, hint[(s*L + l)*stride .. +count[s*L+l]) are the experts that
  * layer truly needs, in priority order. Copied. */

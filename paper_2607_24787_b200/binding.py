@@ -78,6 +78,7 @@ _SIG = {
     "spm_set_plain_lru": [_P, C.c_int],
     "spm_set_timing": [_P, C.c_int],
     "spm_set_ffn_ctas": [_P, C.c_int],
+    "spm_set_batched_path": [_P, C.c_int],
     "spm_set_hint_trace": [_P, _P, _P, C.c_int, C.c_int],
     "spm_set_drop_modulo": [_P, C.c_int],
     "spm_set_deadline_ms": [_P, C.c_int],
@@ -234,6 +235,10 @@ def spm_set_timing(ctx, on):
 
 def spm_set_ffn_ctas(ctx, ctas):
     _check(load().spm_set_ffn_ctas(ctx, ctas), ctx)
+
+
+def spm_set_batched_path(ctx, mode):
+    _check(load().spm_set_batched_path(ctx, mode), ctx)
 
 
 def spm_set_hint_trace(ctx, hint):

@@ -1,0 +1,381 @@
+// Batched decode: slot-indexed grouped SwiGLU expert FFN on the 5th-generation tensor cores.
+//
+// When several sequences are decoded per step, the tokens routed to one expert form a small
+// dense problem  G = X_e Wg^T, U = X_e Wu^T, A = silu(G)*U*w, Y_e = A Wd^T.  Weights stay the
+// streamed operand (they go on the M side of the MMA, 128 rows at a time, read once from their
+// cache slot by TMA), the expert's tokens (padded to 64) are the N side, accumulators live in
+// TMEM. Activations are rounded to bf16 for the tensor cores; accumulation is fp32.
+//
+// Unit of work = (expert, 128 intermediate rows j). For a unit the CTA
+//   phase 1: streams gate[j][:] and up[j][:] over K = hidden in 64-wide blocks together with
+//            the matching block of the expert's token rows, accumulating G^T, U^T [128 x 64] in TMEM;
+//            the epilogue warps read them, apply silu * up * routing weight, and write A^T as bf16
+//            into shared memory (N-contiguous, 128-byte swizzle);
+//   phase 2: streams column j of W_down for 128 hidden units d at a time ([128 j x 128 d], d
+//            contiguous = an M-major A operand) and multiplies by A^T (K = the 128 j), one
+//            accumulator [128 d x 64 tokens] per d-tile, double buffered; the epilogue writes the
+//            rows of real tokens to the partial buffer P[j-tile][token row][d].
+// A combine kernel then adds, per token, its K experts x (I/128) partial rows and the residual in
+// a fixed order. One warp issues TMA, one thread issues tcgen05.mma, four warps run the epilogues;
+// all of them talk through mbarriers, every wait is bounded and an abort flag lets the whole CTA
+// leave together (freeing its TMEM) if a wait ever gives up. No multicast anywhere.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "ptx.cuh"
+#include "../../include/spm.h"
+
+namespace spm {
+
+constexpr int kGgThreads = 192;          // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+constexpr int kGgStages = 4;
+constexpr int kGgTokens = 64;            // N of every MMA: an expert's tokens, zero/garbage padded
+constexpr int kGgTileRows = 128;         // M of every MMA
+constexpr int kGgKBlock = 64;            // bf16 elements per 128-byte swizzled row
+constexpr uint32_t kGgTileBytes = kGgTileRows * 128;          // one [128 x 128 B] weight box
+constexpr uint32_t kGgXBytes = kGgTokens * 128;               // one [64 x 128 B] token box
+constexpr uint32_t kGgStageBytes = 2 * kGgTileBytes + kGgXBytes;   // 40 KB
+constexpr uint32_t kGgActBytes = kGgTileRows * 128;           // A^T: [128 j][64 tokens] bf16
+constexpr uint32_t kGgTmemCols = 256;    // G^T 0..63, U^T 64..127, Y tiles 128..191 and 192..255
+constexpr int kStatusGroupedTimeout = 4;
+
+struct GgUnit {
+    int32_t slot;      // global slot index (layer * slots + slot): 4th coordinate of the weight map
+    int32_t jt;        // 128-row tile of the intermediate dimension
+    int32_t row0;      // first row of this expert in the sorted token-row arrays
+    int32_t ntok;      // tokens of this expert (1..64)
+};
+
+struct GgArgs {
+    const GgUnit* units;
+    int n_units;
+    const float* wrow;     // [rows] routing weight of each sorted token row
+    float* partial;        // [I/128][rows_cap][D]
+    int rows_cap;
+    int D, I;
+    int* status;
+};
+
+// ---- tcgen05 / TMA wrappers ---------------------------------------------------
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]; bf16 inputs, fp32 accumulate; one thread issues.
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
+        "}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// this thread's TMEM lane, 16 consecutive fp32 columns
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor (sm_100 format): start address, leading / stride byte offsets
+// in 16-byte units, version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= uint64_t((addr >> 4) & 0x3fff);
+    d |= uint64_t((lbo_bytes >> 4) & 0x3fff) << 16;
+    d |= uint64_t((sbo_bytes >> 4) & 0x3fff) << 32;
+    d |= uint64_t(1) << 46;      // descriptor version
+    d |= uint64_t(2) << 61;      // SWIZZLE_128B
+    return d;
+}
+
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = 64, operand majors as given.
+__host__ __device__ constexpr uint32_t gg_idesc(bool a_mn_major, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(a_mn_major) << 15) | (uint32_t(b_mn_major) << 16) |
+           (uint32_t(kGgTokens >> 3) << 17) | (uint32_t(kGgTileRows >> 4) << 24);
+}
+
+struct GgAbort {
+    volatile int* flag;     // shared: set by the first wait that gives up
+    int* status;
+};
+
+// bounded wait that also leaves when another role of the CTA has given up
+__device__ __forceinline__ bool gg_wait(uint32_t bar, uint32_t parity, const GgAbort& ab) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*ab.flag) return false;
+        if (global_timer_ns() - t0 > 2000000000ull) {
+            *ab.flag = 1;
+            atomicOr(ab.status, kStatusGroupedTimeout);
+            return false;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kGgThreads, 1)
+ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_constant__ CUtensorMap xmap, const GgArgs a) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    // 1024-byte alignment is what the 128-byte swizzle atoms need
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    unsigned char* stages = smem;                                   // kGgStages x 40 KB
+    unsigned char* act = smem + kGgStages * kGgStageBytes;          // 16 KB
+    uint64_t* bars = reinterpret_cast<uint64_t*>(act + kGgActBytes);
+    uint64_t* full = bars;                    // [stages]  TMA -> MMA
+    uint64_t* empty = full + kGgStages;       // [stages]  MMA -> TMA
+    uint64_t* acc1_full = empty + kGgStages;  // MMA -> epilogue: G^T, U^T complete
+    uint64_t* acc1_empty = acc1_full + 1;     // epilogue -> MMA: G^T, U^T drained
+    uint64_t* act_full = acc1_empty + 1;      // epilogue -> MMA: A^T written
+    uint64_t* act_empty = act_full + 1;       // MMA -> epilogue: phase 2 has consumed A^T
+    uint64_t* acc2_full = act_empty + 1;      // [2] MMA -> epilogue
+    uint64_t* acc2_empty = acc2_full + 2;     // [2] epilogue -> MMA
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc2_empty + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    float* wrow_all = reinterpret_cast<float*>(tmem_slot + 4);      // [4 epilogue warps][64]
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int D = a.D;
+    const int n_kb = D / kGgKBlock;            // phase-1 stages per unit
+    const int n_dt = D / kGgTileRows;          // phase-2 stages per unit
+    GgAbort ab{abort_flag, a.status};
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kGgStages; ++s) { mbar_init(smem_u32(full + s), 1); mbar_init(smem_u32(empty + s), 1); }
+        mbar_init(smem_u32(acc1_full), 1);
+        mbar_init(smem_u32(acc1_empty), 4);     // one arrival per epilogue warp
+        mbar_init(smem_u32(act_full), 4);
+        mbar_init(smem_u32(act_empty), 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(acc2_full + b), 1); mbar_init(smem_u32(acc2_empty + b), 4); }
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kGgTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    // running counters; every role walks the same sequence of units and stages
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            uint32_t it = 0;      // ring position over all stages of all units
+            bool ok = true;
+            for (int u = blockIdx.x; u < a.n_units && ok; u += gridDim.x) {
+                const GgUnit un = a.units[u];
+                for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
+                    const uint32_t s = it % kGgStages;
+                    if (it >= kGgStages) ok = gg_wait(smem_u32(empty + s), ((it / kGgStages) - 1) & 1, ab);
+                    if (!ok) break;
+                    const uint32_t base = smem_u32(stages + s * kGgStageBytes);
+                    const uint32_t fb = smem_u32(full + s);
+                    mbar_arrive_expect_tx(fb, kGgStageBytes);
+                    tma_load_4d(base, &wmap, kb * kGgKBlock, 0, un.jt * kGgTileRows, un.slot, fb);                 // gate rows
+                    tma_load_4d(base + kGgTileBytes, &wmap, kb * kGgKBlock, 1, un.jt * kGgTileRows, un.slot, fb);  // up rows
+                    tma_load_2d(base + 2 * kGgTileBytes, &xmap, kb * kGgKBlock, un.row0, fb);                      // token rows
+                }
+                for (int dt = 0; dt < n_dt && ok; ++dt, ++it) {
+                    const uint32_t s = it % kGgStages;
+                    if (it >= kGgStages) ok = gg_wait(smem_u32(empty + s), ((it / kGgStages) - 1) & 1, ab);
+                    if (!ok) break;
+                    const uint32_t base = smem_u32(stages + s * kGgStageBytes);
+                    const uint32_t fb = smem_u32(full + s);
+                    mbar_arrive_expect_tx(fb, 2 * kGgTileBytes);
+                    tma_load_4d(base, &wmap, dt * kGgTileRows, 2, un.jt * kGgTileRows, un.slot, fb);                      // d 0..63
+                    tma_load_4d(base + kGgTileBytes, &wmap, dt * kGgTileRows + 64, 2, un.jt * kGgTileRows, un.slot, fb); // d 64..127
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            constexpr uint32_t idesc1 = gg_idesc(false, false);   // weights K-major, tokens K-major
+            constexpr uint32_t idesc2 = gg_idesc(true, true);     // W_down column tile M-major, A^T N-major
+            uint32_t it = 0, nu = 0, nd = 0;     // stage counter, unit counter, d-tile counter
+            bool ok = true;
+            for (int u = blockIdx.x; u < a.n_units && ok; u += gridDim.x, ++nu) {
+                if (nu > 0) ok = gg_wait(smem_u32(acc1_empty), (nu - 1) & 1, ab);
+                for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
+                    const uint32_t s = it % kGgStages;
+                    ok = gg_wait(smem_u32(full + s), (it / kGgStages) & 1, ab);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t base = smem_u32(stages + s * kGgStageBytes);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {      // 4 x (K = 16) inside the 64-wide block
+                        const uint64_t bx = smem_desc_sw128(base + 2 * kGgTileBytes + ks * 32, 16, 1024);
+                        tc_mma_bf16(tmem + 0, smem_desc_sw128(base + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
+                        tc_mma_bf16(tmem + 64, smem_desc_sw128(base + kGgTileBytes + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
+                    }
+                    tc_commit(smem_u32(empty + s));
+                }
+                if (!ok) break;
+                tc_commit(smem_u32(acc1_full));
+                ok = gg_wait(smem_u32(act_full), nu & 1, ab);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t act_addr = smem_u32(act);
+                for (int dt = 0; dt < n_dt && ok; ++dt, ++it, ++nd) {
+                    const uint32_t s = it % kGgStages, b = nd & 1;
+                    ok = gg_wait(smem_u32(full + s), (it / kGgStages) & 1, ab);
+                    if (ok && nd >= 2) ok = gg_wait(smem_u32(acc2_empty + b), ((nd >> 1) - 1) & 1, ab);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t base = smem_u32(stages + s * kGgStageBytes);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {      // K = 16 rows j per step, 2048 bytes of each operand
+                        const uint64_t da = smem_desc_sw128(base + ks * 2048, kGgTileBytes, 1024);
+                        const uint64_t db = smem_desc_sw128(act_addr + ks * 2048, kGgActBytes, 1024);
+                        tc_mma_bf16(tmem + 128 + 64 * b, da, db, idesc2, ks != 0);
+                    }
+                    tc_commit(smem_u32(empty + s));
+                    tc_commit(smem_u32(acc2_full + b));
+                }
+                if (!ok) break;
+                tc_commit(smem_u32(act_empty));
+            }
+        }
+    } else {
+        // ---------------- epilogue warps (TMEM lane quarter = warp % 4) ----------------
+        const int q = warp & 3;
+        const int row = q * 32 + lane;                  // accumulator row handled by this thread
+        const uint32_t lane_addr = uint32_t(q * 32) << 16;
+        float* wrow_s = wrow_all + q * kGgTokens;       // this warp's copy: no cross-warp barrier needed
+        uint32_t nu = 0, nd = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < a.n_units && ok; u += gridDim.x, ++nu) {
+            const GgUnit un = a.units[u];
+            // routing weights of this expert's token rows (0 beyond the real tokens)
+            __syncwarp();
+#pragma unroll
+            for (int i = lane; i < kGgTokens; i += 32) wrow_s[i] = i < un.ntok ? a.wrow[un.row0 + i] : 0.f;
+            __syncwarp();
+
+            ok = gg_wait(smem_u32(acc1_full), nu & 1, ab);
+            if (ok && nu > 0) ok = gg_wait(smem_u32(act_empty), (nu - 1) & 1, ab);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            // A^T[j = row][t] = silu(G) * U * w_t, bf16, 16-byte chunks swizzled by (row % 8)
+#pragma unroll
+            for (int c = 0; c < kGgTokens / 16; ++c) {
+                float g[16], up[16];
+                tmem_ld16(tmem + lane_addr + c * 16, g);
+                tmem_ld16(tmem + lane_addr + 64 + c * 16, up);
+                uint32_t packed[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float a0 = g[2 * i] / (1.f + expf(-g[2 * i])) * up[2 * i] * wrow_s[c * 16 + 2 * i];
+                    const float a1 = g[2 * i + 1] / (1.f + expf(-g[2 * i + 1])) * up[2 * i + 1] * wrow_s[c * 16 + 2 * i + 1];
+                    const __nv_bfloat162 p = __floats2bfloat162_rn(a0, a1);
+                    packed[i] = *reinterpret_cast<const uint32_t*>(&p);
+                }
+                unsigned char* rowp = act + row * 128;
+                *reinterpret_cast<uint4*>(rowp + (((2 * c) ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                *reinterpret_cast<uint4*>(rowp + (((2 * c + 1) ^ (row & 7)) << 4)) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+            }
+            fence_proxy_async();            // generic-proxy writes of A^T -> visible to the MMA's async reads
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) { mbar_arrive(smem_u32(acc1_empty)); mbar_arrive(smem_u32(act_full)); }
+
+            // phase 2: one [128 d x 64 tokens] accumulator per d-tile; store the real tokens' rows
+            float* prow = a.partial + (size_t(un.jt) * a.rows_cap + un.row0) * D;
+            for (int dt = 0; dt < n_dt && ok; ++dt, ++nd) {
+                const uint32_t b = nd & 1;
+                ok = __all_sync(0xffffffffu, gg_wait(smem_u32(acc2_full + b), (nd >> 1) & 1, ab));
+                if (!ok) break;
+                tc_fence_after();
+                for (int c = 0; c * 16 < un.ntok; ++c) {
+                    float y[16];
+                    tmem_ld16(tmem + lane_addr + 128 + 64 * b + c * 16, y);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        if (c * 16 + i < un.ntok) prow[size_t(c * 16 + i) * D + dt * kGgTileRows + row] = y[i];
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(acc2_empty + b));
+            }
+        }
+    }
+
+    // everyone meets here (also after an abort); the allocating warp returns the TMEM columns
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, kGgTmemCols);
+}
+
+inline size_t ffn_grouped_smem() {
+    return 1024 + size_t(kGgStages) * kGgStageBytes + kGgActBytes + 256 + 4 * kGgTokens * sizeof(float) + 64;
+}
+
+// Sorted token rows of one wave: Xs[row][:] = bf16(x[token][:]), wrow[row] = w[token][k].
+struct GgRow { int32_t token, k; };
+
+static __global__ void gg_gather_kernel(const float* __restrict__ x, const float* __restrict__ w, const GgRow* __restrict__ rows,
+                                        int n_rows, int D, int K, __nv_bfloat16* __restrict__ xs, float* __restrict__ wrow) {
+    const int r = blockIdx.x;
+    if (r >= n_rows) return;
+    const GgRow ri = rows[r];
+    const float* src = x + size_t(ri.token) * D;
+    __nv_bfloat16* dst = xs + size_t(r) * D;
+    for (int i = threadIdx.x * 4; i < D; i += blockDim.x * 4) {
+        const float4 v = *reinterpret_cast<const float4*>(src + i);
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+        uint2 o;
+        o.x = *reinterpret_cast<const uint32_t*>(&lo);
+        o.y = *reinterpret_cast<const uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(dst + i) = o;
+    }
+    if (threadIdx.x == 0) wrow[r] = w[size_t(ri.token) * K + ri.k];
+}
+
+// h[t][d] += sum over the token's experts of this wave (in k order) and j-tiles (ascending) of
+// P[jt][rowmap[t][k]][d]; rowmap < 0 marks experts that belong to another wave.
+static __global__ void gg_combine_kernel(const float* __restrict__ partial, const int32_t* __restrict__ rowmap, int K, int n_jt,
+                                         int rows_cap, int D, float* h) {
+    const int t = blockIdx.y;
+    const int d = blockIdx.x * blockDim.x + threadIdx.x;
+    if (d >= D) return;
+    float acc = 0.f;
+    for (int k = 0; k < K; ++k) {
+        const int r = rowmap[t * SPM_MAX_TOPK + k];
+        if (r < 0) continue;
+        for (int jt = 0; jt < n_jt; ++jt) acc += __ldcg(partial + (size_t(jt) * rows_cap + r) * D + d);
+    }
+    h[size_t(t) * D + d] += acc;
+}
+
+}  // namespace spm

@@ -15,7 +15,9 @@
 
 #include "../../include/spm.h"
 #include "ffn_gemv.cuh"
+#include "ffn_grouped.cuh"
 #include "router_adapter.cuh"
+#include "tma_maps.h"
 #include "slot_table.h"
 
 using namespace spm;
@@ -53,6 +55,20 @@ struct spm_ctx {
     unsigned long long* ws_clock = nullptr;
     int clock_used = 0;
     double window_us = 0;
+    // batched tensor-core path (bf16, max_batch > 1, no shared experts, I and D multiples of 128)
+    bool tc_ok = false;
+    int batched_path = 0;                 // 0: tensor cores when possible, 1: always the per-token GEMV
+    int rows_cap = 0, n_jt = 0, max_units = 0;
+    CUtensorMap wmap{}, xmap{};
+    __nv_bfloat16* tc_xs = nullptr;
+    float *tc_wrow = nullptr, *tc_partial = nullptr;
+    unsigned char* tc_desc_dev = nullptr;     // kDescRing wave descriptors
+    unsigned char* tc_desc_host = nullptr;    // pinned staging, same layout
+    size_t tc_desc_bytes = 0, tc_off_rows = 0, tc_off_rowmap = 0;
+    std::vector<cudaEvent_t> tc_desc_ev;
+    std::vector<uint8_t> tc_desc_ev_valid;
+    size_t tc_desc_pos = 0;
+    uint64_t tc_launches = 0;
     // mailbox
     Mailbox* mb_host = nullptr;
     Mailbox* mb_dev = nullptr;
@@ -136,6 +152,14 @@ size_t blob_bytes_of(const spm_model_cfg* m) {
 
 constexpr int kMaxCtasBatch1 = 296;
 constexpr int kClockSlots = 4096;     // in-kernel {start, end} pairs between two harvests
+constexpr int kDescRing = 8;          // wave descriptors in flight for the batched tensor-core path
+
+// The grouped tcgen05 kernel handles bf16 weights, more than one sequence per step, no shared
+// experts, and intermediate / hidden sizes that tile by 128.
+bool tc_supported(const spm_model_cfg* m) {
+    return m->dtype == SPM_DTYPE_BF16 && m->max_batch > 1 && m->n_shared == 0 && m->inter % kGgTileRows == 0 &&
+           m->hidden % kGgTileRows == 0;
+}
 static_assert(kMaxCtasBatch1 <= kReduceGroups * kReduceMaxRows, "reduce kernel covers every grid size");
 
 int ffn_grid_for(const spm_ctx* c, int nb) {
@@ -150,6 +174,10 @@ struct Carve {
 
 struct Layout {
     size_t pools, x, logits, u, pihat, w, scores, partial, h, ids, order, clock, counters, status, total;
+    size_t tc_xs, tc_wrow, tc_partial, tc_desc;       // batched tensor-core path only
+    size_t desc_bytes, off_rows, off_rowmap;
+    int rows_cap, n_jt, max_units;
+    bool tc;
 };
 
 Layout layout_of(const spm_model_cfg* m, int S) {
@@ -168,6 +196,19 @@ Layout layout_of(const spm_model_cfg* m, int S) {
     l.ids = c.take(nb * SPM_MAX_TOPK * 4);
     l.order = c.take(n * 4);
     l.clock = c.take(size_t(kClockSlots) * 16);
+    l.tc = tc_supported(m);
+    if (l.tc) {
+        l.rows_cap = m->max_batch * m->top_k;
+        l.n_jt = m->inter / kGgTileRows;
+        l.max_units = std::min(S, m->n_experts) * l.n_jt;
+        l.off_rows = align_up(size_t(l.max_units) * sizeof(GgUnit), 256);
+        l.off_rowmap = l.off_rows + align_up(size_t(l.rows_cap) * sizeof(GgRow), 256);
+        l.desc_bytes = l.off_rowmap + align_up(size_t(m->max_batch) * SPM_MAX_TOPK * 4, 256);
+        l.tc_xs = c.take(size_t(l.rows_cap + kGgTokens) * D * 2);
+        l.tc_wrow = c.take(size_t(l.rows_cap) * 4);
+        l.tc_partial = c.take(size_t(l.n_jt) * l.rows_cap * D * 4);
+        l.tc_desc = c.take(size_t(kDescRing) * l.desc_bytes);
+    }
     l.counters = c.take((nb + 1) * 4);
     l.status = c.take(4);
     l.total = c.off;
@@ -356,6 +397,58 @@ void harvest_ring(spm_ctx* c, size_t i) {
     c->ring_used[i] = 0;
 }
 
+// One wave of the batched tensor-core path: sort the (token, k) pairs of this wave's experts by
+// expert, upload the wave descriptor, then gather -> grouped tcgen05 FFN -> combine.
+int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, const float* w, int nb,
+                        float* h_inout, const std::vector<int16_t>& slot_of_expert, bool first, bool last,
+                        Timing* t, int ring) {
+    const spm_model_cfg& m = c->cfg;
+    const int K = m.top_k;
+    const size_t d = c->tc_desc_pos++ % kDescRing;
+    if (c->tc_desc_ev_valid[d]) CU(c, cudaEventSynchronize(c->tc_desc_ev[d]));   // staging slot free again
+    unsigned char* hd = c->tc_desc_host + d * c->tc_desc_bytes;
+    unsigned char* dd = c->tc_desc_dev + d * c->tc_desc_bytes;
+    GgUnit* units = reinterpret_cast<GgUnit*>(hd);
+    GgRow* rows = reinterpret_cast<GgRow*>(hd + c->tc_off_rows);
+    int32_t* rowmap = reinterpret_cast<int32_t*>(hd + c->tc_off_rowmap);
+    std::fill(rowmap, rowmap + size_t(nb) * SPM_MAX_TOPK, -1);
+    int n_rows = 0, n_units = 0;
+    for (int e = 0; e < m.n_experts; ++e) {
+        if (slot_of_expert[e] < 0) continue;
+        const int row0 = n_rows;
+        for (int tk = 0; tk < nb; ++tk)
+            for (int k = 0; k < K; ++k)
+                if (ids[tk * K + k] == e) {
+                    rowmap[tk * SPM_MAX_TOPK + k] = n_rows;
+                    rows[n_rows++] = GgRow{tk, k};
+                }
+        if (n_rows == row0) continue;
+        for (int jt = 0; jt < c->n_jt; ++jt)
+            units[n_units++] = GgUnit{layer * c->S + slot_of_expert[e], jt, row0, n_rows - row0};
+    }
+    if (n_units == 0) return SPM_OK;
+    CU(c, cudaMemcpyAsync(dd, hd, c->tc_desc_bytes, cudaMemcpyHostToDevice, c->compute));
+    CU(c, cudaEventRecord(c->tc_desc_ev[d], c->compute));
+    c->tc_desc_ev_valid[d] = 1;
+    gg_gather_kernel<<<n_rows, 128, 0, c->compute>>>(x_norm, w, reinterpret_cast<const GgRow*>(dd + c->tc_off_rows), n_rows,
+                                                     m.hidden, K, c->tc_xs, c->tc_wrow);
+    CU(c, cudaGetLastError());
+    if (t && first) CU(c, cudaEventRecord(t->ffn_start[layer], c->compute));
+    if (ring >= 0 && first) CU(c, cudaEventRecord(c->ring_start[ring], c->compute));
+    GgArgs a{reinterpret_cast<const GgUnit*>(dd), n_units, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status};
+    ffn_grouped_kernel<<<std::min(c->num_sms, n_units), kGgThreads, ffn_grouped_smem(), c->compute>>>(c->wmap, c->xmap, a);
+    CU(c, cudaGetLastError());
+    if (t && last) CU(c, cudaEventRecord(t->ffn_end[layer], c->compute));
+    if (ring >= 0 && last) { CU(c, cudaEventRecord(c->ring_end[ring], c->compute)); c->ring_used[ring] = 1; }
+    gg_combine_kernel<<<dim3((m.hidden + 127) / 128, nb), 128, 0, c->compute>>>(
+        c->tc_partial, reinterpret_cast<const int32_t*>(dd + c->tc_off_rowmap), K, c->n_jt, c->rows_cap, m.hidden, h_inout);
+    CU(c, cudaGetLastError());
+    c->kernel_launches += 3;
+    c->ffn_launches++;
+    c->tc_launches++;
+    return SPM_OK;
+}
+
 // Demand resolution, on-demand copies, stream waits and FFN launches of one layer.
 // `t` (may be null) receives the timing events of this layer; `ring` >= 0 selects an event pair
 // of the stand-alone timing ring instead.
@@ -448,24 +541,29 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
                 a.count[tk] = (unsigned char)cnt;
             }
         };
-        if (t && first) CU(c, cudaEventRecord(t->ffn_start[layer], c->compute));
-        if (ring >= 0 && first) CU(c, cudaEventRecord(c->ring_start[ring], c->compute));
-        if (nb == 1) {
-            FfnArgs<1> a{};
-            fill(a);
-            CU(c, launch_gemv<1>(c, a, G, nb));
+        const bool use_tc = nb > 1 && c->tc_ok && c->batched_path == 0;
+        if (use_tc) {
+            if (int rc = launch_grouped_wave(c, layer, x_norm, ids, w, nb, h_inout, slot_of_expert, first, last, t, ring)) return rc;
         } else {
-            FfnArgs<SPM_MAX_BATCH> a{};
-            fill(a);
-            CU(c, launch_gemv<SPM_MAX_BATCH>(c, a, G, nb));
+            if (t && first) CU(c, cudaEventRecord(t->ffn_start[layer], c->compute));
+            if (ring >= 0 && first) CU(c, cudaEventRecord(c->ring_start[ring], c->compute));
+            if (nb == 1) {
+                FfnArgs<1> a{};
+                fill(a);
+                CU(c, launch_gemv<1>(c, a, G, nb));
+            } else {
+                FfnArgs<SPM_MAX_BATCH> a{};
+                fill(a);
+                CU(c, launch_gemv<SPM_MAX_BATCH>(c, a, G, nb));
+            }
+            if (t && last) CU(c, cudaEventRecord(t->ffn_end[layer], c->compute));
+            if (ring >= 0 && last) { CU(c, cudaEventRecord(c->ring_end[ring], c->compute)); c->ring_used[ring] = 1; }
+            ffn_reduce_kernel<<<dim3((m.hidden + kReduceCols - 1) / kReduceCols, nb), kReduceCols * kReduceGroups, 0, c->compute>>>(
+                c->ws_partial, h_inout, h_inout, G, m.hidden);
+            CU(c, cudaGetLastError());
+            c->kernel_launches += 2;
+            c->ffn_launches++;
         }
-        if (t && last) CU(c, cudaEventRecord(t->ffn_end[layer], c->compute));
-        if (ring >= 0 && last) { CU(c, cudaEventRecord(c->ring_end[ring], c->compute)); c->ring_used[ring] = 1; }
-        ffn_reduce_kernel<<<dim3((m.hidden + kReduceCols - 1) / kReduceCols, nb), kReduceCols * kReduceGroups, 0, c->compute>>>(
-            c->ws_partial, h_inout, h_inout, G, m.hidden);
-        CU(c, cudaGetLastError());
-        c->kernel_launches += 2;
-        c->ffn_launches++;
         if (!last) CU(c, cudaEventRecord(c->wave_done, c->compute));
     }
     CU(c, cudaEventRecord(c->pool_free[layer], c->compute));
@@ -501,6 +599,7 @@ int check_status(spm_ctx* c) {
     CU(c, cudaMemcpy(&st, c->ws_status, sizeof st, cudaMemcpyDeviceToHost));
     if (st & kStatusCopyTimeout) return fail(c, SPM_ERR_TIMEOUT, "expert FFN kernel gave up waiting for a weight copy");
     if (st & kStatusBadSlot) return fail(c, SPM_ERR_NOT_RESIDENT, "expert FFN kernel received a slot number outside the pool");
+    if (st & kStatusGroupedTimeout) return fail(c, SPM_ERR_TIMEOUT, "grouped expert FFN kernel gave up waiting on a pipeline barrier");
     return SPM_OK;
 }
 
@@ -611,6 +710,26 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
             if (!cu(cudaEventCreate(&t.k1_done[l]), "cudaEventCreate") || !cu(cudaEventCreate(&t.ffn_start[l]), "cudaEventCreate") ||
                 !cu(cudaEventCreate(&t.ffn_end[l]), "cudaEventCreate")) return bail(SPM_ERR_CUDA);
     }
+    if (lay.tc) {
+        c->rows_cap = lay.rows_cap; c->n_jt = lay.n_jt; c->max_units = lay.max_units;
+        c->tc_xs = reinterpret_cast<__nv_bfloat16*>(base + lay.tc_xs);
+        c->tc_wrow = reinterpret_cast<float*>(base + lay.tc_wrow);
+        c->tc_partial = reinterpret_cast<float*>(base + lay.tc_partial);
+        c->tc_desc_dev = base + lay.tc_desc;
+        c->tc_desc_bytes = lay.desc_bytes; c->tc_off_rows = lay.off_rows; c->tc_off_rowmap = lay.off_rowmap;
+        if (!cu(cudaMemsetAsync(c->tc_xs, 0, size_t(lay.rows_cap + kGgTokens) * cfg->hidden * 2, c->compute), "cudaMemsetAsync")) return bail(SPM_ERR_CUDA);
+        if (!cu(cudaHostAlloc(reinterpret_cast<void**>(&c->tc_desc_host), size_t(kDescRing) * lay.desc_bytes, cudaHostAllocDefault), "cudaHostAlloc(descriptors)")) return bail(SPM_ERR_CUDA);
+        c->tc_desc_ev.resize(kDescRing);
+        c->tc_desc_ev_valid.assign(kDescRing, 0);
+        for (auto& ev : c->tc_desc_ev) if (!cu(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming), "cudaEventCreate")) return bail(SPM_ERR_CUDA);
+        if (!make_weight_map(&c->wmap, c->pools, cfg->hidden, cfg->inter, uint64_t(L) * c->S) ||
+            !make_token_map(&c->xmap, c->tc_xs, cfg->hidden, uint64_t(lay.rows_cap + kGgTokens))) {
+            c->err = "cuTensorMapEncodeTiled failed";
+            return bail(SPM_ERR_CUDA);
+        }
+        if (!cu(cudaFuncSetAttribute(ffn_grouped_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(ffn_grouped_smem())), "cudaFuncSetAttribute")) return bail(SPM_ERR_CUDA);
+        c->tc_ok = true;
+    }
     c->ring_start.resize(64); c->ring_end.resize(64); c->ring_used.assign(64, 0);
     for (size_t i = 0; i < 64; ++i)
         if (!cu(cudaEventCreate(&c->ring_start[i]), "cudaEventCreate") || !cu(cudaEventCreate(&c->ring_end[i]), "cudaEventCreate")) return bail(SPM_ERR_CUDA);
@@ -641,6 +760,8 @@ int spm_destroy(spm_ctx* c) {
         for (auto ev : t.ffn_start) if (ev) cudaEventDestroy(ev);
         for (auto ev : t.ffn_end) if (ev) cudaEventDestroy(ev);
     }
+    for (auto ev : c->tc_desc_ev) if (ev) cudaEventDestroy(ev);
+    if (c->tc_desc_host) cudaFreeHost(c->tc_desc_host);
     for (auto ev : c->ring_start) if (ev) cudaEventDestroy(ev);
     for (auto ev : c->ring_end) if (ev) cudaEventDestroy(ev);
     if (c->mb_host) cudaFreeHost(c->mb_host);
@@ -823,6 +944,11 @@ int spm_set_ffn_ctas(spm_ctx* c, int ctas) {
     if (!c) return SPM_ERR_INVALID_ARG;
     if (ctas < 0 || ctas > kMaxCtasBatch1) return fail(c, SPM_ERR_INVALID_ARG, "ctas %d (max %d)", ctas, kMaxCtasBatch1);
     c->ffn_ctas = ctas;
+    return SPM_OK;
+}
+int spm_set_batched_path(spm_ctx* c, int mode) {
+    if (!c || mode < 0 || mode > 1) return SPM_ERR_INVALID_ARG;
+    c->batched_path = mode;
     return SPM_OK;
 }
 int spm_set_hint_trace(spm_ctx* c, const int32_t* hint, const int32_t* count, int n_steps, int stride) {

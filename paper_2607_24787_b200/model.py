@@ -134,6 +134,7 @@ class OffloadedMoE:
     def set_plain_lru(self, on): B.spm_set_plain_lru(self.ctx, on)
     def set_timing(self, on): B.spm_set_timing(self.ctx, on)
     def set_ffn_ctas(self, g): B.spm_set_ffn_ctas(self.ctx, g)
+    def set_batched_path(self, mode): B.spm_set_batched_path(self.ctx, mode)
     def set_hint_trace(self, hint): B.spm_set_hint_trace(self.ctx, hint)
     def set_drop_modulo(self, m): B.spm_set_drop_modulo(self.ctx, m)
     def profile_window(self): return B.spm_profile_window(self.ctx)
