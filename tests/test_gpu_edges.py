@@ -1,0 +1,108 @@
+"""Edge and degenerate cases of the decode path on the GPU, each against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from helpers import SynthWeights, make_ref
+from oracle import ref_math as M, ref_policy as P
+
+pytestmark = pytest.mark.gpu
+
+
+def dev(a):
+    t = torch.as_tensor(np.ascontiguousarray(a), dtype=torch.float32).cuda()
+    torch.cuda.synchronize()
+    return t
+
+
+def build(cfg, **kw):
+    from paper_2607_24787_b200.build import build as b
+    from paper_2607_24787_b200.synth_model import build_from_synth
+    b()
+    return build_from_synth(cfg, **kw)
+
+
+def compare_run(cfg, steps=6, policy="adapter", tol=4e-5, **kw):
+    m = build(cfg)
+    wts = SynthWeights(cfg)
+    nb = cfg.batch
+    tok = synth.zipf_tokens(cfg, steps=steps)
+    H = synth.embedding_rows(cfg, tok.reshape(-1)).numpy().reshape(steps, nb, cfg.hidden)
+    ref = make_ref(cfg, weights=wts, policy=policy, **kw)
+    m.set_policy(policy)
+    for s in range(steps):
+        out = m.decode_step(dev(H[s]))
+        m.synchronize()
+        want, _ = ref.step(H[s])
+        got = out.cpu().numpy().astype(np.float64)
+        for t in range(nb):
+            assert M.rel_linf(got[t], want[t]) < tol, (s, t)
+    assert m.events() == ref.table.events
+    st = m.stats()
+    m.close()
+    return st
+
+
+def test_single_layer_has_no_adapter():
+    st = compare_run(synth.get_config("tiny", n_layers=1))
+    assert st["prefetch_issued"] == 0 and st["misses"] > 0
+
+
+def test_top_k_equals_n_and_slots_equal_k():
+    # every expert is used by every token: after the first step nothing is ever loaded again
+    st = compare_run(synth.get_config("tiny", n_experts=4, top_k=4, slots=4, budget=2, adapter_rank=3))
+    assert st["misses"] + st["prefetch_issued"] == 2 * 4          # each of the 8 experts is copied exactly once
+
+
+def test_top_1_and_budget_zero():
+    st = compare_run(synth.get_config("tiny", top_k=1, slots=1, budget=0))
+    assert st["prefetch_issued"] == 0
+
+
+def test_budget_larger_than_slots():
+    st = compare_run(synth.get_config("tiny", slots=3, budget=9))
+    assert st["prefetch_issued"] > 0
+
+
+def test_max_hidden_bf16_and_odd_rank():
+    compare_run(synth.get_config("qwen3", n_layers=2, n_experts=9, inter=40, top_k=2, slots=3, budget=1, adapter_rank=7),
+                steps=4, tol=4e-4)
+
+
+def test_shared_experts_batched_use_gemv_path():
+    # shared experts + several sequences: the per-token GEMV kernel (fp32 activations), with waves
+    cfg = synth.get_config("dsvl2", n_layers=2, n_experts=10, inter=64, top_k=3, slots=4, budget=1, batch=5)
+    st = compare_run(cfg, steps=3, tol=4e-4)
+    assert st["waves"] > 0
+
+
+def test_full_batch_fp32():
+    compare_run(synth.get_config("tiny", batch=64, slots=16, budget=2), steps=2)
+
+
+def test_host_deadline_returns_timeout_and_context_survives():
+    """The routing handshake has a host-side deadline: with the compute stream kept busy by unrelated
+    work the call gives up with SPM_ERR_TIMEOUT instead of spinning; nothing on the GPU is disturbed."""
+    from paper_2607_24787_b200 import binding as B
+    cfg = synth.get_config("tiny")
+    m = build(cfg)
+    h = dev(np.ones((1, cfg.hidden)))
+    a = torch.randn(8192, 8192, device="cuda")
+    B.spm_set_deadline_ms(m.ctx, 1)
+    with torch.cuda.stream(m.compute):
+        for _ in range(40):                      # roughly 50 ms of matmuls queued ahead of the router kernel
+            a = a @ a
+            a = a / a.norm()
+    with pytest.raises(B.SpmError) as e:
+        m.decode_step(h)
+    assert e.value.code == -4
+    torch.cuda.synchronize()
+    B.spm_set_deadline_ms(m.ctx, 5000)
+    m.cache_reset()
+    ref = make_ref(cfg, weights=SynthWeights(cfg))
+    out = m.decode_step(h)
+    m.synchronize()
+    want, _ = ref.step(np.ones((1, cfg.hidden)))
+    assert M.rel_linf(out.cpu().numpy(), want) < 4e-5
+    m.close()
