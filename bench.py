@@ -210,6 +210,8 @@ def run_ours(args):
     t_setup = time.time()
     m = build_from_synth(cfg, device=device)                 # budget -1: profiled inside spm_init
     setup_s = time.time() - t_setup
+    if args.stub_us:
+        m.set_attention_stub_us(args.stub_us)
     window_us, t_xfer_us, raw_budget = m.profile_window()
     budget = max(1, raw_budget) if cfg.budget < 0 else cfg.budget
     m.set_budget(budget)
@@ -256,7 +258,7 @@ def run_ours(args):
         "config": {"workload": f"{cfg.name}: L{cfg.n_layers} D{cfg.hidden} n{cfg.n_experts} I{cfg.inter} K{cfg.top_k}"
                                f"+{cfg.n_shared}sh r{cfg.adapter_rank} {cfg.dtype} slots{cfg.slots} batch{cfg.batch}",
                    "policy": "adapter", "budget": budget, "budget_raw": raw_budget, "window_us": window_us,
-                   "t_xfer_us": t_xfer_us, "seed": cfg.seed, "token_ids": "Zipf(1.1)",
+                   "t_xfer_us": t_xfer_us, "attention_stub_us": args.stub_us, "seed": cfg.seed, "token_ids": "Zipf(1.1)",
                    "l2": "inputs larger than L2: every layer streams its own slot pool, 3.6 GB of weights per step",
                    "setup_s": setup_s, "wall_ms_per_step": wall_ms / K},
         "clocks": clk,
@@ -278,6 +280,8 @@ def run_ours(args):
                           "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(cfg.name), "kernel": "ffn_gemv_kernel",
                           "peak_source": f"of {which}", "algorithmic_bytes_per_launch": algo_bytes,
                           "us_per_launch": ffn_us, "in_kernel_window_us": window_us,
+                          "achieved_in_kernel_window": algo_bytes / (window_us * 1e-6) / 1e9 if window_us > 0 else None,
+                          "frac_in_kernel_window": algo_bytes / (window_us * 1e-6) / 1e9 / peak if window_us > 0 else None,
                           "region": f"main arm, {K} timed steps x {cfg.n_layers} launches, each concurrent with a prefetch copy",
                           "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
     result["main_arm"] = main
@@ -301,6 +305,11 @@ def run_ours(args):
         timed_run(m, H_dev, 0, W, world); m.reset_stats()
         el, _, _ = timed_run(m, H_dev, W, n_arm, world)
         arms["perfect_knowledge"] = arm_summary(m, cfg, el, n_arm)
+        # previous token's experts as the prediction (Naive Prefetch)
+        m.set_policy("naive"); m.cache_reset()
+        timed_run(m, H_dev, 0, W, world); m.reset_stats()
+        el, _, _ = timed_run(m, H_dev, W, n_arm, world)
+        arms["naive"] = arm_summary(m, cfg, el, n_arm)
         # prediction and control only (PRED0)
         m.set_policy("pred0"); m.cache_reset()
         timed_run(m, H_dev, 0, W, world); m.reset_stats()
@@ -433,6 +442,62 @@ def ffn_back_to_back(cfg, full, algo_bytes, peak, launches=480):
             "misses": st["misses"]}
 
 
+def run_sweep(args):
+    """Budget x cache-size sweep on the Qwen3-shaped model: for every slots-per-layer value the
+    on-demand arm, and per budget the adapter arm (the configuration's random adapters), a
+    gate-reuse adapter arm (informative predictor) and the perfect-knowledge arm."""
+    from paper_2607_24787_b200.build import build
+    from paper_2607_24787_b200.synth_model import build_from_synth
+    build()
+    device = "cuda:0"
+    torch.cuda.set_device(0)
+    cfg = bench_config(args)
+    K, W = args.steps, args.warmup
+    tok, H = hidden_rows(cfg, W + K, stream=0)
+    H_dev = H.to(device)
+    torch.cuda.synchronize()
+    store, cells = None, []
+    budgets = [int(b) for b in args.sweep_budgets.split(",")]
+    for S in [int(x) for x in args.sweep_slots.split(",")]:
+        for adapter in ("random", "gate_reuse"):
+            m = build_from_synth(cfg, slots=S, budget=1, device=device, store=store, adapter=adapter)
+            store = m.store
+            m.set_timing(1)
+            if args.stub_us:
+                m.set_attention_stub_us(args.stub_us)
+            if adapter == "random":
+                window = m.profile_window()
+
+            def arm(policy, budget, hint=None):
+                m.set_policy(policy); m.set_budget(budget)
+                if hint is not None:
+                    m.set_hint_trace(hint)
+                m.cache_reset()
+                timed_run(m, H_dev, 0, W, 1); m.reset_stats()
+                el, _, _ = timed_run(m, H_dev, W, K, 1)
+                out = arm_summary(m, cfg, el, K)
+                out.update(slots=S, budget=budget, policy=policy if adapter == "random" or policy != "adapter" else "adapter_gate_reuse")
+                return out
+
+            if adapter == "random":
+                cells.append(arm("on_demand", 0))
+                hint = [[[] for _ in range(cfg.n_layers)] for _ in range(W + K)]
+                m.set_policy("on_demand"); m.cache_reset()
+                timed_run(m, H_dev, 0, W + K, 1)
+                for (s_, l_, kind, e_, _) in m.events():
+                    if kind in ("HIT", "HIT_PREFETCHED", "MISS"):
+                        hint[s_][l_].append(e_)
+                for b in budgets:
+                    cells.append(arm("adapter", b))
+                    cells.append(arm("hint_trace", b, hint))
+            else:
+                for b in budgets:
+                    cells.append(arm("adapter", b))
+            m.close()
+    print(json.dumps({"sweep": f"{cfg.name}: {K} steps per cell, seed {cfg.seed}", "attention_stub_us": args.stub_us,
+                      "window_us": window[0], "t_xfer_us": window[1], "budget_raw": window[2], "cells": cells}))
+
+
 # ------------------------------------------------------------------ CPU oracle legs
 class LazyWeights:
     """Oracle weight provider: matrices regenerated from the synthetic generator on first use."""
@@ -552,6 +617,11 @@ def main():
     ap.add_argument("--slots", type=int, default=0, help="override slots per layer")
     ap.add_argument("--arm-steps", type=int, default=128)
     ap.add_argument("--cpu-steps", type=int, default=2)
+    ap.add_argument("--sweep", action="store_true", help="budget x slots sweep (prints one JSON object with all cells)")
+    ap.add_argument("--sweep-budgets", default="1,2,4,8")
+    ap.add_argument("--sweep-slots", default="8,16,32")
+    ap.add_argument("--stub-us", type=int, default=0,
+                    help="attention stand-in of this many microseconds before each layer's router (widens the overlap window)")
     ap.add_argument("--no-arms", action="store_true")
     ap.add_argument("--no-resident", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -562,7 +632,10 @@ def main():
     else:
         if not torch.cuda.is_available():
             raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU implementation")
-        run_ours(args)
+        if args.sweep:
+            run_sweep(args)
+        else:
+            run_ours(args)
 
 
 if __name__ == "__main__":

@@ -60,6 +60,9 @@ extern "C" {
 #define SPM_POLICY_ON_DEMAND  1   /* no prediction, no prefetch (the paper's OFF arm, Table 4)          */
 #define SPM_POLICY_HINT_TRACE 2   /* perfect knowledge: ranking = recorded true next-layer experts      */
 #define SPM_POLICY_PRED0      3   /* predict and select, issue no transfer (the paper's PRED0, Table 4) */
+#define SPM_POLICY_NAIVE      4   /* prediction = the experts the preceding token used at that layer (the
+                                     paper's Naive Prefetch, Table 5), ranked by sum over tokens of
+                                     (K - rank position), ties to the lower id                          */
 
 /* cache event kinds (spm_event.kind) */
 #define SPM_EV_HIT            1   /* needed expert already has a slot                                   */
@@ -217,12 +220,18 @@ int spm_set_hint_trace(spm_ctx* ctx, const int32_t* hint, const int32_t* count,
 /* Fault injection on the host: every prefetch request with (step + expert) % modulo == 0 is
  * lost before it reaches the GPU (0 switches it off). The demand path must then load it. */
 int spm_set_drop_modulo(spm_ctx* ctx, int modulo);
+/* Stand-in for the attention block the synthetic configurations omit: before each layer's router a
+ * kernel that only waits `us` microseconds (0 = off, at most 100000) is enqueued on the compute
+ * stream. It widens the overlap window W_l = t_exec(l+1) - t_pred(l) (Section 3.1) toward the
+ * paper's regime; spm_profile_window adds it to the window it reports. Outputs are unchanged. */
+int spm_set_attention_stub_us(spm_ctx* ctx, int us);
 /* Host deadline of the routing-kernel handshake, in milliseconds (default 5000). */
 int spm_set_deadline_ms(spm_ctx* ctx, int ms);
 
-/* Profile the overlap window (Section 3.3): window_us = median device time of the expert FFN
- * of one layer with K resident experts, t_xfer_us = median time of one expert copy from the
- * pinned store, *budget_raw = floor(window / t_xfer). Uses and then empties the cache. */
+/* Profile the overlap window (Section 3.3): window_us = median device time of the expert FFN of
+ * one layer at max_batch tokens with every needed expert resident (kernel(s) + combine, the same
+ * path a decode step takes), t_xfer_us = median time of one expert copy from the pinned store,
+ * *budget_raw = floor(window / t_xfer). Uses and then empties the cache. */
 int spm_profile_window(spm_ctx* ctx, double* window_us, double* t_xfer_us, int* budget_raw);
 
 int spm_cache_reset(spm_ctx* ctx);                         /* cold cache, step counter, stats, events */

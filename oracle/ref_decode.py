@@ -62,6 +62,7 @@ class RefDecoder:
         self.storage = [dict() for _ in range(n_layers)]   # slot -> (expert, triple)
         self.drop_hook = None     # callable(step, layer, expert) -> bool: lose this prefetch request
         self.keep_records = keep_records
+        self.prev_rank = [[] for _ in range(n_layers)]   # Naive Prefetch: what the preceding step used per layer
 
     # -- transfers into the software slot pool ----------------------------
     def _copy_in(self, layer, expert, slot):
@@ -94,6 +95,7 @@ class RefDecoder:
             ids = np.stack([r[0] for r in routed])
             w = np.stack([r[1] for r in routed])
             rec = LayerRecord(ids=ids, w=w, logits=Z, x=X)
+            this_rank = P.borda_ranking(ids, self.n)
 
             # demand of this layer (Section 3.1, second equation) and on-demand loads
             need = M.batch_demand(ids)
@@ -110,6 +112,8 @@ class RefDecoder:
                     if self.policy == P.HINT_TRACE:
                         ranking = [int(e) for e in hint[l + 1]]
                         sel, protect = tbl.plan(l + 1, ranking, self.M_max, protect_all=True)
+                    elif self.policy == P.NAIVE:
+                        sel, protect = tbl.plan(l + 1, self.prev_rank[l + 1], self.M_max)
                     else:
                         ranking = [int(e) for e in rec.order]
                         sel, protect = tbl.plan(l + 1, ranking, self.M_max)
@@ -144,6 +148,7 @@ class RefDecoder:
                 for trip in shared:
                     y[t] += M.swiglu_expert(*trip, X[t])
             h = h + y
+            self.prev_rank[l] = this_rank          # becomes "the preceding token" for the next step
             rec.h_out = h.copy()
             if self.keep_records:
                 recs.append(rec)

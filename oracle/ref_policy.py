@@ -38,6 +38,7 @@ ADAPTER = "adapter"          # prefetch what the adapter ranks highest
 ON_DEMAND = "on_demand"      # no prediction, no prefetch (the paper's OFF arm)
 HINT_TRACE = "hint_trace"    # perfect knowledge: ranking = the true next-layer experts
 PRED0 = "pred0"              # predict and select, issue nothing (the paper's PRED0 arm)
+NAIVE = "naive"              # prefetch what the preceding token used at that layer (the paper's Naive Prefetch arm)
 
 
 @dataclass
@@ -60,6 +61,20 @@ class Stats:
     touches: int = 0
     waves: int = 0
     planned: int = 0
+
+
+def borda_ranking(ids_per_token, n_experts: int):
+    """Experts used by a batch, ranked by sum over tokens of (K - rank position), ties to the lower id.
+
+    For one token this is the router's own rank order. Used by the Naive Prefetch arm, which
+    replays the previous token's experts as the prediction (Section 4.4, Table 5)."""
+    score = [0] * n_experts
+    for ids in ids_per_token:
+        K = len(ids)
+        for pos, e in enumerate(ids):
+            score[int(e)] += K - pos
+    used = [e for e in range(n_experts) if score[e] > 0]
+    return sorted(used, key=lambda e: (-score[e], e))
 
 
 def select_prefetch(ranking, has_slot, budget: int, slots: int):

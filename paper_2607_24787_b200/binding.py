@@ -18,8 +18,8 @@ SPM_OK = 0
 ERR_NAMES = {-1: "SPM_ERR_INVALID_ARG", -2: "SPM_ERR_CONFIG", -3: "SPM_ERR_CUDA", -4: "SPM_ERR_TIMEOUT",
              -5: "SPM_ERR_NOT_RESIDENT", -6: "SPM_ERR_STATE"}
 DTYPE_FP32, DTYPE_BF16 = 0, 1
-POLICY_ADAPTER, POLICY_ON_DEMAND, POLICY_HINT_TRACE, POLICY_PRED0 = 0, 1, 2, 3
-POLICIES = {"adapter": 0, "on_demand": 1, "hint_trace": 2, "pred0": 3}
+POLICY_ADAPTER, POLICY_ON_DEMAND, POLICY_HINT_TRACE, POLICY_PRED0, POLICY_NAIVE = 0, 1, 2, 3, 4
+POLICIES = {"adapter": 0, "on_demand": 1, "hint_trace": 2, "pred0": 3, "naive": 4}
 EVENT_NAMES = {1: "HIT", 2: "HIT_PREFETCHED", 3: "MISS", 4: "EVICT", 5: "EVICT_WASTED", 6: "PREFETCH",
                7: "TOUCH_PRED", 8: "WAVE", 9: "PLAN", 10: "DROPPED"}
 MAX_BATCH, MAX_TOPK, MAX_EXPERTS = 64, 16, 1024
@@ -82,6 +82,7 @@ _SIG = {
     "spm_set_hint_trace": [_P, _P, _P, C.c_int, C.c_int],
     "spm_set_drop_modulo": [_P, C.c_int],
     "spm_set_deadline_ms": [_P, C.c_int],
+    "spm_set_attention_stub_us": [_P, C.c_int],
     "spm_profile_window": [_P, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int)],
     "spm_cache_reset": [_P],
     "spm_reset_stats": [_P],
@@ -260,6 +261,10 @@ def spm_set_hint_trace(ctx, hint):
 
 def spm_set_drop_modulo(ctx, modulo):
     _check(load().spm_set_drop_modulo(ctx, modulo), ctx)
+
+
+def spm_set_attention_stub_us(ctx, us):
+    _check(load().spm_set_attention_stub_us(ctx, us), ctx)
 
 
 def spm_set_deadline_ms(ctx, ms):

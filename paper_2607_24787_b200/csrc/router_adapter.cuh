@@ -8,10 +8,12 @@
 // One thread-block cluster per token: its CTAs split the n + r weight rows (one warp per row,
 // 16-byte read-only loads all issued before the first use, shuffle reduction) and store the dot
 // products into the leader CTA's shared memory over DSMEM; after one cluster barrier the leader
-// does the token's softmax / Top-K / adapter tail. With several tokens the last leader to
-// finish (atomic ticket) does the batch aggregation. The publishing CTA ranks the priorities,
-// copies ids / order / scores into the host-mapped mailbox, fences at system scope and writes
-// the launch's sequence number, which the host polls.
+// does the token's tails, router (softmax / Top-K) and adapter (up-projection / softmax / ranking)
+// side by side on its two half-blocks. With several tokens the last leader to finish (atomic
+// ticket) does the batch aggregation. Expert ids and the ranking go to the host-mapped mailbox as
+// self-tagged words (sequence number in the upper half) the moment they exist, so the host can
+// act on the ids while the adapter tail is still running; a fenced sequence number follows for
+// callers that also read the untagged scores.
 // Every reduction has a fixed order, so results are bitwise reproducible.
 #pragma once
 
@@ -120,131 +122,235 @@ __device__ __forceinline__ float load_weight(const WT* p, size_t i) {
     return reinterpret_cast<const float*>(p)[i];
 }
 
+// 128-thread (half-block) reduction: shuffle inside warps, 4 warp results through `slot`, one
+// named barrier. Each call site uses its own `slot`, so no barrier is needed before the write.
+__device__ __forceinline__ float half_reduce(float v, float* slot, bool is_max, int bar_id) {
+    const int lane = threadIdx.x & 31, wq = (threadIdx.x >> 5) & 3;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float t = __shfl_xor_sync(0xffffffffu, v, o);
+        v = is_max ? fmaxf(v, t) : v + t;
+    }
+    if (lane == 0) slot[wq] = v;
+    asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+    float r = slot[0];
+#pragma unroll
+    for (int i = 1; i < 4; ++i) r = is_max ? fmaxf(r, slot[i]) : r + slot[i];
+    return r;
+}
+
+// softmax of v[0..n) in shared memory by the 128 threads of one half-block, in place
+__device__ __forceinline__ void half_softmax(float* v, int n, float* slots, int bar_id) {
+    const int ht = threadIdx.x & 127;
+    float m = -INFINITY;
+    for (int e = ht; e < n; e += 128) m = fmaxf(m, v[e]);
+    m = half_reduce(m, slots, true, bar_id);
+    float s = 0.f;
+    for (int e = ht; e < n; e += 128) {
+        const float t = expf(v[e] - m);
+        v[e] = t;
+        s += t;
+    }
+    s = half_reduce(s, slots + 4, false, bar_id);
+    for (int e = ht; e < n; e += 128) v[e] = v[e] / s;
+    asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+}
+
+// Mailbox words carry the launch's sequence number in their upper half, so the host can tell a
+// fresh word from a stale one without any fence between payload and flag.
+__device__ __forceinline__ int32_t tagged(uint32_t seq, int value) { return int32_t((seq << 16) | uint32_t(value)); }
+
 // Grid (kRouterCluster, nb), cluster (kRouterCluster, 1, 1): the CTAs of a cluster split the n + r
 // weight rows of one token and deliver their dot products straight into the leader CTA's shared
-// memory; after one cluster barrier the leader alone runs the softmax / Top-K / adapter tail.
+// memory; after one cluster barrier the leader runs the router tail (softmax, Top-K, renormalise)
+// on its first four warps and the adapter tail (up-projection, softmax, ranking) on the other four.
 template <typename WT>
 __global__ void __launch_bounds__(kRouterThreads)
 router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     constexpr int VEC = 16 / int(sizeof(WT));
     constexpr int MAXIT = 8;        // hidden <= MAXIT * 32 * VEC
+    constexpr int ROWS = 3;         // weight rows a warp fetches before it starts to multiply
     extern __shared__ __align__(16) float sm[];
     float* xs = sm;                 // [D]
     float* zs = xs + a.D;           // [n] logits (leader: filled by the whole cluster)
-    float* ps = zs + a.n;           // [n] probabilities / adapter logits / scores
-    float* us = ps + a.n;           // [r] adapter hidden (leader: filled by the whole cluster)
-    float* scratch = us + a.r;      // [8]
-    float* psel = scratch + kRouterWarps;                       // [K]
+    float* ps = zs + a.n;           // [n] router probabilities
+    float* qs = ps + a.n;           // [n] adapter logits -> probabilities -> priorities
+    float* us = qs + a.n;           // [r] adapter hidden (leader: filled by the whole cluster)
+    float* scratch = us + a.r;      // [16] reduction slots
+    float* psel = scratch + 16;                                 // [K]
     int* isel = reinterpret_cast<int*>(psel + SPM_MAX_TOPK);    // [K]
     float* bs = reinterpret_cast<float*>(isel + SPM_MAX_TOPK);  // [n * r] adapter up-projection (leader)
     __shared__ int s_last;
+    __shared__ float s_tot;
 
+#ifdef SPM_ROUTER_TIMESTAMPS
+    unsigned long long ts[8];
+    ts[0] = global_timer_ns();
+#define SPM_TS(i) ts[i] = global_timer_ns()
+#else
+#define SPM_TS(i)
+#endif
     const int tok = blockIdx.y;
     const uint32_t cr = cluster_ctarank();
     const bool leader = cr == 0;
     const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
     const int D = a.D, n = a.n;
+    const uint32_t tag = a.seq & 0xffffu;
 
     // every CTA of the cluster must be running before anyone writes into the leader's shared
     // memory: arrive now, wait just before the first remote store
     asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
 
-    // leader: start fetching the small adapter up-projection now, it is needed only in the tail
-    if (leader && a.do_adapter) {
-        const WT* B = static_cast<const WT*>(a.adapter_b);
-        for (int i = threadIdx.x; i < n * a.r; i += kRouterThreads) bs[i] = load_weight(B, i);
-    }
-
-    // ---- router input ---------------------------------------------------
+    // ---- router input: hidden row and gain are fetched together, then normalised -----------
     if (a.do_router) {
         const float* ht = a.h + size_t(tok) * D;
+        constexpr int NV4 = MAXIT * 32 * VEC / (kRouterThreads * 4);   // float4 per thread at the largest hidden size
+        float4 hv[NV4], gv[NV4];
+#pragma unroll
+        for (int c = 0; c < NV4; ++c) {
+            const int i = (c * kRouterThreads + threadIdx.x) * 4;
+            if (i < D) {
+                hv[c] = *reinterpret_cast<const float4*>(ht + i);
+                gv[c] = *reinterpret_cast<const float4*>(a.gamma + i);
+            }
+        }
+        // leader: the small adapter up-projection is needed only in the tail; fetch it while the
+        // row and gain are in flight
+        if (leader && a.do_adapter) {
+            const WT* B = static_cast<const WT*>(a.adapter_b);
+            for (int i = threadIdx.x; i < n * a.r; i += kRouterThreads) bs[i] = load_weight(B, i);
+        }
         float ss = 0.f;
-        for (int i = threadIdx.x; i < D; i += kRouterThreads) {
-            const float v = ht[i];
-            xs[i] = v;
-            ss = fmaf(v, v, ss);
+#pragma unroll
+        for (int c = 0; c < NV4; ++c) {
+            const int i = (c * kRouterThreads + threadIdx.x) * 4;
+            if (i < D) {
+                ss = fmaf(hv[c].x, hv[c].x, ss); ss = fmaf(hv[c].y, hv[c].y, ss);
+                ss = fmaf(hv[c].z, hv[c].z, ss); ss = fmaf(hv[c].w, hv[c].w, ss);
+            }
         }
         ss = block_reduce(ss, scratch, false);
         const float inv = 1.0f / sqrtf(ss / float(D) + a.eps);
-        for (int i = threadIdx.x; i < D; i += kRouterThreads) {
-            const float v = xs[i] * a.gamma[i] * inv;
-            xs[i] = v;
-            if (leader && a.x_norm) a.x_norm[size_t(tok) * D + i] = v;
+#pragma unroll
+        for (int c = 0; c < NV4; ++c) {
+            const int i = (c * kRouterThreads + threadIdx.x) * 4;
+            if (i < D) {
+                float4 o;
+                o.x = hv[c].x * gv[c].x * inv; o.y = hv[c].y * gv[c].y * inv;
+                o.z = hv[c].z * gv[c].z * inv; o.w = hv[c].w * gv[c].w * inv;
+                *reinterpret_cast<float4*>(xs + i) = o;
+                if (leader && a.x_norm) *reinterpret_cast<float4*>(a.x_norm + size_t(tok) * D + i) = o;
+            }
         }
     } else {
         const float* xt = a.x_in + size_t(tok) * D;
         for (int i = threadIdx.x; i < D; i += kRouterThreads) xs[i] = xt[i];
+        if (leader && a.do_adapter) {
+            const WT* B = static_cast<const WT*>(a.adapter_b);
+            for (int i = threadIdx.x; i < n * a.r; i += kRouterThreads) bs[i] = load_weight(B, i);
+        }
     }
     __syncthreads();
+    SPM_TS(1);
 
-    // ---- weight rows: router rows then adapter-A rows, one warp per row ----
+    // ---- weight rows: router rows then adapter-A rows, one warp per row, ROWS rows in flight ----
     const int n_r = a.do_router ? n : 0;
     const int rows = n_r + (a.do_adapter ? a.r : 0);
+    constexpr int STRIDE = kRouterCluster * kRouterWarps;
     asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
-    for (int row = int(cr) * kRouterWarps + wi; row < rows; row += kRouterCluster * kRouterWarps) {
-        const WT* wrow = row < n_r ? static_cast<const WT*>(a.router_w) + size_t(row) * D
-                                   : static_cast<const WT*>(a.adapter_a) + size_t(row - n_r) * D;
-        uint4 v[MAXIT];
+    for (int row0 = int(cr) * kRouterWarps + wi; row0 < rows; row0 += ROWS * STRIDE) {
+        uint4 v[ROWS][MAXIT];
 #pragma unroll
-        for (int it = 0; it < MAXIT; ++it) {
-            const int i = (it * 32 + lane) * VEC;
-            if (i < D) v[it] = __ldg(reinterpret_cast<const uint4*>(wrow + i));
-        }
-        float acc = 0.f;
+        for (int rr = 0; rr < ROWS; ++rr) {
+            const int row = row0 + rr * STRIDE;
+            if (row < rows) {
+                const WT* wrow = row < n_r ? static_cast<const WT*>(a.router_w) + size_t(row) * D
+                                           : static_cast<const WT*>(a.adapter_a) + size_t(row - n_r) * D;
 #pragma unroll
-        for (int it = 0; it < MAXIT; ++it) {
-            const int i = (it * 32 + lane) * VEC;
-            if (i < D) {
-                float f[VEC];
-                unpack16(v[it], f);
-#pragma unroll
-                for (int q = 0; q < VEC; ++q) acc = fmaf(f[q], xs[i + q], acc);
+                for (int it = 0; it < MAXIT; ++it) {
+                    const int i = (it * 32 + lane) * VEC;
+                    if (i < D) v[rr][it] = __ldg(reinterpret_cast<const uint4*>(wrow + i));
+                }
             }
         }
-        acc = warp_sum(acc);
-        if (lane == 0) dsmem_store(row < n_r ? zs + row : us + (row - n_r), 0, acc);
+#pragma unroll
+        for (int rr = 0; rr < ROWS; ++rr) {
+            const int row = row0 + rr * STRIDE;
+            if (row < rows) {
+                float acc = 0.f;
+#pragma unroll
+                for (int it = 0; it < MAXIT; ++it) {
+                    const int i = (it * 32 + lane) * VEC;
+                    if (i < D) {
+                        float f[VEC];
+                        unpack16(v[rr][it], f);
+#pragma unroll
+                        for (int q = 0; q < VEC; ++q) acc = fmaf(f[q], xs[i + q], acc);
+                    }
+                }
+                acc = warp_sum(acc);
+                if (lane == 0) dsmem_store(row < n_r ? zs + row : us + (row - n_r), 0, acc);
+            }
+        }
     }
+    SPM_TS(2);
     cluster_sync_all();
     if (!leader) return;
+    SPM_TS(3);
 
-    // ---- tail (leader CTA of the token) -------------------------------------
-    if (a.do_router) {
-        for (int e = threadIdx.x; e < n; e += kRouterThreads) {
+    // ---- tails (leader CTA): router on warps 0-3, adapter on warps 4-7, concurrently ----------
+    Mailbox* mb = a.mailbox;
+    const int half = threadIdx.x >> 7, ht = threadIdx.x & 127;
+    if (half == 0 && a.do_router) {
+        for (int e = ht; e < n; e += 128) {
             const float z = zs[e];
             ps[e] = z;
             a.logits[size_t(tok) * n + e] = z;
             if (a.logits_out) a.logits_out[size_t(tok) * n + e] = z;
         }
-        __syncthreads();
-        block_softmax(ps, n, scratch);          // ps = p, zs = z (ranking is taken on the logits)
-        for (int e = threadIdx.x; e < n; e += kRouterThreads) {
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        half_softmax(ps, n, scratch, 1);          // ps = p, zs = z (ranking is taken on the logits)
+        for (int e = ht; e < n; e += 128) {
             const int rk = rank_of(zs, n, e);
             if (rk < a.K) { isel[rk] = e; psel[rk] = ps[e]; }
         }
-        __syncthreads();
-        if (threadIdx.x == 0) {
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (ht == 0) {
             float tot = 0.f;
             for (int k = 0; k < a.K; ++k) tot += psel[k];
-            for (int k = 0; k < a.K; ++k) {
-                a.ids[size_t(tok) * a.K + k] = isel[k];
-                a.w[size_t(tok) * a.K + k] = a.renorm ? psel[k] / tot : psel[k];
+            s_tot = tot;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (ht < a.K) {
+            a.ids[size_t(tok) * a.K + ht] = isel[ht];
+            a.w[size_t(tok) * a.K + ht] = a.renorm ? psel[ht] / s_tot : psel[ht];
+            mb->ids[tok * a.K + ht] = tagged(tag, isel[ht]);      // the host may start on these at once
+        }
+    }
+    SPM_TS(4);
+    if (half == 1 && a.do_adapter) {
+        for (int e = ht; e < n; e += 128) {
+            float acc = 0.f;
+            for (int q = 0; q < a.r; ++q) acc = fmaf(bs[e * a.r + q], us[q], acc);
+            qs[e] = acc;
+        }
+        asm volatile("bar.sync 2, 128;" ::: "memory");
+        half_softmax(qs, n, scratch + 8, 2);
+        if (a.nb > 1) {
+            for (int e = ht; e < n; e += 128) a.pihat[size_t(tok) * n + e] = qs[e];
+        } else {
+            for (int e = ht; e < n; e += 128) {        // one token: its distribution is the priority vector
+                const int rk = rank_of(qs, n, e);
+                a.order[rk] = e;
+                a.scores[e] = qs[e];
+                mb->order[rk] = tagged(tag, e);
+                mb->scores[e] = qs[e];
             }
         }
     }
-    if (a.do_adapter) {
-        __syncthreads();
-        for (int e = threadIdx.x; e < n; e += kRouterThreads) {
-            float acc = 0.f;
-            for (int q = 0; q < a.r; ++q) acc = fmaf(bs[e * a.r + q], us[q], acc);
-            ps[e] = acc;
-        }
-        __syncthreads();
-        block_softmax(ps, n, scratch);
-        if (a.nb > 1)
-            for (int e = threadIdx.x; e < n; e += kRouterThreads) a.pihat[size_t(tok) * n + e] = ps[e];
-    }
+    SPM_TS(5);
 
-    // ---- several tokens: the last leader to finish aggregates ----------------
+    // ---- several tokens: the last leader to finish aggregates and ranks -------------------------
     if (a.nb > 1) {
         __threadfence();
         __syncthreads();
@@ -256,37 +362,32 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
             for (int e = threadIdx.x; e < n; e += kRouterThreads) {
                 float s = 0.f;
                 for (int t = 0; t < a.nb; ++t) s += __ldcg(a.pihat + size_t(t) * n + e);
-                ps[e] = s;
+                qs[e] = s;
+            }
+            __syncthreads();
+            for (int e = threadIdx.x; e < n; e += kRouterThreads) {
+                const int rk = rank_of(qs, n, e);
+                a.order[rk] = e;
+                a.scores[e] = qs[e];
+                mb->order[rk] = tagged(tag, e);
+                mb->scores[e] = qs[e];
             }
         }
         if (threadIdx.x == 0) a.counters[0] = 0u;
     }
-    __syncthreads();
-
-    Mailbox* mb = a.mailbox;
-    if (a.do_adapter) {
-        for (int e = threadIdx.x; e < n; e += kRouterThreads) {
-            const int rk = rank_of(ps, n, e);
-            a.order[rk] = e;
-            a.scores[e] = ps[e];
-            mb->order[rk] = e;
-            mb->scores[e] = ps[e];
-        }
-    }
-    if (a.do_router) {
-        if (a.nb > 1) {
-            for (int i = threadIdx.x; i < a.nb * a.K; i += kRouterThreads) mb->ids[i] = __ldcg(a.ids + i);
-        } else if (threadIdx.x < a.K) {
-            mb->ids[threadIdx.x] = isel[threadIdx.x];
-        }
-    }
+    SPM_TS(6);
+    // final flag for callers that read untagged payload (scores): fence, then the sequence number
     __threadfence_system();
     __syncthreads();
     if (threadIdx.x == 0) mb->seq = a.seq;
+#ifdef SPM_ROUTER_TIMESTAMPS
+    SPM_TS(7);
+    if (threadIdx.x == 0) for (int i = 0; i < 8; ++i) reinterpret_cast<unsigned long long*>(a.pihat)[i] = ts[i];
+#endif
 }
 
 inline size_t router_smem_bytes(int D, int n, int r) {
-    return sizeof(float) * (size_t(D) + 2 * size_t(n) + size_t(r) + kRouterWarps + 2 * SPM_MAX_TOPK + size_t(n) * r);
+    return sizeof(float) * (size_t(D) + 3 * size_t(n) + size_t(r) + 16 + 2 * SPM_MAX_TOPK + size_t(n) * r);
 }
 
 }  // namespace spm

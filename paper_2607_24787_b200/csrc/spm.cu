@@ -95,6 +95,8 @@ struct spm_ctx {
     std::vector<int32_t> hint, hint_count;
     int hint_steps = 0, hint_stride = 0;
     int drop_modulo = 0;
+    int stub_us = 0;                          // attention stand-in before each layer's router
+    std::vector<std::vector<int32_t>> prev_rank;   // Naive Prefetch: experts the preceding step used, per layer
     std::vector<std::vector<int32_t>> pending_protect;
     std::vector<uint8_t> has_plan;
     std::vector<int32_t> prev_order;          // ranking produced at the previous layer of this step
@@ -323,6 +325,31 @@ int wait_mailbox(spm_ctx* c) {
             auto ms = std::chrono::duration_cast<std::chrono::milliseconds>(std::chrono::steady_clock::now() - t0).count();
             if (ms > c->deadline_ms)
                 return fail(c, SPM_ERR_TIMEOUT, "routing kernel did not report within %d ms", c->deadline_ms);
+        }
+    }
+    std::atomic_thread_fence(std::memory_order_acquire);
+    return SPM_OK;
+}
+
+// Wait (bounded) until `count` self-tagged mailbox words carry the current launch's tag, then
+// return their payloads. The device writes each word as (sequence << 16) | value, so no fence or
+// separate flag is involved: a word is either stale (old tag) or complete.
+int wait_tagged(spm_ctx* c, const volatile int32_t* words, int count, int32_t* out, const char* what) {
+    const uint32_t tag = c->seq & 0xffffu;
+    const auto t0 = std::chrono::steady_clock::now();
+    uint64_t spins = 0;
+    int done = 0;
+    while (done < count) {
+        const uint32_t wv = uint32_t(words[done]);
+        if ((wv >> 16) == tag) { out[done++] = int32_t(wv & 0xffffu); continue; }
+        _mm_pause();
+        if ((++spins & 0x3fff) == 0) {
+            cudaError_t q = cudaStreamQuery(c->compute);
+            if (q != cudaSuccess && q != cudaErrorNotReady)
+                return fail(c, SPM_ERR_CUDA, "compute stream failed while waiting for the %s: %s", what, cudaGetErrorString(q));
+            auto ms = std::chrono::duration_cast<std::chrono::milliseconds>(std::chrono::steady_clock::now() - t0).count();
+            if (ms > c->deadline_ms)
+                return fail(c, SPM_ERR_TIMEOUT, "routing kernel did not deliver the %s within %d ms", what, c->deadline_ms);
         }
     }
     std::atomic_thread_fence(std::memory_order_acquire);
@@ -587,6 +614,22 @@ int do_prefetch(spm_ctx* c, int target, const int32_t* ids, int count, const int
     return SPM_OK;
 }
 
+// Stand-in for the omitted attention block: one thread watches %globaltimer until `ns` have passed.
+__global__ void attention_stub_kernel(unsigned long long ns) {
+    const unsigned long long t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < ns) __nanosleep(200);
+}
+
+// Experts of this step's routing at one layer, ranked by sum over tokens of (K - rank position).
+void borda_rank(const int32_t* ids, int nb, int K, int n, std::vector<int32_t>& out) {
+    std::vector<int32_t> score(n, 0);
+    for (int t = 0; t < nb; ++t)
+        for (int k = 0; k < K; ++k) score[ids[t * K + k]] += K - k;
+    out.clear();
+    for (int e = 0; e < n; ++e) if (score[e] > 0) out.push_back(e);
+    std::stable_sort(out.begin(), out.end(), [&](int32_t x, int32_t y) { return score[x] > score[y]; });
+}
+
 int check_layer(spm_ctx* c, int layer, int nb) {
     if (!c) return SPM_ERR_INVALID_ARG;
     if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, SPM_ERR_INVALID_ARG, "layer %d out of range", layer);
@@ -684,6 +727,7 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
     const int L = cfg->n_layers;
     c->table = new SlotTable(L, cfg->n_experts, c->S, false);
     c->pending_protect.resize(L);
+    c->prev_rank.assign(L, {});
     c->has_plan.assign(L, 0);
     c->layer_stall_us.assign(L, 0.0);
     c->layer_ffn_us.assign(L, 0.0);
@@ -777,7 +821,7 @@ int spm_router_topk(spm_ctx* c, int layer, const float* h, int nb, float* x_norm
     if (int rc = launch_router(c, layer, h, nullptr, nb, x_norm, logits, true, false)) return rc;
     CU(c, cudaMemcpyAsync(w, c->ws_w, size_t(nb) * c->cfg.top_k * 4, cudaMemcpyDeviceToDevice, c->compute));
     if (int rc = wait_mailbox(c)) return rc;
-    memcpy(ids, c->mb_host->ids, size_t(nb) * c->cfg.top_k * 4);
+    for (int i = 0; i < nb * c->cfg.top_k; ++i) ids[i] = c->mb_host->ids[i] & 0xffff;
     return SPM_OK;
 }
 
@@ -788,7 +832,7 @@ int spm_adapter_predict(spm_ctx* c, int layer, const float* x_norm, int nb, floa
     if (int rc = launch_router(c, layer, nullptr, x_norm, nb, nullptr, nullptr, false, true)) return rc;
     if (int rc = wait_mailbox(c)) return rc;
     memcpy(scores, c->mb_host->scores, size_t(c->cfg.n_experts) * 4);
-    memcpy(order, c->mb_host->order, size_t(c->cfg.n_experts) * 4);
+    for (int i = 0; i < c->cfg.n_experts; ++i) order[i] = c->mb_host->order[i] & 0xffff;
     return SPM_OK;
 }
 
@@ -849,12 +893,17 @@ int spm_decode_step(spm_ctx* c, const float* h_in, int nb, float* h_out) {
     const bool predict = c->policy == SPM_POLICY_ADAPTER || c->policy == SPM_POLICY_PRED0;
     c->prev_order_valid = false;
     std::vector<int32_t> ids(size_t(nb) * K);
+    std::vector<int32_t> this_rank;
     for (int l = 0; l < L; ++l) {
         const bool has_adapter = l <= L - 2;
+        if (c->stub_us > 0) {
+            attention_stub_kernel<<<1, 1, 0, c->compute>>>(uint64_t(c->stub_us) * 1000ull);
+            CU(c, cudaGetLastError());
+            c->kernel_launches++;
+        }
         if (int rc = launch_router(c, l, h_out, nullptr, nb, c->ws_x, nullptr, true, predict && has_adapter)) return rc;
         if (t) CU(c, cudaEventRecord(t->k1_done[l], c->compute));
-        if (int rc = wait_mailbox(c)) return rc;
-        memcpy(ids.data(), c->mb_host->ids, ids.size() * 4);
+        if (int rc = wait_tagged(c, c->mb_host->ids, nb * K, ids.data(), "expert ids")) return rc;
 
         if (c->prev_order_valid) {   // ExpertRecall@M of the previous layer's prediction, M = budget
             const int M = std::min(c->budget, n);
@@ -867,6 +916,7 @@ int spm_decode_step(spm_ctx* c, const float* h_in, int nb, float* h_out) {
             }
         }
         if (int rc = run_ffn(c, l, c->ws_x, ids.data(), c->ws_w, nb, h_out, t)) return rc;
+        if (c->policy == SPM_POLICY_NAIVE) borda_rank(ids.data(), nb, K, n, this_rank);
 
         c->prev_order_valid = false;
         if (has_adapter && c->policy != SPM_POLICY_ON_DEMAND) {
@@ -878,8 +928,12 @@ int spm_decode_step(spm_ctx* c, const float* h_in, int nb, float* h_out) {
                 ranking = c->hint.data() + cell * c->hint_stride;
                 n_ranked = c->hint_count[cell];
                 protect_all = true;
+            } else if (c->policy == SPM_POLICY_NAIVE) {
+                ranking = c->prev_rank[l + 1].data();      // what the preceding step used at layer l+1
+                n_ranked = int(c->prev_rank[l + 1].size());
             } else {
-                c->prev_order.assign(c->mb_host->order, c->mb_host->order + n);
+                c->prev_order.resize(n);
+                if (int rc = wait_tagged(c, c->mb_host->order, n, c->prev_order.data(), "expert ranking")) return rc;
                 c->prev_order_valid = true;
                 ranking = c->prev_order.data();
                 n_ranked = n;
@@ -892,6 +946,7 @@ int spm_decode_step(spm_ctx* c, const float* h_in, int nb, float* h_out) {
                                          int(c->protect.size()), nullptr)) return rc;
             }
         }
+        if (c->policy == SPM_POLICY_NAIVE) c->prev_rank[l] = this_rank;
     }
     tb.end_step();
     tb.stats().steps++;
@@ -913,8 +968,8 @@ int spm_decode_step_host(spm_ctx* c, const float* h_in_host, int nb, float* h_ou
 // ---- control --------------------------------------------------------------
 int spm_set_policy(spm_ctx* c, int policy) {
     if (!c) return SPM_ERR_INVALID_ARG;
-    if (policy < SPM_POLICY_ADAPTER || policy > SPM_POLICY_PRED0) return fail(c, SPM_ERR_INVALID_ARG, "policy %d", policy);
-    if (policy != SPM_POLICY_ON_DEMAND && c->cfg.n_layers > 1 && (!c->buf.adapter_a || !c->buf.adapter_b) && policy != SPM_POLICY_HINT_TRACE)
+    if (policy < SPM_POLICY_ADAPTER || policy > SPM_POLICY_NAIVE) return fail(c, SPM_ERR_INVALID_ARG, "policy %d", policy);
+    if ((policy == SPM_POLICY_ADAPTER || policy == SPM_POLICY_PRED0) && c->cfg.n_layers > 1 && (!c->buf.adapter_a || !c->buf.adapter_b))
         return fail(c, SPM_ERR_STATE, "no adapter weights");
     c->policy = policy;
     return SPM_OK;
@@ -972,6 +1027,11 @@ int spm_set_drop_modulo(spm_ctx* c, int modulo) {
     c->drop_modulo = modulo;
     return SPM_OK;
 }
+int spm_set_attention_stub_us(spm_ctx* c, int us) {
+    if (!c || us < 0 || us > 100000) return SPM_ERR_INVALID_ARG;
+    c->stub_us = us;
+    return SPM_OK;
+}
 int spm_set_deadline_ms(spm_ctx* c, int ms) {
     if (!c || ms < 1) return SPM_ERR_INVALID_ARG;
     c->deadline_ms = ms;
@@ -1010,6 +1070,7 @@ int spm_cache_reset(spm_ctx* c) {
     CU(c, cudaStreamSynchronize(c->compute));
     for (auto& t : c->tim) std::fill(t.used.begin(), t.used.end(), 0);
     c->table->reset();
+    for (auto& r : c->prev_rank) r.clear();
     std::fill(c->ring_used.begin(), c->ring_used.end(), 0);
     c->ring_us = 0;
     if (int rc = arm_clock(c)) return rc;
@@ -1030,7 +1091,6 @@ int spm_profile_window(spm_ctx* c, double* window_us, double* t_xfer_us, int* bu
     if (!c || !window_us || !t_xfer_us || !budget_raw) return SPM_ERR_INVALID_ARG;
     if (int rc = spm_cache_reset(c)) return rc;
     const spm_model_cfg& m = c->cfg;
-    const int K = std::min(m.top_k, c->S);
     const int pools = std::min(m.n_layers, 4);
     cudaEvent_t e0, e1;
     CU(c, cudaEventCreate(&e0));
@@ -1040,37 +1100,35 @@ int spm_profile_window(spm_ctx* c, double* window_us, double* t_xfer_us, int* bu
     for (int it = 0; it < 11; ++it) {
         const int layer = it % pools, e = it % m.n_experts;
         CU(c, cudaEventRecord(e0, c->copy));
-        CU(c, cudaMemcpyAsync(slot_ptr(c, layer, it % K), host_blob(c, layer, e), c->blob, cudaMemcpyHostToDevice, c->copy));
+        CU(c, cudaMemcpyAsync(slot_ptr(c, layer, it % c->S), host_blob(c, layer, e), c->blob, cudaMemcpyHostToDevice, c->copy));
         CU(c, cudaEventRecord(e1, c->copy));
         CU(c, cudaEventSynchronize(e1));
         float ms = 0;
         CU(c, cudaEventElapsedTime(&ms, e0, e1));
         if (it >= 2) tx.push_back(ms * 1e3f);
     }
-    // make the first K slots of a few pools valid experts, then time the FFN over them,
-    // cycling through the pools so that the weights come from HBM, not from L2
-    for (int layer = 0; layer < pools; ++layer)
-        for (int s = 0; s < K; ++s)
-            CU(c, cudaMemcpyAsync(slot_ptr(c, layer, s), host_blob(c, layer, s % m.n_experts), c->blob, cudaMemcpyHostToDevice, c->copy));
-    CU(c, cudaStreamSynchronize(c->copy));
-    std::vector<float> wv(K, 1.0f / K);
-    CU(c, cudaMemcpyAsync(c->ws_w, wv.data(), size_t(K) * 4, cudaMemcpyHostToDevice, c->compute));
-    CU(c, cudaMemsetAsync(c->ws_x, 0, size_t(m.hidden) * 4, c->compute));
+    // Window: the expert FFN of one layer at this context's batch size, through the same path a
+    // decode step takes (slot table, kernel choice, combine), with every needed expert resident.
+    // The pools of a few layers are cycled so that the weights come from HBM, not from L2.
+    const int R = std::min(c->S, m.n_experts);
+    const int nb = m.max_batch;
+    {
+        std::vector<int32_t> all(R);
+        for (int e = 0; e < R; ++e) all[e] = e;
+        for (int layer = 0; layer < pools; ++layer)
+            if (int rc = do_prefetch(c, layer, all.data(), R, nullptr, 0, nullptr)) return rc;
+        CU(c, cudaStreamSynchronize(c->copy));
+    }
+    std::vector<int32_t> pids(size_t(nb) * m.top_k);
+    for (size_t i = 0; i < pids.size(); ++i) pids[i] = int32_t(i % size_t(R));
+    std::vector<float> wv(size_t(nb) * m.top_k, 1.0f / m.top_k);
+    CU(c, cudaMemcpyAsync(c->ws_w, wv.data(), wv.size() * 4, cudaMemcpyHostToDevice, c->compute));
+    CU(c, cudaMemsetAsync(c->ws_x, 0, size_t(nb) * m.hidden * 4, c->compute));
+    CU(c, cudaMemsetAsync(c->ws_h, 0, size_t(nb) * m.hidden * 4, c->compute));
     std::vector<float> wt;
-    const int G = ffn_grid_for(c, 1);
     for (int it = 0; it < 14; ++it) {
-        const int layer = it % pools;
-        FfnArgs<1> a{};
-        a.pool = slot_ptr(c, layer, 0);
-        a.shared = m.n_shared ? static_cast<const unsigned char*>(c->buf.shared_experts) + size_t(layer) * m.n_shared * c->blob : nullptr;
-        a.x = c->ws_x; a.w = c->ws_w; a.partial = c->ws_partial; a.status = c->ws_status;
-        a.blob_bytes = c->blob; a.I = m.inter; a.K = m.top_k; a.n_slots = c->S; a.n_shared = m.n_shared;
-        int cnt = 0;
-        for (int k = 0; k < K; ++k) { a.code[cnt] = short(k); a.kidx[cnt] = (unsigned char)k; ++cnt; }
-        for (int s = 0; s < m.n_shared; ++s) { a.code[cnt] = short(-1 - s); a.kidx[cnt] = 255; ++cnt; }
-        a.count[0] = (unsigned char)cnt;
         CU(c, cudaEventRecord(e0, c->compute));
-        CU(c, launch_gemv<1>(c, a, G, 1));
+        if (int rc = run_ffn(c, it % pools, c->ws_x, pids.data(), c->ws_w, nb, c->ws_h, nullptr)) return rc;
         CU(c, cudaEventRecord(e1, c->compute));
         CU(c, cudaEventSynchronize(e1));
         float ms = 0;
@@ -1082,7 +1140,7 @@ int spm_profile_window(spm_ctx* c, double* window_us, double* t_xfer_us, int* bu
     std::sort(tx.begin(), tx.end());
     std::sort(wt.begin(), wt.end());
     *t_xfer_us = tx[tx.size() / 2];
-    *window_us = wt[wt.size() / 2];
+    *window_us = wt[wt.size() / 2] + c->stub_us;
     *budget_raw = int(*window_us / *t_xfer_us);
     if (int rc = check_status(c)) return rc;
     return spm_cache_reset(c);

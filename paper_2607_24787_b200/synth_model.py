@@ -24,13 +24,23 @@ def fill_store(cfg: synth.ModelCfg, store: PinnedStore, device, chunk: int = 32)
 
 
 def build_from_synth(cfg: synth.ModelCfg, slots=None, budget=None, max_batch=None, device="cuda:0",
-                     store: PinnedStore | None = None) -> OffloadedMoE:
-    """Random-init model of the configuration's shape, experts offloaded to pinned host memory."""
+                     store: PinnedStore | None = None, adapter: str = "random") -> OffloadedMoE:
+    """Random-init model of the configuration's shape, experts offloaded to pinned host memory.
+
+    adapter="random": the configuration's N(0, 0.02) rank-r adapters. adapter="gate_reuse": a
+    training-free stand-in for trained adapters, A^l = W_r^{l+1} and Bup = identity (rank n), i.e.
+    the next layer's own gate applied to this layer's router input (data only: same kernels).
+    """
     dev = torch.device(device)
     L = cfg.n_layers
     gamma = torch.ones(L, cfg.hidden, dtype=torch.float32, device=dev)
     router = torch.stack([synth.router_w(cfg, l, dev) for l in range(L)]).contiguous()
-    if L > 1:
+    rank = cfg.adapter_rank
+    if adapter == "gate_reuse" and L > 1:
+        rank = cfg.n_experts
+        a = router[1:].clone().contiguous()
+        b = torch.eye(cfg.n_experts, dtype=router.dtype, device=dev).expand(L - 1, -1, -1).contiguous()
+    elif L > 1:
         a = torch.stack([synth.adapter_a(cfg, l, dev) for l in range(L - 1)]).contiguous()
         b = torch.stack([synth.adapter_b(cfg, l, dev) for l in range(L - 1)]).contiguous()
     else:
@@ -46,7 +56,7 @@ def build_from_synth(cfg: synth.ModelCfg, slots=None, budget=None, max_batch=Non
         store = PinnedStore(L * cfg.n_experts * cfg.expert_bytes)
         fill_store(cfg, store, dev)
     return OffloadedMoE(n_layers=L, hidden=cfg.hidden, n_experts=cfg.n_experts, inter=cfg.inter,
-                        top_k=cfg.top_k, n_shared=cfg.n_shared, adapter_rank=cfg.adapter_rank,
+                        top_k=cfg.top_k, n_shared=cfg.n_shared, adapter_rank=rank,
                         dtype=cfg.dtype, renormalize=cfg.renormalize, rms_eps=cfg.rms_eps,
                         max_batch=cfg.batch if max_batch is None else max_batch,
                         slots=cfg.slots if slots is None else slots,

@@ -169,7 +169,7 @@ def fragile(recs, K, budget):
     return flags
 
 
-@pytest.mark.parametrize("policy", ["adapter", "on_demand", "pred0", "hint_trace"])
+@pytest.mark.parametrize("policy", ["adapter", "on_demand", "pred0", "hint_trace", "naive"])
 def test_decode_step_free_running(setup, policy):
     cfg, m, wts, H = setup
     steps = 24 if cfg.n_experts * cfg.inter * cfg.hidden < 3e6 else 8

@@ -31,13 +31,26 @@ def test_router_preserving_guarantee(tiny):
     hint = ref_decode.true_demand_trace(base_recs)
     arms = [dict(policy=P.ON_DEMAND), dict(policy=P.ADAPTER), dict(policy=P.ADAPTER, budget=4, slots=6),
             dict(policy=P.PRED0), dict(policy=P.HINT_TRACE, hint=hint), dict(policy=P.ADAPTER, plain_lru=True),
-            dict(policy=P.ADAPTER, slots=2, budget=1)]
+            dict(policy=P.ADAPTER, slots=2, budget=1), dict(policy=P.NAIVE, budget=2)]
     for kw in arms:
         _, out, recs = run(cfg, wts, H, **kw)
         assert np.array_equal(out, base), kw                       # bitwise: outputs never depend on the policy
         for a, b in zip(recs, base_recs):
             for ra, rb in zip(a, b):
                 assert np.array_equal(ra.ids, rb.ids) and np.array_equal(ra.w, rb.w)
+
+
+def test_naive_prefetch_replays_the_preceding_token(tiny):
+    cfg, wts, H = tiny
+    assert P.borda_ranking([[5, 2, 9]], 12) == [5, 2, 9]                   # one token: router rank order
+    assert P.borda_ranking([[5, 2], [2, 7]], 12) == [2, 5, 7]              # 2: 1+2, 5: 2, 7: 1
+    assert P.borda_ranking([[1, 0], [0, 1]], 4) == [0, 1]                  # tie -> lower id
+    ref, _, recs = run(cfg, wts, H, policy=P.NAIVE, budget=2, slots=3)
+    ev = ref.table.events
+    assert not [e for e in ev if e[0] == 0 and e[2] == "PREFETCH"]          # no preceding token at step 0
+    for (s, l, kind, e, slot) in ev:
+        if kind == "PREFETCH":
+            assert e in [int(x) for x in recs[s - 1][l].ids[0]]             # only experts the preceding token used there
 
 
 def test_dropped_prefetch_requests_fall_back_to_demand(tiny):
