@@ -183,6 +183,7 @@ def arm_summary(m, cfg, elapsed_ms, steps):
     return {
         "tok_s": steps * cfg.batch / (elapsed_ms / 1e3),
         "stall_us_per_layer": float(stall.sum() / per),
+        "router_done_to_ffn_done_us_per_layer": float((stall.sum() + ffn.sum()) / per),
         "ffn_us_per_launch": st["ffn_us"] / max(st["ffn_launches"], 1),
         "hit_rate": st["hits"] / max(st["hits"] + st["misses"], 1),
         "ready_recall": st["ready_sum"] / max(st["ready_count"], 1),
@@ -305,6 +306,18 @@ def run_ours(args):
         timed_run(m, H_dev, 0, W, world); m.reset_stats()
         el, _, _ = timed_run(m, H_dev, W, n_arm, world)
         arms["perfect_knowledge"] = arm_summary(m, cfg, el, n_arm)
+        # on-demand and perfect knowledge again, with the FFN waiting for its copies on the device
+        if cfg.batch == 1:
+            m.set_device_wait(1)
+            m.set_policy("on_demand"); m.cache_reset()
+            timed_run(m, H_dev, 0, W, world); m.reset_stats()
+            el, _, _ = timed_run(m, H_dev, W, n_arm, world)
+            arms["on_demand_device_wait"] = arm_summary(m, cfg, el, n_arm)
+            m.set_policy("hint_trace"); m.set_hint_trace(hint); m.cache_reset()
+            timed_run(m, H_dev, 0, W, world); m.reset_stats()
+            el, _, _ = timed_run(m, H_dev, W, n_arm, world)
+            arms["perfect_knowledge_device_wait"] = arm_summary(m, cfg, el, n_arm)
+            m.set_device_wait(0)
         # previous token's experts as the prediction (Naive Prefetch)
         m.set_policy("naive"); m.cache_reset()
         timed_run(m, H_dev, 0, W, world); m.reset_stats()

@@ -220,6 +220,13 @@ int spm_set_hint_trace(spm_ctx* ctx, const int32_t* hint, const int32_t* count,
 /* Fault injection on the host: every prefetch request with (step + expert) % modulo == 0 is
  * lost before it reaches the GPU (0 switches it off). The demand path must then load it. */
 int spm_set_drop_modulo(spm_ctx* ctx, int modulo);
+/* Device-side wait for batch-1 expert FFNs (default off). Off: the compute stream waits on the
+ * copy events of the slots a launch reads, then the kernel starts. On: the kernel is launched at
+ * once and each of its CTAs waits (bounded, SPM_ERR_TIMEOUT on expiry) on a per-slot arrival counter
+ * that the copy stream bumps after the expert's bytes have landed, so resident experts are computed
+ * while missing ones are still in flight and no launch latency follows the last copy. Outputs are
+ * bit-identical either way. With it on, the timed FFN duration includes the wait for copies. */
+int spm_set_device_wait(spm_ctx* ctx, int on);
 /* Stand-in for the attention block the synthetic configurations omit: before each layer's router a
  * kernel that only waits `us` microseconds (0 = off, at most 100000) is enqueued on the compute
  * stream. It widens the overlap window W_l = t_exec(l+1) - t_pred(l) (Section 3.1) toward the

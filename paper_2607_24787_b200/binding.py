@@ -83,6 +83,7 @@ _SIG = {
     "spm_set_drop_modulo": [_P, C.c_int],
     "spm_set_deadline_ms": [_P, C.c_int],
     "spm_set_attention_stub_us": [_P, C.c_int],
+    "spm_set_device_wait": [_P, C.c_int],
     "spm_profile_window": [_P, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int)],
     "spm_cache_reset": [_P],
     "spm_reset_stats": [_P],
@@ -261,6 +262,10 @@ def spm_set_hint_trace(ctx, hint):
 
 def spm_set_drop_modulo(ctx, modulo):
     _check(load().spm_set_drop_modulo(ctx, modulo), ctx)
+
+
+def spm_set_device_wait(ctx, on):
+    _check(load().spm_set_device_wait(ctx, int(on)), ctx)
 
 
 def spm_set_attention_stub_us(ctx, us):

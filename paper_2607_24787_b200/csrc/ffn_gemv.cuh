@@ -40,6 +40,8 @@ struct FfnArgs {
     float* partial;                 // [nb][gridDim.x][D]
     int* status;
     unsigned long long* clock;      // optional {earliest CTA start, latest CTA end} in ns (globaltimer)
+    const unsigned* ready;          // optional per-slot arrival counters of this pool (device-side wait)
+    unsigned want[SPM_MAX_TOPK];    // token 0 only: counter value at which entry k's slot holds its expert
     unsigned long long blob_bytes;
     int I, K, n_slots, n_shared;
     unsigned char count[MAXNB];                     // expert entries of token t in this launch
@@ -84,6 +86,7 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
 
     const uint64_t pol = policy_evict_first();
     bool ok = true;
+    unsigned arrived = 0;     // lane 0: entries whose slot is known to hold its expert
 
     auto issue = [&](int i) {
         const int r = r_begin + wi + i * nw;
@@ -93,6 +96,22 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
         const unsigned char* base;
         if (code >= 0) {
             if (code >= a.n_slots) { atomicOr(a.status, kStatusBadSlot); return false; }
+            if (a.ready && !((arrived >> ent) & 1u)) {
+                // Device-side wait: the copy stream bumps the slot's counter after the expert's bytes
+                // have landed. Bounded; on timeout the status word is set and the launch winds down.
+                const unsigned* f = a.ready + code;
+                const unsigned want = a.want[ent];
+                const unsigned long long t0 = global_timer_ns();
+                for (;;) {
+                    unsigned v;
+                    asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(f) : "memory");
+                    if (int(v - want) >= 0) break;
+                    __nanosleep(200);
+                    if (global_timer_ns() - t0 > kWaitLimitNs) { atomicOr(a.status, kStatusCopyTimeout); return false; }
+                }
+                asm volatile("fence.proxy.async;" ::: "memory");   // the weights are read through the async proxy
+                arrived |= 1u << ent;
+            }
             base = a.pool + size_t(code) * a.blob_bytes;
         } else {
             if (-1 - code >= a.n_shared) { atomicOr(a.status, kStatusBadSlot); return false; }

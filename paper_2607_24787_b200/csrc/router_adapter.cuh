@@ -44,13 +44,12 @@ struct RouterArgs {
     float* x_norm;           // out [nb][D]
     float* logits;           // workspace [nb][n]
     float* logits_out;       // optional copy for the caller
-    float* u;                // workspace [nb][r]
     float* pihat;            // workspace [nb][n]
     int32_t* ids;            // out [nb][K]
     float* w;                // out [nb][K]
     float* scores;           // out [n]
     int32_t* order;          // out [n]
-    unsigned* counters;      // [1 + nb], zero between launches
+    unsigned* counters;      // [1] token-leader ticket, zero between launches
     Mailbox* mailbox;        // device view of the host-mapped mailbox
     uint32_t seq;
     int D, n, K, r, nb, renorm, do_router, do_adapter;

@@ -47,7 +47,7 @@ struct spm_ctx {
     int nseg = 0, depth = 2, num_sms = 148, ffn_ctas = 0;
     // arena carve-up
     unsigned char* pools = nullptr;
-    float *ws_x = nullptr, *ws_logits = nullptr, *ws_u = nullptr, *ws_pihat = nullptr, *ws_w = nullptr;
+    float *ws_x = nullptr, *ws_logits = nullptr, *ws_pihat = nullptr, *ws_w = nullptr;
     float *ws_scores = nullptr, *ws_partial = nullptr, *ws_h = nullptr;
     int32_t *ws_ids = nullptr, *ws_order = nullptr;
     unsigned* ws_counters = nullptr;
@@ -96,6 +96,9 @@ struct spm_ctx {
     int hint_steps = 0, hint_stride = 0;
     int drop_modulo = 0;
     int stub_us = 0;                          // attention stand-in before each layer's router
+    bool device_wait = false;                 // batch-1 FFN launched at once, waits for its copies on the device
+    unsigned* ws_slot_gen = nullptr;          // [L][S] arrival counters, bumped by the copy stream
+    std::vector<uint32_t> slot_gen_host;      // value the counter will hold once the latest copy has landed
     std::vector<std::vector<int32_t>> prev_rank;   // Naive Prefetch: experts the preceding step used, per layer
     std::vector<std::vector<int32_t>> pending_protect;
     std::vector<uint8_t> has_plan;
@@ -175,7 +178,7 @@ struct Carve {
 };
 
 struct Layout {
-    size_t pools, x, logits, u, pihat, w, scores, partial, h, ids, order, clock, counters, status, total;
+    size_t pools, slot_gen, x, logits, pihat, w, scores, partial, h, ids, order, clock, counters, status, total;
     size_t tc_xs, tc_wrow, tc_partial, tc_desc;       // batched tensor-core path only
     size_t desc_bytes, off_rows, off_rowmap;
     int rows_cap, n_jt, max_units;
@@ -187,9 +190,9 @@ Layout layout_of(const spm_model_cfg* m, int S) {
     Carve c;
     const size_t nb = m->max_batch, D = m->hidden, n = m->n_experts;
     l.pools = c.take(size_t(m->n_layers) * S * blob_bytes_of(m));
+    l.slot_gen = c.take(size_t(m->n_layers) * S * 4);
     l.x = c.take(nb * D * 4);
     l.logits = c.take(nb * n * 4);
-    l.u = c.take(nb * m->adapter_rank * 4);
     l.pihat = c.take(nb * n * 4);
     l.w = c.take(nb * SPM_MAX_TOPK * 4);
     l.scores = c.take(n * 4);
@@ -211,7 +214,7 @@ Layout layout_of(const spm_model_cfg* m, int S) {
         l.tc_partial = c.take(size_t(l.n_jt) * l.rows_cap * D * 4);
         l.tc_desc = c.take(size_t(kDescRing) * l.desc_bytes);
     }
-    l.counters = c.take((nb + 1) * 4);
+    l.counters = c.take(256);
     l.status = c.take(4);
     l.total = c.off;
     return l;
@@ -274,7 +277,6 @@ int launch_router(spm_ctx* c, int layer, const float* h, const float* x_in, int 
     a.x_norm = x_norm;
     a.logits = c->ws_logits;
     a.logits_out = logits_out;
-    a.u = c->ws_u;
     a.pihat = c->ws_pihat;
     a.ids = c->ws_ids;
     a.w = c->ws_w;
@@ -368,6 +370,14 @@ int issue_copy(spm_ctx* c, int layer, int e, int slot) {
     const size_t k = size_t(layer) * c->S + slot;
     CU(c, cudaMemcpyAsync(slot_ptr(c, layer, slot), host_blob(c, layer, e), c->blob, cudaMemcpyHostToDevice, c->copy));
     CU(c, cudaEventRecord(c->slot_ev[k], c->copy));
+    // stream-ordered counter bump, for launches that wait for their copies on the device
+    if (StreamWriteValue32Fn wr = stream_write32_fn()) {
+        const uint32_t gen = ++c->slot_gen_host[k];
+        if (wr(reinterpret_cast<CUstream>(c->copy), reinterpret_cast<CUdeviceptr>(c->ws_slot_gen + k), gen, 0) != CUDA_SUCCESS)
+            return fail(c, SPM_ERR_CUDA, "cuStreamWriteValue32 failed");
+    } else if (c->device_wait) {
+        return fail(c, SPM_ERR_CUDA, "cuStreamWriteValue32 is not available");
+    }
     c->slot_pending[k] = 1;
     c->h2d_bytes += c->blob;
     return SPM_OK;
@@ -502,6 +512,7 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
     tb.demand(layer, c->need.data(), int(c->need.size()), c->placements, &n_waves);
 
     const int G = ffn_grid_for(c, nb);
+    const bool dev_wait = c->device_wait && nb == 1 && stream_write32_fn() != nullptr;
     std::vector<int16_t>& slot_of_expert = c->wave_slot;   // experts computed in the current wave
     for (int wave = 0; wave < n_waves; ++wave) {
         slot_of_expert.assign(m.n_experts, -1);
@@ -527,6 +538,7 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
             cudaError_t q = cudaEventQuery(c->slot_ev[k]);
             if (q == cudaErrorNotReady) {
                 if (!p.missed) c->extra_late++;
+                if (dev_wait) continue;      // the kernel itself waits for this slot; it stays pending for later launches
                 CU(c, cudaStreamWaitEvent(c->compute, c->slot_ev[k], 0));
             } else if (q != cudaSuccess) {
                 return fail(c, SPM_ERR_CUDA, "copy event query: %s", cudaGetErrorString(q));
@@ -548,6 +560,7 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
             a.partial = c->ws_partial;
             a.status = c->ws_status;
             a.clock = clock_slot;
+            a.ready = dev_wait ? c->ws_slot_gen + size_t(layer) * c->S : nullptr;
             a.blob_bytes = c->blob;
             a.I = m.inter; a.K = K; a.n_slots = c->S; a.n_shared = m.n_shared;
             for (int tk = 0; tk < nb; ++tk) {
@@ -557,6 +570,7 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
                     if (s < 0) continue;
                     a.code[tk * SPM_MAX_TOPK + cnt] = short(s);
                     a.kidx[tk * SPM_MAX_TOPK + cnt] = (unsigned char)k;
+                    if (dev_wait) a.want[cnt] = c->slot_gen_host[size_t(layer) * c->S + s];
                     ++cnt;
                 }
                 if (first)
@@ -710,9 +724,9 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
 
     unsigned char* base = static_cast<unsigned char*>(b->arena);
     c->pools = base + lay.pools;
+    c->ws_slot_gen = reinterpret_cast<unsigned*>(base + lay.slot_gen);
     c->ws_x = reinterpret_cast<float*>(base + lay.x);
     c->ws_logits = reinterpret_cast<float*>(base + lay.logits);
-    c->ws_u = reinterpret_cast<float*>(base + lay.u);
     c->ws_pihat = reinterpret_cast<float*>(base + lay.pihat);
     c->ws_w = reinterpret_cast<float*>(base + lay.w);
     c->ws_scores = reinterpret_cast<float*>(base + lay.scores);
@@ -732,6 +746,7 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
     c->layer_stall_us.assign(L, 0.0);
     c->layer_ffn_us.assign(L, 0.0);
     c->slot_pending.assign(size_t(L) * c->S, 0);
+    c->slot_gen_host.assign(size_t(L) * c->S, 0);
     c->pool_free_valid.assign(L, 0);
 
     auto cu = [&](cudaError_t err, const char* what) {
@@ -740,6 +755,7 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
         return false;
     };
     if (!cu(cudaMemsetAsync(base + lay.counters, 0, lay.total - lay.counters, c->compute), "cudaMemsetAsync")) return bail(SPM_ERR_CUDA);
+    if (!cu(cudaMemsetAsync(c->ws_slot_gen, 0, size_t(L) * c->S * 4, c->compute), "cudaMemsetAsync")) return bail(SPM_ERR_CUDA);
     if (!cu(cudaHostAlloc(reinterpret_cast<void**>(&c->mb_host), sizeof(Mailbox), cudaHostAllocMapped), "cudaHostAlloc(mailbox)")) return bail(SPM_ERR_CUDA);
     memset(c->mb_host, 0, sizeof(Mailbox));
     if (!cu(cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->mb_dev), c->mb_host, 0), "cudaHostGetDevicePointer")) return bail(SPM_ERR_CUDA);
@@ -1025,6 +1041,12 @@ int spm_set_hint_trace(spm_ctx* c, const int32_t* hint, const int32_t* count, in
 int spm_set_drop_modulo(spm_ctx* c, int modulo) {
     if (!c || modulo < 0) return SPM_ERR_INVALID_ARG;
     c->drop_modulo = modulo;
+    return SPM_OK;
+}
+int spm_set_device_wait(spm_ctx* c, int on) {
+    if (!c) return SPM_ERR_INVALID_ARG;
+    if (on && !stream_write32_fn()) return fail(c, SPM_ERR_CUDA, "cuStreamWriteValue32 is not available on this driver");
+    c->device_wait = on != 0;
     return SPM_OK;
 }
 int spm_set_attention_stub_us(spm_ctx* c, int us) {

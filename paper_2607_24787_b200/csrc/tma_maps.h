@@ -25,6 +25,22 @@ inline EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
+// cuStreamWriteValue32: a 32-bit store to device memory in stream order (used to publish "this
+// slot's copy has landed" to kernels that wait on the device side).
+typedef CUresult (*StreamWriteValue32Fn)(CUstream, CUdeviceptr, cuuint32_t, unsigned int);
+
+inline StreamWriteValue32Fn stream_write32_fn() {
+    static StreamWriteValue32Fn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuStreamWriteValue32", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<StreamWriteValue32Fn>(p);
+    }
+    return fn;
+}
+
 // Packed bf16 expert blobs [n_slots][I][3][D] viewed as a 4-D tensor (D, 3, I, n_slots); a box is
 // 64 consecutive elements of D x 128 consecutive rows of one plane of one slot, 128-byte swizzle.
 inline bool make_weight_map(CUtensorMap* map, const void* base, int D, int I, uint64_t n_slots) {

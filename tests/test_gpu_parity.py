@@ -228,6 +228,22 @@ def test_router_preserving_bitwise_on_gpu(setup):
     full.close()
 
 
+def test_device_side_wait_is_bit_identical(setup):
+    """The batch-1 FFN can wait for its copies on the device instead of on stream events: same
+    outputs, same cache events, and the oracle still agrees."""
+    cfg, m, wts, H = setup
+    steps = 8
+    runs = {}
+    for on in (0, 1):
+        m.cache_reset(); m.set_policy("adapter"); m.set_budget(2); m.set_device_wait(on)
+        runs[on] = (run_gpu(m, H, steps), m.events())
+    m.set_device_wait(0)
+    assert np.array_equal(runs[0][0], runs[1][0]) and runs[0][1] == runs[1][1]
+    ref, out_r, _ = run_ref(cfg, wts, H, steps, policy=P.ADAPTER, budget=2)
+    for s in range(steps):
+        assert M.rel_linf(runs[1][0][s], out_r[s]) < 4 * TOL[cfg.dtype]
+
+
 def test_decode_step_host_matches_device(setup):
     cfg, m, wts, H = setup
     m.cache_reset(); m.set_policy("adapter"); m.set_budget(2)
