@@ -213,6 +213,8 @@ def run_ours(args):
     setup_s = time.time() - t_setup
     if args.stub_us:
         m.set_attention_stub_us(args.stub_us)
+    if args.copy_delay_us:
+        m.set_copy_delay_us(args.copy_delay_us)
     window_us, t_xfer_us, raw_budget = m.profile_window()
     budget = max(1, raw_budget) if cfg.budget < 0 else cfg.budget
     m.set_budget(budget)
@@ -259,7 +261,7 @@ def run_ours(args):
         "config": {"workload": f"{cfg.name}: L{cfg.n_layers} D{cfg.hidden} n{cfg.n_experts} I{cfg.inter} K{cfg.top_k}"
                                f"+{cfg.n_shared}sh r{cfg.adapter_rank} {cfg.dtype} slots{cfg.slots} batch{cfg.batch}",
                    "policy": "adapter", "budget": budget, "budget_raw": raw_budget, "window_us": window_us,
-                   "t_xfer_us": t_xfer_us, "attention_stub_us": args.stub_us, "seed": cfg.seed, "token_ids": "Zipf(1.1)",
+                   "t_xfer_us": t_xfer_us, "attention_stub_us": args.stub_us, "copy_delay_us": args.copy_delay_us, "seed": cfg.seed, "token_ids": "Zipf(1.1)",
                    "l2": "inputs larger than L2: every layer streams its own slot pool, 3.6 GB of weights per step",
                    "setup_s": setup_s, "wall_ms_per_step": wall_ms / K},
         "clocks": clk,
@@ -478,6 +480,8 @@ def run_sweep(args):
             m.set_timing(1)
             if args.stub_us:
                 m.set_attention_stub_us(args.stub_us)
+            if args.copy_delay_us:
+                m.set_copy_delay_us(args.copy_delay_us)
             if adapter == "random":
                 window = m.profile_window()
 
@@ -635,6 +639,8 @@ def main():
     ap.add_argument("--sweep-slots", default="8,16,32")
     ap.add_argument("--stub-us", type=int, default=0,
                     help="attention stand-in of this many microseconds before each layer's router (widens the overlap window)")
+    ap.add_argument("--copy-delay-us", type=int, default=0,
+                    help="emulated slower storage tier: extra wait after every expert copy")
     ap.add_argument("--no-arms", action="store_true")
     ap.add_argument("--no-resident", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -220,6 +220,10 @@ int spm_set_hint_trace(spm_ctx* ctx, const int32_t* hint, const int32_t* count,
 /* Fault injection on the host: every prefetch request with (step + expert) % modulo == 0 is
  * lost before it reaches the GPU (0 switches it off). The demand path must then load it. */
 int spm_set_drop_modulo(spm_ctx* ctx, int modulo);
+/* Emulated slower storage tier (the paper's controlled loading delays, Section 4.1): every expert
+ * copy is followed on the copy stream by a wait of `us` microseconds (0 = off, at most 100000)
+ * before the slot counts as loaded. Outputs are unchanged. */
+int spm_set_copy_delay_us(spm_ctx* ctx, int us);
 /* Device-side wait for batch-1 expert FFNs (default off). Off: the compute stream waits on the
  * copy events of the slots a launch reads, then the kernel starts. On: the kernel is launched at
  * once and each of its CTAs waits (bounded, SPM_ERR_TIMEOUT on expiry) on a per-slot arrival counter

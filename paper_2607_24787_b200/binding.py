@@ -84,6 +84,7 @@ _SIG = {
     "spm_set_deadline_ms": [_P, C.c_int],
     "spm_set_attention_stub_us": [_P, C.c_int],
     "spm_set_device_wait": [_P, C.c_int],
+    "spm_set_copy_delay_us": [_P, C.c_int],
     "spm_profile_window": [_P, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int)],
     "spm_cache_reset": [_P],
     "spm_reset_stats": [_P],
@@ -262,6 +263,10 @@ def spm_set_hint_trace(ctx, hint):
 
 def spm_set_drop_modulo(ctx, modulo):
     _check(load().spm_set_drop_modulo(ctx, modulo), ctx)
+
+
+def spm_set_copy_delay_us(ctx, us):
+    _check(load().spm_set_copy_delay_us(ctx, us), ctx)
 
 
 def spm_set_device_wait(ctx, on):

@@ -96,6 +96,7 @@ struct spm_ctx {
     int hint_steps = 0, hint_stride = 0;
     int drop_modulo = 0;
     int stub_us = 0;                          // attention stand-in before each layer's router
+    int copy_delay_us = 0;                    // emulated slower storage tier: extra wait after every expert copy
     bool device_wait = false;                 // batch-1 FFN launched at once, waits for its copies on the device
     unsigned* ws_slot_gen = nullptr;          // [L][S] arrival counters, bumped by the copy stream
     std::vector<uint32_t> slot_gen_host;      // value the counter will hold once the latest copy has landed
@@ -223,12 +224,14 @@ Layout layout_of(const spm_model_cfg* m, int S) {
 // ---- kernel dispatch -------------------------------------------------------
 template <typename WT, int NSEG, int MAXNB>
 cudaError_t launch_gemv_t(const FfnArgs<MAXNB>& a, int G, int nb, int warps, int depth, size_t smem, cudaStream_t st) {
-    static bool attr_set = false;
+    static bool attr_set[64] = {};          // the attribute is per device
     auto kern = ffn_gemv_kernel<WT, NSEG, MAXNB>;
-    if (!attr_set) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kFfnSmemLimit));
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     kern<<<dim3(G, nb), warps * 32, smem, st>>>(a, depth);
     return cudaGetLastError();
@@ -358,6 +361,13 @@ int wait_tagged(spm_ctx* c, const volatile int32_t* words, int count, int32_t* o
     return SPM_OK;
 }
 
+// A kernel that only waits: one thread watches %globaltimer until `ns` have passed. Used as the
+// stand-in for the omitted attention block and as the extra delay of an emulated slower storage tier.
+__global__ void attention_stub_kernel(unsigned long long ns) {
+    const unsigned long long t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < ns) __nanosleep(200);
+}
+
 unsigned char* slot_ptr(spm_ctx* c, int layer, int slot) {
     return c->pools + (size_t(layer) * c->S + slot) * c->blob;
 }
@@ -369,6 +379,10 @@ const unsigned char* host_blob(spm_ctx* c, int layer, int e) {
 int issue_copy(spm_ctx* c, int layer, int e, int slot) {
     const size_t k = size_t(layer) * c->S + slot;
     CU(c, cudaMemcpyAsync(slot_ptr(c, layer, slot), host_blob(c, layer, e), c->blob, cudaMemcpyHostToDevice, c->copy));
+    if (c->copy_delay_us > 0) {
+        attention_stub_kernel<<<1, 1, 0, c->copy>>>(uint64_t(c->copy_delay_us) * 1000ull);   // emulated slower tier
+        CU(c, cudaGetLastError());
+    }
     CU(c, cudaEventRecord(c->slot_ev[k], c->copy));
     // stream-ordered counter bump, for launches that wait for their copies on the device
     if (StreamWriteValue32Fn wr = stream_write32_fn()) {
@@ -626,12 +640,6 @@ int do_prefetch(spm_ctx* c, int target, const int32_t* ids, int count, const int
     }
     if (out_issued) *out_issued = issued;
     return SPM_OK;
-}
-
-// Stand-in for the omitted attention block: one thread watches %globaltimer until `ns` have passed.
-__global__ void attention_stub_kernel(unsigned long long ns) {
-    const unsigned long long t0 = global_timer_ns();
-    while (global_timer_ns() - t0 < ns) __nanosleep(200);
 }
 
 // Experts of this step's routing at one layer, ranked by sum over tokens of (K - rank position).
@@ -1043,6 +1051,11 @@ int spm_set_drop_modulo(spm_ctx* c, int modulo) {
     c->drop_modulo = modulo;
     return SPM_OK;
 }
+int spm_set_copy_delay_us(spm_ctx* c, int us) {
+    if (!c || us < 0 || us > 100000) return SPM_ERR_INVALID_ARG;
+    c->copy_delay_us = us;
+    return SPM_OK;
+}
 int spm_set_device_wait(spm_ctx* c, int on) {
     if (!c) return SPM_ERR_INVALID_ARG;
     if (on && !stream_write32_fn()) return fail(c, SPM_ERR_CUDA, "cuStreamWriteValue32 is not available on this driver");
@@ -1123,6 +1136,7 @@ int spm_profile_window(spm_ctx* c, double* window_us, double* t_xfer_us, int* bu
         const int layer = it % pools, e = it % m.n_experts;
         CU(c, cudaEventRecord(e0, c->copy));
         CU(c, cudaMemcpyAsync(slot_ptr(c, layer, it % c->S), host_blob(c, layer, e), c->blob, cudaMemcpyHostToDevice, c->copy));
+        if (c->copy_delay_us > 0) attention_stub_kernel<<<1, 1, 0, c->copy>>>(uint64_t(c->copy_delay_us) * 1000ull);
         CU(c, cudaEventRecord(e1, c->copy));
         CU(c, cudaEventSynchronize(e1));
         float ms = 0;

@@ -81,6 +81,26 @@ def test_full_batch_fp32():
     compare_run(synth.get_config("tiny", batch=64, slots=16, budget=2), steps=2)
 
 
+def test_timing_knobs_do_not_change_results():
+    """Attention stand-in and emulated storage delay only move time around."""
+    cfg = synth.get_config("tiny")
+    m = build(cfg)
+    tok = synth.zipf_tokens(cfg, steps=4)
+    H = synth.embedding_rows(cfg, tok[:, 0]).numpy()
+    outs = []
+    for stub, delay in ((0, 0), (200, 150)):
+        m.cache_reset(); m.set_attention_stub_us(stub); m.set_copy_delay_us(delay)
+        w = m.profile_window()
+        run = []
+        for s in range(4):
+            out = m.decode_step(dev(H[s:s + 1])); m.synchronize()
+            run.append(out.cpu().numpy())
+        outs.append((np.stack(run), m.events(), w))
+    assert np.array_equal(outs[0][0], outs[1][0]) and outs[0][1] == outs[1][1]
+    assert outs[1][2][0] > outs[0][2][0] + 150 and outs[1][2][1] > outs[0][2][1] + 100    # window and t_xfer grew
+    m.close()
+
+
 def test_host_deadline_returns_timeout_and_context_survives():
     """The routing handshake has a host-side deadline: with the compute stream kept busy by unrelated
     work the call gives up with SPM_ERR_TIMEOUT instead of spinning; nothing on the GPU is disturbed."""
