@@ -54,6 +54,8 @@ extern "C" {
 
 #define SPM_DTYPE_FP32 0
 #define SPM_DTYPE_BF16 1
+#define SPM_DTYPE_Q4   2   /* experts 4-bit (groups of 32 weights + one fp16 scale, value = scale * (q - 8)):
+                              the paper's on-device precision; router, adapter matrices stay bf16 */
 
 /* prefetch policies */
 #define SPM_POLICY_ADAPTER    0   /* rank next-layer experts with the low-rank adapter (the method)    */
@@ -136,7 +138,9 @@ typedef struct {
  *     blob[j][0][0..D) = W_gate[j][:]      j = 0..I-1
  *     blob[j][1][0..D) = W_up[j][:]
  *     blob[j][2][0..D) = W_down[:][j]      (column j of W_down[D][I])
- * Writes 3*I*D*sizeof(element) to *bytes.                                               */
+ * With SPM_DTYPE_Q4 each of these rows is packed as D/2 bytes of nibbles (element 2b in the low
+ * half of byte b, 2b+1 in the high half) followed by D/32 fp16 scales, one per 32 consecutive elements.
+ * Writes the blob size to *bytes: 3*I*D*sizeof(element), or 3*I*(D/2 + D/16) for 4-bit experts. */
 int spm_expert_blob_bytes(const spm_model_cfg* cfg, size_t* bytes);
 
 /* Bytes of device arena needed for `slots_per_layer` routed slots per layer plus workspace. */
@@ -146,7 +150,7 @@ int spm_query_arena(const spm_model_cfg* cfg, int slots_per_layer, size_t* bytes
  * (spm_profile_window is then run once here: max(1, floor(W / t_xfer)); Section 3.3, first
  * paragraphs). Slot tables start empty (cold cache). Fails with SPM_ERR_CONFIG when
  * max_batch == 1 and slots_per_layer < top_k, or when the shape is not supported by the
- * kernels (hidden must be a multiple of 256 (bf16) / 128 (fp32) and <= 8192). */
+ * kernels (hidden must be a multiple of 256 and <= 2048 (bf16, 4-bit) / of 128 and <= 1024 (fp32)). */
 int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget,
              const spm_buffers* buffers, spm_ctx** out);
 int spm_destroy(spm_ctx* ctx);

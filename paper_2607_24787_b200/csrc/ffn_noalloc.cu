@@ -81,7 +81,8 @@ extern "C" int spm_ffn_noalloc(const spm_model_cfg* cfg, const void* blobs, int 
                                const float* w, int count, const float* x_norm, float* h_inout, void* stream,
                                int wait_and_check) {
     if (!cfg || !blobs || !which || !w || !x_norm || !h_inout) return fail(SPM_ERR_INVALID_ARG, "spm_ffn_noalloc: null argument");
-    if (cfg->dtype != SPM_DTYPE_FP32 && cfg->dtype != SPM_DTYPE_BF16) return fail(SPM_ERR_CONFIG, "spm_ffn_noalloc: unknown dtype");
+    if (cfg->dtype != SPM_DTYPE_FP32 && cfg->dtype != SPM_DTYPE_BF16)
+        return fail(SPM_ERR_CONFIG, "spm_ffn_noalloc: only fp32 and bf16 experts are supported");
     const int seg = cfg->dtype == SPM_DTYPE_BF16 ? 256 : 128;
     if (cfg->hidden < seg || cfg->hidden % seg || cfg->hidden / seg > 8 || cfg->hidden > kNoAllocMaxHidden)
         return fail(SPM_ERR_CONFIG, "spm_ffn_noalloc: hidden " + std::to_string(cfg->hidden) + " not supported: a multiple of " +

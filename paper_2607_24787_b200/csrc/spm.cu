@@ -15,6 +15,7 @@
 
 #include "../../include/spm.h"
 #include "ffn_gemv.cuh"
+#include "ffn_gemv_q4.cuh"
 #include "ffn_grouped.cuh"
 #include "router_adapter.cuh"
 #include "tma_maps.h"
@@ -136,8 +137,9 @@ int fail(spm_ctx* c, int code, const char* fmt, ...) {
 
 int check_cfg(const spm_model_cfg* m, int S, spm_ctx* c) {
     if (!m) return fail(c, SPM_ERR_INVALID_ARG, "cfg is null");
-    if (m->dtype != SPM_DTYPE_FP32 && m->dtype != SPM_DTYPE_BF16) return fail(c, SPM_ERR_CONFIG, "unknown dtype %d", m->dtype);
-    const int seg = m->dtype == SPM_DTYPE_BF16 ? 256 : 128;
+    if (m->dtype != SPM_DTYPE_FP32 && m->dtype != SPM_DTYPE_BF16 && m->dtype != SPM_DTYPE_Q4)
+        return fail(c, SPM_ERR_CONFIG, "unknown dtype %d", m->dtype);
+    const int seg = m->dtype == SPM_DTYPE_FP32 ? 128 : 256;
     if (m->n_layers < 1 || m->hidden < seg || m->hidden % seg || m->hidden / seg > 8)
         return fail(c, SPM_ERR_CONFIG, "hidden %d unsupported: need a multiple of %d, at most %d", m->hidden, seg, 8 * seg);
     if (m->n_experts < 1 || m->n_experts > SPM_MAX_EXPERTS) return fail(c, SPM_ERR_CONFIG, "n_experts %d out of range", m->n_experts);
@@ -153,6 +155,7 @@ int check_cfg(const spm_model_cfg* m, int S, spm_ctx* c) {
 }
 
 size_t blob_bytes_of(const spm_model_cfg* m) {
+    if (m->dtype == SPM_DTYPE_Q4) return size_t(3) * m->inter * (size_t(m->hidden) / 2 + size_t(m->hidden) / 16);
     return size_t(3) * m->inter * m->hidden * (m->dtype == SPM_DTYPE_BF16 ? 2 : 4);
 }
 
@@ -252,12 +255,38 @@ cudaError_t launch_gemv_seg(int nseg, const FfnArgs<MAXNB>& a, int G, int nb, in
     return cudaErrorInvalidValue;
 }
 
+template <int NCH, int MAXNB>
+cudaError_t launch_gemv_q4_t(int D, const FfnArgs<MAXNB>& a, int G, int nb, int warps, int depth, size_t smem, cudaStream_t st) {
+    static bool attr_set[64] = {};
+    auto kern = ffn_gemv_q4_kernel<NCH, MAXNB>;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kFfnSmemLimit));
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    kern<<<dim3(G, nb), warps * 32, smem, st>>>(a, depth, D);
+    return cudaGetLastError();
+}
+
+template <int MAXNB>
+cudaError_t launch_gemv_q4(int D, const FfnArgs<MAXNB>& a, int G, int nb, int warps, int depth, size_t smem, cudaStream_t st) {
+    if (D <= 1024) return launch_gemv_q4_t<1, MAXNB>(D, a, G, nb, warps, depth, smem, st);
+    return launch_gemv_q4_t<2, MAXNB>(D, a, G, nb, warps, depth, smem, st);
+}
+
 template <int MAXNB>
 cudaError_t launch_gemv(const spm_ctx* c, const FfnArgs<MAXNB>& a, int G, int nb) {
     int max_cnt = 1;
     for (int t = 0; t < nb; ++t) max_cnt = std::max(max_cnt, int(a.count[t]));
     const int rows_per_cta = (max_cnt * c->cfg.inter + G - 1) / G;
     int warps = 8, depth = 2;
+    if (c->cfg.dtype == SPM_DTYPE_Q4) {
+        size_t smem = 0;
+        ffn_gemv_q4_shape(c->row_bytes, c->cfg.hidden, rows_per_cta, &warps, &depth, &smem);
+        return launch_gemv_q4<MAXNB>(c->cfg.hidden, a, G, nb, warps, depth, smem, c->compute);
+    }
     ffn_gemv_shape(c->row_bytes, rows_per_cta, &warps, &depth);
     const size_t smem = ffn_gemv_smem(c->row_bytes, warps, depth);
     if (c->cfg.dtype == SPM_DTYPE_BF16) return launch_gemv_seg<bf16_t, MAXNB>(c->nseg, a, G, nb, warps, depth, smem, c->compute);
@@ -304,7 +333,7 @@ int launch_router(spm_ctx* c, int layer, const float* h, const float* x_in, int 
     at[0].val.clusterDim.z = 1;
     lc.attrs = at;
     lc.numAttrs = 1;
-    if (m.dtype == SPM_DTYPE_BF16) {
+    if (m.dtype != SPM_DTYPE_FP32) {
         if (smem > 48 * 1024) CU(c, cudaFuncSetAttribute(router_adapter_kernel<bf16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
         CU(c, cudaLaunchKernelEx(&lc, router_adapter_kernel<bf16_t>, a));
     } else {
@@ -526,7 +555,7 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
     tb.demand(layer, c->need.data(), int(c->need.size()), c->placements, &n_waves);
 
     const int G = ffn_grid_for(c, nb);
-    const bool dev_wait = c->device_wait && nb == 1 && stream_write32_fn() != nullptr;
+    const bool dev_wait = c->device_wait && nb == 1 && m.dtype != SPM_DTYPE_Q4 && stream_write32_fn() != nullptr;
     std::vector<int16_t>& slot_of_expert = c->wave_slot;   // experts computed in the current wave
     for (int wave = 0; wave < n_waves; ++wave) {
         slot_of_expert.assign(m.n_experts, -1);
@@ -717,10 +746,10 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
     c->buf = *b;
     c->compute = static_cast<cudaStream_t>(b->compute_stream);
     c->copy = static_cast<cudaStream_t>(b->copy_stream);
-    c->elem = cfg->dtype == SPM_DTYPE_BF16 ? 2 : 4;
+    c->elem = cfg->dtype == SPM_DTYPE_FP32 ? 4 : 2;       // router / adapter element size
     c->blob = blob_bytes_of(cfg);
-    c->row_bytes = size_t(3) * cfg->hidden * c->elem;
-    c->nseg = cfg->hidden / (cfg->dtype == SPM_DTYPE_BF16 ? 256 : 128);
+    c->row_bytes = c->blob / size_t(cfg->inter);
+    c->nseg = cfg->hidden / (cfg->dtype == SPM_DTYPE_FP32 ? 128 : 256);
     c->depth = int((kFfnSmemLimit - 1024) / (4 * c->row_bytes));   // ring depth with the fewest warps
     auto bail = [&](int rc) { g_init_error = c->err; spm_destroy(c); return rc; };
     if (c->depth < 1) { c->err = "hidden too large for the shared-memory ring"; return bail(SPM_ERR_CONFIG); }

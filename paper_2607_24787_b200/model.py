@@ -21,6 +21,18 @@ def pack_experts(gate: torch.Tensor, up: torch.Tensor, down: torch.Tensor) -> to
     return torch.stack((gate, up, down.transpose(1, 2)), dim=2).contiguous()
 
 
+def pack_experts_q4(gate, up, down_t) -> torch.Tensor:
+    """4-bit experts -> packed blobs. Each argument is (q uint8 [ne, I, D] in 0..15, scale fp16
+    [ne, I, D/32]); `down_t` row j is column j of W_down. Returns uint8 [ne, I, 3, D/2 + D/16]:
+    per row D/2 bytes of nibbles (element 2b low, 2b+1 high) then the D/32 fp16 scales."""
+    rows = []
+    for q, scale in (gate, up, down_t):
+        nib = (q[..., 0::2] | (q[..., 1::2] << 4)).to(torch.uint8)
+        sc = scale.contiguous().view(torch.uint8).reshape(*scale.shape[:-1], scale.shape[-1] * 2)
+        rows.append(torch.cat((nib, sc), dim=-1))
+    return torch.stack(rows, dim=2).contiguous()
+
+
 class PinnedStore:
     """Page-locked host buffer from spm_host_alloc, viewed as a flat uint8 torch tensor."""
 
@@ -62,7 +74,7 @@ class OffloadedMoE:
         self.L, self.D, self.n, self.I, self.K = n_layers, hidden, n_experts, inter, top_k
         self.n_shared, self.r, self.slots, self.max_batch = n_shared, adapter_rank, slots, max_batch
         self.cfg = B.make_cfg(n_layers, hidden, n_experts, inter, top_k, n_shared, adapter_rank,
-                              B.DTYPE_BF16 if dtype in ("bf16", torch.bfloat16) else B.DTYPE_FP32,
+                              {"bf16": B.DTYPE_BF16, torch.bfloat16: B.DTYPE_BF16, "q4": B.DTYPE_Q4}.get(dtype, B.DTYPE_FP32),
                               int(renormalize), max_batch, rms_eps)
         self.blob_bytes = B.spm_expert_blob_bytes(self.cfg)
         assert store.nbytes >= n_layers * n_experts * self.blob_bytes

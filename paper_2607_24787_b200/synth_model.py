@@ -6,7 +6,16 @@ import torch
 
 import synth
 
-from .model import OffloadedMoE, PinnedStore, pack_experts
+from .model import OffloadedMoE, PinnedStore, pack_experts, pack_experts_q4
+
+
+def packed_experts(cfg: synth.ModelCfg, layer: int, experts, device) -> torch.Tensor:
+    """Packed blobs (flat uint8 per expert) of the listed experts of one layer."""
+    if cfg.dtype == "q4":
+        g, u, d = synth.expert_q4(cfg, layer, experts, device=device)
+        return pack_experts_q4(g, u, d)
+    g, u, d = synth.expert_matrices(cfg, layer, experts, device=device)
+    return pack_experts(g, u, d).view(torch.uint8)
 
 
 def fill_store(cfg: synth.ModelCfg, store: PinnedStore, device, chunk: int = 32):
@@ -15,11 +24,10 @@ def fill_store(cfg: synth.ModelCfg, store: PinnedStore, device, chunk: int = 32)
     for l in range(cfg.n_layers):
         for e0 in range(0, cfg.n_experts, chunk):
             es = range(e0, min(e0 + chunk, cfg.n_experts))
-            g, u, d = synth.expert_matrices(cfg, l, es, device=device)
-            packed = pack_experts(g, u, d).view(torch.uint8).reshape(-1)
+            packed = packed_experts(cfg, l, es, device).reshape(-1)
             off = (l * cfg.n_experts + e0) * blob
             store.tensor[off:off + packed.numel()].copy_(packed)
-            del g, u, d, packed
+            del packed
     torch.cuda.synchronize(device)
 
 
@@ -49,8 +57,7 @@ def build_from_synth(cfg: synth.ModelCfg, slots=None, budget=None, max_batch=Non
     if cfg.n_shared:
         per_layer = []
         for l in range(L):
-            g, u, d = synth.expert_matrices(cfg, l, range(cfg.n_experts, cfg.n_experts + cfg.n_shared), dev)
-            per_layer.append(pack_experts(g, u, d))
+            per_layer.append(packed_experts(cfg, l, range(cfg.n_experts, cfg.n_experts + cfg.n_shared), dev))
         shared = torch.stack(per_layer).contiguous()
     if store is None:
         store = PinnedStore(L * cfg.n_experts * cfg.expert_bytes)

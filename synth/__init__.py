@@ -15,8 +15,11 @@ from .gen import (  # noqa: F401
     TAG_UP,
     adapter_a,
     adapter_b,
+    dequantize_q4,
     embedding_rows,
     expert_matrices,
+    expert_q4,
+    quantize_q4,
     get_config,
     normal_table,
     router_w,

@@ -50,7 +50,7 @@ class ModelCfg:
     top_k: int
     n_shared: int
     adapter_rank: int
-    dtype: str  # "fp32" or "bf16": storage type of every weight matrix
+    dtype: str  # "fp32" / "bf16": storage type of every weight matrix; "q4": experts 4-bit, the rest bf16
     slots: int  # routed-expert cache slots per layer
     budget: int  # prefetch budget M_max; -1 = derive from the profiled window
     batch: int  # sequences decoded per step
@@ -67,10 +67,13 @@ class ModelCfg:
 
     @property
     def elem_bytes(self) -> int:
+        """Bytes per element of the router / adapter matrices."""
         return 4 if self.dtype == "fp32" else 2
 
     @property
     def expert_bytes(self) -> int:
+        if self.dtype == "q4":      # 32 weights = 16 bytes of nibbles + one fp16 scale: 4.5 bit per weight
+            return 3 * self.inter * (self.hidden // 2 + self.hidden // 16)
         return 3 * self.hidden * self.inter * self.elem_bytes
 
     @property
@@ -85,6 +88,9 @@ CONFIGS = {
     "qwen3": ModelCfg("qwen3", 48, 2048, 128, 768, 8, 0, 16, "bf16", 16, -1, 1, 256, 151936, 1),
     # DeepSeek-VL2-Tiny-shaped MoE decode, 2 always-resident shared experts
     "dsvl2": ModelCfg("dsvl2", 12, 1280, 64, 896, 6, 2, 16, "bf16", 8, -1, 1, 256, 129280, 2),
+    # the same two shapes with 4-bit experts (the paper's on-device setting: 1.94 MB per DeepSeek expert)
+    "qwen3_q4": ModelCfg("qwen3_q4", 48, 2048, 128, 768, 8, 0, 16, "q4", 16, -1, 1, 256, 151936, 1),
+    "dsvl2_q4": ModelCfg("dsvl2_q4", 12, 1280, 64, 896, 6, 2, 16, "q4", 8, -1, 1, 256, 129280, 2),
     # budget / cache sweep on the Qwen3 shape (budget and slots overridden per cell)
     "sweep": ModelCfg("sweep", 48, 2048, 128, 768, 8, 0, 16, "bf16", 16, 1, 1, 512, 151936, 3),
     # batched decode on the Qwen3 shape
@@ -182,12 +188,50 @@ def adapter_b(cfg: ModelCfg, layer: int, device="cpu") -> torch.Tensor:
                         cfg.sigma_w, cfg.torch_dtype, device).view(cfg.n_experts, cfg.adapter_rank)
 
 
+Q4_GROUP = 32
+
+
+def quantize_q4(w: torch.Tensor):
+    """Symmetric 4-bit quantisation along the last dimension in groups of 32 (input preparation).
+
+    Returns (q uint8 in 0..15, scale fp16) with value = scale * (q - 8); scale = max|w| / 7 of the
+    group, rounded to fp16 (1 where the group is all zero)."""
+    g = w.to(torch.float32).reshape(*w.shape[:-1], w.shape[-1] // Q4_GROUP, Q4_GROUP)
+    scale = (g.abs().amax(dim=-1) / 7.0).to(torch.float16)
+    scale = torch.where(scale == 0, torch.ones_like(scale), scale)
+    q = torch.clamp(torch.round(g / scale.to(torch.float32).unsqueeze(-1)) + 8, 0, 15).to(torch.uint8)
+    return q.reshape(w.shape), scale
+
+
+def dequantize_q4(q: torch.Tensor, scale: torch.Tensor) -> torch.Tensor:
+    """fp32 values scale * (q - 8); exact (an fp16 scale times a 4-bit integer fits fp32)."""
+    g = q.to(torch.float32).reshape(*q.shape[:-1], q.shape[-1] // Q4_GROUP, Q4_GROUP) - 8.0
+    return (g * scale.to(torch.float32).unsqueeze(-1)).reshape(q.shape)
+
+
+def expert_q4(cfg: ModelCfg, layer: int, experts, device="cpu"):
+    """4-bit experts: ((q, scale) of gate[ne, I, D], of up[ne, I, D], of down^T[ne, I, D]).
+
+    down^T row j is column j of W_down, so its quantisation groups run along the hidden dimension."""
+    experts = list(experts)
+    ne, I, D = len(experts), cfg.inter, cfg.hidden
+    out = []
+    for tag in (TAG_GATE, TAG_UP, TAG_DOWN):
+        w = synth_normal(cfg.seed, tag, layer, experts, I * D, cfg.sigma_w, torch.bfloat16, device).view(ne, I, D)
+        out.append(quantize_q4(w))
+    return tuple(out)
+
+
 def expert_matrices(cfg: ModelCfg, layer: int, experts, device="cpu"):
     """(gate[ne, I, D], up[ne, I, D], down[ne, D, I]) for the listed experts.
 
     Routed experts are 0..n_experts-1; shared expert s is index n_experts + s.
+    With 4-bit experts these are the de-quantised fp32 values.
     """
     experts = list(experts)
+    if cfg.dtype == "q4":
+        (gq, gs), (uq, us), (dq, dsc) = expert_q4(cfg, layer, experts, device)
+        return dequantize_q4(gq, gs), dequantize_q4(uq, us), dequantize_q4(dq, dsc).transpose(1, 2).contiguous()
     ne, I, D = len(experts), cfg.inter, cfg.hidden
     g = synth_normal(cfg.seed, TAG_GATE, layer, experts, I * D, cfg.sigma_w, cfg.torch_dtype, device)
     u = synth_normal(cfg.seed, TAG_UP, layer, experts, I * D, cfg.sigma_w, cfg.torch_dtype, device)

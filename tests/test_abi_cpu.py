@@ -31,6 +31,7 @@ def test_query_and_config_errors():
     cfg = B.make_cfg(48, 2048, 128, 768, 8, 0, 16, B.DTYPE_BF16)
     assert B.spm_expert_blob_bytes(cfg) == 9437184
     assert B.spm_query_arena(cfg, 16) > 48 * 16 * 9437184
+    assert B.spm_expert_blob_bytes(B.make_cfg(12, 1280, 64, 896, 6, 2, 16, B.DTYPE_Q4)) == 1935360
     with pytest.raises(B.SpmError) as e:
         B.spm_query_arena(cfg, 4)                       # slots < top_k at batch 1
     assert e.value.code == -2

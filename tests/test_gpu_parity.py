@@ -15,7 +15,7 @@ from oracle import ref_decode, ref_math as M, ref_policy as P
 
 pytestmark = pytest.mark.gpu
 
-TOL = {"fp32": 1e-5, "bf16": 1e-4}
+TOL = {"fp32": 1e-5, "bf16": 1e-4, "q4": 1e-4}
 
 
 @pytest.fixture(scope="module")
@@ -45,6 +45,9 @@ SHAPES = {
     # bf16, several 256-wide segments, row count (K+shared)*I not a multiple of the CTA count
     "ds_small": synth.get_config("dsvl2", n_layers=3, n_experts=16, inter=224, slots=8, budget=2),
     "qw_small": synth.get_config("qwen3", n_layers=2, n_experts=24, inter=96, slots=10, budget=3),
+    # 4-bit experts (+ 2 shared), hidden 1280 = 40 groups: the second chunk of a lane is ragged
+    "q4_ds": synth.get_config("dsvl2_q4", n_layers=3, n_experts=16, inter=224, slots=8, budget=2),
+    "q4_qw": synth.get_config("qwen3_q4", n_layers=2, n_experts=24, inter=96, slots=10, budget=3),
     "odd": synth.get_config("tiny", hidden=384, inter=50, n_experts=11, top_k=3, adapter_rank=5, slots=5, seed=7),
 }
 

@@ -51,3 +51,29 @@ def test_config_table():
     assert q.expert_bytes == 9437184 and q.n_layers * q.n_experts * q.expert_bytes == 57982058496
     assert synth.get_config("dsvl2").expert_bytes == 6881280
     assert synth.get_config("tiny").expert_bytes == 393216
+
+
+def test_q4_quantiser_and_packing():
+    w = torch.randn(3, 5, 96) * 0.02
+    w[0, 0, :32] = 0.0                                   # an all-zero group keeps scale 1, codes 8
+    q, s = synth.quantize_q4(w)
+    assert q.dtype == torch.uint8 and q.min() >= 1 and q.max() <= 15 and s.dtype == torch.float16
+    assert s.shape == (3, 5, 3) and torch.all(q[0, 0, :32] == 8) and s[0, 0, 0] == 1
+    deq = synth.dequantize_q4(q, s)
+    err = (deq - w).abs().reshape(3, 5, 3, 32).amax(-1)
+    assert torch.all(err <= s.float() * 0.5 + 1e-7)                       # round to nearest code
+    assert torch.equal(deq, (q.double() - 8).mul(s.double().repeat_interleave(32, -1)).float())   # exact in fp32
+    cfg = synth.get_config("dsvl2_q4")
+    assert cfg.expert_bytes == 1935360                                    # the paper's 1.94 MB per expert
+    assert synth.get_config("qwen3_q4").expert_bytes * 32 == synth.get_config("qwen3").expert_bytes * 9
+    small = cfg.replace(n_layers=1, n_experts=3, inter=8)
+    g, u, d = synth.expert_matrices(small, 0, [1])
+    (gq, gs), (uq, us), (dq, dsc) = synth.expert_q4(small, 0, [1])
+    assert torch.equal(g, synth.dequantize_q4(gq, gs)) and torch.equal(d, synth.dequantize_q4(dq, dsc).transpose(1, 2))
+    from paper_2607_24787_b200.model import pack_experts_q4
+    blob = pack_experts_q4((gq, gs), (uq, us), (dq, dsc))
+    D = small.hidden
+    assert blob.shape == (1, 8, 3, D // 2 + D // 16) and blob.numel() == small.expert_bytes
+    nib = blob[0, 3, 2, :D // 2]
+    assert torch.equal(torch.stack((nib & 15, nib >> 4), -1).reshape(-1), dq[0, 3])
+    assert torch.equal(blob[0, 3, 2, D // 2:].view(torch.float16), dsc[0, 3])
