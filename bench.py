@@ -143,6 +143,14 @@ def hidden_rows(cfg, steps, stream):
     return tok, H.view(steps, cfg.batch, cfg.hidden).contiguous()
 
 
+def ffn_kernel_name(cfg):
+    if cfg.dtype == "q4":
+        return "ffn_gemv_q4_kernel"
+    if cfg.batch > 1 and cfg.n_shared == 0 and cfg.dtype == "bf16":
+        return "ffn_grouped_kernel"
+    return "ffn_gemv_kernel"
+
+
 def bench_config(args):
     """The named configuration; --layers / --slots shrink it for profiler captures and say so in its name."""
     cfg = synth.get_config(args.config)
@@ -280,7 +288,7 @@ def run_ours(args):
     # duration of an HBM-streaming kernel on this machine; `isolated` (below, when the
     # resident leg runs) times the same entry point with no PCIe traffic.
     result["roofline"] = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                          "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(cfg.name), "kernel": "ffn_gemv_kernel",
+                          "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(cfg.name), "kernel": ffn_kernel_name(cfg),
                           "peak_source": f"of {which}", "algorithmic_bytes_per_launch": algo_bytes,
                           "us_per_launch": ffn_us, "in_kernel_window_us": window_us,
                           "achieved_in_kernel_window": algo_bytes / (window_us * 1e-6) / 1e9 if window_us > 0 else None,
@@ -449,7 +457,7 @@ def ffn_back_to_back(cfg, full, algo_bytes, peak, launches=480):
     full.synchronize()
     per_call = e0.elapsed_time(e1) * 1e3 / launches
     ach = mean_bytes / (per_kernel * 1e-6) / 1e9
-    return {"launches": launches, "kernel": "ffn_grouped_kernel" if nb > 1 and cfg.n_shared == 0 else "ffn_gemv_kernel",
+    return {"launches": launches, "kernel": ffn_kernel_name(cfg),
             "algorithmic_bytes_per_launch": mean_bytes, "kernel_us": per_kernel,
             "kernel_window_us": window if window > 0 else None, "call_us_incl_combine": per_call, "gb_s": ach,
             "frac_of_measured_peak": ach / peak,

@@ -33,8 +33,11 @@ __device__ __forceinline__ void unpack_q4_word(uint32_t w, float (&f)[8]) {
     }
 }
 
+constexpr int kQ4MaxWarps = 16;    // activations live in shared memory here, so registers allow 16 warps
+constexpr int kQ4Pad = 36;         // floats per 32-wide group in shared memory: lanes then start 4 banks apart
+
 template <int NCH, int MAXNB>     // NCH = 16-byte nibble chunks (groups of 32 weights) per lane
-__global__ void __launch_bounds__(kFfnMaxThreads, 1)
+__global__ void __launch_bounds__(kQ4MaxWarps * 32, 1)
 ffn_gemv_q4_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth, const int D) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int wi = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -53,7 +56,11 @@ ffn_gemv_q4_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth, co
     const int my_n = span > 0 ? (span + nw - 1) / nw : 0;
 
     unsigned char* ring = smem + size_t(wi) * depth * ROWB;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + ((size_t(nw) * depth * ROWB + 15) & ~size_t(15)));
+    // layout: [ring, reused for the cross-warp reduction][barriers][activations, padded per group]
+    const size_t ring_bytes = size_t(nw) * depth * ROWB, red_bytes = size_t(nw) * n_grp * kQ4Pad * sizeof(float);
+    const size_t area = ((ring_bytes > red_bytes ? ring_bytes : red_bytes) + 15) & ~size_t(15);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + area);
+    float* xs = reinterpret_cast<float*>(smem + area + ((size_t(nw) * depth * 8 + 15) & ~size_t(15)));
     const uint32_t bar0 = smem_u32(bars + wi * depth);
     const uint32_t ring0 = smem_u32(ring);
     if (lane == 0) {
@@ -88,23 +95,15 @@ ffn_gemv_q4_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth, co
             if (!issue(n_issued)) { ok = false; break; }
     }
 
-    // activations of this lane's groups (group g = ch * 32 + lane), their sums, and the partial y
-    float xr[NCH][32], ya[NCH][32];
-    {
-        const float* xt = a.x + size_t(tok) * D;
+    // activations go to shared memory once (group g at xs[g * kQ4Pad ..]); the partial y of this
+    // lane's groups (g = ch * 32 + lane) stays in registers
+    for (int i = threadIdx.x; i < D; i += blockDim.x) xs[(i >> 5) * kQ4Pad + (i & 31)] = a.x[size_t(tok) * D + i];
+    float ya[NCH][32];
 #pragma unroll
-        for (int ch = 0; ch < NCH; ++ch) {
-            const int g = ch * 32 + lane;
+    for (int ch = 0; ch < NCH; ++ch)
 #pragma unroll
-            for (int v = 0; v < 32; v += 4) {
-                float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (g < n_grp) t = *reinterpret_cast<const float4*>(xt + g * 32 + v);
-                xr[ch][v] = t.x; xr[ch][v + 1] = t.y; xr[ch][v + 2] = t.z; xr[ch][v + 3] = t.w;
-            }
-#pragma unroll
-            for (int v = 0; v < 32; ++v) ya[ch][v] = 0.f;
-        }
-    }
+        for (int v = 0; v < 32; ++v) ya[ch][v] = 0.f;
+    __syncthreads();
     ok = __shfl_sync(0xffffffffu, ok, 0);
 
     int cur_ent = -1;
@@ -139,16 +138,20 @@ ffn_gemv_q4_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth, co
                     const float sg = __half2float(*reinterpret_cast<const __half*>(buf + D / 2 + g * 2));
                     const float su = __half2float(*reinterpret_cast<const __half*>(buf + RB + D / 2 + g * 2));
                     const uint32_t wg[4] = {vg.x, vg.y, vg.z, vg.w}, wu[4] = {vu.x, vu.y, vu.z, vu.w};
+                    const float* xg = xs + g * kQ4Pad;
                     float dg = 0.f, du = 0.f;
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         float fg[8], fu[8];
                         unpack_q4_word(wg[q], fg);
                         unpack_q4_word(wu[q], fu);
+                        const float4 x0 = *reinterpret_cast<const float4*>(xg + q * 8);
+                        const float4 x1 = *reinterpret_cast<const float4*>(xg + q * 8 + 4);
+                        const float xv[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
 #pragma unroll
                         for (int v = 0; v < 8; ++v) {
-                            dg = fmaf(fg[v], xr[ch][q * 8 + v], dg);
-                            du = fmaf(fu[v], xr[ch][q * 8 + v], du);
+                            dg = fmaf(fg[v], xv[v], dg);
+                            du = fmaf(fu[v], xv[v], du);
                         }
                     }
                     pg = fmaf(sg, dg, pg);
@@ -196,14 +199,15 @@ ffn_gemv_q4_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth, co
         if (g < n_grp) {
 #pragma unroll
             for (int v = 0; v < 32; v += 4)
-                *reinterpret_cast<float4*>(red + wi * D + g * 32 + v) = make_float4(ya[ch][v], ya[ch][v + 1], ya[ch][v + 2], ya[ch][v + 3]);
+                *reinterpret_cast<float4*>(red + (size_t(wi) * n_grp + g) * kQ4Pad + v) = make_float4(ya[ch][v], ya[ch][v + 1], ya[ch][v + 2], ya[ch][v + 3]);
         }
     }
     __syncthreads();
     float* out = a.partial + (size_t(tok) * G + c) * D;
     for (int d = threadIdx.x; d < D; d += blockDim.x) {
-        float acc = red[d];
-        for (int w2 = 1; w2 < nw; ++w2) acc += red[w2 * D + d];
+        const int o = (d >> 5) * kQ4Pad + (d & 31);
+        float acc = red[o];
+        for (int w2 = 1; w2 < nw; ++w2) acc += red[size_t(w2) * n_grp * kQ4Pad + o];
         out[d] = acc;
     }
     if (a.clock) {
@@ -212,23 +216,22 @@ ffn_gemv_q4_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth, co
     }
 }
 
-// Launch shape for 4-bit rows. The cross-warp reduction needs warps * D floats of shared memory,
-// which for these short rows is more than a shallow ring would take, so the ring depth is raised
-// until it covers it.
+// Launch shape for 4-bit rows: the warp count that leaves the fewest rows on the busiest warp, a
+// ring deep enough to hold a warp's whole share when it fits, and room for the cross-warp reduction.
 inline void ffn_gemv_q4_shape(size_t row_bytes, int D, int rows_per_cta, int* warps, int* depth, size_t* smem) {
     int best_w = 8, best_cost = 1 << 30;
-    for (int w = 4; w <= kFfnMaxWarps; ++w) {
+    for (int w = 4; w <= kQ4MaxWarps; ++w) {
         const int cost = (rows_per_cta + w - 1) / w;
-        if (cost < best_cost || (cost == best_cost && w > best_w)) { best_w = w; best_cost = cost; }
+        if (cost < best_cost || (cost == best_cost && w < best_w)) { best_w = w; best_cost = cost; }
     }
-    int d = 8;
-    while (d > 2 && size_t(best_w) * d * row_bytes > 160 * 1024) --d;
-    size_t ring = size_t(best_w) * d * row_bytes;
-    const size_t red = size_t(best_w) * D * sizeof(float);
-    if (ring < red) ring = red;
+    int d = best_cost < 2 ? 2 : (best_cost > 6 ? 6 : best_cost);
+    while (d > 2 && size_t(best_w) * d * row_bytes > 150 * 1024) --d;
+    size_t area = size_t(best_w) * d * row_bytes;
+    const size_t red = size_t(best_w) * (D / 32) * kQ4Pad * sizeof(float);
+    if (area < red) area = red;
     *warps = best_w;
     *depth = d;
-    *smem = ((ring + 15) & ~size_t(15)) + size_t(best_w) * d * 8 + 16;
+    *smem = ((area + 15) & ~size_t(15)) + ((size_t(best_w) * d * 8 + 15) & ~size_t(15)) + size_t(D / 32) * kQ4Pad * sizeof(float) + 16;
 }
 
 }  // namespace spm
