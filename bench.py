@@ -143,6 +143,19 @@ def hidden_rows(cfg, steps, stream):
     return tok, H.view(steps, cfg.batch, cfg.hidden).contiguous()
 
 
+def affordable_store_layers(cfg, world):
+    """Layers of experts this rank can keep pinned: all of them when 60 % of the host's available memory,
+    split over the ranks of the node, holds the store; otherwise fewer, and the layers repeat (the context
+    is told so through host_store_layers; sizes, copies and kernels are unchanged)."""
+    per_layer = cfg.n_experts * cfg.expert_bytes
+    try:
+        avail = int(open("/proc/meminfo").read().split("MemAvailable:")[1].split()[0]) * 1024
+    except Exception:
+        return cfg.n_layers
+    ranks = int(os.environ.get("LOCAL_WORLD_SIZE", world))
+    return int(max(1, min(cfg.n_layers, (0.6 * avail / max(ranks, 1)) // per_layer)))
+
+
 def ffn_kernel_name(cfg):
     if cfg.dtype == "q4":
         return "ffn_gemv_q4_kernel"
@@ -217,7 +230,8 @@ def run_ours(args):
     cfg = bench_config(args)
     K, W = args.steps, args.warmup
     t_setup = time.time()
-    m = build_from_synth(cfg, device=device)                 # budget -1: profiled inside spm_init
+    store_layers = affordable_store_layers(cfg, world)
+    m = build_from_synth(cfg, device=device, store_layers=store_layers)   # budget -1: profiled inside spm_init
     setup_s = time.time() - t_setup
     if args.stub_us:
         m.set_attention_stub_us(args.stub_us)
@@ -269,7 +283,8 @@ def run_ours(args):
         "config": {"workload": f"{cfg.name}: L{cfg.n_layers} D{cfg.hidden} n{cfg.n_experts} I{cfg.inter} K{cfg.top_k}"
                                f"+{cfg.n_shared}sh r{cfg.adapter_rank} {cfg.dtype} slots{cfg.slots} batch{cfg.batch}",
                    "policy": "adapter", "budget": budget, "budget_raw": raw_budget, "window_us": window_us,
-                   "t_xfer_us": t_xfer_us, "attention_stub_us": args.stub_us, "copy_delay_us": args.copy_delay_us, "seed": cfg.seed, "token_ids": "Zipf(1.1)",
+                   "t_xfer_us": t_xfer_us, "attention_stub_us": args.stub_us, "copy_delay_us": args.copy_delay_us,
+                   "host_store_layers": store_layers, "seed": cfg.seed, "token_ids": "Zipf(1.1)",
                    "l2": "inputs larger than L2: every layer streams its own slot pool, 3.6 GB of weights per step",
                    "setup_s": setup_s, "wall_ms_per_step": wall_ms / K},
         "clocks": clk,
@@ -397,7 +412,8 @@ def h2d_probe(m, cfg):
 def resident_run(cfg, m, H_dev, W, K, peak, algo_bytes, device):
     """All experts resident (slots = n): the HBM-bound ceiling and the FFN kernel without PCIe traffic."""
     from paper_2607_24787_b200.synth_model import build_from_synth
-    full = build_from_synth(cfg, slots=cfg.n_experts, budget=0, device=device, store=m.store, max_batch=cfg.batch)
+    full = build_from_synth(cfg, slots=cfg.n_experts, budget=0, device=device, store=m.store, max_batch=cfg.batch,
+                            store_layers=m.store_layers)
     full.set_policy("on_demand")
     for l in range(cfg.n_layers):                          # preload every expert
         full.prefetch_async(l, np.arange(cfg.n_experts, dtype=np.int32))

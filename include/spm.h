@@ -110,6 +110,10 @@ typedef struct {
     size_t      arena_bytes;     /* >= spm_query_arena()                                         */
     void*       compute_stream;  /* cudaStream_t                                                 */
     void*       copy_stream;     /* cudaStream_t, different from compute_stream                  */
+    int32_t     host_store_layers; /* 0 or L: host_experts holds all L layers. 0 < k < L: it holds only k
+                                      layers and layer l reads the blobs of layer l % k (for hosts that
+                                      cannot pin the whole store; the model then repeats its expert
+                                      weights every k layers, sizes and traffic are unchanged)        */
 } spm_buffers;
 
 typedef struct { int32_t step, layer, kind, expert, slot; } spm_event;

@@ -40,7 +40,7 @@ class Buffers(C.Structure):
     _fields_ = [("rms_gamma", C.c_void_p), ("router_w", C.c_void_p), ("adapter_a", C.c_void_p),
                 ("adapter_b", C.c_void_p), ("shared_experts", C.c_void_p), ("host_experts", C.c_void_p),
                 ("arena", C.c_void_p), ("arena_bytes", C.c_size_t), ("compute_stream", C.c_void_p),
-                ("copy_stream", C.c_void_p)]
+                ("copy_stream", C.c_void_p), ("host_store_layers", C.c_int32)]
 
 
 class Event(C.Structure):

@@ -401,7 +401,9 @@ unsigned char* slot_ptr(spm_ctx* c, int layer, int slot) {
     return c->pools + (size_t(layer) * c->S + slot) * c->blob;
 }
 const unsigned char* host_blob(spm_ctx* c, int layer, int e) {
-    return static_cast<const unsigned char*>(c->buf.host_experts) + (size_t(layer) * c->cfg.n_experts + e) * c->blob;
+    const int k = c->buf.host_store_layers;
+    const int src = (k > 0 && k < c->cfg.n_layers) ? layer % k : layer;
+    return static_cast<const unsigned char*>(c->buf.host_experts) + (size_t(src) * c->cfg.n_experts + e) * c->blob;
 }
 
 // Enqueue one expert transfer on the copy stream and arm the slot's event.
@@ -731,6 +733,7 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
     if (cfg->n_layers > 1 && (!b->adapter_a || !b->adapter_b)) return fail(nullptr, SPM_ERR_INVALID_ARG, "adapter buffers are null");
     if (cfg->n_shared > 0 && !b->shared_experts) return fail(nullptr, SPM_ERR_INVALID_ARG, "shared_experts is null");
     if (b->compute_stream == b->copy_stream) return fail(nullptr, SPM_ERR_INVALID_ARG, "compute and copy stream must differ");
+    if (b->host_store_layers < 0 || b->host_store_layers > cfg->n_layers) return fail(nullptr, SPM_ERR_INVALID_ARG, "host_store_layers out of range");
     if (reinterpret_cast<uintptr_t>(b->arena) % 256) return fail(nullptr, SPM_ERR_INVALID_ARG, "arena must be 256-byte aligned");
     const Layout lay = layout_of(cfg, slots_per_layer);
     if (b->arena_bytes < lay.total) return fail(nullptr, SPM_ERR_INVALID_ARG, "arena too small: %zu < %zu", b->arena_bytes, lay.total);

@@ -66,7 +66,7 @@ class OffloadedMoE:
 
     def __init__(self, *, n_layers, hidden, n_experts, inter, top_k, n_shared, adapter_rank, dtype,
                  renormalize, rms_eps, max_batch, slots, budget, gamma, router_w, adapter_a, adapter_b,
-                 shared_blobs, store: PinnedStore, device="cuda:0"):
+                 shared_blobs, store: PinnedStore, device="cuda:0", store_layers=0):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required: there is no CPU implementation of this path")
         self.device = torch.device(device)
@@ -77,7 +77,8 @@ class OffloadedMoE:
                               {"bf16": B.DTYPE_BF16, torch.bfloat16: B.DTYPE_BF16, "q4": B.DTYPE_Q4}.get(dtype, B.DTYPE_FP32),
                               int(renormalize), max_batch, rms_eps)
         self.blob_bytes = B.spm_expert_blob_bytes(self.cfg)
-        assert store.nbytes >= n_layers * n_experts * self.blob_bytes
+        self.store_layers = store_layers if 0 < store_layers < n_layers else n_layers
+        assert store.nbytes >= self.store_layers * n_experts * self.blob_bytes
         self._keep = [gamma, router_w, adapter_a, adapter_b, shared_blobs, store]
         self.store = store
         self.arena = torch.empty(B.spm_query_arena(self.cfg, slots) + 256, dtype=torch.uint8, device=self.device)
@@ -89,7 +90,8 @@ class OffloadedMoE:
                         adapter_b.data_ptr() if adapter_b is not None else None,
                         shared_blobs.data_ptr() if shared_blobs is not None else None,
                         store.ptr, arena_ptr, self.arena.numel() - 256,
-                        self.compute.cuda_stream, self.copy.cuda_stream)
+                        self.compute.cuda_stream, self.copy.cuda_stream,
+                        0 if self.store_layers == n_layers else self.store_layers)
         torch.cuda.synchronize(self.device)
         self.ctx = B.spm_init(self.cfg, slots, budget, buf)
 

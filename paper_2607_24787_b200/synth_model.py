@@ -18,10 +18,10 @@ def packed_experts(cfg: synth.ModelCfg, layer: int, experts, device) -> torch.Te
     return pack_experts(g, u, d).view(torch.uint8)
 
 
-def fill_store(cfg: synth.ModelCfg, store: PinnedStore, device, chunk: int = 32):
-    """Generate and pack every routed expert of every layer into the pinned host store."""
+def fill_store(cfg: synth.ModelCfg, store: PinnedStore, device, chunk: int = 32, layers=None):
+    """Generate and pack every routed expert of the first `layers` (default all) layers into the pinned host store."""
     blob = cfg.expert_bytes
-    for l in range(cfg.n_layers):
+    for l in range(cfg.n_layers if layers is None else layers):
         for e0 in range(0, cfg.n_experts, chunk):
             es = range(e0, min(e0 + chunk, cfg.n_experts))
             packed = packed_experts(cfg, l, es, device).reshape(-1)
@@ -32,7 +32,7 @@ def fill_store(cfg: synth.ModelCfg, store: PinnedStore, device, chunk: int = 32)
 
 
 def build_from_synth(cfg: synth.ModelCfg, slots=None, budget=None, max_batch=None, device="cuda:0",
-                     store: PinnedStore | None = None, adapter: str = "random") -> OffloadedMoE:
+                     store: PinnedStore | None = None, adapter: str = "random", store_layers: int = 0) -> OffloadedMoE:
     """Random-init model of the configuration's shape, experts offloaded to pinned host memory.
 
     adapter="random": the configuration's N(0, 0.02) rank-r adapters. adapter="gate_reuse": a
@@ -59,9 +59,12 @@ def build_from_synth(cfg: synth.ModelCfg, slots=None, budget=None, max_batch=Non
         for l in range(L):
             per_layer.append(packed_experts(cfg, l, range(cfg.n_experts, cfg.n_experts + cfg.n_shared), dev))
         shared = torch.stack(per_layer).contiguous()
+    # store_layers < L: a host that cannot pin the whole store keeps only that many layers of experts;
+    # layer l then reads the blobs of layer l % store_layers (same sizes and traffic, repeated weights)
+    kl = store_layers if 0 < store_layers < L else L
     if store is None:
-        store = PinnedStore(L * cfg.n_experts * cfg.expert_bytes)
-        fill_store(cfg, store, dev)
+        store = PinnedStore(kl * cfg.n_experts * cfg.expert_bytes)
+        fill_store(cfg, store, dev, layers=kl)
     return OffloadedMoE(n_layers=L, hidden=cfg.hidden, n_experts=cfg.n_experts, inter=cfg.inter,
                         top_k=cfg.top_k, n_shared=cfg.n_shared, adapter_rank=rank,
                         dtype=cfg.dtype, renormalize=cfg.renormalize, rms_eps=cfg.rms_eps,
@@ -69,4 +72,4 @@ def build_from_synth(cfg: synth.ModelCfg, slots=None, budget=None, max_batch=Non
                         slots=cfg.slots if slots is None else slots,
                         budget=cfg.budget if budget is None else budget,
                         gamma=gamma, router_w=router, adapter_a=a, adapter_b=b, shared_blobs=shared,
-                        store=store, device=device)
+                        store=store, device=device, store_layers=kl)

@@ -46,7 +46,7 @@ def test_init_fails_loudly_without_gpu():
     if torch.cuda.is_available():
         pytest.skip("has a GPU")
     cfg = B.make_cfg(2, 256, 16, 128, 2, 0, 8, B.DTYPE_FP32)
-    buf = B.Buffers(256, 256, 256, 256, None, 256, 256, 1 << 40, 1, 2)
+    buf = B.Buffers(256, 256, 256, 256, None, 256, 256, 1 << 40, 1, 2, 0)
     with pytest.raises(B.SpmError) as e:
         B.spm_init(cfg, 4, 2, buf)
     assert e.value.code == -3

@@ -81,6 +81,26 @@ def test_full_batch_fp32():
     compare_run(synth.get_config("tiny", batch=64, slots=16, budget=2), steps=2)
 
 
+def test_partial_host_store_repeats_layers():
+    """A host that cannot pin the whole store keeps k layers of experts; layer l then reads layer l % k."""
+    cfg = synth.get_config("tiny", n_layers=3)
+    m = build(cfg, store_layers=2)
+
+    class Repeating(SynthWeights):
+        def expert(self, l, e):
+            return super().expert(l % 2, e)
+
+    ref = make_ref(cfg, weights=Repeating(cfg))
+    tok = synth.zipf_tokens(cfg, steps=4)
+    H = synth.embedding_rows(cfg, tok[:, 0]).numpy()
+    for s in range(4):
+        out = m.decode_step(dev(H[s:s + 1])); m.synchronize()
+        want, _ = ref.step(H[s:s + 1])
+        assert M.rel_linf(out.cpu().numpy(), want) < 4e-5
+    assert m.events() == ref.table.events
+    m.close()
+
+
 def test_timing_knobs_do_not_change_results():
     """Attention stand-in and emulated storage delay only move time around."""
     cfg = synth.get_config("tiny")
