@@ -316,7 +316,13 @@ int launch_router(spm_ctx* c, int layer, const float* h, const float* x_in, int 
     a.order = c->ws_order;
     a.counters = c->ws_counters;
     a.mailbox = c->mb_dev;
-    a.seq = ++c->seq;
+    // Sequence numbers whose low 16 bits are zero are skipped, and the words this launch will
+    // publish are zeroed first, so a word left by an older launch can never carry the current tag.
+    ++c->seq;
+    if ((c->seq & 0xffffu) == 0) ++c->seq;
+    if (do_router) memset(const_cast<int32_t*>(c->mb_host->ids), 0, size_t(nb) * m.top_k * sizeof(int32_t));
+    if (do_adapter) memset(const_cast<int32_t*>(c->mb_host->order), 0, size_t(m.n_experts) * sizeof(int32_t));
+    a.seq = c->seq;
     a.D = m.hidden; a.n = m.n_experts; a.K = m.top_k; a.r = m.adapter_rank; a.nb = nb;
     a.renorm = m.renormalize; a.do_router = do_router; a.do_adapter = do_adapter;
     a.eps = m.rms_eps;
