@@ -16,7 +16,9 @@
 //            accumulator [128 d x 64 tokens] per d-tile, double buffered; the epilogue writes the
 //            rows of real tokens to the partial buffer P[j-tile][token row][d].
 // A combine kernel then adds, per token, its K experts x (I/128) partial rows and the residual in
-// a fixed order. One warp issues TMA, one thread issues tcgen05.mma, four warps run the epilogues;
+// a fixed order. Phase 1 of the next unit is issued before phase 2 of the current one (two G^T/U^T
+// accumulator pairs), so the weight stream does not pause while the epilogue builds A^T.
+// One warp issues TMA, one thread issues tcgen05.mma, four warps run the epilogues;
 // all of them talk through mbarriers, every wait is bounded and an abort flag lets the whole CTA
 // leave together (freeing its TMEM) if a wait ever gives up. No multicast anywhere.
 #pragma once
@@ -30,7 +32,7 @@
 namespace spm {
 
 constexpr int kGgThreads = 192;          // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
-constexpr int kGgStages = 4;
+constexpr int kGgStages = 5;
 constexpr int kGgTokens = 64;            // N of every MMA: an expert's tokens, zero/garbage padded
 constexpr int kGgTileRows = 128;         // M of every MMA
 constexpr int kGgKBlock = 64;            // bf16 elements per 128-byte swizzled row
@@ -38,7 +40,7 @@ constexpr uint32_t kGgTileBytes = kGgTileRows * 128;          // one [128 x 128 
 constexpr uint32_t kGgXBytes = kGgTokens * 128;               // one [64 x 128 B] token box
 constexpr uint32_t kGgStageBytes = 2 * kGgTileBytes + kGgXBytes;   // 40 KB
 constexpr uint32_t kGgActBytes = kGgTileRows * 128;           // A^T: [128 j][64 tokens] bf16
-constexpr uint32_t kGgTmemCols = 256;    // G^T 0..63, U^T 64..127, Y tiles 128..191 and 192..255
+constexpr uint32_t kGgTmemCols = 512;    // two (G^T, U^T) pairs at 0..127 and 128..255, Y tiles at 256..319 and 320..383
 constexpr int kStatusGroupedTimeout = 4;
 
 struct GgUnit {
@@ -154,9 +156,9 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
     uint64_t* bars = reinterpret_cast<uint64_t*>(act + kGgActBytes);
     uint64_t* full = bars;                    // [stages]  TMA -> MMA
     uint64_t* empty = full + kGgStages;       // [stages]  MMA -> TMA
-    uint64_t* acc1_full = empty + kGgStages;  // MMA -> epilogue: G^T, U^T complete
-    uint64_t* acc1_empty = acc1_full + 1;     // epilogue -> MMA: G^T, U^T drained
-    uint64_t* act_full = acc1_empty + 1;      // epilogue -> MMA: A^T written
+    uint64_t* acc1_full = empty + kGgStages;  // [2] MMA -> epilogue: G^T, U^T of a unit complete
+    uint64_t* acc1_empty = acc1_full + 2;     // [2] epilogue -> MMA: that pair drained
+    uint64_t* act_full = acc1_empty + 2;      // epilogue -> MMA: A^T written
     uint64_t* act_empty = act_full + 1;       // MMA -> epilogue: phase 2 has consumed A^T
     uint64_t* acc2_full = act_empty + 1;      // [2] MMA -> epilogue
     uint64_t* acc2_empty = acc2_full + 2;     // [2] epilogue -> MMA
@@ -168,15 +170,19 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
     const int D = a.D;
     const int n_kb = D / kGgKBlock;            // phase-1 stages per unit
     const int n_dt = D / kGgTileRows;          // phase-2 stages per unit
+    const int my_units = blockIdx.x < a.n_units ? (a.n_units - 1 - int(blockIdx.x)) / int(gridDim.x) + 1 : 0;
     GgAbort ab{abort_flag, a.status};
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kGgStages; ++s) { mbar_init(smem_u32(full + s), 1); mbar_init(smem_u32(empty + s), 1); }
-        mbar_init(smem_u32(acc1_full), 1);
-        mbar_init(smem_u32(acc1_empty), 4);     // one arrival per epilogue warp
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(acc1_full + b), 1);
+            mbar_init(smem_u32(acc1_empty + b), 4);     // one arrival per epilogue warp
+            mbar_init(smem_u32(acc2_full + b), 1);
+            mbar_init(smem_u32(acc2_empty + b), 4);
+        }
         mbar_init(smem_u32(act_full), 4);
         mbar_init(smem_u32(act_empty), 1);
-        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(acc2_full + b), 1); mbar_init(smem_u32(acc2_empty + b), 4); }
         *abort_flag = 0;
         fence_barrier_init();
     }
@@ -186,14 +192,17 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    // running counters; every role walks the same sequence of units and stages
+    // Order of work, identical for the producer and the MMA issuer:
+    //   phase1(0), then for i = 0, 1, ...: phase1(i + 1) if it exists, phase2(i).
+    // Phase 1 of the next unit is issued before phase 2 of the current one, so the weight stream
+    // keeps flowing while the epilogue warps turn G^T, U^T of the current unit into A^T.
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            uint32_t it = 0;      // ring position over all stages of all units
+            uint32_t it = 0;      // ring position over all stages
             bool ok = true;
-            for (int u = blockIdx.x; u < a.n_units && ok; u += gridDim.x) {
-                const GgUnit un = a.units[u];
+            auto load_phase1 = [&](int i) {
+                const GgUnit un = a.units[blockIdx.x + i * gridDim.x];
                 for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
                     const uint32_t s = it % kGgStages;
                     if (it >= kGgStages) ok = gg_wait(smem_u32(empty + s), ((it / kGgStages) - 1) & 1, ab);
@@ -205,6 +214,9 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
                     tma_load_4d(base + kGgTileBytes, &wmap, kb * kGgKBlock, 1, un.jt * kGgTileRows, un.slot, fb);  // up rows
                     tma_load_2d(base + 2 * kGgTileBytes, &xmap, kb * kGgKBlock, un.row0, fb);                      // token rows
                 }
+            };
+            auto load_phase2 = [&](int i) {
+                const GgUnit un = a.units[blockIdx.x + i * gridDim.x];
                 for (int dt = 0; dt < n_dt && ok; ++dt, ++it) {
                     const uint32_t s = it % kGgStages;
                     if (it >= kGgStages) ok = gg_wait(smem_u32(empty + s), ((it / kGgStages) - 1) & 1, ab);
@@ -215,6 +227,11 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
                     tma_load_4d(base, &wmap, dt * kGgTileRows, 2, un.jt * kGgTileRows, un.slot, fb);                      // d 0..63
                     tma_load_4d(base + kGgTileBytes, &wmap, dt * kGgTileRows + 64, 2, un.jt * kGgTileRows, un.slot, fb); // d 64..127
                 }
+            };
+            if (my_units > 0) load_phase1(0);
+            for (int i = 0; i < my_units && ok; ++i) {
+                if (i + 1 < my_units) load_phase1(i + 1);
+                if (ok) load_phase2(i);
             }
         }
     } else if (warp == 1) {
@@ -222,10 +239,12 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
         if (lane == 0) {
             constexpr uint32_t idesc1 = gg_idesc(false, false);   // weights K-major, tokens K-major
             constexpr uint32_t idesc2 = gg_idesc(true, true);     // W_down column tile M-major, A^T N-major
-            uint32_t it = 0, nu = 0, nd = 0;     // stage counter, unit counter, d-tile counter
+            uint32_t it = 0, nd = 0;     // stage counter, d-tile counter
             bool ok = true;
-            for (int u = blockIdx.x; u < a.n_units && ok; u += gridDim.x, ++nu) {
-                if (nu > 0) ok = gg_wait(smem_u32(acc1_empty), (nu - 1) & 1, ab);
+            auto mma_phase1 = [&](int i) {
+                const uint32_t b = i & 1, m = uint32_t(i) >> 1;
+                if (i >= 2) ok = gg_wait(smem_u32(acc1_empty + b), (m - 1) & 1, ab);   // pair drained two units ago
+                const uint32_t acc = tmem + 128 * b;
                 for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
                     const uint32_t s = it % kGgStages;
                     ok = gg_wait(smem_u32(full + s), (it / kGgStages) & 1, ab);
@@ -235,15 +254,16 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {      // 4 x (K = 16) inside the 64-wide block
                         const uint64_t bx = smem_desc_sw128(base + 2 * kGgTileBytes + ks * 32, 16, 1024);
-                        tc_mma_bf16(tmem + 0, smem_desc_sw128(base + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
-                        tc_mma_bf16(tmem + 64, smem_desc_sw128(base + kGgTileBytes + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
+                        tc_mma_bf16(acc, smem_desc_sw128(base + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
+                        tc_mma_bf16(acc + 64, smem_desc_sw128(base + kGgTileBytes + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
                     }
                     tc_commit(smem_u32(empty + s));
                 }
-                if (!ok) break;
-                tc_commit(smem_u32(acc1_full));
-                ok = gg_wait(smem_u32(act_full), nu & 1, ab);
-                if (!ok) break;
+                if (ok) tc_commit(smem_u32(acc1_full + b));
+            };
+            auto mma_phase2 = [&](int i) {
+                ok = gg_wait(smem_u32(act_full), i & 1, ab);
+                if (!ok) return;
                 tc_fence_after();
                 const uint32_t act_addr = smem_u32(act);
                 for (int dt = 0; dt < n_dt && ok; ++dt, ++it, ++nd) {
@@ -257,13 +277,17 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
                     for (int ks = 0; ks < 8; ++ks) {      // K = 16 rows j per step, 2048 bytes of each operand
                         const uint64_t da = smem_desc_sw128(base + ks * 2048, kGgTileBytes, 1024);
                         const uint64_t db = smem_desc_sw128(act_addr + ks * 2048, kGgActBytes, 1024);
-                        tc_mma_bf16(tmem + 128 + 64 * b, da, db, idesc2, ks != 0);
+                        tc_mma_bf16(tmem + 256 + 64 * b, da, db, idesc2, ks != 0);
                     }
                     tc_commit(smem_u32(empty + s));
                     tc_commit(smem_u32(acc2_full + b));
                 }
-                if (!ok) break;
-                tc_commit(smem_u32(act_empty));
+                if (ok) tc_commit(smem_u32(act_empty));
+            };
+            if (my_units > 0) mma_phase1(0);
+            for (int i = 0; i < my_units && ok; ++i) {
+                if (i + 1 < my_units) mma_phase1(i + 1);
+                if (ok) mma_phase2(i);
             }
         }
     } else {
@@ -272,18 +296,19 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
         const int row = q * 32 + lane;                  // accumulator row handled by this thread
         const uint32_t lane_addr = uint32_t(q * 32) << 16;
         float* wrow_s = wrow_all + q * kGgTokens;       // this warp's copy: no cross-warp barrier needed
-        uint32_t nu = 0, nd = 0;
+        uint32_t nd = 0;
         bool ok = true;
-        for (int u = blockIdx.x; u < a.n_units && ok; u += gridDim.x, ++nu) {
-            const GgUnit un = a.units[u];
+        for (int i = 0; i < my_units && ok; ++i) {
+            const GgUnit un = a.units[blockIdx.x + i * gridDim.x];
+            const uint32_t b1 = i & 1;
             // routing weights of this expert's token rows (0 beyond the real tokens)
             __syncwarp();
 #pragma unroll
-            for (int i = lane; i < kGgTokens; i += 32) wrow_s[i] = i < un.ntok ? a.wrow[un.row0 + i] : 0.f;
+            for (int t = lane; t < kGgTokens; t += 32) wrow_s[t] = t < un.ntok ? a.wrow[un.row0 + t] : 0.f;
             __syncwarp();
 
-            ok = gg_wait(smem_u32(acc1_full), nu & 1, ab);
-            if (ok && nu > 0) ok = gg_wait(smem_u32(act_empty), (nu - 1) & 1, ab);
+            ok = gg_wait(smem_u32(acc1_full + b1), (uint32_t(i) >> 1) & 1, ab);
+            if (ok && i > 0) ok = gg_wait(smem_u32(act_empty), (i - 1) & 1, ab);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -291,15 +316,15 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
 #pragma unroll
             for (int c = 0; c < kGgTokens / 16; ++c) {
                 float g[16], up[16];
-                tmem_ld16(tmem + lane_addr + c * 16, g);
-                tmem_ld16(tmem + lane_addr + 64 + c * 16, up);
+                tmem_ld16(tmem + lane_addr + 128 * b1 + c * 16, g);
+                tmem_ld16(tmem + lane_addr + 128 * b1 + 64 + c * 16, up);
                 uint32_t packed[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const float a0 = g[2 * i] / (1.f + expf(-g[2 * i])) * up[2 * i] * wrow_s[c * 16 + 2 * i];
-                    const float a1 = g[2 * i + 1] / (1.f + expf(-g[2 * i + 1])) * up[2 * i + 1] * wrow_s[c * 16 + 2 * i + 1];
+                for (int e = 0; e < 8; ++e) {
+                    const float a0 = g[2 * e] / (1.f + expf(-g[2 * e])) * up[2 * e] * wrow_s[c * 16 + 2 * e];
+                    const float a1 = g[2 * e + 1] / (1.f + expf(-g[2 * e + 1])) * up[2 * e + 1] * wrow_s[c * 16 + 2 * e + 1];
                     const __nv_bfloat162 p = __floats2bfloat162_rn(a0, a1);
-                    packed[i] = *reinterpret_cast<const uint32_t*>(&p);
+                    packed[e] = *reinterpret_cast<const uint32_t*>(&p);
                 }
                 unsigned char* rowp = act + row * 128;
                 *reinterpret_cast<uint4*>(rowp + (((2 * c) ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
@@ -308,7 +333,7 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
             fence_proxy_async();            // generic-proxy writes of A^T -> visible to the MMA's async reads
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) { mbar_arrive(smem_u32(acc1_empty)); mbar_arrive(smem_u32(act_full)); }
+            if (lane == 0) { mbar_arrive(smem_u32(acc1_empty + b1)); mbar_arrive(smem_u32(act_full)); }
 
             // phase 2: one [128 d x 64 tokens] accumulator per d-tile; store the real tokens' rows
             float* prow = a.partial + (size_t(un.jt) * a.rows_cap + un.row0) * D;
@@ -319,10 +344,10 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
                 tc_fence_after();
                 for (int c = 0; c * 16 < un.ntok; ++c) {
                     float y[16];
-                    tmem_ld16(tmem + lane_addr + 128 + 64 * b + c * 16, y);
+                    tmem_ld16(tmem + lane_addr + 256 + 64 * b + c * 16, y);
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        if (c * 16 + i < un.ntok) prow[size_t(c * 16 + i) * D + dt * kGgTileRows + row] = y[i];
+                    for (int e = 0; e < 16; ++e)
+                        if (c * 16 + e < un.ntok) prow[size_t(c * 16 + e) * D + dt * kGgTileRows + row] = y[e];
                 }
                 tc_fence_before();
                 __syncwarp();
