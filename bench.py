@@ -419,6 +419,8 @@ def resident_run(cfg, m, H_dev, W, K, peak, algo_bytes, device):
         full.prefetch_async(l, np.arange(cfg.n_experts, dtype=np.int32))
     full.synchronize()
     full.set_timing(1)
+    # host-driven leg: one host turn per layer, an event pair around every FFN kernel
+    full.set_host_free(0)
     timed_run(full, H_dev, 0, W, 1)
     full.reset_stats()
     el, _, _ = timed_run(full, H_dev, W, K, 1)
@@ -430,6 +432,25 @@ def resident_run(cfg, m, H_dev, W, K, peak, algo_bytes, device):
            "stall_us_per_layer": float(stall.sum() / (max(n, 1) * cfg.n_layers))}
     if cfg.batch == 1:
         out.update(ffn_gb_s=ach, ffn_frac_of_measured_peak=ach / peak)
+    # host-free leg: all layers enqueued without waiting for routing results, kernels launched
+    # ahead of their predecessor's end (no per-kernel events: the in-kernel window is reported)
+    full.set_host_free(1)
+    for policy in ("on_demand", "adapter"):
+        full.set_policy(policy)
+        timed_run(full, H_dev, 0, W, 1)
+        full.reset_stats()
+        el, _, _ = timed_run(full, H_dev, W, K, 1)
+        st = full.stats()
+        leg = {"tok_s": K * cfg.batch / (el / 1e3), "us_per_layer": el * 1e3 / (K * cfg.n_layers),
+               "host_free_steps": st["host_free_steps"], "misses": st["misses"]}
+        if st["host_free_steps"] and st["ffn_window_us"] > 0:
+            win = st["ffn_window_us"] / max(st["ffn_launches"], 1)
+            leg.update(ffn_window_us=win, ffn_gb_s_in_window=algo_bytes / (win * 1e-6) / 1e9,
+                       ffn_frac_in_window=algo_bytes / (win * 1e-6) / 1e9 / peak,
+                       hbm_bound_tok_s=peak * 1e9 / (algo_bytes * cfg.n_layers) * cfg.batch)
+        out["host_free_" + policy] = leg
+    full.set_policy("on_demand")
+    full.set_host_free(0)
     out["ffn_back_to_back"] = ffn_back_to_back(cfg, full, algo_bytes, peak)
     full.close()
     return out
@@ -483,10 +504,11 @@ def ffn_back_to_back(cfg, full, algo_bytes, peak, launches=480):
 
 def run_sweep(args):
     """Budget x cache-size sweep on the Qwen3-shaped model: for every slots-per-layer value the
-    on-demand arm, and per budget the adapter arm (the configuration's random adapters), a
-    gate-reuse adapter arm (informative predictor) and the perfect-knowledge arm."""
+    on-demand arm, and per budget the adapter arm (the configuration's random adapters), adapter
+    arms with structured stand-ins for trained weights (gate reuse, truncated SVD of the next
+    gate, reduced-rank regression on a calibration stream) and the perfect-knowledge arm."""
     from paper_2607_24787_b200.build import build
-    from paper_2607_24787_b200.synth_model import build_from_synth
+    from paper_2607_24787_b200.synth_model import build_from_synth, collect_router_io, fitted_adapters
     build()
     device = "cuda:0"
     torch.cuda.set_device(0)
@@ -497,8 +519,14 @@ def run_sweep(args):
     torch.cuda.synchronize()
     store, cells = None, []
     budgets = [int(b) for b in args.sweep_budgets.split(",")]
+    kinds = args.sweep_adapters.split(",")
+    if "random" not in kinds:
+        kinds.insert(0, "random")            # the on-demand and perfect-knowledge arms ride on this context
+    kinds.sort(key=lambda k: k != "random")
+    fitted = None
     for S in [int(x) for x in args.sweep_slots.split(",")]:
-        for adapter in ("random", "gate_reuse"):
+        for kind in kinds:
+            adapter = fitted if kind == "fit" else kind
             m = build_from_synth(cfg, slots=S, budget=1, device=device, store=store, adapter=adapter)
             store = m.store
             m.set_timing(1)
@@ -506,8 +534,14 @@ def run_sweep(args):
                 m.set_attention_stub_us(args.stub_us)
             if args.copy_delay_us:
                 m.set_copy_delay_us(args.copy_delay_us)
-            if adapter == "random":
+            if kind == "random":
                 window = m.profile_window()
+                if "fit" in kinds and fitted is None:
+                    # calibration stream independent of the evaluated one (its own generator stream)
+                    _, Hc = hidden_rows(cfg, args.calib_steps, stream=777)
+                    X, Z = collect_router_io(m, Hc.to(device))
+                    fitted = fitted_adapters(X, Z, cfg.adapter_rank, cfg.torch_dtype)
+                    del X, Z
 
             def arm(policy, budget, hint=None):
                 m.set_policy(policy); m.set_budget(budget)
@@ -517,16 +551,16 @@ def run_sweep(args):
                 timed_run(m, H_dev, 0, W, 1); m.reset_stats()
                 el, _, _ = timed_run(m, H_dev, W, K, 1)
                 out = arm_summary(m, cfg, el, K)
-                out.update(slots=S, budget=budget, policy=policy if adapter == "random" or policy != "adapter" else "adapter_gate_reuse")
+                out.update(slots=S, budget=budget, policy=policy if kind == "random" or policy != "adapter" else "adapter_" + kind)
                 return out
 
-            if adapter == "random":
+            if kind == "random":
                 cells.append(arm("on_demand", 0))
                 hint = [[[] for _ in range(cfg.n_layers)] for _ in range(W + K)]
                 m.set_policy("on_demand"); m.cache_reset()
                 timed_run(m, H_dev, 0, W + K, 1)
-                for (s_, l_, kind, e_, _) in m.events():
-                    if kind in ("HIT", "HIT_PREFETCHED", "MISS"):
+                for (s_, l_, kind_, e_, _) in m.events():
+                    if kind_ in ("HIT", "HIT_PREFETCHED", "MISS"):
                         hint[s_][l_].append(e_)
                 for b in budgets:
                     cells.append(arm("adapter", b))
@@ -661,6 +695,9 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="budget x slots sweep (prints one JSON object with all cells)")
     ap.add_argument("--sweep-budgets", default="1,2,4,8")
     ap.add_argument("--sweep-slots", default="8,16,32")
+    ap.add_argument("--sweep-adapters", default="random,gate_reuse,svd,fit",
+                    help="adapter weights per sweep arm: random (the configuration), gate_reuse, svd, fit")
+    ap.add_argument("--calib-steps", type=int, default=256, help="tokens of the calibration stream for --sweep-adapters fit")
     ap.add_argument("--stub-us", type=int, default=0,
                     help="attention stand-in of this many microseconds before each layer's router (widens the overlap window)")
     ap.add_argument("--copy-delay-us", type=int, default=0,

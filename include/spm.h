@@ -134,6 +134,7 @@ typedef struct {
     uint64_t ready_count;        /*   ... and the number of terms (ReadyRecall = ready_sum / ready_count) */
     double   recall_sum;         /* sum over (step, layer >= 1, token) of |T ∩ Top_M(s)| / K, M = budget  */
     uint64_t recall_count;       /*   ExpertRecall@M = recall_sum / recall_count  (Section 4.1)          */
+    uint64_t host_free_steps;    /* decode steps enqueued without a host turn (spm_set_host_free)        */
 } spm_stats;
 
 /* ---- packed expert layout ------------------------------------------------
@@ -239,6 +240,19 @@ int spm_set_copy_delay_us(spm_ctx* ctx, int us);
  * while missing ones are still in flight and no launch latency follows the last copy. Outputs are
  * bit-identical either way. With it on, the timed FFN duration includes the wait for copies. */
 int spm_set_device_wait(spm_ctx* ctx, int on);
+/* Host-free decode steps (default on). Once every expert of every layer holds a slot and every
+ * copy has landed (possible only with slots_per_layer >= n_experts), no routing result can change
+ * what the prefetch controller does: each demand is a hit and no selection finds a non-resident
+ * candidate (Section 3.3). spm_decode_step then enqueues all layers without waiting for any routing
+ * result: the routing kernel leaves the slot numbers of the chosen experts in device memory for the
+ * expert kernel that follows, each kernel is launched so that its preamble overlaps the end of its
+ * predecessor, and the ids / rankings go to a ring of host-mapped trace mailboxes from which the
+ * slot table's bookkeeping (hits, LRU ticks, recall statistics, event log) is replayed in order,
+ * at the latest when a call reads or changes that state. Outputs, events and statistics are the
+ * same as with the option off; per-layer event timings are not taken in such steps (the in-kernel
+ * window still is). Steps on the batched tensor-core path are never host-free.
+ * spm_cache_reset() ends the state; it is re-entered once the pools are full again. */
+int spm_set_host_free(spm_ctx* ctx, int on);
 /* Stand-in for the attention block the synthetic configurations omit: before each layer's router a
  * kernel that only waits `us` microseconds (0 = off, at most 100000) is enqueued on the compute
  * stream. It widens the overlap window W_l = t_exec(l+1) - t_pred(l) (Section 3.1) toward the

@@ -52,7 +52,8 @@ class Stats(C.Structure):
                                            "wasted", "prefetch_issued", "touches", "waves", "planned", "dropped",
                                            "late_arrivals", "h2d_bytes", "ffn_launches", "kernel_launches")]
                 + [("ffn_us", C.c_double), ("ffn_window_us", C.c_double), ("stall_us", C.c_double), ("ready_sum", C.c_double),
-                   ("ready_count", C.c_uint64), ("recall_sum", C.c_double), ("recall_count", C.c_uint64)])
+                   ("ready_count", C.c_uint64), ("recall_sum", C.c_double), ("recall_count", C.c_uint64),
+                   ("host_free_steps", C.c_uint64)])
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}
@@ -84,6 +85,7 @@ _SIG = {
     "spm_set_deadline_ms": [_P, C.c_int],
     "spm_set_attention_stub_us": [_P, C.c_int],
     "spm_set_device_wait": [_P, C.c_int],
+    "spm_set_host_free": [_P, C.c_int],
     "spm_set_copy_delay_us": [_P, C.c_int],
     "spm_profile_window": [_P, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int)],
     "spm_cache_reset": [_P],
@@ -271,6 +273,10 @@ def spm_set_copy_delay_us(ctx, us):
 
 def spm_set_device_wait(ctx, on):
     _check(load().spm_set_device_wait(ctx, int(on)), ctx)
+
+
+def spm_set_host_free(ctx, on):
+    _check(load().spm_set_host_free(ctx, int(on)), ctx)
 
 
 def spm_set_attention_stub_us(ctx, us):

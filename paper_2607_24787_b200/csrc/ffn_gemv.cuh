@@ -41,12 +41,28 @@ struct FfnArgs {
     int* status;
     unsigned long long* clock;      // optional {earliest CTA start, latest CTA end} in ns (globaltimer)
     const unsigned* ready;          // optional per-slot arrival counters of this pool (device-side wait)
+    const short* dev_code;          // optional [nb][K] slot numbers left in device memory by the routing kernel:
+                                    // the launch then needs no host knowledge of the routing (count/code/kidx unused;
+                                    // token t has K routed entries followed by the n_shared shared experts)
     unsigned want[SPM_MAX_TOPK];    // token 0 only: counter value at which entry k's slot holds its expert
     unsigned long long blob_bytes;
     int I, K, n_slots, n_shared;
     unsigned char count[MAXNB];                     // expert entries of token t in this launch
     short code[MAXNB * SPM_MAX_TOPK];               // >= 0: slot number; < 0: shared expert -1-s
     unsigned char kidx[MAXNB * SPM_MAX_TOPK];       // column of w[t][.]; 255: weight 1
+
+    __device__ __forceinline__ int entries(int tok) const { return dev_code ? K + n_shared : int(count[tok]); }
+    // slot code of entry `ent`; kBadCode when the device-side table names no slot
+    __device__ __forceinline__ int code_of(int tok, int ent) const {
+        if (!dev_code) return code[tok * SPM_MAX_TOPK + ent];
+        if (ent >= K) return -1 - (ent - K);
+        const int s = __ldcg(dev_code + tok * K + ent);
+        return s >= 0 ? s : (1 << 20);                  // no slot: fails the range check below
+    }
+    __device__ __forceinline__ int kidx_of(int tok, int ent) const {
+        if (!dev_code) return kidx[tok * SPM_MAX_TOPK + ent];
+        return ent < K ? ent : 255;
+    }
 };
 
 template <typename WT, int NSEG, int MAXNB>
@@ -61,13 +77,14 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
     const unsigned long long ts_start = global_timer_ns();
     unsigned long long ts_first = 0, ts_loop = 0;
 #endif
+    grid_dep_launch();
+    const unsigned long long t_entry = global_timer_ns();
     const int wi = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nw = blockDim.x >> 5;      // warps per CTA, chosen by the host to balance rows per warp
-    if (a.clock && threadIdx.x == 0) atomicMin(a.clock, global_timer_ns());
     const int tok = blockIdx.y;
     const int G = gridDim.x, c = blockIdx.x;
     const int I = a.I;
-    const int R = int(a.count[tok]) * I;
+    const int R = a.entries(tok) * I;
     const int r_begin = int((long long)R * c / G);
     const int r_end = int((long long)R * (c + 1) / G);
     const int span = r_end - r_begin - wi;
@@ -83,16 +100,22 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
         fence_barrier_init();
     }
     __syncwarp();
+    // everything above is independent of the preceding kernel; routing results are read below
+    grid_dep_wait();
+    // window start: kernel entry, or the end of the dependency wait when launched ahead of its predecessor's end
+    if (a.clock && threadIdx.x == 0) atomicMin(a.clock, a.dev_code ? global_timer_ns() : t_entry);
 
     const uint64_t pol = policy_evict_first();
     bool ok = true;
     unsigned arrived = 0;     // lane 0: entries whose slot is known to hold its expert
+    int code_ent = -1, code_val = 0;   // lane 0: slot code of the entry being streamed
 
     auto issue = [&](int i) {
         const int r = r_begin + wi + i * nw;
         const int ent = r / I;
         const int j = r - ent * I;
-        const int code = a.code[tok * SPM_MAX_TOPK + ent];
+        if (ent != code_ent) { code_ent = ent; code_val = a.code_of(tok, ent); }
+        const int code = code_val;
         const unsigned char* base;
         if (code >= 0) {
             if (code >= a.n_slots) { atomicOr(a.status, kStatusBadSlot); return false; }
@@ -170,7 +193,7 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
             const int ent = r / I;
             if (ent != cur_ent) {
                 cur_ent = ent;
-                const int kk = a.kidx[tok * SPM_MAX_TOPK + ent];
+                const int kk = a.kidx_of(tok, ent);
                 wk = kk == 255 ? 1.f : a.w[size_t(tok) * a.K + kk];
             }
             const unsigned char* buf = ring + size_t(st) * ROWB;
@@ -256,6 +279,8 @@ constexpr int kReduceMaxRows = 40;     // rows per group: kReduceGroups * kReduc
 static __global__ void __launch_bounds__(kReduceCols * kReduceGroups)
 ffn_reduce_kernel(const float* __restrict__ partial, const float* h_in, float* h_out, int G, int D) {
     __shared__ float part[kReduceGroups][kReduceCols];
+    grid_dep_launch();
+    grid_dep_wait();
     const int tok = blockIdx.y;
     const int col = threadIdx.x % kReduceCols, grp = threadIdx.x / kReduceCols;
     const int d = blockIdx.x * kReduceCols + col;

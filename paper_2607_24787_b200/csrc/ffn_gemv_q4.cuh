@@ -40,16 +40,17 @@ template <int NCH, int MAXNB>     // NCH = 16-byte nibble chunks (groups of 32 w
 __global__ void __launch_bounds__(kQ4MaxWarps * 32, 1)
 ffn_gemv_q4_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth, const int D) {
     extern __shared__ __align__(128) unsigned char smem[];
+    grid_dep_launch();
+    const unsigned long long t_entry = global_timer_ns();
     const int wi = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nw = blockDim.x >> 5;
-    if (a.clock && threadIdx.x == 0) atomicMin(a.clock, global_timer_ns());
     const int tok = blockIdx.y;
     const int G = gridDim.x, c = blockIdx.x;
     const int I = a.I;
     const int n_grp = D / 32;                         // groups per row
     const uint32_t RB = uint32_t(D / 2 + D / 16);     // bytes of one packed row
     const uint32_t ROWB = 3u * RB;
-    const int R = int(a.count[tok]) * I;
+    const int R = a.entries(tok) * I;
     const int r_begin = int((long long)R * c / G);
     const int r_end = int((long long)R * (c + 1) / G);
     const int span = r_end - r_begin - wi;
@@ -68,14 +69,19 @@ ffn_gemv_q4_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth, co
         fence_barrier_init();
     }
     __syncwarp();
+    grid_dep_wait();          // routing results (slot codes, activations, weights) are read from here on
+    // window start: kernel entry, or the end of the dependency wait when launched ahead of its predecessor's end
+    if (a.clock && threadIdx.x == 0) atomicMin(a.clock, a.dev_code ? global_timer_ns() : t_entry);
 
     const uint64_t pol = policy_evict_first();
     bool ok = true;
+    int code_ent = -1, code_val = 0;
     auto issue = [&](int i) {
         const int r = r_begin + wi + i * nw;
         const int ent = r / I;
         const int j = r - ent * I;
-        const int code = a.code[tok * SPM_MAX_TOPK + ent];
+        if (ent != code_ent) { code_ent = ent; code_val = a.code_of(tok, ent); }
+        const int code = code_val;
         const unsigned char* base;
         if (code >= 0) {
             if (code >= a.n_slots) { atomicOr(a.status, kStatusBadSlot); return false; }
@@ -124,7 +130,7 @@ ffn_gemv_q4_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth, co
             const int ent = r / I;
             if (ent != cur_ent) {
                 cur_ent = ent;
-                const int kk = a.kidx[tok * SPM_MAX_TOPK + ent];
+                const int kk = a.kidx_of(tok, ent);
                 wk = kk == 255 ? 1.f : a.w[size_t(tok) * a.K + kk];
             }
             const unsigned char* buf = ring + size_t(st) * ROWB;

@@ -52,7 +52,8 @@ struct GgUnit {
 
 struct GgArgs {
     const GgUnit* units;
-    int n_units;
+    int n_units;           // ... or, when n_units_dev is set, read from device memory (plan built on the device)
+    const int* n_units_dev;
     const float* wrow;     // [rows] routing weight of each sorted token row
     float* partial;        // [I/128][rows_cap][D]
     int rows_cap;
@@ -166,11 +167,11 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     float* wrow_all = reinterpret_cast<float*>(tmem_slot + 4);      // [4 epilogue warps][64]
 
+    grid_dep_launch();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int D = a.D;
     const int n_kb = D / kGgKBlock;            // phase-1 stages per unit
     const int n_dt = D / kGgTileRows;          // phase-2 stages per unit
-    const int my_units = blockIdx.x < a.n_units ? (a.n_units - 1 - int(blockIdx.x)) / int(gridDim.x) + 1 : 0;
     GgAbort ab{abort_flag, a.status};
 
     if (threadIdx.x == 0) {
@@ -191,6 +192,10 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    // barriers and TMEM are set up; everything below reads what the preceding kernels wrote
+    grid_dep_wait();
+    const int n_units = a.n_units_dev ? __ldcg(a.n_units_dev) : a.n_units;
+    const int my_units = int(blockIdx.x) < n_units ? (n_units - 1 - int(blockIdx.x)) / int(gridDim.x) + 1 : 0;
 
     // Order of work, identical for the producer and the MMA issuer:
     //   phase1(0), then for i = 0, 1, ...: phase1(i + 1) if it exists, phase2(i).
@@ -370,7 +375,11 @@ inline size_t ffn_grouped_smem() {
 struct GgRow { int32_t token, k; };
 
 static __global__ void gg_gather_kernel(const float* __restrict__ x, const float* __restrict__ w, const GgRow* __restrict__ rows,
-                                        int n_rows, int D, int K, __nv_bfloat16* __restrict__ xs, float* __restrict__ wrow) {
+                                        int n_rows, const int* n_rows_dev, int D, int K, __nv_bfloat16* __restrict__ xs,
+                                        float* __restrict__ wrow) {
+    grid_dep_launch();
+    grid_dep_wait();
+    if (n_rows_dev) n_rows = __ldcg(n_rows_dev);
     const int r = blockIdx.x;
     if (r >= n_rows) return;
     const GgRow ri = rows[r];
@@ -391,6 +400,8 @@ static __global__ void gg_gather_kernel(const float* __restrict__ x, const float
 // P[jt][rowmap[t][k]][d]; rowmap < 0 marks experts that belong to another wave.
 static __global__ void gg_combine_kernel(const float* __restrict__ partial, const int32_t* __restrict__ rowmap, int K, int n_jt,
                                          int rows_cap, int D, float* h) {
+    grid_dep_launch();
+    grid_dep_wait();
     const int t = blockIdx.y;
     const int d = blockIdx.x * blockDim.x + threadIdx.x;
     if (d >= D) return;
@@ -401,6 +412,62 @@ static __global__ void gg_combine_kernel(const float* __restrict__ partial, cons
         for (int jt = 0; jt < n_jt; ++jt) acc += __ldcg(partial + (size_t(jt) * rows_cap + r) * D + d);
     }
     h[size_t(t) * D + d] += acc;
+}
+
+
+// Wave plan built on the device (all experts resident, one wave): the (token, k) pairs sorted by
+// expert id, then token, then k — the order the host-side planner produces — the units of every
+// routed expert, and the row of each pair for the combine step. One CTA; thread e owns expert e.
+constexpr int kGgPlanThreads = 1024;
+
+static __global__ void __launch_bounds__(kGgPlanThreads)
+gg_plan_kernel(const int32_t* __restrict__ ids, const short* __restrict__ slot_map, int slot_base, int nb, int K, int n,
+               int n_jt, GgUnit* __restrict__ units, GgRow* __restrict__ rows, int32_t* __restrict__ rowmap,
+               int* __restrict__ counts /* {n_units, n_rows} */, int* status) {
+    extern __shared__ int32_t plan_sm[];
+    int32_t* s_ids = plan_sm;                  // [nb * K]
+    int32_t* s_cnt = s_ids + nb * K;           // [n] pairs per expert -> first row
+    int32_t* s_rank = s_cnt + n;               // [n] routed experts before e
+    grid_dep_launch();
+    grid_dep_wait();
+    const int tid = threadIdx.x, total = nb * K;
+    for (int i = tid; i < total; i += blockDim.x) s_ids[i] = __ldcg(ids + i);
+    for (int i = tid; i < nb * SPM_MAX_TOPK; i += blockDim.x) rowmap[i] = -1;
+    __syncthreads();
+    for (int e = tid; e < n; e += blockDim.x) {
+        int cnt = 0;
+        for (int i = 0; i < total; ++i) cnt += s_ids[i] == e;
+        s_cnt[e] = cnt;
+    }
+    __syncthreads();
+    if (tid == 0) {          // exclusive scans over at most SPM_MAX_EXPERTS entries
+        int row = 0, routed = 0;
+        for (int e = 0; e < n; ++e) {
+            const int cnt = s_cnt[e];
+            s_cnt[e] = row;
+            s_rank[e] = cnt > 0 ? routed : -1;
+            row += cnt;
+            routed += cnt > 0;
+        }
+        counts[0] = routed * n_jt;
+        counts[1] = row;
+    }
+    __syncthreads();
+    for (int e = tid; e < n; e += blockDim.x) {
+        if (s_rank[e] < 0) continue;
+        const int row0 = s_cnt[e];
+        int r = row0;
+        for (int i = 0; i < total; ++i)
+            if (s_ids[i] == e) {
+                const int t = i / K, k = i - t * K;
+                rows[r] = GgRow{t, k};
+                rowmap[t * SPM_MAX_TOPK + k] = r;
+                ++r;
+            }
+        const int slot = slot_map[e];
+        if (slot < 0) atomicOr(status, kStatusBadSlot);
+        for (int jt = 0; jt < n_jt; ++jt) units[s_rank[e] * n_jt + jt] = GgUnit{slot_base + (slot < 0 ? 0 : slot), jt, row0, r - row0};
+    }
 }
 
 }  // namespace spm

@@ -65,6 +65,13 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     }
 }
 
+// Programmatic dependent launch. A kernel launched with the programmatic-serialisation attribute
+// may begin before the preceding kernel of its stream has finished; grid_dep_wait() returns once
+// that kernel has completed and its writes are visible (at once in an ordinary launch).
+// grid_dep_launch() lets the next kernel of the stream begin its own preamble early.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ uint64_t policy_evict_first() {
     uint64_t p;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));

@@ -50,7 +50,9 @@ struct RouterArgs {
     float* scores;           // out [n]
     int32_t* order;          // out [n]
     unsigned* counters;      // [1] token-leader ticket, zero between launches
-    Mailbox* mailbox;        // device view of the host-mapped mailbox
+    Mailbox* mailbox;        // device view of a host-mapped mailbox (may be null)
+    const short* slot_map;   // optional [n] slot of each expert of this layer (device memory) ...
+    short* codes_out;        // ... and where to leave the slots of the routed experts, [nb][K]
     uint32_t seq;
     int D, n, K, r, nb, renorm, do_router, do_adapter;
     float eps;
@@ -196,28 +198,59 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     const int D = a.D, n = a.n;
     const uint32_t tag = a.seq & 0xffffu;
 
+    grid_dep_launch();
     // every CTA of the cluster must be running before anyone writes into the leader's shared
     // memory: arrive now, wait just before the first remote store
     asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
 
-    // ---- router input: hidden row and gain are fetched together, then normalised -----------
+    // ---- weights first: none of them depends on the kernel before this one, so in a launch that
+    // overlaps its predecessor they are already in registers when the hidden row becomes readable.
+    // Router rows then adapter-A rows, one warp per row, ROWS rows in flight.
+    const int n_r = a.do_router ? n : 0;
+    const int rows = n_r + (a.do_adapter ? a.r : 0);
+    constexpr int STRIDE = kRouterCluster * kRouterWarps;
+    uint4 v[ROWS][MAXIT];
+    auto load_rows = [&](int row0) {
+#pragma unroll
+        for (int rr = 0; rr < ROWS; ++rr) {
+            const int row = row0 + rr * STRIDE;
+            if (row < rows) {
+                const WT* wrow = row < n_r ? static_cast<const WT*>(a.router_w) + size_t(row) * D
+                                           : static_cast<const WT*>(a.adapter_a) + size_t(row - n_r) * D;
+#pragma unroll
+                for (int it = 0; it < MAXIT; ++it) {
+                    const int i = (it * 32 + lane) * VEC;
+                    if (i < D) v[rr][it] = __ldg(reinterpret_cast<const uint4*>(wrow + i));
+                }
+            }
+        }
+    };
+    int row0 = int(cr) * kRouterWarps + wi;
+    load_rows(row0);
+    constexpr int NV4 = MAXIT * 32 * VEC / (kRouterThreads * 4);   // float4 per thread at the largest hidden size
+    float4 gv[NV4];
     if (a.do_router) {
-        const float* ht = a.h + size_t(tok) * D;
-        constexpr int NV4 = MAXIT * 32 * VEC / (kRouterThreads * 4);   // float4 per thread at the largest hidden size
-        float4 hv[NV4], gv[NV4];
 #pragma unroll
         for (int c = 0; c < NV4; ++c) {
             const int i = (c * kRouterThreads + threadIdx.x) * 4;
-            if (i < D) {
-                hv[c] = *reinterpret_cast<const float4*>(ht + i);
-                gv[c] = *reinterpret_cast<const float4*>(a.gamma + i);
-            }
+            if (i < D) gv[c] = *reinterpret_cast<const float4*>(a.gamma + i);
         }
-        // leader: the small adapter up-projection is needed only in the tail; fetch it while the
-        // row and gain are in flight
-        if (leader && a.do_adapter) {
-            const WT* B = static_cast<const WT*>(a.adapter_b);
-            for (int i = threadIdx.x; i < n * a.r; i += kRouterThreads) bs[i] = load_weight(B, i);
+    }
+    // leader: the small adapter up-projection is needed only in the tail
+    if (leader && a.do_adapter) {
+        const WT* B = static_cast<const WT*>(a.adapter_b);
+        for (int i = threadIdx.x; i < n * a.r; i += kRouterThreads) bs[i] = load_weight(B, i);
+    }
+
+    // ---- router input: the hidden row (written by the preceding kernel) is normalised ----------
+    grid_dep_wait();
+    if (a.do_router) {
+        const float* ht = a.h + size_t(tok) * D;
+        float4 hv[NV4];
+#pragma unroll
+        for (int c = 0; c < NV4; ++c) {
+            const int i = (c * kRouterThreads + threadIdx.x) * 4;
+            if (i < D) hv[c] = *reinterpret_cast<const float4*>(ht + i);
         }
         float ss = 0.f;
 #pragma unroll
@@ -244,34 +277,12 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     } else {
         const float* xt = a.x_in + size_t(tok) * D;
         for (int i = threadIdx.x; i < D; i += kRouterThreads) xs[i] = xt[i];
-        if (leader && a.do_adapter) {
-            const WT* B = static_cast<const WT*>(a.adapter_b);
-            for (int i = threadIdx.x; i < n * a.r; i += kRouterThreads) bs[i] = load_weight(B, i);
-        }
     }
     __syncthreads();
     SPM_TS(1);
 
-    // ---- weight rows: router rows then adapter-A rows, one warp per row, ROWS rows in flight ----
-    const int n_r = a.do_router ? n : 0;
-    const int rows = n_r + (a.do_adapter ? a.r : 0);
-    constexpr int STRIDE = kRouterCluster * kRouterWarps;
     asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
-    for (int row0 = int(cr) * kRouterWarps + wi; row0 < rows; row0 += ROWS * STRIDE) {
-        uint4 v[ROWS][MAXIT];
-#pragma unroll
-        for (int rr = 0; rr < ROWS; ++rr) {
-            const int row = row0 + rr * STRIDE;
-            if (row < rows) {
-                const WT* wrow = row < n_r ? static_cast<const WT*>(a.router_w) + size_t(row) * D
-                                           : static_cast<const WT*>(a.adapter_a) + size_t(row - n_r) * D;
-#pragma unroll
-                for (int it = 0; it < MAXIT; ++it) {
-                    const int i = (it * 32 + lane) * VEC;
-                    if (i < D) v[rr][it] = __ldg(reinterpret_cast<const uint4*>(wrow + i));
-                }
-            }
-        }
+    while (row0 < rows) {
 #pragma unroll
         for (int rr = 0; rr < ROWS; ++rr) {
             const int row = row0 + rr * STRIDE;
@@ -291,6 +302,8 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
                 if (lane == 0) dsmem_store(row < n_r ? zs + row : us + (row - n_r), 0, acc);
             }
         }
+        row0 += ROWS * STRIDE;
+        if (row0 < rows) load_rows(row0);
     }
     SPM_TS(2);
     cluster_sync_all();
@@ -323,7 +336,9 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
         if (ht < a.K) {
             a.ids[size_t(tok) * a.K + ht] = isel[ht];
             a.w[size_t(tok) * a.K + ht] = a.renorm ? psel[ht] / s_tot : psel[ht];
-            mb->ids[tok * a.K + ht] = tagged(tag, isel[ht]);      // the host may start on these at once
+            if (mb) mb->ids[tok * a.K + ht] = tagged(tag, isel[ht]);      // the host may start on these at once
+            // slot numbers for an expert kernel that follows without a host turn
+            if (a.codes_out) a.codes_out[tok * a.K + ht] = a.slot_map[isel[ht]];
         }
     }
     SPM_TS(4);
@@ -342,8 +357,7 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
                 const int rk = rank_of(qs, n, e);
                 a.order[rk] = e;
                 a.scores[e] = qs[e];
-                mb->order[rk] = tagged(tag, e);
-                mb->scores[e] = qs[e];
+                if (mb) { mb->order[rk] = tagged(tag, e); mb->scores[e] = qs[e]; }
             }
         }
     }
@@ -368,8 +382,7 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
                 const int rk = rank_of(qs, n, e);
                 a.order[rk] = e;
                 a.scores[e] = qs[e];
-                mb->order[rk] = tagged(tag, e);
-                mb->scores[e] = qs[e];
+                if (mb) { mb->order[rk] = tagged(tag, e); mb->scores[e] = qs[e]; }
             }
         }
         if (threadIdx.x == 0) a.counters[0] = 0u;
@@ -378,7 +391,7 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     // final flag for callers that read untagged payload (scores): fence, then the sequence number
     __threadfence_system();
     __syncthreads();
-    if (threadIdx.x == 0) mb->seq = a.seq;
+    if (threadIdx.x == 0 && mb) mb->seq = a.seq;
 #ifdef SPM_ROUTER_TIMESTAMPS
     SPM_TS(7);
     if (threadIdx.x == 0) for (int i = 0; i < 8; ++i) reinterpret_cast<unsigned long long*>(a.pihat)[i] = ts[i];

@@ -7,7 +7,9 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <deque>
 #include <string>
+#include <utility>
 #include <vector>
 
 #include <cuda_runtime.h>
@@ -65,6 +67,7 @@ struct spm_ctx {
     float *tc_wrow = nullptr, *tc_partial = nullptr;
     unsigned char* tc_desc_dev = nullptr;     // kDescRing wave descriptors
     unsigned char* tc_desc_host = nullptr;    // pinned staging, same layout
+    int* tc_counts = nullptr;                 // {units, rows} of a wave planned on the device
     size_t tc_desc_bytes = 0, tc_off_rows = 0, tc_off_rowmap = 0;
     std::vector<cudaEvent_t> tc_desc_ev;
     std::vector<uint8_t> tc_desc_ev_valid;
@@ -101,6 +104,18 @@ struct spm_ctx {
     bool device_wait = false;                 // batch-1 FFN launched at once, waits for its copies on the device
     unsigned* ws_slot_gen = nullptr;          // [L][S] arrival counters, bumped by the copy stream
     std::vector<uint32_t> slot_gen_host;      // value the counter will hold once the latest copy has landed
+    // host-free steps: once every expert of every layer is resident, a step is enqueued without
+    // waiting for any routing result; the routing kernel leaves slot numbers for the expert kernel
+    // in device memory and its ids / ranking in a ring of host-mapped trace mailboxes, from which
+    // the slot table's bookkeeping is replayed later, in order
+    bool host_free = true, fast_ready = false;
+    short* ws_slot_map = nullptr;             // [L][n] slot of each expert (valid while fast_ready)
+    short* ws_codes = nullptr;                // [L][max_batch][K] slots of the routed experts of the step in flight
+    Mailbox* tr_host = nullptr;               // [kTraceRing][L]
+    Mailbox* tr_dev = nullptr;
+    std::vector<cudaEvent_t> tr_ev;
+    std::deque<std::pair<int, int>> tr_pending;   // (ring slot, nb) of steps enqueued but not yet replayed
+    uint64_t tr_count = 0, host_free_steps = 0;
     std::vector<std::vector<int32_t>> prev_rank;   // Naive Prefetch: experts the preceding step used, per layer
     std::vector<std::vector<int32_t>> pending_protect;
     std::vector<uint8_t> has_plan;
@@ -162,6 +177,7 @@ size_t blob_bytes_of(const spm_model_cfg* m) {
 constexpr int kMaxCtasBatch1 = 296;
 constexpr int kClockSlots = 4096;     // in-kernel {start, end} pairs between two harvests
 constexpr int kDescRing = 8;          // wave descriptors in flight for the batched tensor-core path
+constexpr int kTraceRing = 8;         // host-free steps whose bookkeeping may be outstanding
 
 // The grouped tcgen05 kernel handles bf16 weights, more than one sequence per step, no shared
 // experts, and intermediate / hidden sizes that tile by 128.
@@ -182,8 +198,8 @@ struct Carve {
 };
 
 struct Layout {
-    size_t pools, slot_gen, x, logits, pihat, w, scores, partial, h, ids, order, clock, counters, status, total;
-    size_t tc_xs, tc_wrow, tc_partial, tc_desc;       // batched tensor-core path only
+    size_t pools, slot_gen, x, logits, pihat, w, scores, partial, h, ids, order, clock, slot_map, codes, counters, status, total;
+    size_t tc_xs, tc_wrow, tc_partial, tc_desc, tc_counts;       // batched tensor-core path only
     size_t desc_bytes, off_rows, off_rowmap;
     int rows_cap, n_jt, max_units;
     bool tc;
@@ -205,6 +221,8 @@ Layout layout_of(const spm_model_cfg* m, int S) {
     l.ids = c.take(nb * SPM_MAX_TOPK * 4);
     l.order = c.take(n * 4);
     l.clock = c.take(size_t(kClockSlots) * 16);
+    l.slot_map = c.take(size_t(m->n_layers) * n * sizeof(short));
+    l.codes = c.take(size_t(m->n_layers) * nb * SPM_MAX_TOPK * sizeof(short));
     l.tc = tc_supported(m);
     if (l.tc) {
         l.rows_cap = m->max_batch * m->top_k;
@@ -217,6 +235,7 @@ Layout layout_of(const spm_model_cfg* m, int S) {
         l.tc_wrow = c.take(size_t(l.rows_cap) * 4);
         l.tc_partial = c.take(size_t(l.n_jt) * l.rows_cap * D * 4);
         l.tc_desc = c.take(size_t(kDescRing) * l.desc_bytes);
+        l.tc_counts = c.take(2 * sizeof(int));
     }
     l.counters = c.take(256);
     l.status = c.take(4);
@@ -225,8 +244,27 @@ Layout layout_of(const spm_model_cfg* m, int S) {
 }
 
 // ---- kernel dispatch -------------------------------------------------------
+// Launch with an optional programmatic-serialisation attribute: the kernel may then start while
+// the preceding kernel of the stream is still running and orders itself with grid_dep_wait().
+template <typename... KArgs, typename... Args>
+cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl, Args&&... args) {
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = grid;
+    lc.blockDim = block;
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    cudaLaunchAttribute at[1];
+    if (pdl) {
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = at;
+        lc.numAttrs = 1;
+    }
+    return cudaLaunchKernelEx(&lc, kern, std::forward<Args>(args)...);
+}
+
 template <typename WT, int NSEG, int MAXNB>
-cudaError_t launch_gemv_t(const FfnArgs<MAXNB>& a, int G, int nb, int warps, int depth, size_t smem, cudaStream_t st) {
+cudaError_t launch_gemv_t(const FfnArgs<MAXNB>& a, int G, int nb, int warps, int depth, size_t smem, cudaStream_t st, bool pdl) {
     static bool attr_set[64] = {};          // the attribute is per device
     auto kern = ffn_gemv_kernel<WT, NSEG, MAXNB>;
     int dev = 0;
@@ -236,27 +274,26 @@ cudaError_t launch_gemv_t(const FfnArgs<MAXNB>& a, int G, int nb, int warps, int
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    kern<<<dim3(G, nb), warps * 32, smem, st>>>(a, depth);
-    return cudaGetLastError();
+    return launch_k(kern, dim3(G, nb), dim3(warps * 32), smem, st, pdl, a, depth);
 }
 
 template <typename WT, int MAXNB>
-cudaError_t launch_gemv_seg(int nseg, const FfnArgs<MAXNB>& a, int G, int nb, int warps, int depth, size_t smem, cudaStream_t st) {
+cudaError_t launch_gemv_seg(int nseg, const FfnArgs<MAXNB>& a, int G, int nb, int warps, int depth, size_t smem, cudaStream_t st, bool pdl) {
     switch (nseg) {
-        case 1: return launch_gemv_t<WT, 1, MAXNB>(a, G, nb, warps, depth, smem, st);
-        case 2: return launch_gemv_t<WT, 2, MAXNB>(a, G, nb, warps, depth, smem, st);
-        case 3: return launch_gemv_t<WT, 3, MAXNB>(a, G, nb, warps, depth, smem, st);
-        case 4: return launch_gemv_t<WT, 4, MAXNB>(a, G, nb, warps, depth, smem, st);
-        case 5: return launch_gemv_t<WT, 5, MAXNB>(a, G, nb, warps, depth, smem, st);
-        case 6: return launch_gemv_t<WT, 6, MAXNB>(a, G, nb, warps, depth, smem, st);
-        case 7: return launch_gemv_t<WT, 7, MAXNB>(a, G, nb, warps, depth, smem, st);
-        case 8: return launch_gemv_t<WT, 8, MAXNB>(a, G, nb, warps, depth, smem, st);
+        case 1: return launch_gemv_t<WT, 1, MAXNB>(a, G, nb, warps, depth, smem, st, pdl);
+        case 2: return launch_gemv_t<WT, 2, MAXNB>(a, G, nb, warps, depth, smem, st, pdl);
+        case 3: return launch_gemv_t<WT, 3, MAXNB>(a, G, nb, warps, depth, smem, st, pdl);
+        case 4: return launch_gemv_t<WT, 4, MAXNB>(a, G, nb, warps, depth, smem, st, pdl);
+        case 5: return launch_gemv_t<WT, 5, MAXNB>(a, G, nb, warps, depth, smem, st, pdl);
+        case 6: return launch_gemv_t<WT, 6, MAXNB>(a, G, nb, warps, depth, smem, st, pdl);
+        case 7: return launch_gemv_t<WT, 7, MAXNB>(a, G, nb, warps, depth, smem, st, pdl);
+        case 8: return launch_gemv_t<WT, 8, MAXNB>(a, G, nb, warps, depth, smem, st, pdl);
     }
     return cudaErrorInvalidValue;
 }
 
 template <int NCH, int MAXNB>
-cudaError_t launch_gemv_q4_t(int D, const FfnArgs<MAXNB>& a, int G, int nb, int warps, int depth, size_t smem, cudaStream_t st) {
+cudaError_t launch_gemv_q4_t(int D, const FfnArgs<MAXNB>& a, int G, int nb, int warps, int depth, size_t smem, cudaStream_t st, bool pdl) {
     static bool attr_set[64] = {};
     auto kern = ffn_gemv_q4_kernel<NCH, MAXNB>;
     int dev = 0;
@@ -266,18 +303,17 @@ cudaError_t launch_gemv_q4_t(int D, const FfnArgs<MAXNB>& a, int G, int nb, int 
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    kern<<<dim3(G, nb), warps * 32, smem, st>>>(a, depth, D);
-    return cudaGetLastError();
+    return launch_k(kern, dim3(G, nb), dim3(warps * 32), smem, st, pdl, a, depth, D);
 }
 
 template <int MAXNB>
-cudaError_t launch_gemv_q4(int D, const FfnArgs<MAXNB>& a, int G, int nb, int warps, int depth, size_t smem, cudaStream_t st) {
-    if (D <= 1024) return launch_gemv_q4_t<1, MAXNB>(D, a, G, nb, warps, depth, smem, st);
-    return launch_gemv_q4_t<2, MAXNB>(D, a, G, nb, warps, depth, smem, st);
+cudaError_t launch_gemv_q4(int D, const FfnArgs<MAXNB>& a, int G, int nb, int warps, int depth, size_t smem, cudaStream_t st, bool pdl) {
+    if (D <= 1024) return launch_gemv_q4_t<1, MAXNB>(D, a, G, nb, warps, depth, smem, st, pdl);
+    return launch_gemv_q4_t<2, MAXNB>(D, a, G, nb, warps, depth, smem, st, pdl);
 }
 
 template <int MAXNB>
-cudaError_t launch_gemv(const spm_ctx* c, const FfnArgs<MAXNB>& a, int G, int nb) {
+cudaError_t launch_gemv(const spm_ctx* c, const FfnArgs<MAXNB>& a, int G, int nb, bool pdl = false) {
     int max_cnt = 1;
     for (int t = 0; t < nb; ++t) max_cnt = std::max(max_cnt, int(a.count[t]));
     const int rows_per_cta = (max_cnt * c->cfg.inter + G - 1) / G;
@@ -285,16 +321,26 @@ cudaError_t launch_gemv(const spm_ctx* c, const FfnArgs<MAXNB>& a, int G, int nb
     if (c->cfg.dtype == SPM_DTYPE_Q4) {
         size_t smem = 0;
         ffn_gemv_q4_shape(c->row_bytes, c->cfg.hidden, rows_per_cta, &warps, &depth, &smem);
-        return launch_gemv_q4<MAXNB>(c->cfg.hidden, a, G, nb, warps, depth, smem, c->compute);
+        return launch_gemv_q4<MAXNB>(c->cfg.hidden, a, G, nb, warps, depth, smem, c->compute, pdl);
     }
     ffn_gemv_shape(c->row_bytes, rows_per_cta, &warps, &depth);
     const size_t smem = ffn_gemv_smem(c->row_bytes, warps, depth);
-    if (c->cfg.dtype == SPM_DTYPE_BF16) return launch_gemv_seg<bf16_t, MAXNB>(c->nseg, a, G, nb, warps, depth, smem, c->compute);
-    return launch_gemv_seg<float, MAXNB>(c->nseg, a, G, nb, warps, depth, smem, c->compute);
+    if (c->cfg.dtype == SPM_DTYPE_BF16) return launch_gemv_seg<bf16_t, MAXNB>(c->nseg, a, G, nb, warps, depth, smem, c->compute, pdl);
+    return launch_gemv_seg<float, MAXNB>(c->nseg, a, G, nb, warps, depth, smem, c->compute, pdl);
 }
 
+// Where a routing launch leaves its results besides the workspace: by default the context's
+// mailbox, which the host polls; a host-free step names a trace mailbox, the device-side slot
+// map and the slot-code row of its layer, and lets the kernel start ahead of its predecessor's end.
+struct RouterRoute {
+    Mailbox* mailbox_dev;
+    const short* slot_map;
+    short* codes_out;
+    bool pdl;
+};
+
 int launch_router(spm_ctx* c, int layer, const float* h, const float* x_in, int nb, float* x_norm,
-                  float* logits_out, bool do_router, bool do_adapter) {
+                  float* logits_out, bool do_router, bool do_adapter, const RouterRoute* route = nullptr) {
     const spm_model_cfg& m = c->cfg;
     RouterArgs a{};
     const size_t D = m.hidden, n = m.n_experts, r = m.adapter_rank;
@@ -315,13 +361,17 @@ int launch_router(spm_ctx* c, int layer, const float* h, const float* x_in, int 
     a.scores = c->ws_scores;
     a.order = c->ws_order;
     a.counters = c->ws_counters;
-    a.mailbox = c->mb_dev;
+    a.mailbox = route ? route->mailbox_dev : c->mb_dev;
+    a.slot_map = route ? route->slot_map : nullptr;
+    a.codes_out = route ? route->codes_out : nullptr;
     // Sequence numbers whose low 16 bits are zero are skipped, and the words this launch will
     // publish are zeroed first, so a word left by an older launch can never carry the current tag.
     ++c->seq;
     if ((c->seq & 0xffffu) == 0) ++c->seq;
-    if (do_router) memset(const_cast<int32_t*>(c->mb_host->ids), 0, size_t(nb) * m.top_k * sizeof(int32_t));
-    if (do_adapter) memset(const_cast<int32_t*>(c->mb_host->order), 0, size_t(m.n_experts) * sizeof(int32_t));
+    if (!route) {
+        if (do_router) memset(const_cast<int32_t*>(c->mb_host->ids), 0, size_t(nb) * m.top_k * sizeof(int32_t));
+        if (do_adapter) memset(const_cast<int32_t*>(c->mb_host->order), 0, size_t(m.n_experts) * sizeof(int32_t));
+    }
     a.seq = c->seq;
     a.D = m.hidden; a.n = m.n_experts; a.K = m.top_k; a.r = m.adapter_rank; a.nb = nb;
     a.renorm = m.renormalize; a.do_router = do_router; a.do_adapter = do_adapter;
@@ -332,13 +382,18 @@ int launch_router(spm_ctx* c, int layer, const float* h, const float* x_in, int 
     lc.blockDim = dim3(kRouterThreads);
     lc.dynamicSmemBytes = smem;
     lc.stream = c->compute;
-    cudaLaunchAttribute at[1];
+    cudaLaunchAttribute at[2];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = kRouterCluster;
     at[0].val.clusterDim.y = 1;
     at[0].val.clusterDim.z = 1;
     lc.attrs = at;
     lc.numAttrs = 1;
+    if (route && route->pdl) {
+        at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[1].val.programmaticStreamSerializationAllowed = 1;
+        lc.numAttrs = 2;
+    }
     if (m.dtype != SPM_DTYPE_FP32) {
         if (smem > 48 * 1024) CU(c, cudaFuncSetAttribute(router_adapter_kernel<bf16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
         CU(c, cudaLaunchKernelEx(&lc, router_adapter_kernel<bf16_t>, a));
@@ -519,11 +574,11 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
     CU(c, cudaEventRecord(c->tc_desc_ev[d], c->compute));
     c->tc_desc_ev_valid[d] = 1;
     gg_gather_kernel<<<n_rows, 128, 0, c->compute>>>(x_norm, w, reinterpret_cast<const GgRow*>(dd + c->tc_off_rows), n_rows,
-                                                     m.hidden, K, c->tc_xs, c->tc_wrow);
+                                                     nullptr, m.hidden, K, c->tc_xs, c->tc_wrow);
     CU(c, cudaGetLastError());
     if (t && first) CU(c, cudaEventRecord(t->ffn_start[layer], c->compute));
     if (ring >= 0 && first) CU(c, cudaEventRecord(c->ring_start[ring], c->compute));
-    GgArgs a{reinterpret_cast<const GgUnit*>(dd), n_units, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status};
+    GgArgs a{reinterpret_cast<const GgUnit*>(dd), n_units, nullptr, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status};
     ffn_grouped_kernel<<<std::min(c->num_sms, n_units), kGgThreads, ffn_grouped_smem(), c->compute>>>(c->wmap, c->xmap, a);
     CU(c, cudaGetLastError());
     if (t && last) CU(c, cudaEventRecord(t->ffn_end[layer], c->compute));
@@ -540,8 +595,10 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
 // Demand resolution, on-demand copies, stream waits and FFN launches of one layer.
 // `t` (may be null) receives the timing events of this layer; `ring` >= 0 selects an event pair
 // of the stand-alone timing ring instead.
+// With `launch` false only the slot table's side runs (the kernels of a host-free step were
+// enqueued earlier); a miss there would mean the step computed with a stale slot map.
 int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, const float* w, int nb,
-            float* h_inout, Timing* t, int ring = -1) {
+            float* h_inout, Timing* t, int ring = -1, bool launch = true) {
     const spm_model_cfg& m = c->cfg;
     const int K = m.top_k;
     SlotTable& tb = *c->table;
@@ -561,6 +618,11 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
     }
     int n_waves = 1;
     tb.demand(layer, c->need.data(), int(c->need.size()), c->placements, &n_waves);
+    if (!launch) {
+        for (const Placement& p : c->placements)
+            if (p.missed) return fail(c, SPM_ERR_STATE, "host-free step met a non-resident expert (layer %d, expert %d)", layer, p.expert);
+        return SPM_OK;
+    }
 
     const int G = ffn_grid_for(c, nb);
     const bool dev_wait = c->device_wait && nb == 1 && m.dtype != SPM_DTYPE_Q4 && stream_write32_fn() != nullptr;
@@ -689,6 +751,210 @@ void borda_rank(const int32_t* ids, int nb, int K, int n, std::vector<int32_t>& 
     std::stable_sort(out.begin(), out.end(), [&](int32_t x, int32_t y) { return score[x] > score[y]; });
 }
 
+
+// The layers of one decode step. With `trace` null the kernels are launched and the routing results
+// awaited layer by layer; with a trace (the mailboxes a host-free step filled) only the host side
+// runs: accounting, slot-table updates, selection — the same calls in the same order.
+int step_layers(spm_ctx* c, float* h_out, int nb, Timing* t, const Mailbox* trace) {
+    const spm_model_cfg& m = c->cfg;
+    const int L = m.n_layers, K = m.top_k, n = m.n_experts;
+    SlotTable& tb = *c->table;
+    const bool predict = c->policy == SPM_POLICY_ADAPTER || c->policy == SPM_POLICY_PRED0;
+    c->prev_order_valid = false;
+    std::vector<int32_t> ids(size_t(nb) * K);
+    std::vector<int32_t> this_rank;
+    for (int l = 0; l < L; ++l) {
+        const bool has_adapter = l <= L - 2;
+        if (!trace) {
+            if (c->stub_us > 0) {
+                attention_stub_kernel<<<1, 1, 0, c->compute>>>(uint64_t(c->stub_us) * 1000ull);
+                CU(c, cudaGetLastError());
+                c->kernel_launches++;
+            }
+            if (int rc = launch_router(c, l, h_out, nullptr, nb, c->ws_x, nullptr, true, predict && has_adapter)) return rc;
+            if (t) CU(c, cudaEventRecord(t->k1_done[l], c->compute));
+            if (int rc = wait_tagged(c, c->mb_host->ids, nb * K, ids.data(), "expert ids")) return rc;
+        } else {
+            for (int i = 0; i < nb * K; ++i) ids[i] = trace[l].ids[i] & 0xffff;
+        }
+
+        if (c->prev_order_valid) {   // ExpertRecall@M of the previous layer's prediction, M = budget
+            const int M = std::min(c->budget, n);
+            for (int tk = 0; tk < nb; ++tk) {
+                int hit = 0;
+                for (int k = 0; k < K; ++k)
+                    for (int q = 0; q < M; ++q) hit += c->prev_order[q] == ids[tk * K + k];
+                c->recall_sum += double(hit) / K;
+                c->recall_count++;
+            }
+        }
+        if (int rc = run_ffn(c, l, c->ws_x, ids.data(), c->ws_w, nb, h_out, t, -1, trace == nullptr)) return rc;
+        if (c->policy == SPM_POLICY_NAIVE) borda_rank(ids.data(), nb, K, n, this_rank);
+
+        c->prev_order_valid = false;
+        if (has_adapter && c->policy != SPM_POLICY_ON_DEMAND) {
+            const int32_t* ranking;
+            int n_ranked;
+            bool protect_all = false;
+            if (c->policy == SPM_POLICY_HINT_TRACE) {
+                const size_t cell = size_t(tb.step()) * L + (l + 1);
+                ranking = c->hint.data() + cell * c->hint_stride;
+                n_ranked = c->hint_count[cell];
+                protect_all = true;
+            } else if (c->policy == SPM_POLICY_NAIVE) {
+                ranking = c->prev_rank[l + 1].data();      // what the preceding step used at layer l+1
+                n_ranked = int(c->prev_rank[l + 1].size());
+            } else {
+                c->prev_order.resize(n);
+                if (!trace) {
+                    if (int rc = wait_tagged(c, c->mb_host->order, n, c->prev_order.data(), "expert ranking")) return rc;
+                } else {
+                    for (int e = 0; e < n; ++e) c->prev_order[e] = trace[l].order[e] & 0xffff;
+                }
+                c->prev_order_valid = true;
+                ranking = c->prev_order.data();
+                n_ranked = n;
+            }
+            tb.plan(l + 1, ranking, n_ranked, c->budget, protect_all, c->sel, c->protect);
+            if (c->policy == SPM_POLICY_PRED0) {
+                tb.plan_only(l + 1, c->sel.data(), int(c->sel.size()));
+            } else {
+                if (int rc = do_prefetch(c, l + 1, c->sel.data(), int(c->sel.size()), c->protect.data(),
+                                         int(c->protect.size()), nullptr)) return rc;
+            }
+        }
+        if (c->policy == SPM_POLICY_NAIVE) c->prev_rank[l] = this_rank;
+    }
+    tb.end_step();
+    tb.stats().steps++;
+    c->tokens += nb;
+    return SPM_OK;
+}
+
+// ---- host-free steps ---------------------------------------------------------
+// Replay the bookkeeping of the oldest enqueued host-free step (waits for its kernels).
+int replay_oldest(spm_ctx* c) {
+    const auto [slot, nb] = c->tr_pending.front();
+    CU(c, cudaEventSynchronize(c->tr_ev[slot]));
+    c->tr_pending.pop_front();
+    return step_layers(c, nullptr, nb, nullptr, c->tr_host + size_t(slot) * c->cfg.n_layers);
+}
+
+int flush_trace(spm_ctx* c) {
+    while (!c->tr_pending.empty())
+        if (int rc = replay_oldest(c)) return rc;
+    return SPM_OK;
+}
+
+// A step may skip the host when no routing result can change what the host would do: every expert
+// of every layer holds a slot and every copy has landed, so any demand is a hit and no selection
+// finds a candidate. On the batched tensor-core path the wave plan is then built by a kernel.
+int host_free_ready(spm_ctx* c, int nb, bool* out) {
+    const spm_model_cfg& m = c->cfg;
+    *out = false;
+    if (!c->host_free || c->S < m.n_experts) return SPM_OK;
+    if (!c->fast_ready) {
+        SlotTable& tb = *c->table;
+        for (int l = 0; l < m.n_layers; ++l)
+            for (int e = 0; e < m.n_experts; ++e)
+                if (tb.slot_of(l, e) < 0) return SPM_OK;
+        for (size_t k = 0; k < c->slot_pending.size(); ++k)
+            if (c->slot_pending[k]) {
+                CU(c, cudaStreamWaitEvent(c->compute, c->slot_ev[k], 0));
+                c->slot_pending[k] = 0;
+            }
+        std::vector<short> map(size_t(m.n_layers) * m.n_experts);
+        for (int l = 0; l < m.n_layers; ++l)
+            for (int e = 0; e < m.n_experts; ++e) map[size_t(l) * m.n_experts + e] = short(tb.slot_of(l, e));
+        CU(c, cudaMemcpyAsync(c->ws_slot_map, map.data(), map.size() * sizeof(short), cudaMemcpyHostToDevice, c->compute));
+        CU(c, cudaStreamSynchronize(c->compute));      // `map` is a temporary
+        c->fast_ready = true;
+    }
+    *out = true;
+    return SPM_OK;
+}
+
+int enqueue_host_free_step(spm_ctx* c, const float* h_in, int nb, float* h_out) {
+    const spm_model_cfg& m = c->cfg;
+    const int L = m.n_layers, K = m.top_k, n = m.n_experts;
+    if (int(c->tr_pending.size()) == kTraceRing)
+        if (int rc = replay_oldest(c)) return rc;
+    const int slot = int(c->tr_count++ % kTraceRing);
+    if (h_out != h_in)
+        CU(c, cudaMemcpyAsync(h_out, h_in, size_t(nb) * m.hidden * 4, cudaMemcpyDeviceToDevice, c->compute));
+    const bool predict = c->policy == SPM_POLICY_ADAPTER || c->policy == SPM_POLICY_PRED0;
+    const int G = ffn_grid_for(c, nb);
+    for (int l = 0; l < L; ++l) {
+        if (c->stub_us > 0) {
+            attention_stub_kernel<<<1, 1, 0, c->compute>>>(uint64_t(c->stub_us) * 1000ull);
+            CU(c, cudaGetLastError());
+            c->kernel_launches++;
+        }
+        short* codes = c->ws_codes + size_t(l) * m.max_batch * SPM_MAX_TOPK;
+        RouterRoute route{c->tr_dev + size_t(slot) * L + l, c->ws_slot_map + size_t(l) * n, codes, true};
+        if (int rc = launch_router(c, l, h_out, nullptr, nb, c->ws_x, nullptr, true, predict && l <= L - 2, &route)) return rc;
+        unsigned long long* clock_slot = nullptr;
+        if (c->timing) {
+            if (c->clock_used == kClockSlots) if (int rc = harvest_clock(c)) return rc;
+            clock_slot = c->ws_clock + 2 * size_t(c->clock_used++);
+        }
+        auto fill = [&](auto& a) {
+            a.pool = slot_ptr(c, l, 0);
+            a.shared = m.n_shared ? static_cast<const unsigned char*>(c->buf.shared_experts) + size_t(l) * m.n_shared * c->blob : nullptr;
+            a.x = c->ws_x;
+            a.w = c->ws_w;
+            a.partial = c->ws_partial;
+            a.status = c->ws_status;
+            a.clock = clock_slot;
+            a.ready = nullptr;
+            a.dev_code = codes;
+            a.blob_bytes = c->blob;
+            a.I = m.inter; a.K = K; a.n_slots = c->S; a.n_shared = m.n_shared;
+            for (int tk = 0; tk < nb; ++tk) a.count[tk] = (unsigned char)(K + m.n_shared);   // launch shape only
+        };
+        if (nb > 1 && c->tc_ok && c->batched_path == 0) {
+            // wave plan on the device, then gather -> grouped tcgen05 FFN -> combine
+            unsigned char* dd = c->tc_desc_dev;        // stream-ordered reuse of the first descriptor slot
+            GgUnit* units = reinterpret_cast<GgUnit*>(dd);
+            GgRow* rows = reinterpret_cast<GgRow*>(dd + c->tc_off_rows);
+            int32_t* rowmap = reinterpret_cast<int32_t*>(dd + c->tc_off_rowmap);
+            CU(c, launch_k(gg_plan_kernel, dim3(1), dim3(kGgPlanThreads), size_t(nb * K + 2 * n) * sizeof(int32_t), c->compute, true,
+                           (const int32_t*)c->ws_ids, (const short*)(c->ws_slot_map + size_t(l) * n), l * c->S, nb, K, n, c->n_jt,
+                           units, rows, rowmap, c->tc_counts, c->ws_status));
+            CU(c, launch_k(gg_gather_kernel, dim3(nb * K), dim3(128), 0, c->compute, true, (const float*)c->ws_x, (const float*)c->ws_w,
+                           (const GgRow*)rows, 0, (const int*)(c->tc_counts + 1), m.hidden, K, c->tc_xs, c->tc_wrow));
+            GgArgs ga{units, 0, c->tc_counts, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status};
+            CU(c, launch_k(ffn_grouped_kernel, dim3(c->num_sms), dim3(kGgThreads), ffn_grouped_smem(), c->compute, true, c->wmap, c->xmap, ga));
+            CU(c, launch_k(gg_combine_kernel, dim3((m.hidden + 127) / 128, nb), dim3(128), 0, c->compute, true,
+                           (const float*)c->tc_partial, (const int32_t*)rowmap, K, c->n_jt, c->rows_cap, m.hidden, h_out));
+            c->kernel_launches += 5;
+            c->ffn_launches++;
+            c->tc_launches++;
+            continue;
+        }
+        if (nb == 1) {
+            FfnArgs<1> a{};
+            fill(a);
+            CU(c, launch_gemv<1>(c, a, G, nb, true));
+        } else {
+            FfnArgs<SPM_MAX_BATCH> a{};
+            fill(a);
+            CU(c, launch_gemv<SPM_MAX_BATCH>(c, a, G, nb, true));
+        }
+        CU(c, launch_k(ffn_reduce_kernel, dim3((m.hidden + kReduceCols - 1) / kReduceCols, nb), dim3(kReduceCols * kReduceGroups), 0,
+                       c->compute, true, (const float*)c->ws_partial, (const float*)h_out, h_out, G, m.hidden));
+        c->kernel_launches += 3;
+        c->ffn_launches++;
+    }
+    CU(c, cudaEventRecord(c->tr_ev[slot], c->compute));
+    c->tr_pending.emplace_back(slot, nb);
+    c->host_free_steps++;
+    // bookkeeping of steps whose kernels have already finished, while the device works on this one
+    while (!c->tr_pending.empty() && cudaEventQuery(c->tr_ev[c->tr_pending.front().first]) == cudaSuccess)
+        if (int rc = replay_oldest(c)) return rc;
+    return SPM_OK;
+}
+
 int check_layer(spm_ctx* c, int layer, int nb) {
     if (!c) return SPM_ERR_INVALID_ARG;
     if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, SPM_ERR_INVALID_ARG, "layer %d out of range", layer);
@@ -781,6 +1047,8 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
     c->ws_ids = reinterpret_cast<int32_t*>(base + lay.ids);
     c->ws_order = reinterpret_cast<int32_t*>(base + lay.order);
     c->ws_clock = reinterpret_cast<unsigned long long*>(base + lay.clock);
+    c->ws_slot_map = reinterpret_cast<short*>(base + lay.slot_map);
+    c->ws_codes = reinterpret_cast<short*>(base + lay.codes);
     c->ws_counters = reinterpret_cast<unsigned*>(base + lay.counters);
     c->ws_status = reinterpret_cast<int*>(base + lay.status);
 
@@ -805,6 +1073,11 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
     if (!cu(cudaHostAlloc(reinterpret_cast<void**>(&c->mb_host), sizeof(Mailbox), cudaHostAllocMapped), "cudaHostAlloc(mailbox)")) return bail(SPM_ERR_CUDA);
     memset(c->mb_host, 0, sizeof(Mailbox));
     if (!cu(cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->mb_dev), c->mb_host, 0), "cudaHostGetDevicePointer")) return bail(SPM_ERR_CUDA);
+    if (!cu(cudaHostAlloc(reinterpret_cast<void**>(&c->tr_host), sizeof(Mailbox) * kTraceRing * L, cudaHostAllocMapped), "cudaHostAlloc(trace)")) return bail(SPM_ERR_CUDA);
+    memset(c->tr_host, 0, sizeof(Mailbox) * kTraceRing * L);
+    if (!cu(cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->tr_dev), c->tr_host, 0), "cudaHostGetDevicePointer")) return bail(SPM_ERR_CUDA);
+    c->tr_ev.resize(kTraceRing);
+    for (auto& ev : c->tr_ev) if (!cu(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming), "cudaEventCreate")) return bail(SPM_ERR_CUDA);
     c->slot_ev.resize(size_t(L) * c->S);
     for (auto& ev : c->slot_ev) if (!cu(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming), "cudaEventCreate")) return bail(SPM_ERR_CUDA);
     c->pool_free.resize(L);
@@ -822,6 +1095,7 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
         c->tc_wrow = reinterpret_cast<float*>(base + lay.tc_wrow);
         c->tc_partial = reinterpret_cast<float*>(base + lay.tc_partial);
         c->tc_desc_dev = base + lay.tc_desc;
+        c->tc_counts = reinterpret_cast<int*>(base + lay.tc_counts);
         c->tc_desc_bytes = lay.desc_bytes; c->tc_off_rows = lay.off_rows; c->tc_off_rowmap = lay.off_rowmap;
         if (!cu(cudaMemsetAsync(c->tc_xs, 0, size_t(lay.rows_cap + kGgTokens) * cfg->hidden * 2, c->compute), "cudaMemsetAsync")) return bail(SPM_ERR_CUDA);
         if (!cu(cudaHostAlloc(reinterpret_cast<void**>(&c->tc_desc_host), size_t(kDescRing) * lay.desc_bytes, cudaHostAllocDefault), "cudaHostAlloc(descriptors)")) return bail(SPM_ERR_CUDA);
@@ -871,6 +1145,8 @@ int spm_destroy(spm_ctx* c) {
     for (auto ev : c->ring_start) if (ev) cudaEventDestroy(ev);
     for (auto ev : c->ring_end) if (ev) cudaEventDestroy(ev);
     if (c->mb_host) cudaFreeHost(c->mb_host);
+    for (auto ev : c->tr_ev) if (ev) cudaEventDestroy(ev);
+    if (c->tr_host) cudaFreeHost(c->tr_host);
     delete c->table;
     delete c;
     return SPM_OK;
@@ -879,6 +1155,7 @@ int spm_destroy(spm_ctx* c) {
 int spm_router_topk(spm_ctx* c, int layer, const float* h, int nb, float* x_norm, int32_t* ids, float* w,
                     float* logits) {
     if (int rc = check_layer(c, layer, nb)) return rc;
+    if (int rc = flush_trace(c)) return rc;
     if (!h || !x_norm || !ids || !w) return fail(c, SPM_ERR_INVALID_ARG, "null argument");
     if (int rc = launch_router(c, layer, h, nullptr, nb, x_norm, logits, true, false)) return rc;
     CU(c, cudaMemcpyAsync(w, c->ws_w, size_t(nb) * c->cfg.top_k * 4, cudaMemcpyDeviceToDevice, c->compute));
@@ -889,6 +1166,7 @@ int spm_router_topk(spm_ctx* c, int layer, const float* h, int nb, float* x_norm
 
 int spm_adapter_predict(spm_ctx* c, int layer, const float* x_norm, int nb, float* scores, int32_t* order) {
     if (int rc = check_layer(c, layer, nb)) return rc;
+    if (int rc = flush_trace(c)) return rc;
     if (layer > c->cfg.n_layers - 2) return fail(c, SPM_ERR_INVALID_ARG, "layer %d has no adapter (L-1 adapters)", layer);
     if (!x_norm || !scores || !order) return fail(c, SPM_ERR_INVALID_ARG, "null argument");
     if (int rc = launch_router(c, layer, nullptr, x_norm, nb, nullptr, nullptr, false, true)) return rc;
@@ -901,6 +1179,7 @@ int spm_adapter_predict(spm_ctx* c, int layer, const float* x_norm, int nb, floa
 int spm_budget_select(spm_ctx* c, int target, const int32_t* order, int n_ranked, int budget, int protect_all,
                       int32_t* out_ids, int* out_count) {
     if (int rc = check_layer(c, target, 1)) return rc;
+    if (int rc = flush_trace(c)) return rc;
     if (!order || !out_ids || !out_count || n_ranked < 0 || n_ranked > c->cfg.n_experts)
         return fail(c, SPM_ERR_INVALID_ARG, "bad ranking argument");
     for (int i = 0; i < n_ranked; ++i)
@@ -915,6 +1194,7 @@ int spm_budget_select(spm_ctx* c, int target, const int32_t* order, int n_ranked
 
 int spm_prefetch_async(spm_ctx* c, int target, const int32_t* ids, int count, int* out_issued) {
     if (int rc = check_layer(c, target, 1)) return rc;
+    if (int rc = flush_trace(c)) return rc;
     if (count < 0 || (count > 0 && !ids)) return fail(c, SPM_ERR_INVALID_ARG, "bad id list");
     for (int i = 0; i < count; ++i)
         if (ids[i] < 0 || ids[i] >= c->cfg.n_experts) return fail(c, SPM_ERR_INVALID_ARG, "expert id %d out of range", ids[i]);
@@ -927,6 +1207,7 @@ int spm_prefetch_async(spm_ctx* c, int target, const int32_t* ids, int count, in
 
 int spm_moe_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, const float* w, int nb, float* h_inout) {
     if (int rc = check_layer(c, layer, nb)) return rc;
+    if (int rc = flush_trace(c)) return rc;
     if (!x_norm || !ids || !w || !h_inout) return fail(c, SPM_ERR_INVALID_ARG, "null argument");
     int ring = -1;
     if (c->timing) {
@@ -940,10 +1221,12 @@ int spm_decode_step(spm_ctx* c, const float* h_in, int nb, float* h_out) {
     if (int rc = check_layer(c, 0, nb)) return rc;
     if (!h_in || !h_out) return fail(c, SPM_ERR_INVALID_ARG, "null argument");
     const spm_model_cfg& m = c->cfg;
-    const int L = m.n_layers, K = m.top_k, n = m.n_experts;
-    SlotTable& tb = *c->table;
-    if (c->policy == SPM_POLICY_HINT_TRACE && tb.step() >= c->hint_steps)
-        return fail(c, SPM_ERR_STATE, "no hint trace for step %d", tb.step());
+    if (c->policy == SPM_POLICY_HINT_TRACE && c->table->step() + int(c->tr_pending.size()) >= c->hint_steps)
+        return fail(c, SPM_ERR_STATE, "no hint trace for step %d", c->table->step() + int(c->tr_pending.size()));
+    bool fast = false;
+    if (int rc = host_free_ready(c, nb, &fast)) return rc;
+    if (fast) return enqueue_host_free_step(c, h_in, nb, h_out);
+    if (int rc = flush_trace(c)) return rc;
     if (h_out != h_in)
         CU(c, cudaMemcpyAsync(h_out, h_in, size_t(nb) * m.hidden * 4, cudaMemcpyDeviceToDevice, c->compute));
     Timing* t = nullptr;
@@ -952,68 +1235,7 @@ int spm_decode_step(spm_ctx* c, const float* h_in, int nb, float* h_out) {
         t = &c->tim[c->tim_cur];
         harvest(c, *t);
     }
-    const bool predict = c->policy == SPM_POLICY_ADAPTER || c->policy == SPM_POLICY_PRED0;
-    c->prev_order_valid = false;
-    std::vector<int32_t> ids(size_t(nb) * K);
-    std::vector<int32_t> this_rank;
-    for (int l = 0; l < L; ++l) {
-        const bool has_adapter = l <= L - 2;
-        if (c->stub_us > 0) {
-            attention_stub_kernel<<<1, 1, 0, c->compute>>>(uint64_t(c->stub_us) * 1000ull);
-            CU(c, cudaGetLastError());
-            c->kernel_launches++;
-        }
-        if (int rc = launch_router(c, l, h_out, nullptr, nb, c->ws_x, nullptr, true, predict && has_adapter)) return rc;
-        if (t) CU(c, cudaEventRecord(t->k1_done[l], c->compute));
-        if (int rc = wait_tagged(c, c->mb_host->ids, nb * K, ids.data(), "expert ids")) return rc;
-
-        if (c->prev_order_valid) {   // ExpertRecall@M of the previous layer's prediction, M = budget
-            const int M = std::min(c->budget, n);
-            for (int tk = 0; tk < nb; ++tk) {
-                int hit = 0;
-                for (int k = 0; k < K; ++k)
-                    for (int q = 0; q < M; ++q) hit += c->prev_order[q] == ids[tk * K + k];
-                c->recall_sum += double(hit) / K;
-                c->recall_count++;
-            }
-        }
-        if (int rc = run_ffn(c, l, c->ws_x, ids.data(), c->ws_w, nb, h_out, t)) return rc;
-        if (c->policy == SPM_POLICY_NAIVE) borda_rank(ids.data(), nb, K, n, this_rank);
-
-        c->prev_order_valid = false;
-        if (has_adapter && c->policy != SPM_POLICY_ON_DEMAND) {
-            const int32_t* ranking;
-            int n_ranked;
-            bool protect_all = false;
-            if (c->policy == SPM_POLICY_HINT_TRACE) {
-                const size_t cell = size_t(tb.step()) * L + (l + 1);
-                ranking = c->hint.data() + cell * c->hint_stride;
-                n_ranked = c->hint_count[cell];
-                protect_all = true;
-            } else if (c->policy == SPM_POLICY_NAIVE) {
-                ranking = c->prev_rank[l + 1].data();      // what the preceding step used at layer l+1
-                n_ranked = int(c->prev_rank[l + 1].size());
-            } else {
-                c->prev_order.resize(n);
-                if (int rc = wait_tagged(c, c->mb_host->order, n, c->prev_order.data(), "expert ranking")) return rc;
-                c->prev_order_valid = true;
-                ranking = c->prev_order.data();
-                n_ranked = n;
-            }
-            tb.plan(l + 1, ranking, n_ranked, c->budget, protect_all, c->sel, c->protect);
-            if (c->policy == SPM_POLICY_PRED0) {
-                tb.plan_only(l + 1, c->sel.data(), int(c->sel.size()));
-            } else {
-                if (int rc = do_prefetch(c, l + 1, c->sel.data(), int(c->sel.size()), c->protect.data(),
-                                         int(c->protect.size()), nullptr)) return rc;
-            }
-        }
-        if (c->policy == SPM_POLICY_NAIVE) c->prev_rank[l] = this_rank;
-    }
-    tb.end_step();
-    tb.stats().steps++;
-    c->tokens += nb;
-    return SPM_OK;
+    return step_layers(c, h_out, nb, t, nullptr);
 }
 
 int spm_decode_step_host(spm_ctx* c, const float* h_in_host, int nb, float* h_out_host) {
@@ -1030,6 +1252,7 @@ int spm_decode_step_host(spm_ctx* c, const float* h_in_host, int nb, float* h_ou
 // ---- control --------------------------------------------------------------
 int spm_set_policy(spm_ctx* c, int policy) {
     if (!c) return SPM_ERR_INVALID_ARG;
+    if (int rc = flush_trace(c)) return rc;
     if (policy < SPM_POLICY_ADAPTER || policy > SPM_POLICY_NAIVE) return fail(c, SPM_ERR_INVALID_ARG, "policy %d", policy);
     if ((policy == SPM_POLICY_ADAPTER || policy == SPM_POLICY_PRED0) && c->cfg.n_layers > 1 && (!c->buf.adapter_a || !c->buf.adapter_b))
         return fail(c, SPM_ERR_STATE, "no adapter weights");
@@ -1038,6 +1261,7 @@ int spm_set_policy(spm_ctx* c, int policy) {
 }
 int spm_set_budget(spm_ctx* c, int budget) {
     if (!c) return SPM_ERR_INVALID_ARG;
+    if (int rc = flush_trace(c)) return rc;
     if (budget < 0) return fail(c, SPM_ERR_INVALID_ARG, "budget %d", budget);
     c->budget = budget;
     return SPM_OK;
@@ -1049,6 +1273,7 @@ int spm_get_budget(spm_ctx* c, int* budget) {
 }
 int spm_set_plain_lru(spm_ctx* c, int on) {
     if (!c) return SPM_ERR_INVALID_ARG;
+    if (int rc = flush_trace(c)) return rc;
     c->table->set_plain_lru(on != 0);
     return SPM_OK;
 }
@@ -1070,6 +1295,7 @@ int spm_set_batched_path(spm_ctx* c, int mode) {
 }
 int spm_set_hint_trace(spm_ctx* c, const int32_t* hint, const int32_t* count, int n_steps, int stride) {
     if (!c) return SPM_ERR_INVALID_ARG;
+    if (int rc = flush_trace(c)) return rc;
     if (!hint || !count || n_steps < 0 || stride < 1) return fail(c, SPM_ERR_INVALID_ARG, "bad hint trace");
     const size_t cells = size_t(n_steps) * c->cfg.n_layers;
     for (size_t i = 0; i < cells; ++i) {
@@ -1086,6 +1312,7 @@ int spm_set_hint_trace(spm_ctx* c, const int32_t* hint, const int32_t* count, in
 }
 int spm_set_drop_modulo(spm_ctx* c, int modulo) {
     if (!c || modulo < 0) return SPM_ERR_INVALID_ARG;
+    if (int rc = flush_trace(c)) return rc;
     c->drop_modulo = modulo;
     return SPM_OK;
 }
@@ -1098,6 +1325,12 @@ int spm_set_device_wait(spm_ctx* c, int on) {
     if (!c) return SPM_ERR_INVALID_ARG;
     if (on && !stream_write32_fn()) return fail(c, SPM_ERR_CUDA, "cuStreamWriteValue32 is not available on this driver");
     c->device_wait = on != 0;
+    return SPM_OK;
+}
+int spm_set_host_free(spm_ctx* c, int on) {
+    if (!c) return SPM_ERR_INVALID_ARG;
+    if (int rc = flush_trace(c)) return rc;
+    c->host_free = on != 0;
     return SPM_OK;
 }
 int spm_set_attention_stub_us(spm_ctx* c, int us) {
@@ -1113,6 +1346,7 @@ int spm_set_deadline_ms(spm_ctx* c, int ms) {
 
 int spm_synchronize(spm_ctx* c) {
     if (!c) return SPM_ERR_INVALID_ARG;
+    if (int rc = flush_trace(c)) return rc;
     CU(c, cudaStreamSynchronize(c->copy));
     CU(c, cudaStreamSynchronize(c->compute));
     return check_status(c);
@@ -1120,6 +1354,7 @@ int spm_synchronize(spm_ctx* c) {
 
 int spm_reset_stats(spm_ctx* c) {
     if (!c) return SPM_ERR_INVALID_ARG;
+    if (int rc = flush_trace(c)) return rc;
     CU(c, cudaStreamSynchronize(c->copy));
     CU(c, cudaStreamSynchronize(c->compute));
     for (auto& t : c->tim) std::fill(t.used.begin(), t.used.end(), 0);
@@ -1132,6 +1367,7 @@ int spm_reset_stats(spm_ctx* c) {
     std::fill(c->layer_ffn_us.begin(), c->layer_ffn_us.end(), 0.0);
     c->timed_steps = 0;
     c->extra_late = c->h2d_bytes = c->ffn_launches = c->kernel_launches = c->tokens = 0;
+    c->host_free_steps = 0;
     c->ready_sum = c->recall_sum = 0;
     c->ready_count = c->recall_count = 0;
     return SPM_OK;
@@ -1139,10 +1375,12 @@ int spm_reset_stats(spm_ctx* c) {
 
 int spm_cache_reset(spm_ctx* c) {
     if (!c) return SPM_ERR_INVALID_ARG;
+    if (int rc = flush_trace(c)) return rc;
     CU(c, cudaStreamSynchronize(c->copy));
     CU(c, cudaStreamSynchronize(c->compute));
     for (auto& t : c->tim) std::fill(t.used.begin(), t.used.end(), 0);
     c->table->reset();
+    c->fast_ready = false;
     for (auto& r : c->prev_rank) r.clear();
     std::fill(c->ring_used.begin(), c->ring_used.end(), 0);
     c->ring_us = 0;
@@ -1156,6 +1394,7 @@ int spm_cache_reset(spm_ctx* c) {
     c->extra_late = c->h2d_bytes = c->ffn_launches = c->kernel_launches = c->tokens = 0;
     c->ready_sum = c->recall_sum = 0;
     c->ready_count = c->recall_count = 0;
+    c->host_free_steps = 0;
     c->prev_order_valid = false;
     return SPM_OK;
 }
@@ -1222,6 +1461,7 @@ int spm_profile_window(spm_ctx* c, double* window_us, double* t_xfer_us, int* bu
 
 int spm_get_stats(spm_ctx* c, spm_stats* out) {
     if (!c || !out) return SPM_ERR_INVALID_ARG;
+    if (int rc = flush_trace(c)) return rc;
     CU(c, cudaStreamSynchronize(c->copy));
     CU(c, cudaStreamSynchronize(c->compute));
     for (auto& t : c->tim) harvest(c, t);
@@ -1239,6 +1479,7 @@ int spm_get_stats(spm_ctx* c, spm_stats* out) {
     for (int l = 0; l < c->cfg.n_layers; ++l) { out->ffn_us += c->layer_ffn_us[l]; out->stall_us += c->layer_stall_us[l]; }
     out->ready_sum = c->ready_sum; out->ready_count = c->ready_count;
     out->recall_sum = c->recall_sum; out->recall_count = c->recall_count;
+    out->host_free_steps = c->host_free_steps;
     return check_status(c);
 }
 
@@ -1253,6 +1494,7 @@ int spm_get_layer_times(spm_ctx* c, double* stall_us, double* ffn_us, uint64_t* 
 
 int spm_get_events(spm_ctx* c, spm_event* out, size_t capacity, size_t* count) {
     if (!c || !count) return SPM_ERR_INVALID_ARG;
+    if (int rc = flush_trace(c)) return rc;
     const auto& ev = c->table->events();
     *count = ev.size();
     if (out) memcpy(out, ev.data(), std::min(capacity, ev.size()) * sizeof(spm_event));
@@ -1261,6 +1503,7 @@ int spm_get_events(spm_ctx* c, spm_event* out, size_t capacity, size_t* count) {
 
 int spm_get_slot_table(spm_ctx* c, int layer, int32_t* slot_expert) {
     if (int rc = check_layer(c, layer, 1)) return rc;
+    if (int rc = flush_trace(c)) return rc;
     if (!slot_expert) return SPM_ERR_INVALID_ARG;
     for (int s = 0; s < c->S; ++s) slot_expert[s] = c->table->expert_in(layer, s);
     return SPM_OK;

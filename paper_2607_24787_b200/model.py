@@ -153,6 +153,7 @@ class OffloadedMoE:
     def set_drop_modulo(self, m): B.spm_set_drop_modulo(self.ctx, m)
     def set_attention_stub_us(self, us): B.spm_set_attention_stub_us(self.ctx, us)
     def set_device_wait(self, on): B.spm_set_device_wait(self.ctx, on)
+    def set_host_free(self, on): B.spm_set_host_free(self.ctx, on)
     def set_copy_delay_us(self, us): B.spm_set_copy_delay_us(self.ctx, us)
     def profile_window(self): return B.spm_profile_window(self.ctx)
     def cache_reset(self): B.spm_cache_reset(self.ctx)

@@ -6,6 +6,7 @@ import torch
 
 import synth
 
+from .adapter_fit import reduced_rank_fit, svd_adapter
 from .model import OffloadedMoE, PinnedStore, pack_experts, pack_experts_q4
 
 
@@ -31,20 +32,61 @@ def fill_store(cfg: synth.ModelCfg, store: PinnedStore, device, chunk: int = 32,
     torch.cuda.synchronize(device)
 
 
+def collect_router_io(m: OffloadedMoE, H_dev: torch.Tensor):
+    """Calibration pass for fitted adapters: decodes the rows of H_dev [steps, 1, D] layer by layer
+    through the stand-alone entry points and records, per layer, the router input x and the native
+    router logits z. Returns (X [L, steps, D], Z [L, steps, n]) fp32 on the device."""
+    steps = H_dev.shape[0]
+    X = torch.empty(m.L, steps, m.D, dtype=torch.float32, device=m.device)
+    Z = torch.empty(m.L, steps, m.n, dtype=torch.float32, device=m.device)
+    for s in range(steps):
+        h = H_dev[s].clone()
+        torch.cuda.synchronize(m.device)
+        for l in range(m.L):
+            x, ids, w, logits = m.router_topk(l, h, want_logits=True)
+            m.moe_ffn(l, x, ids, w, h)
+            m.synchronize()
+            X[l, s].copy_(x[0])
+            Z[l, s].copy_(logits[0])
+    torch.cuda.synchronize(m.device)
+    return X, Z
+
+
+def fitted_adapters(X: torch.Tensor, Z: torch.Tensor, rank: int, dtype: torch.dtype, ridge: float = 1e-3):
+    """Reduced-rank regression of layer l+1's router logits on layer l's router input, per layer.
+    Returns (A [L-1, rank, D], B_up [L-1, n, rank]) in `dtype`."""
+    a_all, b_all = [], []
+    for l in range(X.shape[0] - 1):
+        a, b = reduced_rank_fit(X[l], Z[l + 1], rank, ridge)
+        a_all.append(a.to(dtype))
+        b_all.append(b.to(dtype))
+    return torch.stack(a_all).contiguous(), torch.stack(b_all).contiguous()
+
+
 def build_from_synth(cfg: synth.ModelCfg, slots=None, budget=None, max_batch=None, device="cuda:0",
-                     store: PinnedStore | None = None, adapter: str = "random", store_layers: int = 0) -> OffloadedMoE:
+                     store: PinnedStore | None = None, adapter="random", store_layers: int = 0) -> OffloadedMoE:
     """Random-init model of the configuration's shape, experts offloaded to pinned host memory.
 
     adapter="random": the configuration's N(0, 0.02) rank-r adapters. adapter="gate_reuse": a
     training-free stand-in for trained adapters, A^l = W_r^{l+1} and Bup = identity (rank n), i.e.
-    the next layer's own gate applied to this layer's router input (data only: same kernels).
+    the next layer's own gate applied to this layer's router input. adapter="svd": the rank-r
+    truncated SVD of W_r^{l+1}. adapter=(A, B_up): given tensors [L-1, r, D] and [L-1, n, r], e.g.
+    from fitted_adapters(). All of these are data only: the same kernels run them.
     """
     dev = torch.device(device)
     L = cfg.n_layers
     gamma = torch.ones(L, cfg.hidden, dtype=torch.float32, device=dev)
     router = torch.stack([synth.router_w(cfg, l, dev) for l in range(L)]).contiguous()
     rank = cfg.adapter_rank
-    if adapter == "gate_reuse" and L > 1:
+    if isinstance(adapter, tuple) and L > 1:
+        a, b = (t.to(device=dev, dtype=router.dtype).contiguous() for t in adapter)
+        rank = a.shape[1]
+        assert a.shape == (L - 1, rank, cfg.hidden) and b.shape == (L - 1, cfg.n_experts, rank)
+    elif adapter == "svd" and L > 1:
+        pairs = [svd_adapter(router[l + 1], rank) for l in range(L - 1)]
+        a = torch.stack([p[0] for p in pairs]).to(router.dtype).contiguous()
+        b = torch.stack([p[1] for p in pairs]).to(router.dtype).contiguous()
+    elif adapter == "gate_reuse" and L > 1:
         rank = cfg.n_experts
         a = router[1:].clone().contiguous()
         b = torch.eye(cfg.n_experts, dtype=router.dtype, device=dev).expand(L - 1, -1, -1).contiguous()
