@@ -441,8 +441,11 @@ def resident_run(cfg, m, H_dev, W, K, peak, algo_bytes, device):
         full.reset_stats()
         el, _, _ = timed_run(full, H_dev, W, K, 1)
         st = full.stats()
+        nl = max(st["ffn_launches"], 1)
         leg = {"tok_s": K * cfg.batch / (el / 1e3), "us_per_layer": el * 1e3 / (K * cfg.n_layers),
-               "host_free_steps": st["host_free_steps"], "misses": st["misses"]}
+               "host_free_steps": st["host_free_steps"], "misses": st["misses"],
+               "router_window_us": st["router_window_us"] / nl, "reduce_window_us": st["reduce_window_us"] / nl,
+               "idle_between_kernels_us_per_layer": st["gap_us"] / nl}
         if st["host_free_steps"] and st["ffn_window_us"] > 0:
             win = st["ffn_window_us"] / max(st["ffn_launches"], 1)
             leg.update(ffn_window_us=win, ffn_gb_s_in_window=algo_bytes / (win * 1e-6) / 1e9,

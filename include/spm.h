@@ -135,6 +135,9 @@ typedef struct {
     double   recall_sum;         /* sum over (step, layer >= 1, token) of |T ∩ Top_M(s)| / K, M = budget  */
     uint64_t recall_count;       /*   ExpertRecall@M = recall_sum / recall_count  (Section 4.1)          */
     uint64_t host_free_steps;    /* decode steps enqueued without a host turn (spm_set_host_free)        */
+    double router_window_us;     /* in-kernel windows of the routing kernels (first leader past its launch      */
+    double reduce_window_us;     /*   dependency -> last leader done) and of the combine kernels, timing on     */
+    double gap_us;               /* device idle time between consecutive clocked kernels of the compute stream  */
 } spm_stats;
 
 /* ---- packed expert layout ------------------------------------------------

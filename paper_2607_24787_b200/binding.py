@@ -53,7 +53,8 @@ class Stats(C.Structure):
                                            "late_arrivals", "h2d_bytes", "ffn_launches", "kernel_launches")]
                 + [("ffn_us", C.c_double), ("ffn_window_us", C.c_double), ("stall_us", C.c_double), ("ready_sum", C.c_double),
                    ("ready_count", C.c_uint64), ("recall_sum", C.c_double), ("recall_count", C.c_uint64),
-                   ("host_free_steps", C.c_uint64)])
+                   ("host_free_steps", C.c_uint64), ("router_window_us", C.c_double), ("reduce_window_us", C.c_double),
+                   ("gap_us", C.c_double)])
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}

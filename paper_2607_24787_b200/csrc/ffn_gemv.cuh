@@ -277,10 +277,12 @@ constexpr int kReduceGroups = 8;
 constexpr int kReduceMaxRows = 40;     // rows per group: kReduceGroups * kReduceMaxRows >= max G
 
 static __global__ void __launch_bounds__(kReduceCols * kReduceGroups)
-ffn_reduce_kernel(const float* __restrict__ partial, const float* h_in, float* h_out, int G, int D) {
+ffn_reduce_kernel(const float* __restrict__ partial, const float* h_in, float* h_out, int G, int D,
+                  unsigned long long* clock = nullptr) {
     __shared__ float part[kReduceGroups][kReduceCols];
     grid_dep_launch();
     grid_dep_wait();
+    if (clock && threadIdx.x == 0) atomicMin(clock, global_timer_ns());
     const int tok = blockIdx.y;
     const int col = threadIdx.x % kReduceCols, grp = threadIdx.x / kReduceCols;
     const int d = blockIdx.x * kReduceCols + col;
@@ -300,6 +302,10 @@ ffn_reduce_kernel(const float* __restrict__ partial, const float* h_in, float* h
 #pragma unroll
         for (int g = 1; g < kReduceGroups; ++g) tot += part[g][col];
         h_out[size_t(tok) * D + d] = h_in[size_t(tok) * D + d] + tot;
+    }
+    if (clock) {
+        __syncthreads();
+        if (threadIdx.x == 0) atomicMax(clock + 1, global_timer_ns());
     }
 }
 

@@ -53,6 +53,11 @@ struct RouterArgs {
     Mailbox* mailbox;        // device view of a host-mapped mailbox (may be null)
     const short* slot_map;   // optional [n] slot of each expert of this layer (device memory) ...
     short* codes_out;        // ... and where to leave the slots of the routed experts, [nb][K]
+    unsigned long long* clock;   // optional {first leader past its dependency wait, last leader done} in ns
+    const float* partial;    // optional [nb][G][D] partial rows of the preceding expert kernel: the hidden row is
+    int G;                   //   then h + sum of them (summed here instead of by a combine kernel) ...
+    float* h_out;            //   ... and written back here ([nb][D], may alias h)
+    int publish_seq;         // fence and publish the sequence number for hosts that read untagged payload
     uint32_t seq;
     int D, n, K, r, nb, renorm, do_router, do_adapter;
     float eps;
@@ -94,12 +99,23 @@ __device__ __forceinline__ void block_softmax(float* v, int n, float* scratch) {
 // position of element e in the ordering (value descending, index ascending)
 __device__ __forceinline__ int rank_of(const float* v, int n, int e) {
     const float ve = v[e];
-    int c = 0;
-    for (int j = 0; j < n; ++j) c += (v[j] > ve) || (v[j] == ve && j < e);
+    int c = 0, j = 0;
+    if ((reinterpret_cast<uintptr_t>(v) & 15) == 0) {
+        for (; j + 4 <= n; j += 4) {
+            const float4 t = *reinterpret_cast<const float4*>(v + j);
+            c += (t.x > ve) || (t.x == ve && j < e);
+            c += (t.y > ve) || (t.y == ve && j + 1 < e);
+            c += (t.z > ve) || (t.z == ve && j + 2 < e);
+            c += (t.w > ve) || (t.w == ve && j + 3 < e);
+        }
+    }
+    for (; j < n; ++j) c += (v[j] > ve) || (v[j] == ve && j < e);
     return c;
 }
 
 constexpr int kRouterCluster = 8;   // CTAs per token, one thread-block cluster
+constexpr int kReduceGroupsR = 8;   // runs of partial rows (= warps of a CTA); must equal the combine kernel's group count
+constexpr int kReduceChunkR = 20;   // partial rows a lane keeps in flight
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -166,7 +182,7 @@ __device__ __forceinline__ int32_t tagged(uint32_t seq, int value) { return int3
 // memory; after one cluster barrier the leader runs the router tail (softmax, Top-K, renormalise)
 // on its first four warps and the adapter tail (up-projection, softmax, ranking) on the other four.
 template <typename WT>
-__global__ void __launch_bounds__(kRouterThreads)
+__global__ void __launch_bounds__(kRouterThreads, 1)
 router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     constexpr int VEC = 16 / int(sizeof(WT));
     constexpr int MAXIT = 8;        // hidden <= MAXIT * 32 * VEC
@@ -181,11 +197,12 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     float* psel = scratch + 16;                                 // [K]
     int* isel = reinterpret_cast<int*>(psel + SPM_MAX_TOPK);    // [K]
     float* bs = reinterpret_cast<float*>(isel + SPM_MAX_TOPK);  // [n * r] adapter up-projection (leader)
+    float* part = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(bs + a.n * a.r) + 15) & ~uintptr_t(15));   // [kReduceGroupsR][D / cluster] group sums of partial rows
+    short* smap = reinterpret_cast<short*>(part + a.D);          // [n] slot of each expert (leader)
     __shared__ int s_last;
-    __shared__ float s_tot;
 
 #ifdef SPM_ROUTER_TIMESTAMPS
-    unsigned long long ts[8];
+    unsigned long long ts[12] = {};
     ts[0] = global_timer_ns();
 #define SPM_TS(i) ts[i] = global_timer_ns()
 #else
@@ -204,29 +221,41 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
 
     // ---- weights first: none of them depends on the kernel before this one, so in a launch that
-    // overlaps its predecessor they are already in registers when the hidden row becomes readable.
-    // Router rows then adapter-A rows, one warp per row, ROWS rows in flight.
+    // overlaps its predecessor they are already in registers (or on their way into L2) when the
+    // hidden row becomes readable. Router rows then adapter-A rows, one warp per row, ROWS rows in flight.
     const int n_r = a.do_router ? n : 0;
     const int rows = n_r + (a.do_adapter ? a.r : 0);
     constexpr int STRIDE = kRouterCluster * kRouterWarps;
+    const bool fused = a.partial != nullptr;      // this launch also sums the preceding expert kernel's partial rows
     uint4 v[ROWS][MAXIT];
+    auto row_ptr = [&](int row) {
+        return row < n_r ? static_cast<const WT*>(a.router_w) + size_t(row) * D
+                         : static_cast<const WT*>(a.adapter_a) + size_t(row - n_r) * D;
+    };
     auto load_rows = [&](int row0) {
 #pragma unroll
         for (int rr = 0; rr < ROWS; ++rr) {
             const int row = row0 + rr * STRIDE;
-            if (row < rows) {
-                const WT* wrow = row < n_r ? static_cast<const WT*>(a.router_w) + size_t(row) * D
-                                           : static_cast<const WT*>(a.adapter_a) + size_t(row - n_r) * D;
 #pragma unroll
-                for (int it = 0; it < MAXIT; ++it) {
-                    const int i = (it * 32 + lane) * VEC;
-                    if (i < D) v[rr][it] = __ldg(reinterpret_cast<const uint4*>(wrow + i));
-                }
+            for (int it = 0; it < MAXIT; ++it) {
+                const int i = (it * 32 + lane) * VEC;
+                v[rr][it] = (row < rows && i < D) ? __ldg(reinterpret_cast<const uint4*>(row_ptr(row) + i)) : make_uint4(0, 0, 0, 0);
             }
         }
     };
     int row0 = int(cr) * kRouterWarps + wi;
-    load_rows(row0);
+    if (!fused) {
+        load_rows(row0);
+    } else {
+        // the registers are needed for the partial rows first: start the weights on their way into L2
+#pragma unroll
+        for (int rr = 0; rr < ROWS; ++rr) {
+            const int row = row0 + rr * STRIDE;
+            if (row < rows)
+                for (int i = lane * 128; i < D * int(sizeof(WT)); i += 32 * 128)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(row_ptr(row)) + i));
+        }
+    }
     constexpr int NV4 = MAXIT * 32 * VEC / (kRouterThreads * 4);   // float4 per thread at the largest hidden size
     float4 gv[NV4];
     if (a.do_router) {
@@ -236,16 +265,72 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
             if (i < D) gv[c] = *reinterpret_cast<const float4*>(a.gamma + i);
         }
     }
-    // leader: the small adapter up-projection is needed only in the tail
+    // leader: the small adapter up-projection and the slot map are needed only in the tail
     if (leader && a.do_adapter) {
         const WT* B = static_cast<const WT*>(a.adapter_b);
         for (int i = threadIdx.x; i < n * a.r; i += kRouterThreads) bs[i] = load_weight(B, i);
     }
+    if (leader && a.slot_map)
+        for (int i = threadIdx.x; i < n; i += kRouterThreads) smap[i] = a.slot_map[i];
 
-    // ---- router input: the hidden row (written by the preceding kernel) is normalised ----------
+    // ---- router input: the hidden row (written by the preceding kernels) is normalised ----------
     grid_dep_wait();
+    SPM_TS(8);
+    if (a.clock && leader && threadIdx.x == 0) atomicMin(a.clock, global_timer_ns());
+    bool cluster_started = false;      // the start-of-kernel cluster barrier has been waited for
+    if (fused) {
+        // h = h + sum over the expert kernel's CTAs of their partial rows, in the combine kernel's
+        // order: kReduceGroupsR runs of consecutive rows, each summed front to back, the runs then
+        // added in order, the residual last. This CTA owns D / cluster columns; warp g sums run g.
+        const int slice = D / kRouterCluster, nq = slice / 4;
+        const int col0 = int(cr) * slice;
+        const int per = (a.G + kReduceGroupsR - 1) / kReduceGroupsR;
+        const int c0 = wi * per, c1 = min(a.G, c0 + per);
+        float hin = 0.f;
+        if (threadIdx.x < slice) hin = a.h[size_t(tok) * D + col0 + threadIdx.x];
+        const float* pbase = a.partial + size_t(tok) * a.G * D + col0;
+        // a lane owns column quads lane and lane + 32 of the slice; all rows of its run are in
+        // flight together for both before the first addition
+        constexpr int QPL = 2;
+        for (int r0 = c0; r0 < c1 || r0 == c0; r0 += kReduceChunkR) {
+            float4 t[QPL][kReduceChunkR];
+#pragma unroll
+            for (int j = 0; j < QPL; ++j) {
+                const int q = lane + 32 * j;
+#pragma unroll
+                for (int i = 0; i < kReduceChunkR; ++i)
+                    t[j][i] = (q < nq && r0 + i < c1) ? __ldcg(reinterpret_cast<const float4*>(pbase + size_t(r0 + i) * D) + q)
+                                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int j = 0; j < QPL; ++j) {
+                const int q = lane + 32 * j;
+                if (q >= nq) continue;
+                float4 acc = r0 == c0 ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<const float4*>(part + wi * slice + q * 4);
+#pragma unroll
+                for (int i = 0; i < kReduceChunkR; ++i) { acc.x += t[j][i].x; acc.y += t[j][i].y; acc.z += t[j][i].z; acc.w += t[j][i].w; }
+                *reinterpret_cast<float4*>(part + wi * slice + q * 4) = acc;
+            }
+        }
+        __syncthreads();
+        asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+        cluster_started = true;
+        if (threadIdx.x < slice) {
+            float tot = part[threadIdx.x];
+#pragma unroll
+            for (int g = 1; g < kReduceGroupsR; ++g) tot += part[g * slice + threadIdx.x];
+            const float hv1 = hin + tot;
+            a.h_out[size_t(tok) * D + col0 + threadIdx.x] = hv1;
+#pragma unroll
+            for (uint32_t dst = 0; dst < kRouterCluster; ++dst) dsmem_store(xs + col0 + threadIdx.x, dst, hv1);
+        }
+        load_rows(row0);                 // L2 hits by now; in flight across the barrier and the normalisation
+        SPM_TS(9);
+        cluster_sync_all();              // every CTA holds the whole updated row in xs
+        SPM_TS(10);
+    }
     if (a.do_router) {
-        const float* ht = a.h + size_t(tok) * D;
+        const float* ht = fused ? xs : a.h + size_t(tok) * D;
         float4 hv[NV4];
 #pragma unroll
         for (int c = 0; c < NV4; ++c) {
@@ -281,26 +366,37 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     __syncthreads();
     SPM_TS(1);
 
-    asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+    if (!cluster_started) asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
     while (row0 < rows) {
+        // per row the products are accumulated in element order; the rows of a batch share each
+        // 16-byte read of the activations
+        float acc[ROWS];
+#pragma unroll
+        for (int rr = 0; rr < ROWS; ++rr) acc[rr] = 0.f;
+#pragma unroll
+        for (int it = 0; it < MAXIT; ++it) {
+            const int i = (it * 32 + lane) * VEC;
+            if (i < D) {
+                float xv[VEC];
+#pragma unroll
+                for (int q = 0; q < VEC; q += 4) {
+                    const float4 t = *reinterpret_cast<const float4*>(xs + i + q);
+                    xv[q] = t.x; xv[q + 1] = t.y; xv[q + 2] = t.z; xv[q + 3] = t.w;
+                }
+#pragma unroll
+                for (int rr = 0; rr < ROWS; ++rr) {
+                    float f[VEC];
+                    unpack16(v[rr][it], f);
+#pragma unroll
+                    for (int q = 0; q < VEC; ++q) acc[rr] = fmaf(f[q], xv[q], acc[rr]);
+                }
+            }
+        }
 #pragma unroll
         for (int rr = 0; rr < ROWS; ++rr) {
             const int row = row0 + rr * STRIDE;
-            if (row < rows) {
-                float acc = 0.f;
-#pragma unroll
-                for (int it = 0; it < MAXIT; ++it) {
-                    const int i = (it * 32 + lane) * VEC;
-                    if (i < D) {
-                        float f[VEC];
-                        unpack16(v[rr][it], f);
-#pragma unroll
-                        for (int q = 0; q < VEC; ++q) acc = fmaf(f[q], xs[i + q], acc);
-                    }
-                }
-                acc = warp_sum(acc);
-                if (lane == 0) dsmem_store(row < n_r ? zs + row : us + (row - n_r), 0, acc);
-            }
+            const float tot = warp_sum(acc[rr]);
+            if (row < rows && lane == 0) dsmem_store(row < n_r ? zs + row : us + (row - n_r), 0, tot);
         }
         row0 += ROWS * STRIDE;
         if (row0 < rows) load_rows(row0);
@@ -327,18 +423,14 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
             if (rk < a.K) { isel[rk] = e; psel[rk] = ps[e]; }
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (ht == 0) {
+        if (ht < a.K) {
             float tot = 0.f;
             for (int k = 0; k < a.K; ++k) tot += psel[k];
-            s_tot = tot;
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (ht < a.K) {
             a.ids[size_t(tok) * a.K + ht] = isel[ht];
-            a.w[size_t(tok) * a.K + ht] = a.renorm ? psel[ht] / s_tot : psel[ht];
+            a.w[size_t(tok) * a.K + ht] = a.renorm ? psel[ht] / tot : psel[ht];
             if (mb) mb->ids[tok * a.K + ht] = tagged(tag, isel[ht]);      // the host may start on these at once
             // slot numbers for an expert kernel that follows without a host turn
-            if (a.codes_out) a.codes_out[tok * a.K + ht] = a.slot_map[isel[ht]];
+            if (a.codes_out) a.codes_out[tok * a.K + ht] = smap[isel[ht]];
         }
     }
     SPM_TS(4);
@@ -367,7 +459,10 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     if (a.nb > 1) {
         __threadfence();
         __syncthreads();
-        if (threadIdx.x == 0) s_last = atomicAdd(&a.counters[0], 1u) == unsigned(a.nb - 1);
+        if (threadIdx.x == 0) {
+            if (a.clock) atomicMax(a.clock + 1, global_timer_ns());
+            s_last = atomicAdd(&a.counters[0], 1u) == unsigned(a.nb - 1);
+        }
         __syncthreads();
         if (!s_last) return;
         __threadfence();
@@ -389,17 +484,22 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     }
     SPM_TS(6);
     // final flag for callers that read untagged payload (scores): fence, then the sequence number
-    __threadfence_system();
-    __syncthreads();
-    if (threadIdx.x == 0 && mb) mb->seq = a.seq;
+    if (a.publish_seq) {
+        __threadfence_system();
+        __syncthreads();
+        if (threadIdx.x == 0 && mb) mb->seq = a.seq;
+    }
+    if (threadIdx.x == 0 && a.clock) atomicMax(a.clock + 1, global_timer_ns());
 #ifdef SPM_ROUTER_TIMESTAMPS
     SPM_TS(7);
-    if (threadIdx.x == 0) for (int i = 0; i < 8; ++i) reinterpret_cast<unsigned long long*>(a.pihat)[i] = ts[i];
+    if (threadIdx.x == 0 || threadIdx.x == 128)
+        for (int i = 0; i < 12; ++i) reinterpret_cast<unsigned long long*>(a.pihat)[(threadIdx.x >> 7) * 12 + i] = ts[i];
 #endif
 }
 
 inline size_t router_smem_bytes(int D, int n, int r) {
-    return sizeof(float) * (size_t(D) + 3 * size_t(n) + size_t(r) + 16 + 2 * SPM_MAX_TOPK + size_t(n) * r);
+    return sizeof(float) * (2 * size_t(D) + 3 * size_t(n) + size_t(r) + 16 + 2 * SPM_MAX_TOPK + size_t(n) * r) +
+           ((size_t(n) * sizeof(short) + 15) & ~size_t(15)) + 16;
 }
 
 }  // namespace spm

@@ -33,6 +33,8 @@ struct bf16_t { uint16_t v; };
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+enum ClockKind : uint8_t { kClkFfn = 0, kClkRouter = 1, kClkReduce = 2 };   // owners of in-kernel clock slots
+
 struct Timing {            // CUDA events of one step, per layer
     std::vector<cudaEvent_t> k1_done, ffn_start, ffn_end;
     std::vector<uint8_t> used;
@@ -57,7 +59,8 @@ struct spm_ctx {
     int* ws_status = nullptr;
     unsigned long long* ws_clock = nullptr;
     int clock_used = 0;
-    double window_us = 0;
+    std::vector<uint8_t> clock_kind;          // which kernel each armed clock slot belongs to (ClockKind)
+    double window_us = 0, router_window_us = 0, reduce_window_us = 0, gap_us = 0;
     // batched tensor-core path (bf16, max_batch > 1, no shared experts, I and D multiples of 128)
     bool tc_ok = false;
     int batched_path = 0;                 // 0: tensor cores when possible, 1: always the per-token GEMV
@@ -143,6 +146,8 @@ int fail(spm_ctx* c, int code, const char* fmt, ...) {
     return code;
 }
 
+int take_clock(spm_ctx* c, ClockKind kind, unsigned long long** out);
+
 #define CU(c, call)                                                                        \
     do {                                                                                   \
         cudaError_t e_ = (call);                                                           \
@@ -175,7 +180,7 @@ size_t blob_bytes_of(const spm_model_cfg* m) {
 }
 
 constexpr int kMaxCtasBatch1 = 296;
-constexpr int kClockSlots = 4096;     // in-kernel {start, end} pairs between two harvests
+constexpr int kClockSlots = 12288;    // in-kernel {start, end} pairs between two harvests
 constexpr int kDescRing = 8;          // wave descriptors in flight for the batched tensor-core path
 constexpr int kTraceRing = 8;         // host-free steps whose bookkeeping may be outstanding
 
@@ -186,6 +191,7 @@ bool tc_supported(const spm_model_cfg* m) {
            m->hidden % kGgTileRows == 0;
 }
 static_assert(kMaxCtasBatch1 <= kReduceGroups * kReduceMaxRows, "reduce kernel covers every grid size");
+static_assert(kReduceGroups == kReduceGroupsR && kReduceGroupsR == kRouterWarps, "the routing kernel folds partial rows in the combine kernel's order");
 
 int ffn_grid_for(const spm_ctx* c, int nb) {
     if (nb == 1) return c->ffn_ctas > 0 ? std::min(c->ffn_ctas, kMaxCtasBatch1) : c->num_sms;
@@ -337,10 +343,12 @@ struct RouterRoute {
     const short* slot_map;
     short* codes_out;
     bool pdl;
+    const float* partial;      // partial rows of the preceding layer's expert kernel to fold into the hidden row, or null
+    int G;
 };
 
 int launch_router(spm_ctx* c, int layer, const float* h, const float* x_in, int nb, float* x_norm,
-                  float* logits_out, bool do_router, bool do_adapter, const RouterRoute* route = nullptr) {
+                  float* logits_out, bool do_router, bool do_adapter, const RouterRoute* route = nullptr, bool publish_seq = true) {
     const spm_model_cfg& m = c->cfg;
     RouterArgs a{};
     const size_t D = m.hidden, n = m.n_experts, r = m.adapter_rank;
@@ -364,6 +372,11 @@ int launch_router(spm_ctx* c, int layer, const float* h, const float* x_in, int 
     a.mailbox = route ? route->mailbox_dev : c->mb_dev;
     a.slot_map = route ? route->slot_map : nullptr;
     a.codes_out = route ? route->codes_out : nullptr;
+    a.partial = route ? route->partial : nullptr;
+    a.G = route ? route->G : 0;
+    a.h_out = const_cast<float*>(h);
+    a.publish_seq = publish_seq;
+    if (int rc = take_clock(c, kClkRouter, &a.clock)) return rc;
     // Sequence numbers whose low 16 bits are zero are skipped, and the words this launch will
     // publish are zeroed first, so a word left by an older launch can never carry the current tag.
     ++c->seq;
@@ -511,16 +524,32 @@ void harvest(spm_ctx* c, Timing& t) {
 }
 
 // Read back the in-kernel {first start, last end} pairs written so far and re-arm the slots.
+// Slots are handed out in stream order, so the distance from one kernel's end to the next one's
+// start is the idle time between them on the device (launch gaps, host turns, waits for copies).
 int harvest_clock(spm_ctx* c) {
     if (c->clock_used == 0) return SPM_OK;
     std::vector<unsigned long long> h(size_t(c->clock_used) * 2);
     CU(c, cudaStreamSynchronize(c->compute));
     CU(c, cudaMemcpy(h.data(), c->ws_clock, h.size() * 8, cudaMemcpyDeviceToHost));
-    for (int i = 0; i < c->clock_used; ++i)
-        if (h[2 * i + 1] > h[2 * i]) c->window_us += double(h[2 * i + 1] - h[2 * i]) * 1e-3;
+    for (int i = 0; i < c->clock_used; ++i) {
+        if (h[2 * i + 1] <= h[2 * i]) continue;
+        const double us = double(h[2 * i + 1] - h[2 * i]) * 1e-3;
+        (c->clock_kind[i] == kClkFfn ? c->window_us : c->clock_kind[i] == kClkRouter ? c->router_window_us : c->reduce_window_us) += us;
+        if (i > 0 && h[2 * i - 1] > h[2 * i - 2] && h[2 * i] > h[2 * i - 1]) c->gap_us += double(h[2 * i] - h[2 * i - 1]) * 1e-3;
+    }
     for (int i = 0; i < c->clock_used; ++i) { h[2 * i] = ~0ull; h[2 * i + 1] = 0; }
     CU(c, cudaMemcpy(c->ws_clock, h.data(), h.size() * 8, cudaMemcpyHostToDevice));
     c->clock_used = 0;
+    return SPM_OK;
+}
+
+// Next clock slot for a kernel of the given kind (null when timing is off).
+int take_clock(spm_ctx* c, ClockKind kind, unsigned long long** out) {
+    *out = nullptr;
+    if (!c->timing) return SPM_OK;
+    if (c->clock_used == kClockSlots) if (int rc = harvest_clock(c)) return rc;
+    c->clock_kind[c->clock_used] = kind;
+    *out = c->ws_clock + 2 * size_t(c->clock_used++);
     return SPM_OK;
 }
 
@@ -660,11 +689,9 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
         }
 
         const bool first = wave == 0, last = wave == n_waves - 1;
+        const bool use_tc = nb > 1 && c->tc_ok && c->batched_path == 0;
         unsigned long long* clock_slot = nullptr;
-        if (c->timing) {
-            if (c->clock_used == kClockSlots) if (int rc = harvest_clock(c)) return rc;
-            clock_slot = c->ws_clock + 2 * size_t(c->clock_used++);
-        }
+        if (!use_tc) if (int rc = take_clock(c, kClkFfn, &clock_slot)) return rc;
         auto fill = [&](auto& a) {
             a.pool = slot_ptr(c, layer, 0);
             a.shared = m.n_shared ? static_cast<const unsigned char*>(c->buf.shared_experts) + size_t(layer) * m.n_shared * c->blob : nullptr;
@@ -695,7 +722,6 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
                 a.count[tk] = (unsigned char)cnt;
             }
         };
-        const bool use_tc = nb > 1 && c->tc_ok && c->batched_path == 0;
         if (use_tc) {
             if (int rc = launch_grouped_wave(c, layer, x_norm, ids, w, nb, h_inout, slot_of_expert, first, last, t, ring)) return rc;
         } else {
@@ -712,8 +738,10 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
             }
             if (t && last) CU(c, cudaEventRecord(t->ffn_end[layer], c->compute));
             if (ring >= 0 && last) { CU(c, cudaEventRecord(c->ring_end[ring], c->compute)); c->ring_used[ring] = 1; }
+            unsigned long long* reduce_clock = nullptr;
+            if (int rc = take_clock(c, kClkReduce, &reduce_clock)) return rc;
             ffn_reduce_kernel<<<dim3((m.hidden + kReduceCols - 1) / kReduceCols, nb), kReduceCols * kReduceGroups, 0, c->compute>>>(
-                c->ws_partial, h_inout, h_inout, G, m.hidden);
+                c->ws_partial, h_inout, h_inout, G, m.hidden, reduce_clock);
             CU(c, cudaGetLastError());
             c->kernel_launches += 2;
             c->ffn_launches++;
@@ -771,7 +799,7 @@ int step_layers(spm_ctx* c, float* h_out, int nb, Timing* t, const Mailbox* trac
                 CU(c, cudaGetLastError());
                 c->kernel_launches++;
             }
-            if (int rc = launch_router(c, l, h_out, nullptr, nb, c->ws_x, nullptr, true, predict && has_adapter)) return rc;
+            if (int rc = launch_router(c, l, h_out, nullptr, nb, c->ws_x, nullptr, true, predict && has_adapter, nullptr, false)) return rc;
             if (t) CU(c, cudaEventRecord(t->k1_done[l], c->compute));
             if (int rc = wait_tagged(c, c->mb_host->ids, nb * K, ids.data(), "expert ids")) return rc;
         } else {
@@ -891,13 +919,15 @@ int enqueue_host_free_step(spm_ctx* c, const float* h_in, int nb, float* h_out) 
             c->kernel_launches++;
         }
         short* codes = c->ws_codes + size_t(l) * m.max_batch * SPM_MAX_TOPK;
-        RouterRoute route{c->tr_dev + size_t(slot) * L + l, c->ws_slot_map + size_t(l) * n, codes, true};
-        if (int rc = launch_router(c, l, h_out, nullptr, nb, c->ws_x, nullptr, true, predict && l <= L - 2, &route)) return rc;
+        // On the GEMV path the routing kernel of layer l + 1 also folds layer l's partial rows into the
+        // hidden row, so only the last layer needs the combine kernel.
+        const bool use_tc = nb > 1 && c->tc_ok && c->batched_path == 0;
+        const bool fold = !use_tc && l > 0 && c->stub_us == 0;
+        RouterRoute route{c->tr_dev + size_t(slot) * L + l, c->ws_slot_map + size_t(l) * n, codes, true,
+                          fold ? c->ws_partial : nullptr, G};
+        if (int rc = launch_router(c, l, h_out, nullptr, nb, c->ws_x, nullptr, true, predict && l <= L - 2, &route, false)) return rc;
         unsigned long long* clock_slot = nullptr;
-        if (c->timing) {
-            if (c->clock_used == kClockSlots) if (int rc = harvest_clock(c)) return rc;
-            clock_slot = c->ws_clock + 2 * size_t(c->clock_used++);
-        }
+        if (!use_tc) if (int rc = take_clock(c, kClkFfn, &clock_slot)) return rc;
         auto fill = [&](auto& a) {
             a.pool = slot_ptr(c, l, 0);
             a.shared = m.n_shared ? static_cast<const unsigned char*>(c->buf.shared_experts) + size_t(l) * m.n_shared * c->blob : nullptr;
@@ -912,7 +942,7 @@ int enqueue_host_free_step(spm_ctx* c, const float* h_in, int nb, float* h_out) 
             a.I = m.inter; a.K = K; a.n_slots = c->S; a.n_shared = m.n_shared;
             for (int tk = 0; tk < nb; ++tk) a.count[tk] = (unsigned char)(K + m.n_shared);   // launch shape only
         };
-        if (nb > 1 && c->tc_ok && c->batched_path == 0) {
+        if (use_tc) {
             // wave plan on the device, then gather -> grouped tcgen05 FFN -> combine
             unsigned char* dd = c->tc_desc_dev;        // stream-ordered reuse of the first descriptor slot
             GgUnit* units = reinterpret_cast<GgUnit*>(dd);
@@ -941,9 +971,14 @@ int enqueue_host_free_step(spm_ctx* c, const float* h_in, int nb, float* h_out) 
             fill(a);
             CU(c, launch_gemv<SPM_MAX_BATCH>(c, a, G, nb, true));
         }
-        CU(c, launch_k(ffn_reduce_kernel, dim3((m.hidden + kReduceCols - 1) / kReduceCols, nb), dim3(kReduceCols * kReduceGroups), 0,
-                       c->compute, true, (const float*)c->ws_partial, (const float*)h_out, h_out, G, m.hidden));
-        c->kernel_launches += 3;
+        if (l == L - 1 || c->stub_us > 0) {
+            unsigned long long* reduce_clock = nullptr;
+            if (int rc = take_clock(c, kClkReduce, &reduce_clock)) return rc;
+            CU(c, launch_k(ffn_reduce_kernel, dim3((m.hidden + kReduceCols - 1) / kReduceCols, nb), dim3(kReduceCols * kReduceGroups), 0,
+                           c->compute, true, (const float*)c->ws_partial, (const float*)h_out, h_out, G, m.hidden, reduce_clock));
+            c->kernel_launches++;
+        }
+        c->kernel_launches += 2;
         c->ffn_launches++;
     }
     CU(c, cudaEventRecord(c->tr_ev[slot], c->compute));
@@ -1115,6 +1150,7 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
         if (!cu(cudaEventCreate(&c->ring_start[i]), "cudaEventCreate") || !cu(cudaEventCreate(&c->ring_end[i]), "cudaEventCreate")) return bail(SPM_ERR_CUDA);
     if (!cu(cudaStreamSynchronize(c->compute), "cudaStreamSynchronize")) return bail(SPM_ERR_CUDA);
 
+    c->clock_kind.assign(kClockSlots, kClkFfn);
     if (arm_clock(c) != SPM_OK) return bail(SPM_ERR_CUDA);
     c->budget = budget < 0 ? 1 : budget;
     if (budget < 0) {
@@ -1362,7 +1398,7 @@ int spm_reset_stats(spm_ctx* c) {
     std::fill(c->ring_used.begin(), c->ring_used.end(), 0);
     c->ring_us = 0;
     if (int rc = arm_clock(c)) return rc;
-    c->window_us = 0;
+    c->window_us = c->router_window_us = c->reduce_window_us = c->gap_us = 0;
     std::fill(c->layer_stall_us.begin(), c->layer_stall_us.end(), 0.0);
     std::fill(c->layer_ffn_us.begin(), c->layer_ffn_us.end(), 0.0);
     c->timed_steps = 0;
@@ -1385,7 +1421,7 @@ int spm_cache_reset(spm_ctx* c) {
     std::fill(c->ring_used.begin(), c->ring_used.end(), 0);
     c->ring_us = 0;
     if (int rc = arm_clock(c)) return rc;
-    c->window_us = 0;
+    c->window_us = c->router_window_us = c->reduce_window_us = c->gap_us = 0;
     std::fill(c->slot_pending.begin(), c->slot_pending.end(), 0);
     std::fill(c->has_plan.begin(), c->has_plan.end(), 0);
     std::fill(c->layer_stall_us.begin(), c->layer_stall_us.end(), 0.0);
@@ -1474,6 +1510,9 @@ int spm_get_stats(spm_ctx* c, spm_stats* out) {
     out->kernel_launches = c->kernel_launches;
     if (int rc = harvest_clock(c)) return rc;
     out->ffn_window_us = c->window_us;
+    out->router_window_us = c->router_window_us;
+    out->reduce_window_us = c->reduce_window_us;
+    out->gap_us = c->gap_us;
     out->ffn_us = c->ring_us;
     out->stall_us = 0;
     for (int l = 0; l < c->cfg.n_layers; ++l) { out->ffn_us += c->layer_ffn_us[l]; out->stall_us += c->layer_stall_us[l]; }
