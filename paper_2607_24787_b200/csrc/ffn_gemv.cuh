@@ -78,7 +78,7 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
     unsigned long long ts_first = 0, ts_loop = 0;
 #endif
     grid_dep_launch();
-    const unsigned long long t_entry = global_timer_ns();
+    const unsigned long long t_entry = (a.clock && threadIdx.x == 0) ? global_timer_ns() : 0ull;
     const int wi = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nw = blockDim.x >> 5;      // warps per CTA, chosen by the host to balance rows per warp
     const int tok = blockIdx.y;
@@ -107,39 +107,43 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
 
     const uint64_t pol = policy_evict_first();
     bool ok = true;
-    unsigned arrived = 0;     // lane 0: entries whose slot is known to hold its expert
-    int code_ent = -1, code_val = 0;   // lane 0: slot code of the entry being streamed
+    int src_ent = -1;                          // lane 0: entry being streamed and where its blob starts
+    const unsigned char* src_base = nullptr;   //         (null: the entry cannot be served)
+
+    // Blob of entry `ent`, resolved once per entry: slot number (launch arguments, or the routing
+    // kernel's device-side codes), range check, and with device-side waiting the arrival of its copy.
+    auto resolve = [&](int ent) -> const unsigned char* {
+        const int code = a.code_of(tok, ent);
+        if (code < 0) {
+            if (-1 - code >= a.n_shared) { atomicOr(a.status, kStatusBadSlot); return nullptr; }
+            return a.shared + size_t(-1 - code) * a.blob_bytes;
+        }
+        if (code >= a.n_slots) { atomicOr(a.status, kStatusBadSlot); return nullptr; }
+        if (a.ready) {
+            // Device-side wait: the copy stream bumps the slot's counter after the expert's bytes
+            // have landed. Bounded; on timeout the status word is set and the launch winds down.
+            const unsigned* f = a.ready + code;
+            const unsigned want = a.want[ent];
+            const unsigned long long t0 = global_timer_ns();
+            for (;;) {
+                unsigned v;
+                asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(f) : "memory");
+                if (int(v - want) >= 0) break;
+                __nanosleep(200);
+                if (global_timer_ns() - t0 > kWaitLimitNs) { atomicOr(a.status, kStatusCopyTimeout); return nullptr; }
+            }
+            asm volatile("fence.proxy.async;" ::: "memory");   // the weights are read through the async proxy
+        }
+        return a.pool + size_t(code) * a.blob_bytes;
+    };
 
     auto issue = [&](int i) {
         const int r = r_begin + wi + i * nw;
         const int ent = r / I;
         const int j = r - ent * I;
-        if (ent != code_ent) { code_ent = ent; code_val = a.code_of(tok, ent); }
-        const int code = code_val;
-        const unsigned char* base;
-        if (code >= 0) {
-            if (code >= a.n_slots) { atomicOr(a.status, kStatusBadSlot); return false; }
-            if (a.ready && !((arrived >> ent) & 1u)) {
-                // Device-side wait: the copy stream bumps the slot's counter after the expert's bytes
-                // have landed. Bounded; on timeout the status word is set and the launch winds down.
-                const unsigned* f = a.ready + code;
-                const unsigned want = a.want[ent];
-                const unsigned long long t0 = global_timer_ns();
-                for (;;) {
-                    unsigned v;
-                    asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(f) : "memory");
-                    if (int(v - want) >= 0) break;
-                    __nanosleep(200);
-                    if (global_timer_ns() - t0 > kWaitLimitNs) { atomicOr(a.status, kStatusCopyTimeout); return false; }
-                }
-                asm volatile("fence.proxy.async;" ::: "memory");   // the weights are read through the async proxy
-                arrived |= 1u << ent;
-            }
-            base = a.pool + size_t(code) * a.blob_bytes;
-        } else {
-            if (-1 - code >= a.n_shared) { atomicOr(a.status, kStatusBadSlot); return false; }
-            base = a.shared + size_t(-1 - code) * a.blob_bytes;
-        }
+        if (ent != src_ent) { src_ent = ent; src_base = resolve(ent); }
+        const unsigned char* base = src_base;
+        if (!base) return false;
         const int st = i % depth;
         mbar_arrive_expect_tx(bar0 + 8u * st, ROWB);
         bulk_g2s(ring0 + uint32_t(st) * ROWB, base + size_t(j) * ROWB, ROWB, bar0 + 8u * st, pol);
@@ -260,10 +264,12 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
         if (threadIdx.x == 0) atomicMax(a.clock + 1, global_timer_ns());
     }
 #ifdef SPM_FFN_TIMESTAMPS
-    // profiling aid: per-warp phase times, appended behind the partial rows
+    // profiling aid: per-warp phase times and the SM id, appended behind the partial rows
     if (lane == 0) {
-        unsigned long long* ts = reinterpret_cast<unsigned long long*>(a.partial + size_t(gridDim.y) * G * D) + (size_t(c) * nw + wi) * 4;
-        ts[0] = ts_start; ts[1] = ts_first; ts[2] = ts_loop; ts[3] = global_timer_ns();
+        unsigned long long* ts = reinterpret_cast<unsigned long long*>(a.partial + size_t(gridDim.y) * G * D) + (size_t(c) * nw + wi) * 5;
+        unsigned smid;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        ts[0] = ts_start; ts[1] = ts_first; ts[2] = ts_loop; ts[3] = global_timer_ns(); ts[4] = smid;
     }
 #endif
 }

@@ -41,7 +41,7 @@ __global__ void __launch_bounds__(kQ4MaxWarps * 32, 1)
 ffn_gemv_q4_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth, const int D) {
     extern __shared__ __align__(128) unsigned char smem[];
     grid_dep_launch();
-    const unsigned long long t_entry = global_timer_ns();
+    const unsigned long long t_entry = (a.clock && threadIdx.x == 0) ? global_timer_ns() : 0ull;
     const int wi = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nw = blockDim.x >> 5;
     const int tok = blockIdx.y;
@@ -75,21 +75,24 @@ ffn_gemv_q4_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth, co
 
     const uint64_t pol = policy_evict_first();
     bool ok = true;
-    int code_ent = -1, code_val = 0;
+    int src_ent = -1;                          // lane 0: entry being streamed and where its blob starts
+    const unsigned char* src_base = nullptr;   //         (null: the entry cannot be served)
+    auto resolve = [&](int ent) -> const unsigned char* {
+        const int code = a.code_of(tok, ent);
+        if (code < 0) {
+            if (-1 - code >= a.n_shared) { atomicOr(a.status, kStatusBadSlot); return nullptr; }
+            return a.shared + size_t(-1 - code) * a.blob_bytes;
+        }
+        if (code >= a.n_slots) { atomicOr(a.status, kStatusBadSlot); return nullptr; }
+        return a.pool + size_t(code) * a.blob_bytes;
+    };
     auto issue = [&](int i) {
         const int r = r_begin + wi + i * nw;
         const int ent = r / I;
         const int j = r - ent * I;
-        if (ent != code_ent) { code_ent = ent; code_val = a.code_of(tok, ent); }
-        const int code = code_val;
-        const unsigned char* base;
-        if (code >= 0) {
-            if (code >= a.n_slots) { atomicOr(a.status, kStatusBadSlot); return false; }
-            base = a.pool + size_t(code) * a.blob_bytes;
-        } else {
-            if (-1 - code >= a.n_shared) { atomicOr(a.status, kStatusBadSlot); return false; }
-            base = a.shared + size_t(-1 - code) * a.blob_bytes;
-        }
+        if (ent != src_ent) { src_ent = ent; src_base = resolve(ent); }
+        const unsigned char* base = src_base;
+        if (!base) return false;
         const int st = i % depth;
         mbar_arrive_expect_tx(bar0 + 8u * st, ROWB);
         bulk_g2s(ring0 + uint32_t(st) * ROWB, base + size_t(j) * ROWB, ROWB, bar0 + 8u * st, pol);

@@ -405,13 +405,22 @@ static __global__ void gg_combine_kernel(const float* __restrict__ partial, cons
     const int t = blockIdx.y;
     const int d = blockIdx.x * blockDim.x + threadIdx.x;
     if (d >= D) return;
+    const float h_in = h[size_t(t) * D + d];
     float acc = 0.f;
+    constexpr int JB = 8;                 // j-tiles fetched together
     for (int k = 0; k < K; ++k) {
         const int r = rowmap[t * SPM_MAX_TOPK + k];
         if (r < 0) continue;
-        for (int jt = 0; jt < n_jt; ++jt) acc += __ldcg(partial + (size_t(jt) * rows_cap + r) * D + d);
+        for (int j0 = 0; j0 < n_jt; j0 += JB) {
+            float v[JB];
+#pragma unroll
+            for (int j = 0; j < JB; ++j)
+                v[j] = j0 + j < n_jt ? __ldcg(partial + (size_t(j0 + j) * rows_cap + r) * D + d) : 0.f;
+#pragma unroll
+            for (int j = 0; j < JB; ++j) if (j0 + j < n_jt) acc += v[j];
+        }
     }
-    h[size_t(t) * D + d] += acc;
+    h[size_t(t) * D + d] = h_in + acc;
 }
 
 

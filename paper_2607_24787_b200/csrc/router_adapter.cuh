@@ -181,8 +181,10 @@ __device__ __forceinline__ int32_t tagged(uint32_t seq, int value) { return int3
 // weight rows of one token and deliver their dot products straight into the leader CTA's shared
 // memory; after one cluster barrier the leader runs the router tail (softmax, Top-K, renormalise)
 // on its first four warps and the adapter tail (up-projection, softmax, ranking) on the other four.
-template <typename WT>
-__global__ void __launch_bounds__(kRouterThreads, 1)
+// MINB = 1: all registers to one CTA per SM (the fold keeps 40 partial-row quads in flight);
+// MINB = 2: register budget halved so two CTAs share an SM, for batches with more CTAs than SMs.
+template <typename WT, int MINB>
+__global__ void __launch_bounds__(kRouterThreads, MINB)
 router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     constexpr int VEC = 16 / int(sizeof(WT));
     constexpr int MAXIT = 8;        // hidden <= MAXIT * 32 * VEC
@@ -226,7 +228,7 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     const int n_r = a.do_router ? n : 0;
     const int rows = n_r + (a.do_adapter ? a.r : 0);
     constexpr int STRIDE = kRouterCluster * kRouterWarps;
-    const bool fused = a.partial != nullptr;      // this launch also sums the preceding expert kernel's partial rows
+    const bool fused = MINB == 1 && a.partial != nullptr;   // this launch also sums the preceding expert kernel's partial rows
     uint4 v[ROWS][MAXIT];
     auto row_ptr = [&](int row) {
         return row < n_r ? static_cast<const WT*>(a.router_w) + size_t(row) * D
@@ -278,7 +280,7 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     SPM_TS(8);
     if (a.clock && leader && threadIdx.x == 0) atomicMin(a.clock, global_timer_ns());
     bool cluster_started = false;      // the start-of-kernel cluster barrier has been waited for
-    if (fused) {
+    if constexpr (MINB == 1) if (fused) {
         // h = h + sum over the expert kernel's CTAs of their partial rows, in the combine kernel's
         // order: kReduceGroupsR runs of consecutive rows, each summed front to back, the runs then
         // added in order, the residual last. This CTA owns D / cluster columns; warp g sums run g.

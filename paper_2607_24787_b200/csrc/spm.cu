@@ -407,13 +407,17 @@ int launch_router(spm_ctx* c, int layer, const float* h, const float* x_in, int 
         at[1].val.programmaticStreamSerializationAllowed = 1;
         lc.numAttrs = 2;
     }
-    if (m.dtype != SPM_DTYPE_FP32) {
-        if (smem > 48 * 1024) CU(c, cudaFuncSetAttribute(router_adapter_kernel<bf16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
-        CU(c, cudaLaunchKernelEx(&lc, router_adapter_kernel<bf16_t>, a));
-    } else {
-        if (smem > 48 * 1024) CU(c, cudaFuncSetAttribute(router_adapter_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
-        CU(c, cudaLaunchKernelEx(&lc, router_adapter_kernel<float>, a));
-    }
+    // more CTAs than SMs: the variant compiled for two CTAs per SM halves the number of waves
+    const bool dense = kRouterCluster * nb > c->num_sms && !a.partial;
+    auto go = [&](auto kern) -> int {
+        if (smem > 48 * 1024) CU(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+        CU(c, cudaLaunchKernelEx(&lc, kern, a));
+        return SPM_OK;
+    };
+    int rc;
+    if (m.dtype != SPM_DTYPE_FP32) rc = dense ? go(router_adapter_kernel<bf16_t, 2>) : go(router_adapter_kernel<bf16_t, 1>);
+    else rc = dense ? go(router_adapter_kernel<float, 2>) : go(router_adapter_kernel<float, 1>);
+    if (rc) return rc;
     CU(c, cudaGetLastError());
     c->kernel_launches++;
     return SPM_OK;
