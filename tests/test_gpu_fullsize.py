@@ -104,3 +104,37 @@ def test_one_full_depth_step_and_properties(qwen):
     again = m.decode_step(h)
     m.synchronize()                                        # the step runs on the library's stream, not torch's
     assert np.array_equal(f64(again)[0], outs[2])               # cold cache, other policy: identical output
+
+
+def test_fully_resident_host_free_steps_give_the_offloaded_bits(qwen):
+    # the router-preserving guarantee at full size: 16 slots per layer with prefetching against all
+    # 128 experts resident (host-free steps, 54 GiB of slots), same tokens -> identical outputs
+    from paper_2607_24787_b200.synth_model import build_from_synth
+    cfg, m = qwen
+    if torch.cuda.mem_get_info()[0] < 70 * 2 ** 30:
+        pytest.skip("not enough device memory for 128 slots per layer")
+    tok = synth.zipf_tokens(cfg, steps=4)
+    H = synth.embedding_rows(cfg, tok[:, 0])
+    m.cache_reset(); m.set_policy("adapter")
+    offloaded = []
+    for s in range(4):
+        h = H[s:s + 1].cuda(); torch.cuda.synchronize()
+        out = m.decode_step(h)
+        m.synchronize()
+        offloaded.append(out.cpu().numpy())
+    full = build_from_synth(cfg, slots=cfg.n_experts, budget=1, store=m.store)
+    try:
+        for l in range(cfg.n_layers):
+            assert full.prefetch_async(l, np.arange(cfg.n_experts, dtype=np.int32)) == cfg.n_experts
+        full.synchronize()
+        outs = []
+        for s in range(4):                                  # enqueued back to back, no synchronisation in between
+            h = H[s:s + 1].cuda(); torch.cuda.synchronize()
+            outs.append(full.decode_step(h))
+        full.synchronize()
+        st = full.stats()
+        assert st["host_free_steps"] == 4 and st["misses"] == 0 and st["hits"] == 4 * cfg.n_layers * cfg.top_k
+        for s in range(4):
+            assert np.array_equal(outs[s].cpu().numpy(), offloaded[s]), s
+    finally:
+        full.close()
