@@ -403,79 +403,95 @@ static __global__ void gg_combine_kernel(const float* __restrict__ partial, cons
     grid_dep_launch();
     grid_dep_wait();
     const int t = blockIdx.y;
-    const int d = blockIdx.x * blockDim.x + threadIdx.x;
+    const int d = (blockIdx.x * blockDim.x + threadIdx.x) * 4;     // four columns per thread
     if (d >= D) return;
-    const float h_in = h[size_t(t) * D + d];
-    float acc = 0.f;
+    const float4 h_in = *reinterpret_cast<const float4*>(h + size_t(t) * D + d);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     constexpr int JB = 8;                 // j-tiles fetched together
     for (int k = 0; k < K; ++k) {
         const int r = rowmap[t * SPM_MAX_TOPK + k];
         if (r < 0) continue;
         for (int j0 = 0; j0 < n_jt; j0 += JB) {
-            float v[JB];
+            float4 v[JB];
 #pragma unroll
             for (int j = 0; j < JB; ++j)
-                v[j] = j0 + j < n_jt ? __ldcg(partial + (size_t(j0 + j) * rows_cap + r) * D + d) : 0.f;
+                v[j] = j0 + j < n_jt ? __ldcg(reinterpret_cast<const float4*>(partial + (size_t(j0 + j) * rows_cap + r) * D + d))
+                                     : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-            for (int j = 0; j < JB; ++j) if (j0 + j < n_jt) acc += v[j];
+            for (int j = 0; j < JB; ++j)
+                if (j0 + j < n_jt) { acc.x += v[j].x; acc.y += v[j].y; acc.z += v[j].z; acc.w += v[j].w; }
         }
     }
-    h[size_t(t) * D + d] = h_in + acc;
+    *reinterpret_cast<float4*>(h + size_t(t) * D + d) = make_float4(h_in.x + acc.x, h_in.y + acc.y, h_in.z + acc.z, h_in.w + acc.w);
 }
-
 
 // Wave plan built on the device (all experts resident, one wave): the (token, k) pairs sorted by
 // expert id, then token, then k — the order the host-side planner produces — the units of every
-// routed expert, and the row of each pair for the combine step. One CTA; thread e owns expert e.
-constexpr int kGgPlanThreads = 1024;
+// routed expert, and the row of each pair for the combine step. One CTA, one thread per pair:
+// a pair's row is (pairs of lower experts) + (same-expert pairs in lower warps) + (same-expert
+// pairs in lower lanes of its warp), the last from a warp match, the others from small prefix sums.
+constexpr int kGgPlanThreads = 1024;     // >= SPM_MAX_BATCH * SPM_MAX_TOPK pairs
+static_assert(kGgPlanThreads >= SPM_MAX_BATCH * SPM_MAX_TOPK, "one thread per (token, k) pair");
+
+inline size_t gg_plan_smem(int n) { return (size_t(kGgPlanThreads / 32) * n + 3 * size_t(n)) * sizeof(int32_t); }
 
 static __global__ void __launch_bounds__(kGgPlanThreads)
 gg_plan_kernel(const int32_t* __restrict__ ids, const short* __restrict__ slot_map, int slot_base, int nb, int K, int n,
                int n_jt, GgUnit* __restrict__ units, GgRow* __restrict__ rows, int32_t* __restrict__ rowmap,
                int* __restrict__ counts /* {n_units, n_rows} */, int* status) {
     extern __shared__ int32_t plan_sm[];
-    int32_t* s_ids = plan_sm;                  // [nb * K]
-    int32_t* s_cnt = s_ids + nb * K;           // [n] pairs per expert -> first row
-    int32_t* s_rank = s_cnt + n;               // [n] routed experts before e
+    constexpr int NW = kGgPlanThreads / 32;
+    int32_t* tab = plan_sm;                    // [NW][n] same-expert pairs per warp -> exclusive prefix over warps
+    int32_t* cnt = tab + NW * n;               // [n] pairs per expert
+    int32_t* start = cnt + n;                  // [n] first row of the expert
+    int32_t* rank = start + n;                 // [n] routed experts before e, -1 if not routed
     grid_dep_launch();
+    const int tid = threadIdx.x, lane = tid & 31, wi = tid >> 5, total = nb * K;
+    for (int i = tid; i < NW * n; i += kGgPlanThreads) tab[i] = 0;      // independent of the preceding kernel
     grid_dep_wait();
-    const int tid = threadIdx.x, total = nb * K;
-    for (int i = tid; i < total; i += blockDim.x) s_ids[i] = __ldcg(ids + i);
-    for (int i = tid; i < nb * SPM_MAX_TOPK; i += blockDim.x) rowmap[i] = -1;
+    const int e = tid < total ? __ldcg(ids + tid) : -1;
+    for (int i = tid; i < nb * SPM_MAX_TOPK; i += kGgPlanThreads) rowmap[i] = -1;
     __syncthreads();
-    for (int e = tid; e < n; e += blockDim.x) {
-        int cnt = 0;
-        for (int i = 0; i < total; ++i) cnt += s_ids[i] == e;
-        s_cnt[e] = cnt;
+    const unsigned same = __match_any_sync(0xffffffffu, e);
+    const int before = __popc(same & ((1u << lane) - 1u));
+    if (e >= 0 && before == 0) tab[wi * n + e] = __popc(same);
+    __syncthreads();
+    for (int x = tid; x < n; x += kGgPlanThreads) {
+        int run = 0;
+        for (int w2 = 0; w2 < NW; ++w2) { const int c = tab[w2 * n + x]; tab[w2 * n + x] = run; run += c; }
+        cnt[x] = run;
     }
     __syncthreads();
-    if (tid == 0) {          // exclusive scans over at most SPM_MAX_EXPERTS entries
+    if (wi == 0) {           // exclusive scans over the experts: rows and routed-expert ranks
         int row = 0, routed = 0;
-        for (int e = 0; e < n; ++e) {
-            const int cnt = s_cnt[e];
-            s_cnt[e] = row;
-            s_rank[e] = cnt > 0 ? routed : -1;
-            row += cnt;
-            routed += cnt > 0;
+        for (int x0 = 0; x0 < n; x0 += 32) {
+            const int x = x0 + lane;
+            const int c = x < n ? cnt[x] : 0, r = c > 0;
+            int pc = c, pr = r;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int tc = __shfl_up_sync(0xffffffffu, pc, o), tr = __shfl_up_sync(0xffffffffu, pr, o);
+                if (lane >= o) { pc += tc; pr += tr; }
+            }
+            if (x < n) { start[x] = row + pc - c; rank[x] = r ? routed + pr - r : -1; }
+            row += __shfl_sync(0xffffffffu, pc, 31);
+            routed += __shfl_sync(0xffffffffu, pr, 31);
         }
-        counts[0] = routed * n_jt;
-        counts[1] = row;
+        if (lane == 0) { counts[0] = routed * n_jt; counts[1] = row; }
     }
     __syncthreads();
-    for (int e = tid; e < n; e += blockDim.x) {
-        if (s_rank[e] < 0) continue;
-        const int row0 = s_cnt[e];
-        int r = row0;
-        for (int i = 0; i < total; ++i)
-            if (s_ids[i] == e) {
-                const int t = i / K, k = i - t * K;
-                rows[r] = GgRow{t, k};
-                rowmap[t * SPM_MAX_TOPK + k] = r;
-                ++r;
-            }
-        const int slot = slot_map[e];
-        if (slot < 0) atomicOr(status, kStatusBadSlot);
-        for (int jt = 0; jt < n_jt; ++jt) units[s_rank[e] * n_jt + jt] = GgUnit{slot_base + (slot < 0 ? 0 : slot), jt, row0, r - row0};
+    if (e >= 0) {
+        const int r = start[e] + tab[wi * n + e] + before;
+        const int t = tid / K, k = tid - t * K;
+        rows[r] = GgRow{t, k};
+        rowmap[t * SPM_MAX_TOPK + k] = r;
+    }
+    for (int x = tid; x < n * n_jt; x += kGgPlanThreads) {
+        const int ex = x / n_jt, jt = x - ex * n_jt;
+        if (rank[ex] < 0) continue;
+        const int slot = slot_map[ex];
+        if (slot < 0 && jt == 0) atomicOr(status, kStatusBadSlot);
+        units[rank[ex] * n_jt + jt] = GgUnit{slot_base + (slot < 0 ? 0 : slot), jt, start[ex], cnt[ex]};
     }
 }
 

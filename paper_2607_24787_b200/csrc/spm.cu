@@ -616,7 +616,7 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
     CU(c, cudaGetLastError());
     if (t && last) CU(c, cudaEventRecord(t->ffn_end[layer], c->compute));
     if (ring >= 0 && last) { CU(c, cudaEventRecord(c->ring_end[ring], c->compute)); c->ring_used[ring] = 1; }
-    gg_combine_kernel<<<dim3((m.hidden + 127) / 128, nb), 128, 0, c->compute>>>(
+    gg_combine_kernel<<<dim3((m.hidden / 4 + 127) / 128, nb), 128, 0, c->compute>>>(
         c->tc_partial, reinterpret_cast<const int32_t*>(dd + c->tc_off_rowmap), K, c->n_jt, c->rows_cap, m.hidden, h_inout);
     CU(c, cudaGetLastError());
     c->kernel_launches += 3;
@@ -952,14 +952,14 @@ int enqueue_host_free_step(spm_ctx* c, const float* h_in, int nb, float* h_out) 
             GgUnit* units = reinterpret_cast<GgUnit*>(dd);
             GgRow* rows = reinterpret_cast<GgRow*>(dd + c->tc_off_rows);
             int32_t* rowmap = reinterpret_cast<int32_t*>(dd + c->tc_off_rowmap);
-            CU(c, launch_k(gg_plan_kernel, dim3(1), dim3(kGgPlanThreads), size_t(nb * K + 2 * n) * sizeof(int32_t), c->compute, true,
+            CU(c, launch_k(gg_plan_kernel, dim3(1), dim3(kGgPlanThreads), gg_plan_smem(n), c->compute, true,
                            (const int32_t*)c->ws_ids, (const short*)(c->ws_slot_map + size_t(l) * n), l * c->S, nb, K, n, c->n_jt,
                            units, rows, rowmap, c->tc_counts, c->ws_status));
             CU(c, launch_k(gg_gather_kernel, dim3(nb * K), dim3(128), 0, c->compute, true, (const float*)c->ws_x, (const float*)c->ws_w,
                            (const GgRow*)rows, 0, (const int*)(c->tc_counts + 1), m.hidden, K, c->tc_xs, c->tc_wrow));
             GgArgs ga{units, 0, c->tc_counts, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status};
             CU(c, launch_k(ffn_grouped_kernel, dim3(c->num_sms), dim3(kGgThreads), ffn_grouped_smem(), c->compute, true, c->wmap, c->xmap, ga));
-            CU(c, launch_k(gg_combine_kernel, dim3((m.hidden + 127) / 128, nb), dim3(128), 0, c->compute, true,
+            CU(c, launch_k(gg_combine_kernel, dim3((m.hidden / 4 + 127) / 128, nb), dim3(128), 0, c->compute, true,
                            (const float*)c->tc_partial, (const int32_t*)rowmap, K, c->n_jt, c->rows_cap, m.hidden, h_out));
             c->kernel_launches += 5;
             c->ffn_launches++;
@@ -1147,6 +1147,8 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
             return bail(SPM_ERR_CUDA);
         }
         if (!cu(cudaFuncSetAttribute(ffn_grouped_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(ffn_grouped_smem())), "cudaFuncSetAttribute")) return bail(SPM_ERR_CUDA);
+        if (gg_plan_smem(cfg->n_experts) > 48 * 1024 &&
+            !cu(cudaFuncSetAttribute(gg_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(gg_plan_smem(cfg->n_experts))), "cudaFuncSetAttribute")) return bail(SPM_ERR_CUDA);
         c->tc_ok = true;
     }
     c->ring_start.resize(64); c->ring_end.resize(64); c->ring_used.assign(64, 0);
