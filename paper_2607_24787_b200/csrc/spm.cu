@@ -84,6 +84,7 @@ struct spm_ctx {
     // per-slot copy events
     std::vector<cudaEvent_t> slot_ev;
     std::vector<uint8_t> slot_pending;
+    std::vector<size_t> slot_dep;             // slot whose event covers the batch this slot's latest copy belongs to
     std::vector<cudaEvent_t> pool_free;       // recorded after the last FFN that read pool l
     std::vector<uint8_t> pool_free_valid;
     cudaEvent_t wave_done = nullptr;
@@ -484,23 +485,28 @@ const unsigned char* host_blob(spm_ctx* c, int layer, int e) {
     return static_cast<const unsigned char*>(c->buf.host_experts) + (size_t(src) * c->cfg.n_experts + e) * c->blob;
 }
 
-// Enqueue one expert transfer on the copy stream and arm the slot's event.
-int issue_copy(spm_ctx* c, int layer, int e, int slot) {
+// Enqueue one expert transfer on the copy stream. Transfers are issued in batches (the misses of a
+// wave, the selections of a prefetch) that are awaited as a whole, so only the last transfer of a
+// batch records an event (`lead` = the slot whose event covers the batch): every stream operation
+// between two copies costs a few microseconds of link time. With device-side waiting each transfer
+// also bumps its slot's arrival counter, because the kernel then waits slot by slot.
+int issue_copy(spm_ctx* c, int layer, int e, int slot, size_t lead, bool last_of_batch) {
     const size_t k = size_t(layer) * c->S + slot;
     CU(c, cudaMemcpyAsync(slot_ptr(c, layer, slot), host_blob(c, layer, e), c->blob, cudaMemcpyHostToDevice, c->copy));
     if (c->copy_delay_us > 0) {
         attention_stub_kernel<<<1, 1, 0, c->copy>>>(uint64_t(c->copy_delay_us) * 1000ull);   // emulated slower tier
         CU(c, cudaGetLastError());
     }
-    CU(c, cudaEventRecord(c->slot_ev[k], c->copy));
-    // stream-ordered counter bump, for launches that wait for their copies on the device
-    if (StreamWriteValue32Fn wr = stream_write32_fn()) {
+    if (last_of_batch) CU(c, cudaEventRecord(c->slot_ev[lead], c->copy));
+    if (c->device_wait) {
+        // stream-ordered counter bump, for launches that wait for their copies on the device
+        StreamWriteValue32Fn wr = stream_write32_fn();
+        if (!wr) return fail(c, SPM_ERR_CUDA, "cuStreamWriteValue32 is not available");
         const uint32_t gen = ++c->slot_gen_host[k];
         if (wr(reinterpret_cast<CUstream>(c->copy), reinterpret_cast<CUdeviceptr>(c->ws_slot_gen + k), gen, 0) != CUDA_SUCCESS)
             return fail(c, SPM_ERR_CUDA, "cuStreamWriteValue32 failed");
-    } else if (c->device_wait) {
-        return fail(c, SPM_ERR_CUDA, "cuStreamWriteValue32 is not available");
     }
+    c->slot_dep[k] = lead;
     c->slot_pending[k] = 1;
     c->h2d_bytes += c->blob;
     return SPM_OK;
@@ -662,18 +668,21 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
     std::vector<int16_t>& slot_of_expert = c->wave_slot;   // experts computed in the current wave
     for (int wave = 0; wave < n_waves; ++wave) {
         slot_of_expert.assign(m.n_experts, -1);
-        bool any_copy = false;
+        int n_missed = 0, last_missed = -1;
         for (size_t i = 0; i < c->placements.size(); ++i) {
             const Placement& p = c->placements[i];
             if (p.wave != wave) continue;
             slot_of_expert[p.expert] = int16_t(p.slot);
-            if (p.missed) {
-                if (!any_copy) {
-                    if (int rc = order_copy_after_readers(c, layer)) return rc;
-                    if (wave > 0) CU(c, cudaStreamWaitEvent(c->copy, c->wave_done, 0));
-                    any_copy = true;
-                }
-                if (int rc = issue_copy(c, layer, p.expert, p.slot)) return rc;
+            if (p.missed) { ++n_missed; last_missed = int(i); }
+        }
+        if (n_missed > 0) {
+            if (int rc = order_copy_after_readers(c, layer)) return rc;
+            if (wave > 0) CU(c, cudaStreamWaitEvent(c->copy, c->wave_done, 0));
+            const size_t lead = size_t(layer) * c->S + c->placements[last_missed].slot;
+            for (size_t i = 0; i < c->placements.size(); ++i) {
+                const Placement& p = c->placements[i];
+                if (p.wave != wave || !p.missed) continue;
+                if (int rc = issue_copy(c, layer, p.expert, p.slot, lead, int(i) == last_missed)) return rc;
             }
         }
         for (size_t i = 0; i < c->placements.size(); ++i) {
@@ -681,11 +690,12 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
             if (p.wave != wave) continue;
             const size_t k = size_t(layer) * c->S + p.slot;
             if (!c->slot_pending[k]) continue;
-            cudaError_t q = cudaEventQuery(c->slot_ev[k]);
+            const size_t dep = c->slot_dep[k];       // (an event re-recorded by a later batch only waits longer)
+            cudaError_t q = cudaEventQuery(c->slot_ev[dep]);
             if (q == cudaErrorNotReady) {
                 if (!p.missed) c->extra_late++;
                 if (dev_wait) continue;      // the kernel itself waits for this slot; it stays pending for later launches
-                CU(c, cudaStreamWaitEvent(c->compute, c->slot_ev[k], 0));
+                CU(c, cudaStreamWaitEvent(c->compute, c->slot_ev[dep], 0));
             } else if (q != cudaSuccess) {
                 return fail(c, SPM_ERR_CUDA, "copy event query: %s", cudaGetErrorString(q));
             }
@@ -765,9 +775,12 @@ int do_prefetch(spm_ctx* c, int target, const int32_t* ids, int count, const int
     const int issued = tb.prefetch(target, ids, count, protect, n_protect, c->drop_modulo, c->slots_tmp.data());
     if (issued > 0) {
         if (int rc = order_copy_after_readers(c, target)) return rc;
+        int last = -1;
+        for (int i = 0; i < count; ++i) if (c->slots_tmp[i] >= 0) last = i;
+        const size_t lead = size_t(target) * c->S + c->slots_tmp[last];
         for (int i = 0; i < count; ++i)
             if (c->slots_tmp[i] >= 0)
-                if (int rc = issue_copy(c, target, ids[i], c->slots_tmp[i])) return rc;
+                if (int rc = issue_copy(c, target, ids[i], c->slots_tmp[i], lead, i == last)) return rc;
     }
     if (out_issued) *out_issued = issued;
     return SPM_OK;
@@ -795,16 +808,23 @@ int step_layers(spm_ctx* c, float* h_out, int nb, Timing* t, const Mailbox* trac
     c->prev_order_valid = false;
     std::vector<int32_t> ids(size_t(nb) * K);
     std::vector<int32_t> this_rank;
+    // The routing kernel of layer l + 1 depends only on layer l's kernels, so it is enqueued as soon as
+    // they are and before the host plans and issues layer l + 1's prefetch (several driver calls):
+    // the device never waits for that host work. The mailbox words of layer l are read before.
+    auto enqueue_router = [&](int l) -> int {
+        if (c->stub_us > 0) {
+            attention_stub_kernel<<<1, 1, 0, c->compute>>>(uint64_t(c->stub_us) * 1000ull);
+            CU(c, cudaGetLastError());
+            c->kernel_launches++;
+        }
+        if (int rc = launch_router(c, l, h_out, nullptr, nb, c->ws_x, nullptr, true, predict && l <= L - 2, nullptr, false)) return rc;
+        if (t) CU(c, cudaEventRecord(t->k1_done[l], c->compute));
+        return SPM_OK;
+    };
+    if (!trace) if (int rc = enqueue_router(0)) return rc;
     for (int l = 0; l < L; ++l) {
         const bool has_adapter = l <= L - 2;
         if (!trace) {
-            if (c->stub_us > 0) {
-                attention_stub_kernel<<<1, 1, 0, c->compute>>>(uint64_t(c->stub_us) * 1000ull);
-                CU(c, cudaGetLastError());
-                c->kernel_launches++;
-            }
-            if (int rc = launch_router(c, l, h_out, nullptr, nb, c->ws_x, nullptr, true, predict && has_adapter, nullptr, false)) return rc;
-            if (t) CU(c, cudaEventRecord(t->k1_done[l], c->compute));
             if (int rc = wait_tagged(c, c->mb_host->ids, nb * K, ids.data(), "expert ids")) return rc;
         } else {
             for (int i = 0; i < nb * K; ++i) ids[i] = trace[l].ids[i] & 0xffff;
@@ -824,6 +844,10 @@ int step_layers(spm_ctx* c, float* h_out, int nb, Timing* t, const Mailbox* trac
         if (c->policy == SPM_POLICY_NAIVE) borda_rank(ids.data(), nb, K, n, this_rank);
 
         c->prev_order_valid = false;
+        const bool reads_order = has_adapter && (c->policy == SPM_POLICY_ADAPTER || c->policy == SPM_POLICY_PRED0);
+        if (!trace && !reads_order && l + 1 < L) {       // nothing left to read from layer l's mailbox
+            if (int rc = enqueue_router(l + 1)) return rc;
+        }
         if (has_adapter && c->policy != SPM_POLICY_ON_DEMAND) {
             const int32_t* ranking;
             int n_ranked;
@@ -840,6 +864,7 @@ int step_layers(spm_ctx* c, float* h_out, int nb, Timing* t, const Mailbox* trac
                 c->prev_order.resize(n);
                 if (!trace) {
                     if (int rc = wait_tagged(c, c->mb_host->order, n, c->prev_order.data(), "expert ranking")) return rc;
+                    if (int rc = enqueue_router(l + 1)) return rc;      // has_adapter: layer l + 1 exists
                 } else {
                     for (int e = 0; e < n; ++e) c->prev_order[e] = trace[l].order[e] & 0xffff;
                 }
@@ -892,7 +917,7 @@ int host_free_ready(spm_ctx* c, int nb, bool* out) {
                 if (tb.slot_of(l, e) < 0) return SPM_OK;
         for (size_t k = 0; k < c->slot_pending.size(); ++k)
             if (c->slot_pending[k]) {
-                CU(c, cudaStreamWaitEvent(c->compute, c->slot_ev[k], 0));
+                CU(c, cudaStreamWaitEvent(c->compute, c->slot_ev[c->slot_dep[k]], 0));
                 c->slot_pending[k] = 0;
             }
         std::vector<short> map(size_t(m.n_layers) * m.n_experts);
@@ -1099,6 +1124,7 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
     c->layer_stall_us.assign(L, 0.0);
     c->layer_ffn_us.assign(L, 0.0);
     c->slot_pending.assign(size_t(L) * c->S, 0);
+    c->slot_dep.assign(size_t(L) * c->S, 0);
     c->slot_gen_host.assign(size_t(L) * c->S, 0);
     c->pool_free_valid.assign(L, 0);
 
@@ -1366,6 +1392,12 @@ int spm_set_copy_delay_us(spm_ctx* c, int us) {
 int spm_set_device_wait(spm_ctx* c, int on) {
     if (!c) return SPM_ERR_INVALID_ARG;
     if (on && !stream_write32_fn()) return fail(c, SPM_ERR_CUDA, "cuStreamWriteValue32 is not available on this driver");
+    if (int rc = flush_trace(c)) return rc;
+    if ((on != 0) != c->device_wait) {
+        // transfers issued in the other mode carry no arrival counters (or no per-slot meaning): let them land first
+        CU(c, cudaStreamSynchronize(c->copy));
+        std::fill(c->slot_pending.begin(), c->slot_pending.end(), 0);
+    }
     c->device_wait = on != 0;
     return SPM_OK;
 }
