@@ -237,11 +237,12 @@ int spm_set_drop_modulo(spm_ctx* ctx, int modulo);
  * before the slot counts as loaded. Outputs are unchanged. */
 int spm_set_copy_delay_us(spm_ctx* ctx, int us);
 /* Device-side wait for batch-1 expert FFNs (default off). Off: the compute stream waits on the
- * copy events of the slots a launch reads, then the kernel starts. On: the kernel is launched at
- * once and each of its CTAs waits (bounded, SPM_ERR_TIMEOUT on expiry) on a per-slot arrival counter
- * that the copy stream bumps after the expert's bytes have landed, so resident experts are computed
- * while missing ones are still in flight and no launch latency follows the last copy. Outputs are
- * bit-identical either way. With it on, the timed FFN duration includes the wait for copies. */
+ * event of the batch of copies that fills the slots a launch reads, then the kernel starts. On: the
+ * kernel is launched at once and its warps wait (bounded, SPM_ERR_TIMEOUT on expiry) on an arrival
+ * counter that the copy stream bumps after the last copy of that batch has landed, so rows of
+ * resident experts are streamed while missing ones are still in flight and no launch latency
+ * follows the last copy. Outputs are bit-identical either way. With it on, the timed FFN duration
+ * includes the wait for copies. Switching the option waits for both streams. */
 int spm_set_device_wait(spm_ctx* ctx, int on);
 /* Host-free decode steps (default on). Once every expert of every layer holds a slot and every
  * copy has landed (possible only with slots_per_layer >= n_experts), no routing result can change

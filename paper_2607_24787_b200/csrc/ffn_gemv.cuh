@@ -44,7 +44,8 @@ struct FfnArgs {
     const short* dev_code;          // optional [nb][K] slot numbers left in device memory by the routing kernel:
                                     // the launch then needs no host knowledge of the routing (count/code/kidx unused;
                                     // token t has K routed entries followed by the n_shared shared experts)
-    unsigned want[SPM_MAX_TOPK];    // token 0 only: counter value at which entry k's slot holds its expert
+    unsigned want[SPM_MAX_TOPK];    // token 0 only: entry k's expert has landed once ready[watch[k]] >= want[k]
+    short watch[SPM_MAX_TOPK];      //   (the counter of the slot that leads the batch of copies entry k's slot was filled by)
     unsigned long long blob_bytes;
     int I, K, n_slots, n_shared;
     unsigned char count[MAXNB];                     // expert entries of token t in this launch
@@ -122,7 +123,7 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
         if (a.ready) {
             // Device-side wait: the copy stream bumps the slot's counter after the expert's bytes
             // have landed. Bounded; on timeout the status word is set and the launch winds down.
-            const unsigned* f = a.ready + code;
+            const unsigned* f = a.ready + a.watch[ent];
             const unsigned want = a.want[ent];
             const unsigned long long t0 = global_timer_ns();
             for (;;) {

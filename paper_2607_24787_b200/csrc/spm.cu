@@ -107,7 +107,8 @@ struct spm_ctx {
     int copy_delay_us = 0;                    // emulated slower storage tier: extra wait after every expert copy
     bool device_wait = false;                 // batch-1 FFN launched at once, waits for its copies on the device
     unsigned* ws_slot_gen = nullptr;          // [L][S] arrival counters, bumped by the copy stream
-    std::vector<uint32_t> slot_gen_host;      // value the counter will hold once the latest copy has landed
+    std::vector<uint32_t> slot_gen_host;      // arrival counter of a slot as a batch leader: batches it has led so far
+    std::vector<uint32_t> slot_want;          // counter value of its batch leader at which a slot's latest copy has landed
     // host-free steps: once every expert of every layer is resident, a step is enqueued without
     // waiting for any routing result; the routing kernel leaves slot numbers for the expert kernel
     // in device memory and its ids / ranking in a ring of host-mapped trace mailboxes, from which
@@ -488,8 +489,8 @@ const unsigned char* host_blob(spm_ctx* c, int layer, int e) {
 // Enqueue one expert transfer on the copy stream. Transfers are issued in batches (the misses of a
 // wave, the selections of a prefetch) that are awaited as a whole, so only the last transfer of a
 // batch records an event (`lead` = the slot whose event covers the batch): every stream operation
-// between two copies costs a few microseconds of link time. With device-side waiting each transfer
-// also bumps its slot's arrival counter, because the kernel then waits slot by slot.
+// between two copies costs a few microseconds of link time. With device-side waiting the last
+// transfer also bumps the lead slot's arrival counter, which the kernel watches for the whole batch.
 int issue_copy(spm_ctx* c, int layer, int e, int slot, size_t lead, bool last_of_batch) {
     const size_t k = size_t(layer) * c->S + slot;
     CU(c, cudaMemcpyAsync(slot_ptr(c, layer, slot), host_blob(c, layer, e), c->blob, cudaMemcpyHostToDevice, c->copy));
@@ -497,15 +498,18 @@ int issue_copy(spm_ctx* c, int layer, int e, int slot, size_t lead, bool last_of
         attention_stub_kernel<<<1, 1, 0, c->copy>>>(uint64_t(c->copy_delay_us) * 1000ull);   // emulated slower tier
         CU(c, cudaGetLastError());
     }
-    if (last_of_batch) CU(c, cudaEventRecord(c->slot_ev[lead], c->copy));
-    if (c->device_wait) {
-        // stream-ordered counter bump, for launches that wait for their copies on the device
-        StreamWriteValue32Fn wr = stream_write32_fn();
-        if (!wr) return fail(c, SPM_ERR_CUDA, "cuStreamWriteValue32 is not available");
-        const uint32_t gen = ++c->slot_gen_host[k];
-        if (wr(reinterpret_cast<CUstream>(c->copy), reinterpret_cast<CUdeviceptr>(c->ws_slot_gen + k), gen, 0) != CUDA_SUCCESS)
-            return fail(c, SPM_ERR_CUDA, "cuStreamWriteValue32 failed");
+    if (last_of_batch) {
+        CU(c, cudaEventRecord(c->slot_ev[lead], c->copy));
+        if (c->device_wait) {
+            // stream-ordered bump of the lead slot's arrival counter, for launches that wait on the device
+            StreamWriteValue32Fn wr = stream_write32_fn();
+            if (!wr) return fail(c, SPM_ERR_CUDA, "cuStreamWriteValue32 is not available");
+            if (wr(reinterpret_cast<CUstream>(c->copy), reinterpret_cast<CUdeviceptr>(c->ws_slot_gen + lead), c->slot_gen_host[lead] + 1, 0) != CUDA_SUCCESS)
+                return fail(c, SPM_ERR_CUDA, "cuStreamWriteValue32 failed");
+        }
+        ++c->slot_gen_host[lead];        // every slot of the batch was given this value as its target below
     }
+    c->slot_want[k] = c->slot_gen_host[lead] + (last_of_batch ? 0 : 1);
     c->slot_dep[k] = lead;
     c->slot_pending[k] = 1;
     c->h2d_bytes += c->blob;
@@ -724,7 +728,11 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
                     if (s < 0) continue;
                     a.code[tk * SPM_MAX_TOPK + cnt] = short(s);
                     a.kidx[tk * SPM_MAX_TOPK + cnt] = (unsigned char)k;
-                    if (dev_wait) a.want[cnt] = c->slot_gen_host[size_t(layer) * c->S + s];
+                    if (dev_wait) {
+                        const size_t ks = size_t(layer) * c->S + s;
+                        a.want[cnt] = c->slot_want[ks];
+                        a.watch[cnt] = short(c->slot_dep[ks] - size_t(layer) * c->S);
+                    }
                     ++cnt;
                 }
                 if (first)
@@ -1126,6 +1134,7 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
     c->slot_pending.assign(size_t(L) * c->S, 0);
     c->slot_dep.assign(size_t(L) * c->S, 0);
     c->slot_gen_host.assign(size_t(L) * c->S, 0);
+    c->slot_want.assign(size_t(L) * c->S, 0);
     c->pool_free_valid.assign(L, 0);
 
     auto cu = [&](cudaError_t err, const char* what) {
@@ -1396,7 +1405,10 @@ int spm_set_device_wait(spm_ctx* c, int on) {
     if ((on != 0) != c->device_wait) {
         // transfers issued in the other mode carry no arrival counters (or no per-slot meaning): let them land first
         CU(c, cudaStreamSynchronize(c->copy));
+        CU(c, cudaStreamSynchronize(c->compute));
         std::fill(c->slot_pending.begin(), c->slot_pending.end(), 0);
+        // batches led while the option was off did not bump the device-side counters
+        if (on) CU(c, cudaMemcpy(c->ws_slot_gen, c->slot_gen_host.data(), c->slot_gen_host.size() * sizeof(uint32_t), cudaMemcpyHostToDevice));
     }
     c->device_wait = on != 0;
     return SPM_OK;
