@@ -383,7 +383,7 @@ int launch_router(spm_ctx* c, int layer, const float* h, const float* x_in, int 
     // publish are zeroed first, so a word left by an older launch can never carry the current tag.
     ++c->seq;
     if ((c->seq & 0xffffu) == 0) ++c->seq;
-    if (!route) {
+    if (!route || route->mailbox_dev == c->mb_dev) {
         if (do_router) memset(const_cast<int32_t*>(c->mb_host->ids), 0, size_t(nb) * m.top_k * sizeof(int32_t));
         if (do_adapter) memset(const_cast<int32_t*>(c->mb_host->order), 0, size_t(m.n_experts) * sizeof(int32_t));
     }
@@ -640,8 +640,10 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
 // of the stand-alone timing ring instead.
 // With `launch` false only the slot table's side runs (the kernels of a host-free step were
 // enqueued earlier); a miss there would mean the step computed with a stale slot map.
+// With `leave_partial` the partial rows of the last wave stay in the workspace for the next
+// layer's routing kernel to fold into the hidden row (GEMV path only; reported through *left).
 int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, const float* w, int nb,
-            float* h_inout, Timing* t, int ring = -1, bool launch = true) {
+            float* h_inout, Timing* t, int ring = -1, bool launch = true, bool leave_partial = false, bool* left = nullptr) {
     const spm_model_cfg& m = c->cfg;
     const int K = m.top_k;
     SlotTable& tb = *c->table;
@@ -760,12 +762,17 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
             }
             if (t && last) CU(c, cudaEventRecord(t->ffn_end[layer], c->compute));
             if (ring >= 0 && last) { CU(c, cudaEventRecord(c->ring_end[ring], c->compute)); c->ring_used[ring] = 1; }
-            unsigned long long* reduce_clock = nullptr;
-            if (int rc = take_clock(c, kClkReduce, &reduce_clock)) return rc;
-            ffn_reduce_kernel<<<dim3((m.hidden + kReduceCols - 1) / kReduceCols, nb), kReduceCols * kReduceGroups, 0, c->compute>>>(
-                c->ws_partial, h_inout, h_inout, G, m.hidden, reduce_clock);
-            CU(c, cudaGetLastError());
-            c->kernel_launches += 2;
+            if (last && leave_partial) {
+                if (left) *left = true;
+                c->kernel_launches += 1;
+            } else {
+                unsigned long long* reduce_clock = nullptr;
+                if (int rc = take_clock(c, kClkReduce, &reduce_clock)) return rc;
+                ffn_reduce_kernel<<<dim3((m.hidden + kReduceCols - 1) / kReduceCols, nb), kReduceCols * kReduceGroups, 0, c->compute>>>(
+                    c->ws_partial, h_inout, h_inout, G, m.hidden, reduce_clock);
+                CU(c, cudaGetLastError());
+                c->kernel_launches += 2;
+            }
             c->ffn_launches++;
         }
         if (!last) CU(c, cudaEventRecord(c->wave_done, c->compute));
@@ -819,16 +826,22 @@ int step_layers(spm_ctx* c, float* h_out, int nb, Timing* t, const Mailbox* trac
     // The routing kernel of layer l + 1 depends only on layer l's kernels, so it is enqueued as soon as
     // they are and before the host plans and issues layer l + 1's prefetch (several driver calls):
     // the device never waits for that host work. The mailbox words of layer l are read before.
+    bool partial_left = false;       // the preceding layer's partial rows are still to be folded into the hidden row
     auto enqueue_router = [&](int l) -> int {
         if (c->stub_us > 0) {
             attention_stub_kernel<<<1, 1, 0, c->compute>>>(uint64_t(c->stub_us) * 1000ull);
             CU(c, cudaGetLastError());
             c->kernel_launches++;
         }
-        if (int rc = launch_router(c, l, h_out, nullptr, nb, c->ws_x, nullptr, true, predict && l <= L - 2, nullptr, false)) return rc;
+        RouterRoute fold{c->mb_dev, nullptr, nullptr, false, c->ws_partial, ffn_grid_for(c, nb)};
+        if (int rc = launch_router(c, l, h_out, nullptr, nb, c->ws_x, nullptr, true, predict && l <= L - 2,
+                                   partial_left ? &fold : nullptr, false)) return rc;
+        partial_left = false;
         if (t) CU(c, cudaEventRecord(t->k1_done[l], c->compute));
         return SPM_OK;
     };
+    // GEMV path: only the last layer runs the combine kernel, the others leave it to the next routing kernel
+    const bool gemv_path = !(nb > 1 && c->tc_ok && c->batched_path == 0);
     if (!trace) if (int rc = enqueue_router(0)) return rc;
     for (int l = 0; l < L; ++l) {
         const bool has_adapter = l <= L - 2;
@@ -848,7 +861,8 @@ int step_layers(spm_ctx* c, float* h_out, int nb, Timing* t, const Mailbox* trac
                 c->recall_count++;
             }
         }
-        if (int rc = run_ffn(c, l, c->ws_x, ids.data(), c->ws_w, nb, h_out, t, -1, trace == nullptr)) return rc;
+        if (int rc = run_ffn(c, l, c->ws_x, ids.data(), c->ws_w, nb, h_out, t, -1, trace == nullptr,
+                             gemv_path && l + 1 < L && c->stub_us == 0, &partial_left)) return rc;
         if (c->policy == SPM_POLICY_NAIVE) borda_rank(ids.data(), nb, K, n, this_rank);
 
         c->prev_order_valid = false;
