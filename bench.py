@@ -9,8 +9,10 @@ adapter, budget selection, asynchronous prefetch, on-demand loads, slot-indexed 
 
   value : decode tokens/s, hidden rows already in HBM, timed with CUDA events on the compute stream
   e2e   : the same through spm_decode_step_host (pinned host rows in, host rows out, every step)
-  roofline : expert-FFN kernel, algorithmic weight bytes / mean device time of its launches inside
-             the timed region, against the measured HBM copy bandwidth
+  roofline : expert-FFN kernel, algorithmic weight bytes / mean device time of its launches (CUDA
+             event pair per launch, the kernel timed by itself on a fully-resident context; the
+             same pair inside the main arm and the in-kernel windows are given beside it),
+             against the measured HBM copy bandwidth
   cpu_baseline : the CPU oracle timed on this machine's host cores on a bounded sample
 
 `--impl reference` times the CPU oracle instead (rank 0 only).
@@ -361,17 +363,26 @@ def run_ours(args):
         try:
             result["resident"] = resident_run(cfg, m, H_dev, W, min(K, args.arm_steps), peak, algo_bytes, device)
             b2b = result["resident"]["ffn_back_to_back"]
-            result["roofline"]["isolated"] = {
+            iso = {
                 "kernel": b2b["kernel"], "achieved": b2b["gb_s"], "frac": b2b["frac_of_measured_peak"],
                 "us_per_launch": b2b["kernel_us"], "algorithmic_bytes_per_launch": b2b["algorithmic_bytes_per_launch"],
                 "in_kernel_window_us": b2b["kernel_window_us"],
+                "achieved_in_kernel_window": b2b["gb_s_in_kernel_window"],
                 "frac_in_kernel_window": (b2b["gb_s_in_kernel_window"] or 0) / peak,
-                "region": f"{b2b['launches']} spm_moe_ffn launches back to back, all experts resident, event pair per launch"}
-            if cfg.batch > 1:      # in the batched run a launch's bytes vary with the demand: report the isolated leg
-                result["roofline"].update(achieved=b2b["gb_s"], frac=b2b["frac_of_measured_peak"],
-                                          us_per_launch=b2b["kernel_us"], kernel=b2b["kernel"],
-                                          algorithmic_bytes_per_launch=b2b["algorithmic_bytes_per_launch"],
-                                          region=result["roofline"]["isolated"]["region"], traffic=None)
+                "frac_of_nominal_8TBs": b2b["gb_s"] / NOMINAL_HBM_GBS,
+                "region": f"{b2b['launches']} spm_moe_ffn launches back to back on the compute stream, all experts resident "
+                          f"(pools of all layers cycled, nothing served from L2), CUDA event pair per launch"}
+            # The headline is the kernel timed by itself (burst peak as denominator). Inside the main arm every
+            # launch follows a wait for PCIe copies and overlaps the next prefetch copy; an event pair there
+            # measures mostly launch latency behind the busy link (the in-kernel window stays the same), so
+            # that figure is kept beside it, not as the kernel's roofline.
+            main_view = {k: result["roofline"][k] for k in ("achieved", "frac", "us_per_launch", "in_kernel_window_us",
+                                                            "achieved_in_kernel_window", "frac_in_kernel_window", "region")}
+            if cfg.batch > 1:      # a batched launch's bytes vary with the demand: only the isolated leg has a byte count
+                main_view = {"us_per_launch": result["roofline"]["us_per_launch"], "region": result["roofline"]["region"]}
+                result["roofline"]["traffic"] = None
+            result["roofline"].update(iso)
+            result["roofline"]["in_main_arm"] = main_view
         except Exception as e:   # noqa: BLE001 (reported, not hidden)
             result["resident"] = {"error": str(e)[:200]}
 
