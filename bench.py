@@ -386,6 +386,13 @@ def run_ours(args):
         except Exception as e:   # noqa: BLE001 (reported, not hidden)
             result["resident"] = {"error": str(e)[:200]}
 
+    # second denominator: what a kernel that only reads reaches on this device (the copy figure pays for writes too)
+    try:
+        ro = m.measure_read_bandwidth(4 << 30)
+        result["roofline"]["read_only_stream_gb_s"] = ro
+        result["roofline"]["frac_of_read_only_stream"] = result["roofline"]["achieved"] / ro
+    except Exception as e:   # noqa: BLE001 (pools smaller than 256 MiB: nothing to measure)
+        result["roofline"]["read_only_stream_gb_s"] = None
     if world == 1 and rank == 0 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(cfg, H[W:W + args.cpu_steps].numpy(), device, budget)
     m.close()

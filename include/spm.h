@@ -270,6 +270,13 @@ int spm_set_deadline_ms(spm_ctx* ctx, int ms);
  * path a decode step takes), t_xfer_us = median time of one expert copy from the pinned store,
  * *budget_raw = floor(window / t_xfer). Uses and then empties the cache. */
 int spm_profile_window(spm_ctx* ctx, double* window_us, double* t_xfer_us, int* budget_raw);
+/* Read-only HBM streaming rate of this device, as a second denominator beside the copy bandwidth:
+ * a kernel that only reads (16-byte loads, grid of 4 CTAs per SM, every loaded word folded into a
+ * checksum that is written once per thread) streams the first `bytes` of the slot pools (clamped
+ * to their size, rounded down to 16 bytes; at least 256 MiB is needed so that L2 does not serve
+ * it) `reps` >= 1 times on the compute stream; *gb_s is the best repetition by CUDA event pair.
+ * The pool contents are not modified. Waits for the compute stream. */
+int spm_measure_read_bandwidth(spm_ctx* ctx, size_t bytes, int reps, double* gb_s);
 
 int spm_cache_reset(spm_ctx* ctx);                         /* cold cache, step counter, stats, events */
 int spm_reset_stats(spm_ctx* ctx);                         /* counters, timings and event log only; cache kept */

@@ -89,6 +89,7 @@ _SIG = {
     "spm_set_host_free": [_P, C.c_int],
     "spm_set_copy_delay_us": [_P, C.c_int],
     "spm_profile_window": [_P, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int)],
+    "spm_measure_read_bandwidth": [_P, C.c_size_t, C.c_int, C.POINTER(C.c_double)],
     "spm_cache_reset": [_P],
     "spm_reset_stats": [_P],
     "spm_get_stats": [_P, C.POINTER(Stats)],
@@ -293,6 +294,12 @@ def spm_profile_window(ctx):
     w, t, b = C.c_double(), C.c_double(), C.c_int()
     _check(load().spm_profile_window(ctx, C.byref(w), C.byref(t), C.byref(b)), ctx)
     return w.value, t.value, b.value
+
+
+def spm_measure_read_bandwidth(ctx, nbytes, reps=5) -> float:
+    g = C.c_double()
+    _check(load().spm_measure_read_bandwidth(ctx, nbytes, reps, C.byref(g)), ctx)
+    return g.value
 
 
 def spm_cache_reset(ctx):

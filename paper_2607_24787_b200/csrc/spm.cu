@@ -470,6 +470,20 @@ int wait_tagged(spm_ctx* c, const volatile int32_t* words, int count, int32_t* o
     return SPM_OK;
 }
 
+// Read-only streaming probe: every thread folds its 16-byte words into a checksum.
+__global__ void __launch_bounds__(512)
+read_probe_kernel(const uint4* __restrict__ p, size_t n16, unsigned* sink) {
+    unsigned acc = 0;
+    const size_t stride = size_t(gridDim.x) * blockDim.x;
+    size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    for (; i + 3 * stride < n16; i += 4 * stride) {      // four independent loads in flight per thread
+        const uint4 a = __ldcs(p + i), b = __ldcs(p + i + stride), c2 = __ldcs(p + i + 2 * stride), d = __ldcs(p + i + 3 * stride);
+        acc ^= a.x ^ a.y ^ a.z ^ a.w ^ b.x ^ b.y ^ b.z ^ b.w ^ c2.x ^ c2.y ^ c2.z ^ c2.w ^ d.x ^ d.y ^ d.z ^ d.w;
+    }
+    for (; i < n16; i += stride) { const uint4 a = __ldcs(p + i); acc ^= a.x ^ a.y ^ a.z ^ a.w; }
+    if (acc == 0x9e3779b9u) *sink = acc;      // keeps the loads alive; practically never taken
+}
+
 // A kernel that only waits: one thread watches %globaltimer until `ns` have passed. Used as the
 // stand-in for the omitted attention block and as the extra delay of an emulated slower storage tier.
 __global__ void attention_stub_kernel(unsigned long long ns) {
@@ -1557,6 +1571,33 @@ int spm_profile_window(spm_ctx* c, double* window_us, double* t_xfer_us, int* bu
     *budget_raw = int(*window_us / *t_xfer_us);
     if (int rc = check_status(c)) return rc;
     return spm_cache_reset(c);
+}
+
+int spm_measure_read_bandwidth(spm_ctx* c, size_t bytes, int reps, double* gb_s) {
+    if (!c || !gb_s || reps < 1) return SPM_ERR_INVALID_ARG;
+    if (int rc = flush_trace(c)) return rc;
+    const size_t pool_bytes = size_t(c->cfg.n_layers) * c->S * c->blob;
+    bytes = std::min(bytes, pool_bytes) / 16 * 16;
+    if (bytes < (size_t(256) << 20)) return fail(c, SPM_ERR_INVALID_ARG, "need at least 256 MiB of slot pools to measure beyond L2");
+    cudaEvent_t e0, e1;
+    CU(c, cudaEventCreate(&e0));
+    CU(c, cudaEventCreate(&e1));
+    float best = 0.f;
+    for (int r = 0; r < reps + 1; ++r) {        // first repetition is a warm-up
+        CU(c, cudaEventRecord(e0, c->compute));
+        read_probe_kernel<<<4 * c->num_sms, 512, 0, c->compute>>>(reinterpret_cast<const uint4*>(c->pools), bytes / 16,
+                                                                  reinterpret_cast<unsigned*>(c->ws_counters + 8));
+        CU(c, cudaGetLastError());
+        CU(c, cudaEventRecord(e1, c->compute));
+        CU(c, cudaEventSynchronize(e1));
+        float ms = 0.f;
+        CU(c, cudaEventElapsedTime(&ms, e0, e1));
+        if (r > 0) best = std::max(best, float(double(bytes) / (double(ms) * 1e-3) / 1e9));
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    *gb_s = best;
+    return SPM_OK;
 }
 
 int spm_get_stats(spm_ctx* c, spm_stats* out) {

@@ -156,6 +156,7 @@ class OffloadedMoE:
     def set_host_free(self, on): B.spm_set_host_free(self.ctx, on)
     def set_copy_delay_us(self, us): B.spm_set_copy_delay_us(self.ctx, us)
     def profile_window(self): return B.spm_profile_window(self.ctx)
+    def measure_read_bandwidth(self, nbytes, reps=5): return B.spm_measure_read_bandwidth(self.ctx, nbytes, reps)
     def cache_reset(self): B.spm_cache_reset(self.ctx)
     def reset_stats(self): B.spm_reset_stats(self.ctx)
     def stats(self): return B.spm_get_stats(self.ctx)

@@ -146,3 +146,15 @@ def test_host_deadline_returns_timeout_and_context_survives():
     want, _ = ref.step(np.ones((1, cfg.hidden)))
     assert M.rel_linf(out.cpu().numpy(), want) < 4e-5
     m.close()
+
+
+def test_read_bandwidth_probe_and_its_limits():
+    cfg = synth.get_config("qwen3", n_layers=2, slots=24)          # 2 x 24 x 9 MiB = 432 MiB of pools
+    m = build(cfg)
+    before = [list(m.slot_table(l)) for l in range(cfg.n_layers)]
+    g = m.measure_read_bandwidth(1 << 40, reps=3)                    # clamped to the pools
+    assert 1000.0 < g < 12000.0, g                                   # GB/s: above PCIe, below any HBM3e figure
+    assert before == [list(m.slot_table(l)) for l in range(cfg.n_layers)]
+    with pytest.raises(Exception):
+        m.measure_read_bandwidth(1 << 20)                            # too small to get past L2
+    m.close()
