@@ -279,6 +279,19 @@ int spm_profile_window(spm_ctx* ctx, double* window_us, double* t_xfer_us, int* 
 int spm_measure_read_bandwidth(spm_ctx* ctx, size_t bytes, int reps, double* gb_s);
 
 int spm_cache_reset(spm_ctx* ctx);                         /* cold cache, step counter, stats, events */
+/* Checkpoint / resume of the expert cache (Section 3.3's availability state; integers only, no
+ * weights): which expert holds which slot, LRU ticks, prefetch-origin and first-use flags, the
+ * global tick and the step counter, as 2 + 4 * n_layers * slots_per_layer 64-bit words.
+ * export: `state` HOST [capacity] or NULL to query; *count receives the number of words; with a
+ *   buffer that is too small nothing is written and SPM_ERR_INVALID_ARG is returned. Waits for
+ *   outstanding bookkeeping, not for the GPU.
+ * import: into a context of the same shape (else SPM_ERR_INVALID_ARG, context unchanged): waits
+ *   for both streams, installs the table, clears statistics and the event log, and copies every
+ *   listed expert from the host store into its slot on the copy stream (the next launch that
+ *   reads a slot waits for it as for any other copy). Decoding then continues exactly as the
+ *   exporting context would have: same hits, misses, evictions, outputs. */
+int spm_cache_export(spm_ctx* ctx, int64_t* state, size_t capacity, size_t* count);
+int spm_cache_import(spm_ctx* ctx, const int64_t* state, size_t count);
 int spm_reset_stats(spm_ctx* ctx);                         /* counters, timings and event log only; cache kept */
 int spm_get_stats(spm_ctx* ctx, spm_stats* out);           /* waits for timed work to finish */
 /* Per-layer sums since the last reset: stall_us[L], ffn_us[L], and the number of steps in them. */
@@ -349,6 +362,9 @@ int spm_sim_end_step(spm_sim* sim);
 int spm_sim_events(spm_sim* sim, spm_event* out, size_t capacity, size_t* count);
 int spm_sim_stats(spm_sim* sim, spm_stats* out);
 int spm_sim_slot_table(spm_sim* sim, int layer, int32_t* slot_expert /* [slots] */);
+/* Same checkpoint words as spm_cache_export / spm_cache_import, for the host-only table. */
+int spm_sim_export(spm_sim* sim, int64_t* state, size_t capacity, size_t* count);
+int spm_sim_import(spm_sim* sim, const int64_t* state, size_t count);
 
 #ifdef __cplusplus
 }

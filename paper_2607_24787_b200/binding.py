@@ -110,6 +110,10 @@ _SIG = {
     "spm_sim_events": [_P, _P, C.c_size_t, C.POINTER(C.c_size_t)],
     "spm_sim_stats": [_P, C.POINTER(Stats)],
     "spm_sim_slot_table": [_P, C.c_int, _P],
+    "spm_sim_export": [_P, _P, C.c_size_t, C.POINTER(C.c_size_t)],
+    "spm_sim_import": [_P, _P, C.c_size_t],
+    "spm_cache_export": [_P, _P, C.c_size_t, C.POINTER(C.c_size_t)],
+    "spm_cache_import": [_P, _P, C.c_size_t],
 }
 EXPORTS = sorted(list(_SIG) + ["spm_last_error"])
 
@@ -306,6 +310,20 @@ def spm_cache_reset(ctx):
     _check(load().spm_cache_reset(ctx), ctx)
 
 
+def spm_cache_export(ctx) -> np.ndarray:
+    """The expert cache's checkpoint words (int64)."""
+    n = C.c_size_t()
+    _check(load().spm_cache_export(ctx, None, 0, C.byref(n)), ctx)
+    out = np.empty(n.value, np.int64)
+    _check(load().spm_cache_export(ctx, _ptr(out), out.size, C.byref(n)), ctx)
+    return out
+
+
+def spm_cache_import(ctx, state):
+    state = np.ascontiguousarray(state, np.int64)
+    _check(load().spm_cache_import(ctx, _ptr(state), state.size), ctx)
+
+
 def spm_reset_stats(ctx):
     _check(load().spm_reset_stats(ctx), ctx)
 
@@ -428,3 +446,14 @@ class Sim:
         out = np.empty(self.S, np.int32)
         _check(load().spm_sim_slot_table(self.h, layer, _ptr(out)))
         return [int(e) for e in out]
+
+    def export_state(self) -> np.ndarray:
+        n = C.c_size_t()
+        _check(load().spm_sim_export(self.h, None, 0, C.byref(n)))
+        out = np.empty(n.value, np.int64)
+        _check(load().spm_sim_export(self.h, _ptr(out), out.size, C.byref(n)))
+        return out
+
+    def import_state(self, state):
+        state = np.ascontiguousarray(state, np.int64)
+        _check(load().spm_sim_import(self.h, _ptr(state), state.size))

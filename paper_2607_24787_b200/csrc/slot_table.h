@@ -9,6 +9,7 @@
 // Pure C++ (no CUDA): the GPU context and the host-only simulator share this class.
 #pragma once
 
+#include <cstddef>
 #include <cstdint>
 #include <vector>
 
@@ -160,6 +161,48 @@ public:
             log(layer, SPM_EV_PLAN, ids[i], -1);
             stats_.planned++;
         }
+    }
+
+    // Checkpoint of the table as 64-bit words (no weights): {tick, step}, then per slot of every
+    // layer {expert or -1, LRU tick, origin, used}. Accounting (statistics, event log) is not part of it.
+    static size_t state_words(int n_layers, int slots) { return 2 + size_t(4) * n_layers * slots; }
+    size_t state_words() const { return state_words(L_, S_); }
+    void export_state(int64_t* out) const {
+        out[0] = int64_t(tick_);
+        out[1] = step_;
+        for (size_t k = 0; k < size_t(L_) * S_; ++k) {
+            out[2 + 4 * k] = slot_expert_[k];
+            out[3 + 4 * k] = int64_t(slot_tick_[k]);
+            out[4 + 4 * k] = slot_origin_[k];
+            out[5 + 4 * k] = slot_used_[k];
+        }
+    }
+    // Returns false (table untouched) when the words do not describe a valid table of this shape:
+    // expert ids in range and at most once per layer, ticks not above the global tick, flags 0/1.
+    bool import_state(const int64_t* in, size_t count) {
+        if (count != state_words() || in[0] < 0 || in[1] < 0 || in[1] > INT32_MAX) return false;
+        std::vector<int32_t> es(size_t(L_) * n_, -1);
+        for (int l = 0; l < L_; ++l)
+            for (int sl = 0; sl < S_; ++sl) {
+                const size_t k = size_t(l) * S_ + sl;
+                const int64_t e = in[2 + 4 * k], tk = in[3 + 4 * k], og = in[4 + 4 * k], us = in[5 + 4 * k];
+                if (e < -1 || e >= n_ || tk < 0 || tk > in[0] || og < 0 || og > 1 || us < 0 || us > 1) return false;
+                if (e >= 0) {
+                    if (es[size_t(l) * n_ + e] >= 0) return false;
+                    es[size_t(l) * n_ + e] = sl;
+                }
+            }
+        tick_ = uint64_t(in[0]);
+        step_ = int32_t(in[1]);
+        for (size_t k = 0; k < size_t(L_) * S_; ++k) {
+            slot_expert_[k] = int32_t(in[2 + 4 * k]);
+            slot_tick_[k] = uint64_t(in[3 + 4 * k]);
+            slot_origin_[k] = uint8_t(in[4 + 4 * k]);
+            slot_used_[k] = uint8_t(in[5 + 4 * k]);
+        }
+        expert_slot_ = es;
+        reset_accounting();
+        return true;
     }
 
 private:

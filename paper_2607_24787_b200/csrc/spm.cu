@@ -1513,6 +1513,39 @@ int spm_cache_reset(spm_ctx* c) {
     return SPM_OK;
 }
 
+int spm_cache_export(spm_ctx* c, int64_t* state, size_t capacity, size_t* count) {
+    if (!c || !count) return SPM_ERR_INVALID_ARG;
+    if (int rc = flush_trace(c)) return rc;
+    *count = c->table->state_words();
+    if (!state) return SPM_OK;
+    if (capacity < *count) return fail(c, SPM_ERR_INVALID_ARG, "state buffer too small: %zu < %zu words", capacity, *count);
+    c->table->export_state(state);
+    return SPM_OK;
+}
+
+int spm_cache_import(spm_ctx* c, const int64_t* state, size_t count) {
+    if (!c || !state) return SPM_ERR_INVALID_ARG;
+    if (count != c->table->state_words()) return fail(c, SPM_ERR_INVALID_ARG, "state has %zu words, this context needs %zu", count, c->table->state_words());
+    {   // validate on a scratch table first so that a bad state leaves the context untouched
+        SlotTable probe(c->cfg.n_layers, c->cfg.n_experts, c->S, false);
+        if (!probe.import_state(state, count)) return fail(c, SPM_ERR_INVALID_ARG, "state does not describe a valid slot table of this shape");
+    }
+    if (int rc = spm_cache_reset(c)) return rc;          // waits for both streams, clears accounting and pending copies
+    c->table->import_state(state, count);
+    for (int l = 0; l < c->cfg.n_layers; ++l) {
+        int last = -1;
+        for (int sl = 0; sl < c->S; ++sl) if (c->table->expert_in(l, sl) >= 0) last = sl;
+        if (last < 0) continue;
+        const size_t lead = size_t(l) * c->S + last;
+        for (int sl = 0; sl <= last; ++sl) {
+            const int e = c->table->expert_in(l, sl);
+            if (e >= 0) if (int rc = issue_copy(c, l, e, sl, lead, sl == last)) return rc;
+        }
+    }
+    c->h2d_bytes = 0;        // restoring the cache is not decode traffic
+    return SPM_OK;
+}
+
 int spm_profile_window(spm_ctx* c, double* window_us, double* t_xfer_us, int* budget_raw) {
     if (!c || !window_us || !t_xfer_us || !budget_raw) return SPM_ERR_INVALID_ARG;
     if (int rc = spm_cache_reset(c)) return rc;
@@ -1747,6 +1780,20 @@ int spm_sim_stats(spm_sim* s, spm_stats* out) {
     if (!s || !out) return SPM_ERR_INVALID_ARG;
     *out = s->table.stats();
     return SPM_OK;
+}
+
+int spm_sim_export(spm_sim* s, int64_t* state, size_t capacity, size_t* count) {
+    if (!s || !count) return SPM_ERR_INVALID_ARG;
+    *count = s->table.state_words();
+    if (!state) return SPM_OK;
+    if (capacity < *count) return SPM_ERR_INVALID_ARG;
+    s->table.export_state(state);
+    return SPM_OK;
+}
+
+int spm_sim_import(spm_sim* s, const int64_t* state, size_t count) {
+    if (!s || !state) return SPM_ERR_INVALID_ARG;
+    return s->table.import_state(state, count) ? SPM_OK : SPM_ERR_INVALID_ARG;
 }
 
 int spm_sim_slot_table(spm_sim* s, int layer, int32_t* slot_expert) {

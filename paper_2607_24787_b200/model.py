@@ -158,6 +158,8 @@ class OffloadedMoE:
     def profile_window(self): return B.spm_profile_window(self.ctx)
     def measure_read_bandwidth(self, nbytes, reps=5): return B.spm_measure_read_bandwidth(self.ctx, nbytes, reps)
     def cache_reset(self): B.spm_cache_reset(self.ctx)
+    def cache_export(self): return B.spm_cache_export(self.ctx)
+    def cache_import(self, state): B.spm_cache_import(self.ctx, state)
     def reset_stats(self): B.spm_reset_stats(self.ctx)
     def stats(self): return B.spm_get_stats(self.ctx)
     def layer_times(self): return B.spm_get_layer_times(self.ctx, self.L)

@@ -110,3 +110,45 @@ def test_sim_rejects_bad_arguments():
     with pytest.raises(B.SpmError):
         sim.plan(1, [0, 1, 8], 2)
     sim.close()
+
+
+def test_checkpoint_words_match_the_oracle_state_and_resume_identically():
+    # export after a run = the oracle's table word for word; a fresh table that imports it and is
+    # driven on gives the events an uninterrupted table gives
+    L, n, K, S, budget, steps = 3, 24, 3, 6, 2, 60
+    rng = np.random.default_rng(11)
+    trace = [[sorted({int(e) for e in rng.permutation(n)[:K]}) for _ in range(L)] for _ in range(steps)]
+    ranks = [[[int(e) for e in rng.permutation(n)] for _ in range(L)] for _ in range(steps)]
+    ref = P.SlotPolicy(L, n, S, False)
+    sim = B.Sim(L, n, S, False)
+    half = steps // 2
+    drive(ref, trace[:half], ranks[:half], L, budget, "adapter")
+    drive(sim, trace[:half], ranks[:half], L, budget, "adapter")
+    words = sim.export_state()
+    assert words.size == 2 + 4 * L * S and words[0] == ref.tick and words[1] == ref.step == half
+    for l in range(L):
+        for s in range(S):
+            w = words[2 + 4 * (l * S + s):6 + 4 * (l * S + s)]
+            p = ref.pools[l]
+            assert list(w) == [p.slot_expert[s], p.slot_tick[s], p.slot_origin[s], p.slot_used[s]], (l, s)
+    resumed = B.Sim(L, n, S, False)
+    resumed.import_state(words)
+    n_before = len(sim.events())
+    drive(sim, trace[half:], ranks[half:], L, budget, "adapter")
+    drive(resumed, trace[half:], ranks[half:], L, budget, "adapter")
+    assert resumed.events() == sim.events()[n_before:]
+    assert [resumed.slot_table(l) for l in range(L)] == [sim.slot_table(l) for l in range(L)]
+    # invalid states are refused and leave the table as it was
+    keep = resumed.export_state()
+    for bad in (words[:-1], np.concatenate((words, [0])), np.where(np.arange(words.size) == 2, n, words),
+                np.where(np.arange(words.size) == 3, words[0] + 1, words)):
+        with pytest.raises(B.SpmError):
+            resumed.import_state(bad)
+    dup = words.copy()
+    dup[2 + 4] = dup[2]                    # the same expert in two slots of layer 0
+    if dup[2] >= 0:
+        with pytest.raises(B.SpmError):
+            resumed.import_state(dup)
+    assert np.array_equal(resumed.export_state(), keep)
+    for x in (sim, resumed):
+        x.close()

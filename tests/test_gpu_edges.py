@@ -158,3 +158,36 @@ def test_read_bandwidth_probe_and_its_limits():
     with pytest.raises(Exception):
         m.measure_read_bandwidth(1 << 20)                            # too small to get past L2
     m.close()
+
+
+def test_cache_checkpoint_resumes_a_run_bit_for_bit():
+    # export the cache state mid-run, import it into a fresh context: the rest of the run gives the
+    # same outputs, events and slot tables as the uninterrupted one and as the oracle
+    cfg = synth.get_config("tiny", slots=5, budget=2)
+    steps, half = 16, 7
+    tok = synth.zipf_tokens(cfg, steps=steps)
+    H = synth.embedding_rows(cfg, tok.reshape(-1)).numpy().reshape(steps, 1, cfg.hidden)
+    ref = make_ref(cfg, weights=SynthWeights(cfg), policy="adapter")
+    a = build(cfg)
+    outs = []
+    for s in range(steps):
+        if s == half:
+            state = a.cache_export()
+            mark = len(a.events())
+        outs.append(a.decode_step(dev(H[s])))
+        a.synchronize()
+        want, _ = ref.step(H[s])
+        assert M.rel_linf(outs[-1].cpu().numpy().astype(np.float64)[0], want[0]) < 4e-5
+    assert a.events() == ref.table.events
+    b = build(cfg)
+    b.cache_import(state)
+    assert b.stats()["h2d_bytes"] == 0 and b.events() == []
+    for s in range(half, steps):
+        out = b.decode_step(dev(H[s]))
+        b.synchronize()
+        assert np.array_equal(out.cpu().numpy(), outs[s].cpu().numpy()), s
+    assert b.events() == a.events()[mark:]
+    assert [list(b.slot_table(l)) for l in range(cfg.n_layers)] == [list(a.slot_table(l)) for l in range(cfg.n_layers)]
+    with pytest.raises(Exception):
+        b.cache_import(state[:-1])
+    a.close(); b.close()
