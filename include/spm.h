@@ -292,6 +292,12 @@ int spm_cache_reset(spm_ctx* ctx);                         /* cold cache, step c
  *   exporting context would have: same hits, misses, evictions, outputs. */
 int spm_cache_export(spm_ctx* ctx, int64_t* state, size_t capacity, size_t* count);
 int spm_cache_import(spm_ctx* ctx, const int64_t* state, size_t count);
+/* Debug aid: checks the slot table's structural invariants (slot -> expert and expert -> slot are
+ * inverse maps, no expert in two slots of a layer, no LRU tick ahead of the global tick) and, when
+ * `with_device` is non-zero, waits for the compute stream and checks the kernels' status word
+ * (bad slot number, copy or pipeline time-out). SPM_OK, or SPM_ERR_STATE / the status error with a
+ * message in spm_last_error. */
+int spm_check_invariants(spm_ctx* ctx, int with_device);
 int spm_reset_stats(spm_ctx* ctx);                         /* counters, timings and event log only; cache kept */
 int spm_get_stats(spm_ctx* ctx, spm_stats* out);           /* waits for timed work to finish */
 /* Per-layer sums since the last reset: stall_us[L], ffn_us[L], and the number of steps in them. */
@@ -363,6 +369,7 @@ int spm_sim_events(spm_sim* sim, spm_event* out, size_t capacity, size_t* count)
 int spm_sim_stats(spm_sim* sim, spm_stats* out);
 int spm_sim_slot_table(spm_sim* sim, int layer, int32_t* slot_expert /* [slots] */);
 /* Same checkpoint words as spm_cache_export / spm_cache_import, for the host-only table. */
+int spm_sim_check(spm_sim* sim);                            /* SPM_OK, or SPM_ERR_STATE when the table's invariants fail */
 int spm_sim_export(spm_sim* sim, int64_t* state, size_t capacity, size_t* count);
 int spm_sim_import(spm_sim* sim, const int64_t* state, size_t count);
 

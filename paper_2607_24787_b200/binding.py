@@ -110,6 +110,8 @@ _SIG = {
     "spm_sim_events": [_P, _P, C.c_size_t, C.POINTER(C.c_size_t)],
     "spm_sim_stats": [_P, C.POINTER(Stats)],
     "spm_sim_slot_table": [_P, C.c_int, _P],
+    "spm_sim_check": [_P],
+    "spm_check_invariants": [_P, C.c_int],
     "spm_sim_export": [_P, _P, C.c_size_t, C.POINTER(C.c_size_t)],
     "spm_sim_import": [_P, _P, C.c_size_t],
     "spm_cache_export": [_P, _P, C.c_size_t, C.POINTER(C.c_size_t)],
@@ -310,6 +312,10 @@ def spm_cache_reset(ctx):
     _check(load().spm_cache_reset(ctx), ctx)
 
 
+def spm_check_invariants(ctx, with_device=True):
+    _check(load().spm_check_invariants(ctx, int(with_device)), ctx)
+
+
 def spm_cache_export(ctx) -> np.ndarray:
     """The expert cache's checkpoint words (int64)."""
     n = C.c_size_t()
@@ -446,6 +452,9 @@ class Sim:
         out = np.empty(self.S, np.int32)
         _check(load().spm_sim_slot_table(self.h, layer, _ptr(out)))
         return [int(e) for e in out]
+
+    def check(self):
+        _check(load().spm_sim_check(self.h))
 
     def export_state(self) -> np.ndarray:
         n = C.c_size_t()

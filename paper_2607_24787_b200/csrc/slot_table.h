@@ -163,6 +163,27 @@ public:
         }
     }
 
+    // Structural invariants of the table: slot -> expert and expert -> slot are inverse maps, no
+    // expert sits in two slots of a layer, no tick lies ahead of the global tick, flags are 0/1.
+    // Returns -1 when they hold, else the index (layer * slots + slot, or L*S + layer*n + expert
+    // for a dangling expert entry) of the first violation.
+    long long check() const {
+        for (int l = 0; l < L_; ++l) {
+            for (int sl = 0; sl < S_; ++sl) {
+                const size_t k = size_t(l) * S_ + sl;
+                const int e = slot_expert_[k];
+                if (e < -1 || e >= n_ || slot_tick_[k] > tick_ || slot_origin_[k] > 1 || slot_used_[k] > 1) return (long long)k;
+                if (e >= 0 && expert_slot_[size_t(l) * n_ + e] != sl) return (long long)k;
+            }
+            for (int e = 0; e < n_; ++e) {
+                const int sl = expert_slot_[size_t(l) * n_ + e];
+                if (sl < -1 || sl >= S_ || (sl >= 0 && slot_expert_[size_t(l) * S_ + sl] != e))
+                    return (long long)(size_t(L_) * S_ + size_t(l) * n_ + e);
+            }
+        }
+        return -1;
+    }
+
     // Checkpoint of the table as 64-bit words (no weights): {tick, step}, then per slot of every
     // layer {expert or -1, LRU tick, origin, used}. Accounting (statistics, event log) is not part of it.
     static size_t state_words(int n_layers, int slots) { return 2 + size_t(4) * n_layers * slots; }

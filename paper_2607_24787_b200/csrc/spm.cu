@@ -1513,6 +1513,18 @@ int spm_cache_reset(spm_ctx* c) {
     return SPM_OK;
 }
 
+int spm_check_invariants(spm_ctx* c, int with_device) {
+    if (!c) return SPM_ERR_INVALID_ARG;
+    if (int rc = flush_trace(c)) return rc;
+    const long long bad = c->table->check();
+    if (bad >= 0) return fail(c, SPM_ERR_STATE, "slot table invariant violated at index %lld", bad);
+    if (with_device) {
+        CU(c, cudaStreamSynchronize(c->compute));
+        return check_status(c);
+    }
+    return SPM_OK;
+}
+
 int spm_cache_export(spm_ctx* c, int64_t* state, size_t capacity, size_t* count) {
     if (!c || !count) return SPM_ERR_INVALID_ARG;
     if (int rc = flush_trace(c)) return rc;
@@ -1780,6 +1792,11 @@ int spm_sim_stats(spm_sim* s, spm_stats* out) {
     if (!s || !out) return SPM_ERR_INVALID_ARG;
     *out = s->table.stats();
     return SPM_OK;
+}
+
+int spm_sim_check(spm_sim* s) {
+    if (!s) return SPM_ERR_INVALID_ARG;
+    return s->table.check() < 0 ? SPM_OK : SPM_ERR_STATE;
 }
 
 int spm_sim_export(spm_sim* s, int64_t* state, size_t capacity, size_t* count) {

@@ -158,6 +158,7 @@ class OffloadedMoE:
     def profile_window(self): return B.spm_profile_window(self.ctx)
     def measure_read_bandwidth(self, nbytes, reps=5): return B.spm_measure_read_bandwidth(self.ctx, nbytes, reps)
     def cache_reset(self): B.spm_cache_reset(self.ctx)
+    def check_invariants(self, with_device=True): B.spm_check_invariants(self.ctx, with_device)
     def cache_export(self): return B.spm_cache_export(self.ctx)
     def cache_import(self, state): B.spm_cache_import(self.ctx, state)
     def reset_stats(self): B.spm_reset_stats(self.ctx)

@@ -73,6 +73,7 @@ def drive(policy_obj, trace, ranks, L, budget, mode, drop=0):
             policy_obj.step += 1
         else:
             policy_obj.end_step()
+            policy_obj.check()                 # structural invariants of the library's table after every step
 
 
 @pytest.mark.parametrize("mode,S,budget,nb,plain,drop", [

@@ -39,6 +39,7 @@ def compare_run(cfg, steps=6, policy="adapter", tol=4e-5, **kw):
         for t in range(nb):
             assert M.rel_linf(got[t], want[t]) < tol, (s, t)
     assert m.events() == ref.table.events
+    m.check_invariants()
     st = m.stats()
     m.close()
     return st
