@@ -51,6 +51,7 @@ extern "C" {
 #define SPM_ERR_TIMEOUT       (-4)  /* routing kernel did not report within the deadline      */
 #define SPM_ERR_NOT_RESIDENT  (-5)  /* an expert handed to the FFN has no loaded slot         */
 #define SPM_ERR_STATE         (-6)  /* call made in the wrong order (e.g. no hint trace set)  */
+#define SPM_ERR_NUMERIC       (-7)  /* a routing kernel met a non-finite logit (NaN / Inf in h or weights) */
 
 #define SPM_DTYPE_FP32 0
 #define SPM_DTYPE_BF16 1

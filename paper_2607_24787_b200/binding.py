@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(HERE, "libspm.so")
 
 SPM_OK = 0
 ERR_NAMES = {-1: "SPM_ERR_INVALID_ARG", -2: "SPM_ERR_CONFIG", -3: "SPM_ERR_CUDA", -4: "SPM_ERR_TIMEOUT",
-             -5: "SPM_ERR_NOT_RESIDENT", -6: "SPM_ERR_STATE"}
+             -5: "SPM_ERR_NOT_RESIDENT", -6: "SPM_ERR_STATE", -7: "SPM_ERR_NUMERIC"}
 DTYPE_FP32, DTYPE_BF16, DTYPE_Q4 = 0, 1, 2
 POLICY_ADAPTER, POLICY_ON_DEMAND, POLICY_HINT_TRACE, POLICY_PRED0, POLICY_NAIVE = 0, 1, 2, 3, 4
 POLICIES = {"adapter": 0, "on_demand": 1, "hint_trace": 2, "pred0": 3, "naive": 4}

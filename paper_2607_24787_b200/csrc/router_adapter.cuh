@@ -54,6 +54,7 @@ struct RouterArgs {
     const short* slot_map;   // optional [n] slot of each expert of this layer (device memory) ...
     short* codes_out;        // ... and where to leave the slots of the routed experts, [nb][K]
     unsigned long long* clock;   // optional {first leader past its dependency wait, last leader done} in ns
+    int* status;             // optional status word: kStatusNonFinite is set when a router logit is NaN or Inf
     const float* partial;    // optional [nb][G][D] partial rows of the preceding expert kernel: the hidden row is
     int G;                   //   then h + sum of them (summed here instead of by a combine kernel) ...
     float* h_out;            //   ... and written back here ([nb][D], may alias h)
@@ -114,6 +115,7 @@ __device__ __forceinline__ int rank_of(const float* v, int n, int e) {
 }
 
 constexpr int kRouterCluster = 8;   // CTAs per token, one thread-block cluster
+constexpr int kStatusNonFinite = 8; // status bit (the expert kernels own bits 1, 2 and 4)
 constexpr int kReduceGroupsR = 8;   // runs of partial rows (= warps of a CTA); must equal the combine kernel's group count
 constexpr int kReduceChunkR = 20;   // partial rows a lane keeps in flight
 
@@ -412,8 +414,14 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     Mailbox* mb = a.mailbox;
     const int half = threadIdx.x >> 7, ht = threadIdx.x & 127;
     if (half == 0 && a.do_router) {
+        if (ht < a.K) { isel[ht] = 0; psel[ht] = 0.f; }     // stays in range even if NaN logits leave a rank unfilled
         for (int e = ht; e < n; e += 128) {
-            const float z = zs[e];
+            float z = zs[e];
+            if (!isfinite(z)) {      // ids of this token are meaningless then; keep the ordering total so every rank is filled
+                if (a.status) atomicOr(a.status, kStatusNonFinite);
+                z = -3.0e38f;
+                zs[e] = z;
+            }
             ps[e] = z;
             a.logits[size_t(tok) * n + e] = z;
             if (a.logits_out) a.logits_out[size_t(tok) * n + e] = z;
@@ -440,6 +448,10 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
         for (int e = ht; e < n; e += 128) {
             float acc = 0.f;
             for (int q = 0; q < a.r; ++q) acc = fmaf(bs[e * a.r + q], us[q], acc);
+            if (!isfinite(acc)) {
+                if (a.status) atomicOr(a.status, kStatusNonFinite);
+                acc = -3.0e38f;
+            }
             qs[e] = acc;
         }
         asm volatile("bar.sync 2, 128;" ::: "memory");

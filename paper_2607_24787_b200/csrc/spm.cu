@@ -371,6 +371,7 @@ int launch_router(spm_ctx* c, int layer, const float* h, const float* x_in, int 
     a.scores = c->ws_scores;
     a.order = c->ws_order;
     a.counters = c->ws_counters;
+    a.status = c->ws_status;
     a.mailbox = route ? route->mailbox_dev : c->mb_dev;
     a.slot_map = route ? route->slot_map : nullptr;
     a.codes_out = route ? route->codes_out : nullptr;
@@ -1065,9 +1066,12 @@ int check_layer(spm_ctx* c, int layer, int nb) {
 int check_status(spm_ctx* c) {
     int st = 0;
     CU(c, cudaMemcpy(&st, c->ws_status, sizeof st, cudaMemcpyDeviceToHost));
+    if (st == 0) return SPM_OK;
+    CU(c, cudaMemset(c->ws_status, 0, sizeof st));      // reported once; the context stays usable
     if (st & kStatusCopyTimeout) return fail(c, SPM_ERR_TIMEOUT, "expert FFN kernel gave up waiting for a weight copy");
     if (st & kStatusBadSlot) return fail(c, SPM_ERR_NOT_RESIDENT, "expert FFN kernel received a slot number outside the pool");
     if (st & kStatusGroupedTimeout) return fail(c, SPM_ERR_TIMEOUT, "grouped expert FFN kernel gave up waiting on a pipeline barrier");
+    if (st & kStatusNonFinite) return fail(c, SPM_ERR_NUMERIC, "a routing kernel met a non-finite logit (NaN or Inf in the hidden rows or the weights)");
     return SPM_OK;
 }
 

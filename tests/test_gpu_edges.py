@@ -192,3 +192,25 @@ def test_cache_checkpoint_resumes_a_run_bit_for_bit():
     with pytest.raises(Exception):
         b.cache_import(state[:-1])
     a.close(); b.close()
+
+
+def test_non_finite_hidden_row_is_reported_not_propagated_silently():
+    from paper_2607_24787_b200 import binding as B
+    cfg = synth.get_config("tiny")
+    m = build(cfg)
+    tok = synth.zipf_tokens(cfg, steps=2)
+    H = synth.embedding_rows(cfg, tok.reshape(-1)).numpy().reshape(2, 1, cfg.hidden)
+    bad = H[0].copy()
+    bad[0, 7] = np.inf
+    m.decode_step(dev(bad))
+    with pytest.raises(B.SpmError) as e:
+        m.synchronize()
+    assert e.value.code == -7
+    # reported once; the context keeps working
+    m.cache_reset()
+    out = m.decode_step(dev(H[1]))
+    m.synchronize()
+    ref = make_ref(cfg, weights=SynthWeights(cfg), policy="adapter")
+    want, _ = ref.step(H[1])
+    assert M.rel_linf(out.cpu().numpy().astype(np.float64)[0], want[0]) < 4e-5
+    m.close()
