@@ -211,6 +211,7 @@ def arm_summary(m, cfg, elapsed_ms, steps):
         "hit_rate": st["hits"] / max(st["hits"] + st["misses"], 1),
         "ready_recall": st["ready_sum"] / max(st["ready_count"], 1),
         "expert_recall_at_budget": (st["recall_sum"] / st["recall_count"]) if st["recall_count"] else None,
+        "expert_recall_at_half_k_k_k_plus_2": [r / st["recall_count"] for r in st["recall_at"]] if st["recall_count"] else None,
         "copies_per_token": (st["misses"] + st["prefetch_issued"]) / max(steps * cfg.batch, 1),
         "prefetch_issued": st["prefetch_issued"], "prefetch_used": st["hits_prefetched"], "prefetch_wasted": st["wasted"],
         "late_arrivals": st["late_arrivals"],

@@ -139,6 +139,8 @@ typedef struct {
     double router_window_us;     /* in-kernel windows of the routing kernels (first leader past its launch      */
     double reduce_window_us;     /*   dependency -> last leader done) and of the combine kernels, timing on     */
     double gap_us;               /* device idle time between consecutive clocked kernels of the compute stream  */
+    double recall_at[3];         /* sums like recall_sum for M = max(1, K/2), K, K+2 (the coverage levels of
+                                    the paper's model-level table); divide by recall_count                    */
 } spm_stats;
 
 /* ---- packed expert layout ------------------------------------------------

@@ -54,10 +54,12 @@ class Stats(C.Structure):
                 + [("ffn_us", C.c_double), ("ffn_window_us", C.c_double), ("stall_us", C.c_double), ("ready_sum", C.c_double),
                    ("ready_count", C.c_uint64), ("recall_sum", C.c_double), ("recall_count", C.c_uint64),
                    ("host_free_steps", C.c_uint64), ("router_window_us", C.c_double), ("reduce_window_us", C.c_double),
-                   ("gap_us", C.c_double)])
+                   ("gap_us", C.c_double), ("recall_at", C.c_double * 3)])
 
     def as_dict(self):
-        return {k: getattr(self, k) for k, _ in self._fields_}
+        d = {k: getattr(self, k) for k, _ in self._fields_}
+        d["recall_at"] = list(d["recall_at"])
+        return d
 
 
 # symbol -> argument types (all return int except spm_last_error)

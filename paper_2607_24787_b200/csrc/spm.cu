@@ -132,6 +132,7 @@ struct spm_ctx {
     std::vector<int16_t> wave_slot;
     uint64_t extra_late = 0, h2d_bytes = 0, ffn_launches = 0, kernel_launches = 0, tokens = 0;
     double ready_sum = 0, recall_sum = 0;
+    double recall_at[3] = {0, 0, 0};          // ExpertRecall@M for M = K/2, K, K+2 (same terms as recall_sum)
     uint64_t ready_count = 0, recall_count = 0;
     std::string err;
 };
@@ -874,6 +875,14 @@ int step_layers(spm_ctx* c, float* h_out, int nb, Timing* t, const Mailbox* trac
                     for (int q = 0; q < M; ++q) hit += c->prev_order[q] == ids[tk * K + k];
                 c->recall_sum += double(hit) / K;
                 c->recall_count++;
+                const int Ms[3] = {std::max(1, K / 2), K, K + 2};      // the coverage levels the paper tabulates
+                for (int j = 0; j < 3; ++j) {
+                    int h2 = 0;
+                    const int Mj = std::min(Ms[j], n);
+                    for (int k = 0; k < K; ++k)
+                        for (int q = 0; q < Mj; ++q) h2 += c->prev_order[q] == ids[tk * K + k];
+                    c->recall_at[j] += double(h2) / K;
+                }
             }
         }
         if (int rc = run_ffn(c, l, c->ws_x, ids.data(), c->ws_w, nb, h_out, t, -1, trace == nullptr,
@@ -1487,6 +1496,7 @@ int spm_reset_stats(spm_ctx* c) {
     c->extra_late = c->h2d_bytes = c->ffn_launches = c->kernel_launches = c->tokens = 0;
     c->host_free_steps = 0;
     c->ready_sum = c->recall_sum = 0;
+    c->recall_at[0] = c->recall_at[1] = c->recall_at[2] = 0;
     c->ready_count = c->recall_count = 0;
     return SPM_OK;
 }
@@ -1511,6 +1521,7 @@ int spm_cache_reset(spm_ctx* c) {
     c->timed_steps = 0;
     c->extra_late = c->h2d_bytes = c->ffn_launches = c->kernel_launches = c->tokens = 0;
     c->ready_sum = c->recall_sum = 0;
+    c->recall_at[0] = c->recall_at[1] = c->recall_at[2] = 0;
     c->ready_count = c->recall_count = 0;
     c->host_free_steps = 0;
     c->prev_order_valid = false;
@@ -1672,6 +1683,7 @@ int spm_get_stats(spm_ctx* c, spm_stats* out) {
     for (int l = 0; l < c->cfg.n_layers; ++l) { out->ffn_us += c->layer_ffn_us[l]; out->stall_us += c->layer_stall_us[l]; }
     out->ready_sum = c->ready_sum; out->ready_count = c->ready_count;
     out->recall_sum = c->recall_sum; out->recall_count = c->recall_count;
+    for (int j = 0; j < 3; ++j) out->recall_at[j] = c->recall_at[j];
     out->host_free_steps = c->host_free_steps;
     return check_status(c);
 }

@@ -203,6 +203,10 @@ def test_decode_step_free_running(setup, policy):
         rr = np.mean([M.expert_recall_at_m(recs[s][l + 1].ids, recs[s][l].scores, min(budget, cfg.n_experts), cfg.top_k)
                       for s in range(steps) for l in range(cfg.n_layers - 1)])
         assert abs(st["recall_sum"] / st["recall_count"] - rr) < 1e-9
+        for j, Mj in enumerate((max(1, cfg.top_k // 2), cfg.top_k, cfg.top_k + 2)):      # the paper's coverage levels
+            rj = np.mean([M.expert_recall_at_m(recs[s][l + 1].ids, recs[s][l].scores, min(Mj, cfg.n_experts), cfg.top_k)
+                          for s in range(steps) for l in range(cfg.n_layers - 1)])
+            assert abs(st["recall_at"][j] / st["recall_count"] - rj) < 1e-9, Mj
     rdy = np.mean([recs[s][l].ready for s in range(steps) for l in range(1, cfg.n_layers)])
     assert abs(st["ready_sum"] / st["ready_count"] - rdy) < 1e-9
 
