@@ -97,21 +97,32 @@ __device__ __forceinline__ void block_softmax(float* v, int n, float* scratch) {
     __syncthreads();
 }
 
-// position of element e in the ordering (value descending, index ascending)
-__device__ __forceinline__ int rank_of(const float* v, int n, int e) {
-    const float ve = v[e];
-    int c = 0, j = 0;
-    if ((reinterpret_cast<uintptr_t>(v) & 15) == 0) {
+// Order-preserving integer image of a finite float (-0 counts as +0): a < b  <=>  key(a) < key(b).
+__device__ __forceinline__ int order_key(float v) {
+    const int b = __float_as_int(v + 0.0f);
+    return b ^ ((b >> 31) & 0x7fffffff);
+}
+
+// Position of element e in the ordering (key descending, index ascending) of k[0..n): the number
+// of elements that beat it. Element j beats e when k[j] > k[e], or k[j] == k[e] and j < e, i.e.
+// when k[j] > k[e] - (j < e): branch-free, four independent counters. Keys never equal INT_MIN
+// (that image belongs to a NaN, and non-finite values are replaced before ranking).
+__device__ __forceinline__ int rank_of_key(const int* k, int n, int e) {
+    const int ke = k[e];
+    int c0 = 0, c1 = 0, c2 = 0, c3 = 0, j = 0;
+    if ((reinterpret_cast<uintptr_t>(k) & 15) == 0) {
+#pragma unroll 4
         for (; j + 4 <= n; j += 4) {
-            const float4 t = *reinterpret_cast<const float4*>(v + j);
-            c += (t.x > ve) || (t.x == ve && j < e);
-            c += (t.y > ve) || (t.y == ve && j + 1 < e);
-            c += (t.z > ve) || (t.z == ve && j + 2 < e);
-            c += (t.w > ve) || (t.w == ve && j + 3 < e);
+            const int4 t = *reinterpret_cast<const int4*>(k + j);
+            const int d = e - j;                       // element j + i precedes e  <=>  i < d
+            c0 += t.x > ke - int(0 < d);
+            c1 += t.y > ke - int(1 < d);
+            c2 += t.z > ke - int(2 < d);
+            c3 += t.w > ke - int(3 < d);
         }
     }
-    for (; j < n; ++j) c += (v[j] > ve) || (v[j] == ve && j < e);
-    return c;
+    for (; j < n; ++j) c0 += k[j] > ke - int(j < e);
+    return c0 + c1 + c2 + c3;
 }
 
 constexpr int kRouterCluster = 8;   // CTAs per token, one thread-block cluster
@@ -420,16 +431,16 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
             if (!isfinite(z)) {      // ids of this token are meaningless then; keep the ordering total so every rank is filled
                 if (a.status) atomicOr(a.status, kStatusNonFinite);
                 z = -3.0e38f;
-                zs[e] = z;
             }
             ps[e] = z;
+            reinterpret_cast<int*>(zs)[e] = order_key(z);       // the ranking below works on these
             a.logits[size_t(tok) * n + e] = z;
             if (a.logits_out) a.logits_out[size_t(tok) * n + e] = z;
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
-        half_softmax(ps, n, scratch, 1);          // ps = p, zs = z (ranking is taken on the logits)
+        half_softmax(ps, n, scratch, 1);          // ps = p, zs = order keys of z (ranking is taken on the logits)
         for (int e = ht; e < n; e += 128) {
-            const int rk = rank_of(zs, n, e);
+            const int rk = rank_of_key(reinterpret_cast<const int*>(zs), n, e);
             if (rk < a.K) { isel[rk] = e; psel[rk] = ps[e]; }
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -460,7 +471,7 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
             for (int e = ht; e < n; e += 128) a.pihat[size_t(tok) * n + e] = qs[e];
         } else {
             for (int e = ht; e < n; e += 128) {        // one token: its distribution is the priority vector
-                const int rk = rank_of(qs, n, e);
+                const int rk = rank_of_key(reinterpret_cast<const int*>(qs), n, e);   // non-negative floats order like their bits
                 a.order[rk] = e;
                 a.scores[e] = qs[e];
                 if (mb) { mb->order[rk] = tagged(tag, e); mb->scores[e] = qs[e]; }
@@ -488,7 +499,7 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
             }
             __syncthreads();
             for (int e = threadIdx.x; e < n; e += kRouterThreads) {
-                const int rk = rank_of(qs, n, e);
+                const int rk = rank_of_key(reinterpret_cast<const int*>(qs), n, e);
                 a.order[rk] = e;
                 a.scores[e] = qs[e];
                 if (mb) { mb->order[rk] = tagged(tag, e); mb->scores[e] = qs[e]; }
