@@ -7,8 +7,8 @@
  *      T = Top_K(z);  w_e = p_e / sum_{j in T} p_j            [Section 3.1, first equation]
  *   2. batch demand T_batch = union of the tokens' Top-K sets  [Section 3.1, second equation];
  *      experts of T_batch without a cache slot are copied on demand from the pinned
- *      host store ("any required expert that is not available is loaded on demand",
- *      Section 3.3, last paragraph)
+ *      host store (the fallback that Section 3.3's last paragraph prescribes for every
+ *      needed expert the prefetch did not bring in)
  *   3. adapter (l <= L-2):  z^ = Bup (A x);  pi^ = softmax(z^);  s_e = sum over tokens of pi^_e
  *      [Section 3.2, equations 1, 3, 4]; the experts of layer l+1 are ranked by s
  *   4. budgeted selection  P = Top_{M_max}({ s_e : e not available, not in transfer }),

@@ -130,6 +130,7 @@ struct spm_ctx {
     std::vector<Placement> placements;
     std::vector<int32_t> need, sel, protect, slots_tmp;
     std::vector<int16_t> wave_slot;
+    std::vector<int32_t> plan_first;
     uint64_t extra_late = 0, h2d_bytes = 0, ffn_launches = 0, kernel_launches = 0, tokens = 0;
     double ready_sum = 0, recall_sum = 0;
     double recall_at[3] = {0, 0, 0};          // ExpertRecall@M for M = K/2, K, K+2 (same terms as recall_sum)
@@ -614,20 +615,28 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
     GgRow* rows = reinterpret_cast<GgRow*>(hd + c->tc_off_rows);
     int32_t* rowmap = reinterpret_cast<int32_t*>(hd + c->tc_off_rowmap);
     std::fill(rowmap, rowmap + size_t(nb) * SPM_MAX_TOPK, -1);
+    // counting sort of the wave's (token, k) pairs by expert: rows of an expert keep token-major order
     int n_rows = 0, n_units = 0;
+    std::vector<int32_t>& row_of = c->plan_first;       // per expert: pairs in this wave, then the next free row of its run
+    row_of.assign(size_t(m.n_experts) + 1, 0);
+    for (int i = 0; i < nb * K; ++i)
+        if (slot_of_expert[ids[i]] >= 0) ++row_of[ids[i] + 1];
     for (int e = 0; e < m.n_experts; ++e) {
-        if (slot_of_expert[e] < 0) continue;
-        const int row0 = n_rows;
-        for (int tk = 0; tk < nb; ++tk)
-            for (int k = 0; k < K; ++k)
-                if (ids[tk * K + k] == e) {
-                    rowmap[tk * SPM_MAX_TOPK + k] = n_rows;
-                    rows[n_rows++] = GgRow{tk, k};
-                }
-        if (n_rows == row0) continue;
+        const int cnt = row_of[e + 1];
+        row_of[e + 1] = row_of[e] + cnt;
+        if (cnt == 0) continue;
         for (int jt = 0; jt < c->n_jt; ++jt)
-            units[n_units++] = GgUnit{layer * c->S + slot_of_expert[e], jt, row0, n_rows - row0};
+            units[n_units++] = GgUnit{layer * c->S + slot_of_expert[e], jt, row_of[e], cnt};
     }
+    n_rows = row_of[m.n_experts];
+    for (int tk = 0; tk < nb; ++tk)
+        for (int k = 0; k < K; ++k) {
+            const int e = ids[tk * K + k];
+            if (slot_of_expert[e] < 0) continue;
+            const int r = row_of[e]++;
+            rowmap[tk * SPM_MAX_TOPK + k] = r;
+            rows[r] = GgRow{tk, k};
+        }
     if (n_units == 0) return SPM_OK;
     CU(c, cudaMemcpyAsync(dd, hd, c->tc_desc_bytes, cudaMemcpyHostToDevice, c->compute));
     CU(c, cudaEventRecord(c->tc_desc_ev[d], c->compute));
