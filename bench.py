@@ -470,6 +470,15 @@ def resident_run(cfg, m, H_dev, W, K, peak, algo_bytes, device):
             leg.update(ffn_window_us=win, ffn_gb_s_in_window=algo_bytes / (win * 1e-6) / 1e9,
                        ffn_frac_in_window=algo_bytes / (win * 1e-6) / 1e9 / peak,
                        hbm_bound_tok_s=peak * 1e9 / (algo_bytes * cfg.n_layers) * cfg.batch)
+        # the same without per-kernel clocks, launch by launch and replayed from CUDA graphs
+        full.set_timing(0)
+        for replay, key in ((0, "tok_s_untimed_launches"), (1, "tok_s_untimed_graph_replay")):
+            full.set_graph_replay(replay)
+            timed_run(full, H_dev, 0, W, 1)
+            el2, _, _ = timed_run(full, H_dev, W, K, 1)
+            leg[key] = K * cfg.batch / (el2 / 1e3)
+        full.set_graph_replay(1)
+        full.set_timing(1)
         out["host_free_" + policy] = leg
     full.set_policy("on_demand")
     full.set_host_free(0)

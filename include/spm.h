@@ -260,6 +260,12 @@ int spm_set_device_wait(spm_ctx* ctx, int on);
  * window still is). Steps on the batched tensor-core path are never host-free.
  * spm_cache_reset() ends the state; it is re-entered once the pools are full again. */
 int spm_set_host_free(spm_ctx* ctx, int on);
+/* Replay host-free steps from CUDA graphs (default on): the launches of such a step are the same
+ * every time for a given trace slot, batch size, output buffer and launch geometry, so each
+ * combination is captured once (after one step enqueued launch by launch) and replayed with a
+ * single submission. Off, or with timing / an attention stand-in set, every kernel is launched
+ * individually. Results are identical. */
+int spm_set_graph_replay(spm_ctx* ctx, int on);
 /* Stand-in for the attention block the synthetic configurations omit: before each layer's router a
  * kernel that only waits `us` microseconds (0 = off, at most 100000) is enqueued on the compute
  * stream. It widens the overlap window W_l = t_exec(l+1) - t_pred(l) (Section 3.1) toward the

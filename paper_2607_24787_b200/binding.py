@@ -89,6 +89,7 @@ _SIG = {
     "spm_set_attention_stub_us": [_P, C.c_int],
     "spm_set_device_wait": [_P, C.c_int],
     "spm_set_host_free": [_P, C.c_int],
+    "spm_set_graph_replay": [_P, C.c_int],
     "spm_set_copy_delay_us": [_P, C.c_int],
     "spm_profile_window": [_P, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int)],
     "spm_measure_read_bandwidth": [_P, C.c_size_t, C.c_int, C.POINTER(C.c_double)],
@@ -287,6 +288,10 @@ def spm_set_device_wait(ctx, on):
 
 def spm_set_host_free(ctx, on):
     _check(load().spm_set_host_free(ctx, int(on)), ctx)
+
+
+def spm_set_graph_replay(ctx, on):
+    _check(load().spm_set_graph_replay(ctx, int(on)), ctx)
 
 
 def spm_set_attention_stub_us(ctx, us):

@@ -121,6 +121,13 @@ struct spm_ctx {
     std::vector<cudaEvent_t> tr_ev;
     std::deque<std::pair<int, int>> tr_pending;   // (ring slot, nb) of steps enqueued but not yet replayed
     uint64_t tr_count = 0, host_free_steps = 0;
+    struct HostFreeGraph {                    // a captured host-free step and what one replay adds to the launch counters
+        int slot, nb; const float* h_out; bool predict; int G, batched_path;
+        uint64_t kernels, ffns, tcs;
+        cudaGraphExec_t exec;
+    };
+    std::vector<HostFreeGraph> hf_graphs;
+    bool graph_replay = true, hf_warm = false;
     std::vector<std::vector<int32_t>> prev_rank;   // Naive Prefetch: experts the preceding step used, per layer
     std::vector<std::vector<int32_t>> pending_protect;
     std::vector<uint8_t> has_plan;
@@ -986,15 +993,10 @@ int host_free_ready(spm_ctx* c, int nb, bool* out) {
     return SPM_OK;
 }
 
-int enqueue_host_free_step(spm_ctx* c, const float* h_in, int nb, float* h_out) {
+// The kernels of all layers of one host-free step, enqueued on the compute stream (or captured).
+int enqueue_host_free_layers(spm_ctx* c, int nb, float* h_out, int slot, bool predict) {
     const spm_model_cfg& m = c->cfg;
     const int L = m.n_layers, K = m.top_k, n = m.n_experts;
-    if (int(c->tr_pending.size()) == kTraceRing)
-        if (int rc = replay_oldest(c)) return rc;
-    const int slot = int(c->tr_count++ % kTraceRing);
-    if (h_out != h_in)
-        CU(c, cudaMemcpyAsync(h_out, h_in, size_t(nb) * m.hidden * 4, cudaMemcpyDeviceToDevice, c->compute));
-    const bool predict = c->policy == SPM_POLICY_ADAPTER || c->policy == SPM_POLICY_PRED0;
     const int G = ffn_grid_for(c, nb);
     for (int l = 0; l < L; ++l) {
         if (c->stub_us > 0) {
@@ -1064,6 +1066,56 @@ int enqueue_host_free_step(spm_ctx* c, const float* h_in, int nb, float* h_out) 
         }
         c->kernel_launches += 2;
         c->ffn_launches++;
+    }
+    return SPM_OK;
+}
+
+// A host-free step is the same sequence of launches every time (for a given trace slot, batch size,
+// output buffer, prediction on/off and launch geometry), so it is captured once into a CUDA graph
+// and replayed: one submission instead of 2-5 per layer. Steps with timing or an attention
+// stand-in are enqueued launch by launch.
+int enqueue_host_free_step(spm_ctx* c, const float* h_in, int nb, float* h_out) {
+    const spm_model_cfg& m = c->cfg;
+    if (int(c->tr_pending.size()) == kTraceRing)
+        if (int rc = replay_oldest(c)) return rc;
+    const int slot = int(c->tr_count++ % kTraceRing);
+    if (h_out != h_in)
+        CU(c, cudaMemcpyAsync(h_out, h_in, size_t(nb) * m.hidden * 4, cudaMemcpyDeviceToDevice, c->compute));
+    const bool predict = c->policy == SPM_POLICY_ADAPTER || c->policy == SPM_POLICY_PRED0;
+    bool done = false;
+    if (c->graph_replay && !c->timing && c->stub_us == 0) {
+        const int G = ffn_grid_for(c, nb);
+        spm_ctx::HostFreeGraph* g = nullptr;
+        for (auto& x : c->hf_graphs)
+            if (x.slot == slot && x.nb == nb && x.h_out == h_out && x.predict == predict && x.G == G && x.batched_path == c->batched_path) g = &x;
+        if (!g && c->hf_warm && c->hf_graphs.size() < 64) {
+            // (the first host-free step ran launch by launch, so every kernel attribute is already set)
+            spm_ctx::HostFreeGraph ng{slot, nb, h_out, predict, G, c->batched_path, 0, 0, 0, nullptr};
+            const uint64_t k0 = c->kernel_launches, f0 = c->ffn_launches, t0 = c->tc_launches;
+            cudaGraph_t graph = nullptr;
+            CU(c, cudaStreamBeginCapture(c->compute, cudaStreamCaptureModeRelaxed));
+            const int rc = enqueue_host_free_layers(c, nb, h_out, slot, predict);
+            const cudaError_t ce = cudaStreamEndCapture(c->compute, &graph);
+            ng.kernels = c->kernel_launches - k0; ng.ffns = c->ffn_launches - f0; ng.tcs = c->tc_launches - t0;
+            c->kernel_launches = k0; c->ffn_launches = f0; c->tc_launches = t0;
+            if (rc == SPM_OK && ce == cudaSuccess && graph && cudaGraphInstantiate(&ng.exec, graph, 0) == cudaSuccess) {
+                c->hf_graphs.push_back(ng);
+                g = &c->hf_graphs.back();
+            } else {
+                cudaGetLastError();
+                c->graph_replay = false;       // capture is not possible here: keep enqueueing launch by launch
+            }
+            if (graph) cudaGraphDestroy(graph);
+        }
+        if (g) {
+            CU(c, cudaGraphLaunch(g->exec, c->compute));
+            c->kernel_launches += g->kernels; c->ffn_launches += g->ffns; c->tc_launches += g->tcs;
+            done = true;
+        }
+    }
+    if (!done) {
+        if (int rc = enqueue_host_free_layers(c, nb, h_out, slot, predict)) return rc;
+        c->hf_warm = true;
     }
     CU(c, cudaEventRecord(c->tr_ev[slot], c->compute));
     c->tr_pending.emplace_back(slot, nb);
@@ -1273,6 +1325,7 @@ int spm_destroy(spm_ctx* c) {
     for (auto ev : c->ring_end) if (ev) cudaEventDestroy(ev);
     if (c->mb_host) cudaFreeHost(c->mb_host);
     for (auto ev : c->tr_ev) if (ev) cudaEventDestroy(ev);
+    for (auto& g : c->hf_graphs) if (g.exec) cudaGraphExecDestroy(g.exec);
     if (c->tr_host) cudaFreeHost(c->tr_host);
     delete c->table;
     delete c;
@@ -1467,6 +1520,11 @@ int spm_set_host_free(spm_ctx* c, int on) {
     if (!c) return SPM_ERR_INVALID_ARG;
     if (int rc = flush_trace(c)) return rc;
     c->host_free = on != 0;
+    return SPM_OK;
+}
+int spm_set_graph_replay(spm_ctx* c, int on) {
+    if (!c) return SPM_ERR_INVALID_ARG;
+    c->graph_replay = on != 0;
     return SPM_OK;
 }
 int spm_set_attention_stub_us(spm_ctx* c, int us) {

@@ -154,6 +154,7 @@ class OffloadedMoE:
     def set_attention_stub_us(self, us): B.spm_set_attention_stub_us(self.ctx, us)
     def set_device_wait(self, on): B.spm_set_device_wait(self.ctx, on)
     def set_host_free(self, on): B.spm_set_host_free(self.ctx, on)
+    def set_graph_replay(self, on): B.spm_set_graph_replay(self.ctx, on)
     def set_copy_delay_us(self, us): B.spm_set_copy_delay_us(self.ctx, us)
     def profile_window(self): return B.spm_profile_window(self.ctx)
     def measure_read_bandwidth(self, nbytes, reps=5): return B.spm_measure_read_bandwidth(self.ctx, nbytes, reps)

@@ -176,3 +176,24 @@ def test_host_free_tensor_core_path_equals_host_driven(case):
     for s in range(steps):
         assert np.array_equal(a[s], b[s]), s
     assert ev_a == ev_b and st_a == st_b
+
+
+@pytest.mark.parametrize("name", ["tiny", "ds_small", "tiny_b3"])
+def test_graph_replay_gives_the_same_bits_and_bookkeeping(name):
+    cfg = SHAPES[name]
+    steps = 24                      # three laps of the trace ring: every slot's graph is captured, then replayed
+    H = rows(cfg, steps)
+    results = []
+    for replay in (1, 0):
+        m = build(cfg)
+        m.set_graph_replay(replay)
+        preload(cfg, m)
+        outs = run(m, H)
+        st = m.stats()
+        assert st["host_free_steps"] == steps
+        results.append((outs, m.events(), {k: st[k] for k in ("hits", "touches", "steps", "tokens", "kernel_launches", "ffn_launches", "recall_sum")}))
+        m.close()
+    (a, ev_a, st_a), (b, ev_b, st_b) = results
+    for s in range(steps):
+        assert np.array_equal(a[s], b[s]), s
+    assert ev_a == ev_b and st_a == st_b
