@@ -474,7 +474,8 @@ def resident_run(cfg, m, H_dev, W, K, peak, algo_bytes, device):
         full.set_timing(0)
         for replay, key in ((0, "tok_s_untimed_launches"), (1, "tok_s_untimed_graph_replay")):
             full.set_graph_replay(replay)
-            timed_run(full, H_dev, 0, W, 1)
+            for _ in range(1 + 9 // max(W, 1)):       # one step launch by launch, then one capture per trace slot (8)
+                timed_run(full, H_dev, 0, W, 1)
             el2, _, _ = timed_run(full, H_dev, W, K, 1)
             leg[key] = K * cfg.batch / (el2 / 1e3)
         full.set_graph_replay(1)
