@@ -1093,9 +1093,12 @@ int enqueue_host_free_step(spm_ctx* c, const float* h_in, int nb, float* h_out) 
             spm_ctx::HostFreeGraph ng{slot, nb, h_out, predict, G, c->batched_path, 0, 0, 0, nullptr};
             const uint64_t k0 = c->kernel_launches, f0 = c->ffn_launches, t0 = c->tc_launches;
             cudaGraph_t graph = nullptr;
-            CU(c, cudaStreamBeginCapture(c->compute, cudaStreamCaptureModeRelaxed));
-            const int rc = enqueue_host_free_layers(c, nb, h_out, slot, predict);
-            const cudaError_t ce = cudaStreamEndCapture(c->compute, &graph);
+            int rc = SPM_ERR_CUDA;
+            cudaError_t ce = cudaStreamBeginCapture(c->compute, cudaStreamCaptureModeRelaxed);   // (fails on the legacy default stream)
+            if (ce == cudaSuccess) {
+                rc = enqueue_host_free_layers(c, nb, h_out, slot, predict);
+                ce = cudaStreamEndCapture(c->compute, &graph);
+            }
             ng.kernels = c->kernel_launches - k0; ng.ffns = c->ffn_launches - f0; ng.tcs = c->tc_launches - t0;
             c->kernel_launches = k0; c->ffn_launches = f0; c->tc_launches = t0;
             if (rc == SPM_OK && ce == cudaSuccess && graph && cudaGraphInstantiate(&ng.exec, graph, 0) == cudaSuccess) {
