@@ -159,10 +159,10 @@ def affordable_store_layers(cfg, world):
 
 
 def ffn_kernel_name(cfg):
+    if cfg.batch > 1 and cfg.n_shared == 0 and cfg.dtype in ("bf16", "q4"):
+        return "ffn_grouped_q4_kernel" if cfg.dtype == "q4" else "ffn_grouped_kernel"
     if cfg.dtype == "q4":
         return "ffn_gemv_q4_kernel"
-    if cfg.batch > 1 and cfg.n_shared == 0 and cfg.dtype == "bf16":
-        return "ffn_grouped_kernel"
     return "ffn_gemv_kernel"
 
 
@@ -655,20 +655,30 @@ def make_oracle(cfg, wts, budget, slots=None, policy="adapter"):
                       budget, policy=policy, renormalize=bool(cfg.renormalize), rms_eps=cfg.rms_eps, keep_records=False)
 
 
-def cpu_baseline(cfg, H, device, budget):
+def cpu_baseline(cfg, H, device, budget, mem_budget=40e9):
     """The oracle, as it stands, on a bounded sample: a few decode steps of the same token stream.
-    Weights are generated before the clock starts (a dry pass fills the provider's cache)."""
-    wts = LazyWeights(cfg, device if torch.cuda.is_available() else "cpu")
-    warm = make_oracle(cfg, wts, 0, slots=cfg.n_experts, policy="on_demand")
+    Weights are generated before the clock starts (an untimed pass of the same step fills the
+    provider's cache, which is emptied after the step). The fp64 matrices of one step stay below
+    `mem_budget` bytes: a batched step touches nearly every expert of every layer, so there the
+    sample is the first Ls layers and tokens/s is scaled by Ls / n_layers."""
+    per_layer = min(cfg.n_experts, cfg.batch * cfg.top_k) * 3 * cfg.inter * cfg.hidden * 8
+    Ls = int(max(1, min(cfg.n_layers, mem_budget // max(per_layer, 1))))
+    sub = cfg.replace(n_layers=Ls) if Ls < cfg.n_layers else cfg
+    wts = LazyWeights(sub, device if torch.cuda.is_available() else "cpu")
+    warm = make_oracle(sub, wts, 0, slots=cfg.n_experts, policy="on_demand")
+    ref = make_oracle(sub, wts, budget)
+    dt = 0.0
     for s in range(H.shape[0]):
-        warm.step(H[s])
-    ref = make_oracle(cfg, wts, budget)
-    t0 = time.perf_counter()
-    for s in range(H.shape[0]):
+        warm.step(H[s])                      # untimed: fills the weight cache for this step
+        t0 = time.perf_counter()
         ref.step(H[s])
-    dt = time.perf_counter() - t0
-    return {"value": H.shape[0] * cfg.batch / dt, "unit": "tokens/s", "cores": oracle_threads(), "kind": "oracle",
-            "sample": f"{H.shape[0]} decode steps (all {cfg.n_layers} layers) of the bench token stream, "
+        dt += time.perf_counter() - t0
+        wts.cache = {k: v for k, v in wts.cache.items() if k[0] != "e"}   # bound memory
+    layers = f"all {cfg.n_layers} layers" if Ls == cfg.n_layers else \
+        f"the first {Ls} of {cfg.n_layers} layers, tokens/s scaled by {Ls}/{cfg.n_layers}"
+    return {"value": H.shape[0] * cfg.batch * (Ls / cfg.n_layers) / dt, "unit": "tokens/s", "cores": oracle_threads(),
+            "kind": "oracle",
+            "sample": f"{H.shape[0]} decode steps ({layers}) of the bench token stream, "
                       f"numpy fp64, weights pre-generated; {dt:.2f} s"}
 
 

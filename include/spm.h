@@ -223,9 +223,10 @@ int spm_set_plain_lru(spm_ctx* ctx, int on);              /* 1: no predicted-use
 int spm_set_timing(spm_ctx* ctx, int on);                 /* record CUDA events around FFN / stalls */
 int spm_set_ffn_ctas(spm_ctx* ctx, int ctas);             /* CTAs per token of the GEMV FFN (0 = default) */
 /* Expert FFN used when nb > 1. 0 (default): the grouped tensor-core kernel (tcgen05, bf16
- * activations, fp32 accumulation) whenever the shape allows it (bf16 weights, no shared experts,
- * inter and hidden multiples of 128), else the GEMV kernel once per token. 1: always the GEMV
- * kernel per token (fp32 activations). */
+ * activations, fp32 accumulation) whenever the shape allows it (bf16 or 4-bit weights, no shared
+ * experts, inter a multiple of 128, hidden a multiple of 128 for bf16 and of 256 for 4-bit
+ * weights, which are expanded to bf16 on the way to the tensor cores), else the GEMV kernel once
+ * per token. 1: always the GEMV kernel per token (fp32 activations). */
 int spm_set_batched_path(spm_ctx* ctx, int mode);
 /* Perfect-knowledge ranking for SPM_POLICY_HINT_TRACE: for step s (counted from the last
  * spm_cache_reset) and layer l, hint[(s*L + l)*stride .. +count[s*L+l]) are the experts that
@@ -257,7 +258,8 @@ int spm_set_device_wait(spm_ctx* ctx, int on);
  * slot table's bookkeeping (hits, LRU ticks, recall statistics, event log) is replayed in order,
  * at the latest when a call reads or changes that state. Outputs, events and statistics are the
  * same as with the option off; per-layer event timings are not taken in such steps (the in-kernel
- * window still is). Steps on the batched tensor-core path are never host-free.
+ * window still is). On the batched tensor-core path the wave plan (token rows sorted by expert,
+ * work units, combine map) is then built by a kernel instead of the host.
  * spm_cache_reset() ends the state; it is re-entered once the pools are full again. */
 int spm_set_host_free(spm_ctx* ctx, int on);
 /* Replay host-free steps from CUDA graphs (default on): the launches of such a step are the same

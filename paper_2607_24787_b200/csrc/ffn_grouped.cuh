@@ -376,7 +376,7 @@ struct GgRow { int32_t token, k; };
 
 static __global__ void gg_gather_kernel(const float* __restrict__ x, const float* __restrict__ w, const GgRow* __restrict__ rows,
                                         int n_rows, const int* n_rows_dev, int D, int K, __nv_bfloat16* __restrict__ xs,
-                                        float* __restrict__ wrow) {
+                                        float* __restrict__ wrow, int perm8) {
     grid_dep_launch();
     grid_dep_wait();
     if (n_rows_dev) n_rows = __ldcg(n_rows_dev);
@@ -385,13 +385,29 @@ static __global__ void gg_gather_kernel(const float* __restrict__ x, const float
     const GgRow ri = rows[r];
     const float* src = x + size_t(ri.token) * D;
     __nv_bfloat16* dst = xs + size_t(r) * D;
-    for (int i = threadIdx.x * 4; i < D; i += blockDim.x * 4) {
-        const float4 v = *reinterpret_cast<const float4*>(src + i);
-        const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
-        uint2 o;
-        o.x = *reinterpret_cast<const uint32_t*>(&lo);
-        o.y = *reinterpret_cast<const uint32_t*>(&hi);
-        *reinterpret_cast<uint2*>(dst + i) = o;
+    if (perm8) {
+        // columns 8g .. 8g+7 are stored in the order 0 4 1 5 2 6 3 7: the order in which the 4-bit
+        // kernel unpacks a word of eight weights, so that its operand needs no re-ordering
+        for (int i = threadIdx.x * 8; i < D; i += blockDim.x * 8) {
+            const float4 v0 = *reinterpret_cast<const float4*>(src + i), v1 = *reinterpret_cast<const float4*>(src + i + 4);
+            const __nv_bfloat162 p0 = __floats2bfloat162_rn(v0.x, v1.x), p1 = __floats2bfloat162_rn(v0.y, v1.y);
+            const __nv_bfloat162 p2 = __floats2bfloat162_rn(v0.z, v1.z), p3 = __floats2bfloat162_rn(v0.w, v1.w);
+            uint4 o;
+            o.x = *reinterpret_cast<const uint32_t*>(&p0);
+            o.y = *reinterpret_cast<const uint32_t*>(&p1);
+            o.z = *reinterpret_cast<const uint32_t*>(&p2);
+            o.w = *reinterpret_cast<const uint32_t*>(&p3);
+            *reinterpret_cast<uint4*>(dst + i) = o;
+        }
+    } else {
+        for (int i = threadIdx.x * 4; i < D; i += blockDim.x * 4) {
+            const float4 v = *reinterpret_cast<const float4*>(src + i);
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+            uint2 o;
+            o.x = *reinterpret_cast<const uint32_t*>(&lo);
+            o.y = *reinterpret_cast<const uint32_t*>(&hi);
+            *reinterpret_cast<uint2*>(dst + i) = o;
+        }
     }
     if (threadIdx.x == 0) wrow[r] = w[size_t(ri.token) * K + ri.k];
 }

@@ -1,0 +1,375 @@
+// Batched decode with 4-bit experts: the grouped SwiGLU expert FFN of ffn_grouped.cuh fed from
+// packed 4-bit blobs (groups of 32 weights + one fp16 scale, see ffn_gemv_q4.cuh).
+//
+// The tensor cores take bf16 operands, so a fourth role is added between the TMA producer and the
+// MMA issuer: eight de-quantisation warps (two threads per weight row of the 128-row tile, one per
+// 16 KB operand tile) turn each packed tile into the bf16 tile the MMA expects, written with the
+// 128-byte swizzle a TMA load of bf16 data would have produced, so descriptors, accumulators,
+// epilogues and the work order are those of the bf16 kernel. The conversion stays in packed bf16
+// arithmetic: a nibble q is OR-ed into the mantissa of 128.0 (exact 128 + q), 136 is subtracted
+// (exact q - 8) and the result is multiplied by the group's scale rounded to bf16:
+// weight = bf16_rn(bf16_rn(scale) * (q - 8)), two instructions per pair of weights.
+//
+// Three rings. Packed stages (TMA -> de-quantisation) hold 64 bytes of nibbles per row, i.e. two
+// K-blocks of gate and up rows (phase 1) or one d-tile of the W_down column tile (phase 2), and
+// every second one also the 16 bytes of scales per row that cover it and its successor. Most of
+// the shared memory goes to this ring: a 4-bit tile is a quarter of its bf16 image, so the bytes
+// in flight towards HBM, not the operand stages, decide the streaming rate. Operand stages
+// (de-quantisation -> MMA) hold the two bf16 tiles of one item (one K-block of 64, or one d-tile
+// of 128). Token-row stages (TMA -> MMA) hold the bf16 token rows of one K-block. Every wait is
+// bounded and shares the abort flag of the CTA; no multicast.
+#pragma once
+
+#include "ffn_gemv_q4.cuh"
+#include "ffn_grouped.cuh"
+
+namespace spm {
+
+constexpr int kQgThreads = 448;          // warp 0 TMA, warp 1 MMA + TMEM, warps 2-5 epilogue, warps 6-13 de-quantisation
+constexpr int kQgDequantWarps = 8;
+constexpr int kQgOperandStages = 2;      // 2 x 16 KB bf16 tiles each
+constexpr int kQgPackedStages = 6;
+constexpr int kQgTokenStages = 2;        // 8 KB each
+constexpr uint32_t kQgOperandBytes = 2 * kGgTileBytes;
+constexpr uint32_t kQgHalfBytes = 8192;  // [128 rows][64 B] of nibbles
+constexpr uint32_t kQgNibBytes = 2 * kQgHalfBytes;   // phase 1: gate + up; phase 2: one such tile
+constexpr uint32_t kQgScaleBytes = 2048; // [128 rows][16 B] = 8 fp16 scales per row
+constexpr uint32_t kQgPackedBytes = kQgNibBytes + 2 * kQgScaleBytes;
+
+// 8 nibbles of one word -> 8 bf16 (scale * (q - 8)) as one 16-byte chunk. Nibbles p and p + 4 sit at
+// the same position of the two 16-bit halves, so four packed operations give the pairs (e0,e4)
+// (e1,e5) (e2,e6) (e3,e7), and the chunk is stored in that order: element positions 0..7 of a group of
+// eight hold weights 0 4 1 5 2 6 3 7. Where the group runs along the contraction (first GEMM) the
+// token rows are gathered in the same order; where it runs along the output rows (second GEMM) the
+// epilogue maps the accumulator row back (qg_unpermute).
+__device__ __forceinline__ uint4 dequant_chunk(uint32_t w, __nv_bfloat162 scale2) {
+    const uint32_t off_bits = 0x43084308u;                       // bf16x2 {136, 136}
+    const __nv_bfloat162 off = *reinterpret_cast<const __nv_bfloat162*>(&off_bits);
+    uint32_t r[4];
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+        const uint32_t bits = ((w >> (4 * p)) & 0x000f000fu) | 0x43004300u;     // bf16x2 {128 + q_p, 128 + q_{p+4}}
+        const __nv_bfloat162 v = __hmul2(__hsub2(*reinterpret_cast<const __nv_bfloat162*>(&bits), off), scale2);
+        r[p] = *reinterpret_cast<const uint32_t*>(&v);
+    }
+    return make_uint4(r[0], r[1], r[2], r[3]);
+}
+
+__device__ __forceinline__ int qg_unpermute(int m) { return (m & ~7) | ((m & 7) >> 1) | ((m & 1) << 2); }
+
+__device__ __forceinline__ __nv_bfloat162 scale_at(const uint4& v, int i) {      // i-th fp16 of a 16-byte vector, as bf16x2
+    const uint32_t w = i < 2 ? v.x : i < 4 ? v.y : i < 6 ? v.z : v.w;
+    return __float2bfloat162_rn(__half2float(__ushort_as_half((unsigned short)((i & 1) ? (w >> 16) : (w & 0xffffu)))));
+}
+
+// The super-items (one packed stage each) of a CTA in work order: phase1(0), then for i = 0, 1, ...:
+// phase1(i + 1) if it exists, phase2(i). A phase-1 super-item is two K-blocks, a phase-2 one a d-tile.
+struct QgSeq {
+    int my_units, p1, p2;          // units of this CTA, super-items per phase
+    int u1 = 0, i = 0, idx = 0;    // unit whose phase 1 / phase 2 is being walked, position inside the phase
+    bool phase1 = true, done = false;
+    __device__ QgSeq(int units, int n1, int n2) : my_units(units), p1(n1), p2(n2) { done = units == 0; }
+    __device__ int unit() const { return phase1 ? u1 : i; }
+    __device__ void next() {
+        if (++idx < (phase1 ? p1 : p2)) return;
+        idx = 0;
+        if (phase1) {
+            if (u1 == 0 && my_units > 1) { u1 = 1; return; }     // after phase1(0): phase1(1), then phase2(0)
+            phase1 = false;                                       // after phase1(i + 1): phase2(i)
+        } else {
+            if (++i >= my_units) { done = true; return; }
+            if (i + 1 < my_units) { u1 = i + 1; phase1 = true; }
+        }
+    }
+};
+
+__global__ void __launch_bounds__(kQgThreads, 1)
+ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_constant__ CUtensorMap sc16,
+                      const __grid_constant__ CUtensorMap xmap, const GgArgs a) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    unsigned char* mst = smem;                                               // operand stages
+    unsigned char* act = mst + kQgOperandStages * kQgOperandBytes;           // A^T, 16 KB
+    unsigned char* xst = act + kGgActBytes;                                  // token-row stages
+    unsigned char* qst = xst + kQgTokenStages * kGgXBytes;                   // packed stages
+    uint64_t* bars = reinterpret_cast<uint64_t*>(qst + kQgPackedStages * kQgPackedBytes);
+    uint64_t* qfull = bars;                          // [packed]   TMA -> de-quantisation
+    uint64_t* qempty = qfull + kQgPackedStages;      // [packed]   de-quantisation -> TMA
+    uint64_t* xfull = qempty + kQgPackedStages;      // [token]    TMA -> MMA
+    uint64_t* xempty = xfull + kQgTokenStages;       // [token]    MMA -> TMA
+    uint64_t* mfull = xempty + kQgTokenStages;       // [operand]  de-quantisation -> MMA
+    uint64_t* mempty = mfull + kQgOperandStages;     // [operand]  MMA -> de-quantisation
+    uint64_t* acc1_full = mempty + kQgOperandStages; // [2]
+    uint64_t* acc1_empty = acc1_full + 2;            // [2]
+    uint64_t* act_full = acc1_empty + 2;
+    uint64_t* act_empty = act_full + 1;
+    uint64_t* acc2_full = act_empty + 1;             // [2]
+    uint64_t* acc2_empty = acc2_full + 2;            // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc2_empty + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    float* wrow_all = reinterpret_cast<float*>(tmem_slot + 4);               // [4 epilogue warps][64]
+
+    grid_dep_launch();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int D = a.D;
+    const int n_kb = D / kGgKBlock;
+    const int n_dt = D / kGgTileRows;
+    GgAbort ab{abort_flag, a.status};
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kQgPackedStages; ++s) { mbar_init(smem_u32(qfull + s), 1); mbar_init(smem_u32(qempty + s), kQgDequantWarps); }
+        for (int s = 0; s < kQgTokenStages; ++s) { mbar_init(smem_u32(xfull + s), 1); mbar_init(smem_u32(xempty + s), 1); }
+        for (int s = 0; s < kQgOperandStages; ++s) { mbar_init(smem_u32(mfull + s), kQgDequantWarps); mbar_init(smem_u32(mempty + s), 1); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(acc1_full + b), 1);
+            mbar_init(smem_u32(acc1_empty + b), 4);
+            mbar_init(smem_u32(acc2_full + b), 1);
+            mbar_init(smem_u32(acc2_empty + b), 4);
+        }
+        mbar_init(smem_u32(act_full), 4);
+        mbar_init(smem_u32(act_empty), 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kGgTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    grid_dep_wait();
+    const int n_units = a.n_units_dev ? __ldcg(a.n_units_dev) : a.n_units;
+    const int my_units = int(blockIdx.x) < n_units ? (n_units - 1 - int(blockIdx.x)) / int(gridDim.x) + 1 : 0;
+    const int sc_x0 = D / 2;                         // byte offset of the scales inside a packed row
+    const int p1_supers = n_kb / 2, p2_supers = n_dt;
+
+    if (warp == 0) {
+        // ---------------- TMA producer: packed stages one super-item ahead of the token rows ----------------
+        if (lane == 0) {
+            uint32_t np = 0, nx = 0;      // packed stages / token-row stages issued so far
+            bool ok = true;
+            auto load_packed = [&](const QgSeq& q) {
+                const GgUnit un = a.units[blockIdx.x + q.unit() * gridDim.x];
+                const uint32_t ps = np % kQgPackedStages;
+                if (np >= uint32_t(kQgPackedStages)) ok = gg_wait(smem_u32(qempty + ps), ((np / kQgPackedStages) - 1) & 1, ab);
+                if (!ok) return;
+                const uint32_t qb = smem_u32(qst + ps * kQgPackedBytes), fq = smem_u32(qfull + ps);
+                const int r0 = un.jt * kGgTileRows;
+                const bool with_scales = (q.idx & 1) == 0;        // 16 bytes of scales cover two super-items
+                if (q.phase1) {
+                    mbar_arrive_expect_tx(fq, 2 * kQgHalfBytes + (with_scales ? 2 * kQgScaleBytes : 0));
+                    tma_load_4d(qb, &nib64, q.idx * 64, 0, r0, un.slot, fq);
+                    tma_load_4d(qb + kQgHalfBytes, &nib64, q.idx * 64, 1, r0, un.slot, fq);
+                    if (with_scales) {
+                        tma_load_4d(qb + kQgNibBytes, &sc16, sc_x0 + (q.idx >> 1) * 16, 0, r0, un.slot, fq);
+                        tma_load_4d(qb + kQgNibBytes + kQgScaleBytes, &sc16, sc_x0 + (q.idx >> 1) * 16, 1, r0, un.slot, fq);
+                    }
+                } else {
+                    mbar_arrive_expect_tx(fq, kQgHalfBytes + (with_scales ? kQgScaleBytes : 0));
+                    tma_load_4d(qb, &nib64, q.idx * 64, 2, r0, un.slot, fq);
+                    if (with_scales) tma_load_4d(qb + kQgNibBytes, &sc16, sc_x0 + (q.idx >> 1) * 16, 2, r0, un.slot, fq);
+                }
+                ++np;
+            };
+            auto load_tokens = [&](const QgSeq& q) {      // the two K-blocks of a phase-1 super-item
+                if (!q.phase1) return;
+                const GgUnit un = a.units[blockIdx.x + q.unit() * gridDim.x];
+                for (int j = 0; j < 2 && ok; ++j, ++nx) {
+                    const uint32_t xs = nx % kQgTokenStages;
+                    if (nx >= uint32_t(kQgTokenStages)) ok = gg_wait(smem_u32(xempty + xs), ((nx / kQgTokenStages) - 1) & 1, ab);
+                    if (!ok) return;
+                    const uint32_t fx = smem_u32(xfull + xs);
+                    mbar_arrive_expect_tx(fx, kGgXBytes);
+                    tma_load_2d(smem_u32(xst + xs * kGgXBytes), &xmap, (q.idx * 2 + j) * kGgKBlock, un.row0, fx);
+                }
+            };
+            QgSeq cur(my_units, p1_supers, p2_supers);
+            if (!cur.done) load_packed(cur);
+            while (!cur.done && ok) {
+                QgSeq nxt = cur;
+                nxt.next();
+                if (!nxt.done) load_packed(nxt);
+                if (ok) load_tokens(cur);
+                cur = nxt;
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (as in the bf16 kernel; operands and token rows on separate rings) ----------------
+        if (lane == 0) {
+            constexpr uint32_t idesc1 = gg_idesc(false, false);
+            constexpr uint32_t idesc2 = gg_idesc(true, true);
+            uint32_t t = 0, nx = 0, nd = 0;     // operand items, token-row stages, d-tiles consumed so far
+            bool ok = true;
+            auto mma_phase1 = [&](int i) {
+                const uint32_t b = i & 1, m = uint32_t(i) >> 1;
+                if (i >= 2) ok = gg_wait(smem_u32(acc1_empty + b), (m - 1) & 1, ab);
+                const uint32_t acc = tmem + 128 * b;
+                for (int kb = 0; kb < n_kb && ok; ++kb, ++t, ++nx) {
+                    const uint32_t s = t % kQgOperandStages, xs = nx % kQgTokenStages;
+                    ok = gg_wait(smem_u32(mfull + s), (t / kQgOperandStages) & 1, ab);
+                    if (ok) ok = gg_wait(smem_u32(xfull + xs), (nx / kQgTokenStages) & 1, ab);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t base = smem_u32(mst + s * kQgOperandBytes), xb = smem_u32(xst + xs * kGgXBytes);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint64_t bx = smem_desc_sw128(xb + ks * 32, 16, 1024);
+                        tc_mma_bf16(acc, smem_desc_sw128(base + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
+                        tc_mma_bf16(acc + 64, smem_desc_sw128(base + kGgTileBytes + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
+                    }
+                    tc_commit(smem_u32(mempty + s));
+                    tc_commit(smem_u32(xempty + xs));
+                }
+                if (ok) tc_commit(smem_u32(acc1_full + b));
+            };
+            auto mma_phase2 = [&](int i) {
+                ok = gg_wait(smem_u32(act_full), i & 1, ab);
+                if (!ok) return;
+                tc_fence_after();
+                const uint32_t act_addr = smem_u32(act);
+                for (int dt = 0; dt < n_dt && ok; ++dt, ++t, ++nd) {
+                    const uint32_t s = t % kQgOperandStages, b = nd & 1;
+                    ok = gg_wait(smem_u32(mfull + s), (t / kQgOperandStages) & 1, ab);
+                    if (ok && nd >= 2) ok = gg_wait(smem_u32(acc2_empty + b), ((nd >> 1) - 1) & 1, ab);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t base = smem_u32(mst + s * kQgOperandBytes);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint64_t da = smem_desc_sw128(base + ks * 2048, kGgTileBytes, 1024);
+                        const uint64_t db = smem_desc_sw128(act_addr + ks * 2048, kGgActBytes, 1024);
+                        tc_mma_bf16(tmem + 256 + 64 * b, da, db, idesc2, ks != 0);
+                    }
+                    tc_commit(smem_u32(mempty + s));
+                    tc_commit(smem_u32(acc2_full + b));
+                }
+                if (ok) tc_commit(smem_u32(act_empty));
+            };
+            if (my_units > 0) mma_phase1(0);
+            for (int i = 0; i < my_units && ok; ++i) {
+                if (i + 1 < my_units) mma_phase1(i + 1);
+                if (ok) mma_phase2(i);
+            }
+        }
+    } else if (warp >= 6) {
+        // ---------------- de-quantisation warps: two threads per weight row, one per operand tile ----------------
+        const int dq = warp - 6;
+        const int r = (dq & 3) * 32 + lane;          // row of the 128-row tile
+        const int tile = dq >> 2;                    // phase 1: 0 = gate, 1 = up; phase 2: 0 = d 0..63, 1 = d 64..127 of the d-tile
+        const uint32_t sw = uint32_t(r & 7);         // 128-byte swizzle of the bf16 operand rows
+        const uint32_t sq = uint32_t((r >> 1) & 3);  // 64-byte swizzle of the packed rows
+        uint32_t t = 0, np = 0;                      // operand items written, packed stages consumed
+        bool ok = true;
+        uint4 sc = make_uint4(0, 0, 0, 0);           // this row's 8 scales for the current pair of super-items
+        for (QgSeq q(my_units, p1_supers, p2_supers); !q.done && ok; q.next(), ++np) {
+            const uint32_t ps = np % kQgPackedStages;
+            ok = __all_sync(0xffffffffu, gg_wait(smem_u32(qfull + ps), (np / kQgPackedStages) & 1, ab));
+            if (!ok) break;
+            const unsigned char* qb = qst + ps * kQgPackedBytes;
+            const unsigned char* nrow = qb + (q.phase1 ? tile * kQgHalfBytes : 0) + r * 64;    // this row's 64 bytes of nibbles
+            if ((q.idx & 1) == 0)
+                sc = *reinterpret_cast<const uint4*>(qb + kQgNibBytes + (q.phase1 ? tile * kQgScaleBytes : 0) + r * 16);
+            const int items = q.phase1 ? 2 : 1;
+            for (int j = 0; j < items && ok; ++j, ++t) {
+                // phase 1: K-block j of the super-item = packed chunks 2j, 2j+1 of the row;
+                // phase 2: the d-tile, this thread's half = packed chunks 2*tile, 2*tile+1.
+                // A packed chunk (16 bytes, 32 weights) has one scale: number 4 * (idx & 1) + chunk of `sc`.
+                const int c0 = q.phase1 ? 2 * j : 2 * tile;
+                const uint4 n0 = *reinterpret_cast<const uint4*>(nrow + ((uint32_t(c0) ^ sq) << 4));
+                const uint4 n1 = *reinterpret_cast<const uint4*>(nrow + ((uint32_t(c0 + 1) ^ sq) << 4));
+                const int g = 4 * (q.idx & 1) + c0;
+                const __nv_bfloat162 s0 = scale_at(sc, g), s1 = scale_at(sc, g + 1);
+                const uint32_t ms = t % kQgOperandStages;
+                if (t >= uint32_t(kQgOperandStages))
+                    ok = __all_sync(0xffffffffu, gg_wait(smem_u32(mempty + ms), ((t / kQgOperandStages) - 1) & 1, ab));
+                if (!ok) break;
+                unsigned char* row = mst + ms * kQgOperandBytes + tile * kGgTileBytes + r * 128;
+                const uint32_t w0[4] = {n0.x, n0.y, n0.z, n0.w}, w1[4] = {n1.x, n1.y, n1.z, n1.w};
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    *reinterpret_cast<uint4*>(row + ((uint32_t(c) ^ sw) << 4)) = dequant_chunk(w0[c], s0);
+                    *reinterpret_cast<uint4*>(row + ((uint32_t(c + 4) ^ sw) << 4)) = dequant_chunk(w1[c], s1);
+                }
+                fence_proxy_async();          // generic-proxy writes -> visible to the MMA's async reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(mfull + ms));
+            }
+            if (!ok) break;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(qempty + ps));
+        }
+    } else {
+        // ---------------- epilogue warps (as in the bf16 kernel) ----------------
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const uint32_t lane_addr = uint32_t(q * 32) << 16;
+        float* wrow_s = wrow_all + q * kGgTokens;
+        uint32_t nd = 0;
+        bool ok = true;
+        for (int i = 0; i < my_units && ok; ++i) {
+            const GgUnit un = a.units[blockIdx.x + i * gridDim.x];
+            const uint32_t b1 = i & 1;
+            __syncwarp();
+#pragma unroll
+            for (int tk = lane; tk < kGgTokens; tk += 32) wrow_s[tk] = tk < un.ntok ? a.wrow[un.row0 + tk] : 0.f;
+            __syncwarp();
+            ok = gg_wait(smem_u32(acc1_full + b1), (uint32_t(i) >> 1) & 1, ab);
+            if (ok && i > 0) ok = gg_wait(smem_u32(act_empty), (i - 1) & 1, ab);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < kGgTokens / 16; ++c) {
+                float g[16], up[16];
+                tmem_ld16(tmem + lane_addr + 128 * b1 + c * 16, g);
+                tmem_ld16(tmem + lane_addr + 128 * b1 + 64 + c * 16, up);
+                uint32_t packed[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float a0 = g[2 * e] / (1.f + expf(-g[2 * e])) * up[2 * e] * wrow_s[c * 16 + 2 * e];
+                    const float a1 = g[2 * e + 1] / (1.f + expf(-g[2 * e + 1])) * up[2 * e + 1] * wrow_s[c * 16 + 2 * e + 1];
+                    const __nv_bfloat162 p = __floats2bfloat162_rn(a0, a1);
+                    packed[e] = *reinterpret_cast<const uint32_t*>(&p);
+                }
+                unsigned char* rowp = act + row * 128;
+                *reinterpret_cast<uint4*>(rowp + (((2 * c) ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                *reinterpret_cast<uint4*>(rowp + (((2 * c + 1) ^ (row & 7)) << 4)) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) { mbar_arrive(smem_u32(acc1_empty + b1)); mbar_arrive(smem_u32(act_full)); }
+
+            float* prow = a.partial + (size_t(un.jt) * a.rows_cap + un.row0) * D;
+            for (int dt = 0; dt < n_dt && ok; ++dt, ++nd) {
+                const uint32_t b = nd & 1;
+                ok = __all_sync(0xffffffffu, gg_wait(smem_u32(acc2_full + b), (nd >> 1) & 1, ab));
+                if (!ok) break;
+                tc_fence_after();
+                const int d = dt * kGgTileRows + qg_unpermute(row);       // accumulator row -> output column
+                for (int c = 0; c * 16 < un.ntok; ++c) {
+                    float y[16];
+                    tmem_ld16(tmem + lane_addr + 256 + 64 * b + c * 16, y);
+#pragma unroll
+                    for (int e = 0; e < 16; ++e)
+                        if (c * 16 + e < un.ntok) prow[size_t(c * 16 + e) * D + d] = y[e];
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(acc2_empty + b));
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, kGgTmemCols);
+}
+
+inline size_t ffn_grouped_q4_smem() {
+    return 1024 + size_t(kQgOperandStages) * kQgOperandBytes + kGgActBytes + size_t(kQgTokenStages) * kGgXBytes +
+           size_t(kQgPackedStages) * kQgPackedBytes + 512 + 4 * kGgTokens * sizeof(float) + 64;
+}
+static_assert(1024 + kQgOperandStages * kQgOperandBytes + kGgActBytes + kQgTokenStages * kGgXBytes +
+              kQgPackedStages * kQgPackedBytes + 512 + 4 * kGgTokens * 4 + 64 <= 232448, "shared memory of the 4-bit grouped kernel");
+
+}  // namespace spm

@@ -19,6 +19,7 @@
 #include "ffn_gemv.cuh"
 #include "ffn_gemv_q4.cuh"
 #include "ffn_grouped.cuh"
+#include "ffn_grouped_q4.cuh"
 #include "router_adapter.cuh"
 #include "tma_maps.h"
 #include "slot_table.h"
@@ -66,6 +67,7 @@ struct spm_ctx {
     int batched_path = 0;                 // 0: tensor cores when possible, 1: always the per-token GEMV
     int rows_cap = 0, n_jt = 0, max_units = 0;
     CUtensorMap wmap{}, xmap{};
+    CUtensorMap qmapn{}, qmapsc{};            // 4-bit blobs: nibble box of 128 bytes, scale box of 16 bytes
     __nv_bfloat16* tc_xs = nullptr;
     float *tc_wrow = nullptr, *tc_partial = nullptr;
     unsigned char* tc_desc_dev = nullptr;     // kDescRing wave descriptors
@@ -195,11 +197,13 @@ constexpr int kClockSlots = 12288;    // in-kernel {start, end} pairs between tw
 constexpr int kDescRing = 8;          // wave descriptors in flight for the batched tensor-core path
 constexpr int kTraceRing = 8;         // host-free steps whose bookkeeping may be outstanding
 
-// The grouped tcgen05 kernel handles bf16 weights, more than one sequence per step, no shared
-// experts, and intermediate / hidden sizes that tile by 128.
+// The grouped tcgen05 kernels handle bf16 or 4-bit weights, more than one sequence per step, no
+// shared experts, and intermediate / hidden sizes that tile by 128.
 bool tc_supported(const spm_model_cfg* m) {
-    return m->dtype == SPM_DTYPE_BF16 && m->max_batch > 1 && m->n_shared == 0 && m->inter % kGgTileRows == 0 &&
-           m->hidden % kGgTileRows == 0;
+    // the 4-bit kernel takes the scales of 256 columns (16 bytes per row) at a time
+    const int col_step = m->dtype == SPM_DTYPE_Q4 ? 2 * kGgTileRows : kGgTileRows;
+    return (m->dtype == SPM_DTYPE_BF16 || m->dtype == SPM_DTYPE_Q4) && m->max_batch > 1 && m->n_shared == 0 &&
+           m->inter % kGgTileRows == 0 && m->hidden % col_step == 0;
 }
 static_assert(kMaxCtasBatch1 <= kReduceGroups * kReduceMaxRows, "reduce kernel covers every grid size");
 static_assert(kReduceGroups == kReduceGroupsR && kReduceGroupsR == kRouterWarps, "the routing kernel folds partial rows in the combine kernel's order");
@@ -649,12 +653,16 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
     CU(c, cudaEventRecord(c->tc_desc_ev[d], c->compute));
     c->tc_desc_ev_valid[d] = 1;
     gg_gather_kernel<<<n_rows, 128, 0, c->compute>>>(x_norm, w, reinterpret_cast<const GgRow*>(dd + c->tc_off_rows), n_rows,
-                                                     nullptr, m.hidden, K, c->tc_xs, c->tc_wrow);
+                                                     nullptr, m.hidden, K, c->tc_xs, c->tc_wrow, m.dtype == SPM_DTYPE_Q4 ? 1 : 0);
     CU(c, cudaGetLastError());
     if (t && first) CU(c, cudaEventRecord(t->ffn_start[layer], c->compute));
     if (ring >= 0 && first) CU(c, cudaEventRecord(c->ring_start[ring], c->compute));
     GgArgs a{reinterpret_cast<const GgUnit*>(dd), n_units, nullptr, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status};
-    ffn_grouped_kernel<<<std::min(c->num_sms, n_units), kGgThreads, ffn_grouped_smem(), c->compute>>>(c->wmap, c->xmap, a);
+    if (m.dtype == SPM_DTYPE_Q4)
+        ffn_grouped_q4_kernel<<<std::min(c->num_sms, n_units), kQgThreads, ffn_grouped_q4_smem(), c->compute>>>(
+            c->qmapn, c->qmapsc, c->xmap, a);
+    else
+        ffn_grouped_kernel<<<std::min(c->num_sms, n_units), kGgThreads, ffn_grouped_smem(), c->compute>>>(c->wmap, c->xmap, a);
     CU(c, cudaGetLastError());
     if (t && last) CU(c, cudaEventRecord(t->ffn_end[layer], c->compute));
     if (ring >= 0 && last) { CU(c, cudaEventRecord(c->ring_end[ring], c->compute)); c->ring_used[ring] = 1; }
@@ -1038,9 +1046,14 @@ int enqueue_host_free_layers(spm_ctx* c, int nb, float* h_out, int slot, bool pr
                            (const int32_t*)c->ws_ids, (const short*)(c->ws_slot_map + size_t(l) * n), l * c->S, nb, K, n, c->n_jt,
                            units, rows, rowmap, c->tc_counts, c->ws_status));
             CU(c, launch_k(gg_gather_kernel, dim3(nb * K), dim3(128), 0, c->compute, true, (const float*)c->ws_x, (const float*)c->ws_w,
-                           (const GgRow*)rows, 0, (const int*)(c->tc_counts + 1), m.hidden, K, c->tc_xs, c->tc_wrow));
+                           (const GgRow*)rows, 0, (const int*)(c->tc_counts + 1), m.hidden, K, c->tc_xs, c->tc_wrow,
+                           m.dtype == SPM_DTYPE_Q4 ? 1 : 0));
             GgArgs ga{units, 0, c->tc_counts, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status};
-            CU(c, launch_k(ffn_grouped_kernel, dim3(c->num_sms), dim3(kGgThreads), ffn_grouped_smem(), c->compute, true, c->wmap, c->xmap, ga));
+            if (m.dtype == SPM_DTYPE_Q4)
+                CU(c, launch_k(ffn_grouped_q4_kernel, dim3(c->num_sms), dim3(kQgThreads), ffn_grouped_q4_smem(), c->compute, true,
+                               c->qmapn, c->qmapsc, c->xmap, ga));
+            else
+                CU(c, launch_k(ffn_grouped_kernel, dim3(c->num_sms), dim3(kGgThreads), ffn_grouped_smem(), c->compute, true, c->wmap, c->xmap, ga));
             CU(c, launch_k(gg_combine_kernel, dim3((m.hidden / 4 + 127) / 128, nb), dim3(128), 0, c->compute, true,
                            (const float*)c->tc_partial, (const int32_t*)rowmap, K, c->n_jt, c->rows_cap, m.hidden, h_out));
             c->kernel_launches += 5;
@@ -1281,12 +1294,15 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
         c->tc_desc_ev.resize(kDescRing);
         c->tc_desc_ev_valid.assign(kDescRing, 0);
         for (auto& ev : c->tc_desc_ev) if (!cu(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming), "cudaEventCreate")) return bail(SPM_ERR_CUDA);
-        if (!make_weight_map(&c->wmap, c->pools, cfg->hidden, cfg->inter, uint64_t(L) * c->S) ||
-            !make_token_map(&c->xmap, c->tc_xs, cfg->hidden, uint64_t(lay.rows_cap + kGgTokens))) {
+        const bool maps_ok = cfg->dtype == SPM_DTYPE_Q4
+            ? make_q4_maps(&c->qmapn, &c->qmapsc, c->pools, cfg->hidden, cfg->inter, uint64_t(L) * c->S)
+            : make_weight_map(&c->wmap, c->pools, cfg->hidden, cfg->inter, uint64_t(L) * c->S);
+        if (!maps_ok || !make_token_map(&c->xmap, c->tc_xs, cfg->hidden, uint64_t(lay.rows_cap + kGgTokens))) {
             c->err = "cuTensorMapEncodeTiled failed";
             return bail(SPM_ERR_CUDA);
         }
         if (!cu(cudaFuncSetAttribute(ffn_grouped_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(ffn_grouped_smem())), "cudaFuncSetAttribute")) return bail(SPM_ERR_CUDA);
+        if (!cu(cudaFuncSetAttribute(ffn_grouped_q4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(ffn_grouped_q4_smem())), "cudaFuncSetAttribute")) return bail(SPM_ERR_CUDA);
         if (gg_plan_smem(cfg->n_experts) > 48 * 1024 &&
             !cu(cudaFuncSetAttribute(gg_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(gg_plan_smem(cfg->n_experts))), "cudaFuncSetAttribute")) return bail(SPM_ERR_CUDA);
         c->tc_ok = true;

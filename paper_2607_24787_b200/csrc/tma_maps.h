@@ -68,4 +68,23 @@ inline bool make_token_map(CUtensorMap* map, const void* base, int D, uint64_t r
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Packed 4-bit expert blobs [n_slots][I][3][RB bytes] (RB = D/2 nibble bytes + D/16 scale bytes per
+// row) viewed as a 4-D byte tensor (RB, 3, I, n_slots). Two box shapes over the same memory:
+// 64 nibble bytes (128 weights) x 128 rows with the 64-byte swizzle, and 16 scale bytes x 128 rows.
+inline bool make_q4_maps(CUtensorMap* nib64, CUtensorMap* sc16, const void* base, int D, int I, uint64_t n_slots) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t rb = cuuint64_t(D) / 2 + cuuint64_t(D) / 16;
+    const cuuint64_t dims[4] = {rb, 3, cuuint64_t(I), n_slots};
+    const cuuint64_t strides[3] = {rb, rb * 3, rb * 3 * cuuint64_t(I)};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const cuuint32_t box_n[4] = {64, 1, 128, 1}, box_s[4] = {16, 1, 128, 1};
+    return fn(nib64, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box_n, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS &&
+           fn(sc16, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box_s, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace spm

@@ -95,6 +95,8 @@ CONFIGS = {
     "sweep": ModelCfg("sweep", 48, 2048, 128, 768, 8, 0, 16, "bf16", 16, 1, 1, 512, 151936, 3),
     # batched decode on the Qwen3 shape
     "batched": ModelCfg("batched", 48, 2048, 128, 768, 8, 0, 16, "bf16", 32, -1, 64, 128, 151936, 4),
+    # ... and with 4-bit experts
+    "batched_q4": ModelCfg("batched_q4", 48, 2048, 128, 768, 8, 0, 16, "q4", 32, -1, 64, 128, 151936, 4),
 }
 
 

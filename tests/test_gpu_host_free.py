@@ -151,6 +151,7 @@ TC_CASES = {
     "wide": synth.get_config("qwen3", n_layers=2, hidden=1280, n_experts=16, inter=384, top_k=3, slots=16, budget=2, batch=64),
     "many_tokens": synth.get_config("qwen3", n_layers=3, hidden=512, n_experts=8, inter=128, top_k=2, slots=8, budget=1, batch=64),
     "ragged_batch": synth.get_config("qwen3", n_layers=2, hidden=256, n_experts=24, inter=256, top_k=4, slots=24, budget=2, batch=17),
+    "q4_wide": synth.get_config("qwen3_q4", n_layers=2, hidden=1280, n_experts=16, inter=384, top_k=3, slots=16, budget=2, batch=64),
 }
 
 
