@@ -125,6 +125,14 @@ __host__ __device__ constexpr uint32_t gg_idesc(bool a_mn_major, bool b_mn_major
            (uint32_t(kGgTokens >> 3) << 17) | (uint32_t(kGgTileRows >> 4) << 24);
 }
 
+// The same with N given at run time (a multiple of 16, at most kGgTokens): a unit with few tokens
+// asks the tensor core for only that many columns.
+__device__ __forceinline__ uint32_t gg_idesc_n(bool a_mn_major, bool b_mn_major, uint32_t n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(a_mn_major) << 15) | (uint32_t(b_mn_major) << 16) |
+           ((n >> 3) << 17) | (uint32_t(kGgTileRows >> 4) << 24);
+}
+__device__ __forceinline__ uint32_t gg_pad_tokens(int ntok) { return uint32_t(max(16, (ntok + 15) & ~15)); }
+
 struct GgAbort {
     volatile int* flag;     // shared: set by the first wait that gives up
     int* status;
@@ -203,34 +211,43 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
     // keeps flowing while the epilogue warps turn G^T, U^T of the current unit into A^T.
     if (warp == 0) {
         // ---------------- TMA producer ----------------
-        if (lane == 0) {
+        // The producer and the MMA issuer are walked by their whole warp in uniform control flow and
+        // one elected lane issues: addresses and descriptors then stay in uniform registers (issued
+        // from inside a one-lane branch, each tcgen05.mma cost the issuing thread about 90 cycles).
+        {
             uint32_t it = 0;      // ring position over all stages
             bool ok = true;
             auto load_phase1 = [&](int i) {
                 const GgUnit un = a.units[blockIdx.x + i * gridDim.x];
                 for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
                     const uint32_t s = it % kGgStages;
-                    if (it >= kGgStages) ok = gg_wait(smem_u32(empty + s), ((it / kGgStages) - 1) & 1, ab);
+                    if (it >= kGgStages) ok = __all_sync(0xffffffffu, gg_wait(smem_u32(empty + s), ((it / kGgStages) - 1) & 1, ab));
                     if (!ok) break;
                     const uint32_t base = smem_u32(stages + s * kGgStageBytes);
                     const uint32_t fb = smem_u32(full + s);
-                    mbar_arrive_expect_tx(fb, kGgStageBytes);
-                    tma_load_4d(base, &wmap, kb * kGgKBlock, 0, un.jt * kGgTileRows, un.slot, fb);                 // gate rows
-                    tma_load_4d(base + kGgTileBytes, &wmap, kb * kGgKBlock, 1, un.jt * kGgTileRows, un.slot, fb);  // up rows
-                    tma_load_2d(base + 2 * kGgTileBytes, &xmap, kb * kGgKBlock, un.row0, fb);                      // token rows
+                    if (elect_one()) {
+                        mbar_arrive_expect_tx(fb, kGgStageBytes);
+                        tma_load_4d(base, &wmap, kb * kGgKBlock, 0, un.jt * kGgTileRows, un.slot, fb);                 // gate rows
+                        tma_load_4d(base + kGgTileBytes, &wmap, kb * kGgKBlock, 1, un.jt * kGgTileRows, un.slot, fb);  // up rows
+                        tma_load_2d(base + 2 * kGgTileBytes, &xmap, kb * kGgKBlock, un.row0, fb);                      // token rows
+                    }
+                    __syncwarp();
                 }
             };
             auto load_phase2 = [&](int i) {
                 const GgUnit un = a.units[blockIdx.x + i * gridDim.x];
                 for (int dt = 0; dt < n_dt && ok; ++dt, ++it) {
                     const uint32_t s = it % kGgStages;
-                    if (it >= kGgStages) ok = gg_wait(smem_u32(empty + s), ((it / kGgStages) - 1) & 1, ab);
+                    if (it >= kGgStages) ok = __all_sync(0xffffffffu, gg_wait(smem_u32(empty + s), ((it / kGgStages) - 1) & 1, ab));
                     if (!ok) break;
                     const uint32_t base = smem_u32(stages + s * kGgStageBytes);
                     const uint32_t fb = smem_u32(full + s);
-                    mbar_arrive_expect_tx(fb, 2 * kGgTileBytes);
-                    tma_load_4d(base, &wmap, dt * kGgTileRows, 2, un.jt * kGgTileRows, un.slot, fb);                      // d 0..63
-                    tma_load_4d(base + kGgTileBytes, &wmap, dt * kGgTileRows + 64, 2, un.jt * kGgTileRows, un.slot, fb); // d 64..127
+                    if (elect_one()) {
+                        mbar_arrive_expect_tx(fb, 2 * kGgTileBytes);
+                        tma_load_4d(base, &wmap, dt * kGgTileRows, 2, un.jt * kGgTileRows, un.slot, fb);                      // d 0..63
+                        tma_load_4d(base + kGgTileBytes, &wmap, dt * kGgTileRows + 64, 2, un.jt * kGgTileRows, un.slot, fb); // d 64..127
+                    }
+                    __syncwarp();
                 }
             };
             if (my_units > 0) load_phase1(0);
@@ -241,53 +258,64 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            constexpr uint32_t idesc1 = gg_idesc(false, false);   // weights K-major, tokens K-major
-            constexpr uint32_t idesc2 = gg_idesc(true, true);     // W_down column tile M-major, A^T N-major
+        {
             uint32_t it = 0, nd = 0;     // stage counter, d-tile counter
             bool ok = true;
+            auto wait_all = [&](uint64_t* bar, uint32_t parity) { ok = __all_sync(0xffffffffu, ok && gg_wait(smem_u32(bar), parity, ab)); };
             auto mma_phase1 = [&](int i) {
                 const uint32_t b = i & 1, m = uint32_t(i) >> 1;
-                if (i >= 2) ok = gg_wait(smem_u32(acc1_empty + b), (m - 1) & 1, ab);   // pair drained two units ago
+                // weights K-major, tokens K-major; N = the unit's tokens rounded up to 16
+                const uint32_t idesc1 = gg_idesc_n(false, false, gg_pad_tokens(a.units[blockIdx.x + i * gridDim.x].ntok));
+                if (i >= 2) wait_all(acc1_empty + b, (m - 1) & 1);   // pair drained two units ago
                 const uint32_t acc = tmem + 128 * b;
                 for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
                     const uint32_t s = it % kGgStages;
-                    ok = gg_wait(smem_u32(full + s), (it / kGgStages) & 1, ab);
+                    wait_all(full + s, (it / kGgStages) & 1);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t base = smem_u32(stages + s * kGgStageBytes);
+                    if (elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {      // 4 x (K = 16) inside the 64-wide block
-                        const uint64_t bx = smem_desc_sw128(base + 2 * kGgTileBytes + ks * 32, 16, 1024);
-                        tc_mma_bf16(acc, smem_desc_sw128(base + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
-                        tc_mma_bf16(acc + 64, smem_desc_sw128(base + kGgTileBytes + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
+                        for (int ks = 0; ks < 4; ++ks) {      // 4 x (K = 16) inside the 64-wide block
+                            const uint64_t bx = smem_desc_sw128(base + 2 * kGgTileBytes + ks * 32, 16, 1024);
+                            tc_mma_bf16(acc, smem_desc_sw128(base + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
+                            tc_mma_bf16(acc + 64, smem_desc_sw128(base + kGgTileBytes + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
+                        }
+                        tc_commit(smem_u32(empty + s));
                     }
-                    tc_commit(smem_u32(empty + s));
+                    __syncwarp();
                 }
-                if (ok) tc_commit(smem_u32(acc1_full + b));
+                if (ok && elect_one()) tc_commit(smem_u32(acc1_full + b));
+                __syncwarp();
             };
             auto mma_phase2 = [&](int i) {
-                ok = gg_wait(smem_u32(act_full), i & 1, ab);
+                // W_down column tile M-major, A^T N-major
+                const uint32_t idesc2 = gg_idesc_n(true, true, gg_pad_tokens(a.units[blockIdx.x + i * gridDim.x].ntok));
+                wait_all(act_full, i & 1);
                 if (!ok) return;
                 tc_fence_after();
                 const uint32_t act_addr = smem_u32(act);
                 for (int dt = 0; dt < n_dt && ok; ++dt, ++it, ++nd) {
                     const uint32_t s = it % kGgStages, b = nd & 1;
-                    ok = gg_wait(smem_u32(full + s), (it / kGgStages) & 1, ab);
-                    if (ok && nd >= 2) ok = gg_wait(smem_u32(acc2_empty + b), ((nd >> 1) - 1) & 1, ab);
+                    wait_all(full + s, (it / kGgStages) & 1);
+                    if (nd >= 2) wait_all(acc2_empty + b, ((nd >> 1) - 1) & 1);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t base = smem_u32(stages + s * kGgStageBytes);
+                    if (elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {      // K = 16 rows j per step, 2048 bytes of each operand
-                        const uint64_t da = smem_desc_sw128(base + ks * 2048, kGgTileBytes, 1024);
-                        const uint64_t db = smem_desc_sw128(act_addr + ks * 2048, kGgActBytes, 1024);
-                        tc_mma_bf16(tmem + 256 + 64 * b, da, db, idesc2, ks != 0);
+                        for (int ks = 0; ks < 8; ++ks) {      // K = 16 rows j per step, 2048 bytes of each operand
+                            const uint64_t da = smem_desc_sw128(base + ks * 2048, kGgTileBytes, 1024);
+                            const uint64_t db = smem_desc_sw128(act_addr + ks * 2048, kGgActBytes, 1024);
+                            tc_mma_bf16(tmem + 256 + 64 * b, da, db, idesc2, ks != 0);
+                        }
+                        tc_commit(smem_u32(empty + s));
+                        tc_commit(smem_u32(acc2_full + b));
                     }
-                    tc_commit(smem_u32(empty + s));
-                    tc_commit(smem_u32(acc2_full + b));
+                    __syncwarp();
                 }
-                if (ok) tc_commit(smem_u32(act_empty));
+                if (ok && elect_one()) tc_commit(smem_u32(act_empty));
+                __syncwarp();
             };
             if (my_units > 0) mma_phase1(0);
             for (int i = 0; i < my_units && ok; ++i) {
@@ -318,8 +346,10 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
             if (!ok) break;
             tc_fence_after();
             // A^T[j = row][t] = silu(G) * U * w_t, bf16, 16-byte chunks swizzled by (row % 8)
+            const int n_pad = int(gg_pad_tokens(un.ntok));      // columns the MMAs of this unit wrote
 #pragma unroll
             for (int c = 0; c < kGgTokens / 16; ++c) {
+                if (c * 16 >= n_pad) break;
                 float g[16], up[16];
                 tmem_ld16(tmem + lane_addr + 128 * b1 + c * 16, g);
                 tmem_ld16(tmem + lane_addr + 128 * b1 + 64 + c * 16, up);

@@ -25,10 +25,12 @@
 
 namespace spm {
 
-constexpr int kQgThreads = 448;          // warp 0 TMA, warp 1 MMA + TMEM, warps 2-5 epilogue, warps 6-13 de-quantisation
+constexpr int kQgThreads = 480;          // warp 0 TMA (packed weights), 1 MMA + TMEM, 2-5 epilogue, 6-13 de-quantisation, 14 TMA (token rows)
 constexpr int kQgDequantWarps = 8;
-constexpr int kQgOperandStages = 2;      // 2 x 16 KB bf16 tiles each
-constexpr int kQgPackedStages = 6;
+constexpr int kQgGroups = 4;             // de-quantisation groups of two warps; group g expands the items with t % 4 == g
+constexpr int kQgGroupWarps = kQgDequantWarps / kQgGroups;
+constexpr int kQgOperandStages = 4;      // 2 x 16 KB bf16 tiles each
+constexpr int kQgPackedStages = 3;
 constexpr int kQgTokenStages = 2;        // 8 KB each
 constexpr uint32_t kQgOperandBytes = 2 * kGgTileBytes;
 constexpr uint32_t kQgHalfBytes = 8192;  // [128 rows][64 B] of nibbles
@@ -119,7 +121,7 @@ ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_co
     if (threadIdx.x == 0) {
         for (int s = 0; s < kQgPackedStages; ++s) { mbar_init(smem_u32(qfull + s), 1); mbar_init(smem_u32(qempty + s), kQgDequantWarps); }
         for (int s = 0; s < kQgTokenStages; ++s) { mbar_init(smem_u32(xfull + s), 1); mbar_init(smem_u32(xempty + s), 1); }
-        for (int s = 0; s < kQgOperandStages; ++s) { mbar_init(smem_u32(mfull + s), kQgDequantWarps); mbar_init(smem_u32(mempty + s), 1); }
+        for (int s = 0; s < kQgOperandStages; ++s) { mbar_init(smem_u32(mfull + s), kQgGroupWarps); mbar_init(smem_u32(mempty + s), 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(acc1_full + b), 1);
             mbar_init(smem_u32(acc1_empty + b), 4);
@@ -143,106 +145,101 @@ ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_co
     const int p1_supers = n_kb / 2, p2_supers = n_dt;
 
     if (warp == 0) {
-        // ---------------- TMA producer: packed stages one super-item ahead of the token rows ----------------
-        if (lane == 0) {
-            uint32_t np = 0, nx = 0;      // packed stages / token-row stages issued so far
+        // ---------------- TMA producer of the packed weights: runs ahead as far as the packed ring allows ----------------
+        // The whole warp walks the loop in uniform control flow and one elected lane issues.
+        {
+            uint32_t np = 0;              // packed stages issued so far
             bool ok = true;
             auto load_packed = [&](const QgSeq& q) {
                 const GgUnit un = a.units[blockIdx.x + q.unit() * gridDim.x];
                 const uint32_t ps = np % kQgPackedStages;
-                if (np >= uint32_t(kQgPackedStages)) ok = gg_wait(smem_u32(qempty + ps), ((np / kQgPackedStages) - 1) & 1, ab);
+                if (np >= uint32_t(kQgPackedStages))
+                    ok = __all_sync(0xffffffffu, gg_wait(smem_u32(qempty + ps), ((np / kQgPackedStages) - 1) & 1, ab));
                 if (!ok) return;
                 const uint32_t qb = smem_u32(qst + ps * kQgPackedBytes), fq = smem_u32(qfull + ps);
                 const int r0 = un.jt * kGgTileRows;
                 const bool with_scales = (q.idx & 1) == 0;        // 16 bytes of scales cover two super-items
-                if (q.phase1) {
-                    mbar_arrive_expect_tx(fq, 2 * kQgHalfBytes + (with_scales ? 2 * kQgScaleBytes : 0));
-                    tma_load_4d(qb, &nib64, q.idx * 64, 0, r0, un.slot, fq);
-                    tma_load_4d(qb + kQgHalfBytes, &nib64, q.idx * 64, 1, r0, un.slot, fq);
-                    if (with_scales) {
-                        tma_load_4d(qb + kQgNibBytes, &sc16, sc_x0 + (q.idx >> 1) * 16, 0, r0, un.slot, fq);
-                        tma_load_4d(qb + kQgNibBytes + kQgScaleBytes, &sc16, sc_x0 + (q.idx >> 1) * 16, 1, r0, un.slot, fq);
+                if (elect_one()) {
+                    if (q.phase1) {
+                        mbar_arrive_expect_tx(fq, 2 * kQgHalfBytes + (with_scales ? 2 * kQgScaleBytes : 0));
+                        tma_load_4d(qb, &nib64, q.idx * 64, 0, r0, un.slot, fq);
+                        tma_load_4d(qb + kQgHalfBytes, &nib64, q.idx * 64, 1, r0, un.slot, fq);
+                        if (with_scales) {
+                            tma_load_4d(qb + kQgNibBytes, &sc16, sc_x0 + (q.idx >> 1) * 16, 0, r0, un.slot, fq);
+                            tma_load_4d(qb + kQgNibBytes + kQgScaleBytes, &sc16, sc_x0 + (q.idx >> 1) * 16, 1, r0, un.slot, fq);
+                        }
+                    } else {
+                        mbar_arrive_expect_tx(fq, kQgHalfBytes + (with_scales ? kQgScaleBytes : 0));
+                        tma_load_4d(qb, &nib64, q.idx * 64, 2, r0, un.slot, fq);
+                        if (with_scales) tma_load_4d(qb + kQgNibBytes, &sc16, sc_x0 + (q.idx >> 1) * 16, 2, r0, un.slot, fq);
                     }
-                } else {
-                    mbar_arrive_expect_tx(fq, kQgHalfBytes + (with_scales ? kQgScaleBytes : 0));
-                    tma_load_4d(qb, &nib64, q.idx * 64, 2, r0, un.slot, fq);
-                    if (with_scales) tma_load_4d(qb + kQgNibBytes, &sc16, sc_x0 + (q.idx >> 1) * 16, 2, r0, un.slot, fq);
                 }
+                __syncwarp();
                 ++np;
             };
-            auto load_tokens = [&](const QgSeq& q) {      // the two K-blocks of a phase-1 super-item
-                if (!q.phase1) return;
-                const GgUnit un = a.units[blockIdx.x + q.unit() * gridDim.x];
-                for (int j = 0; j < 2 && ok; ++j, ++nx) {
-                    const uint32_t xs = nx % kQgTokenStages;
-                    if (nx >= uint32_t(kQgTokenStages)) ok = gg_wait(smem_u32(xempty + xs), ((nx / kQgTokenStages) - 1) & 1, ab);
-                    if (!ok) return;
-                    const uint32_t fx = smem_u32(xfull + xs);
-                    mbar_arrive_expect_tx(fx, kGgXBytes);
-                    tma_load_2d(smem_u32(xst + xs * kGgXBytes), &xmap, (q.idx * 2 + j) * kGgKBlock, un.row0, fx);
-                }
-            };
-            QgSeq cur(my_units, p1_supers, p2_supers);
-            if (!cur.done) load_packed(cur);
-            while (!cur.done && ok) {
-                QgSeq nxt = cur;
-                nxt.next();
-                if (!nxt.done) load_packed(nxt);
-                if (ok) load_tokens(cur);
-                cur = nxt;
-            }
+            for (QgSeq q(my_units, p1_supers, p2_supers); !q.done && ok; q.next()) load_packed(q);
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer (as in the bf16 kernel; operands and token rows on separate rings) ----------------
-        if (lane == 0) {
-            constexpr uint32_t idesc1 = gg_idesc(false, false);
-            constexpr uint32_t idesc2 = gg_idesc(true, true);
+        // The whole warp walks the loop in uniform control flow and one elected lane issues.
+        {
             uint32_t t = 0, nx = 0, nd = 0;     // operand items, token-row stages, d-tiles consumed so far
             bool ok = true;
+            auto wait_all = [&](uint64_t* bar, uint32_t parity) { ok = __all_sync(0xffffffffu, ok && gg_wait(smem_u32(bar), parity, ab)); };
             auto mma_phase1 = [&](int i) {
                 const uint32_t b = i & 1, m = uint32_t(i) >> 1;
-                if (i >= 2) ok = gg_wait(smem_u32(acc1_empty + b), (m - 1) & 1, ab);
+                const uint32_t idesc1 = gg_idesc_n(false, false, gg_pad_tokens(a.units[blockIdx.x + i * gridDim.x].ntok));
+                if (i >= 2) wait_all(acc1_empty + b, (m - 1) & 1);
                 const uint32_t acc = tmem + 128 * b;
                 for (int kb = 0; kb < n_kb && ok; ++kb, ++t, ++nx) {
                     const uint32_t s = t % kQgOperandStages, xs = nx % kQgTokenStages;
-                    ok = gg_wait(smem_u32(mfull + s), (t / kQgOperandStages) & 1, ab);
-                    if (ok) ok = gg_wait(smem_u32(xfull + xs), (nx / kQgTokenStages) & 1, ab);
+                    wait_all(mfull + s, (t / kQgOperandStages) & 1);
+                    wait_all(xfull + xs, (nx / kQgTokenStages) & 1);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t base = smem_u32(mst + s * kQgOperandBytes), xb = smem_u32(xst + xs * kGgXBytes);
+                    if (elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        const uint64_t bx = smem_desc_sw128(xb + ks * 32, 16, 1024);
-                        tc_mma_bf16(acc, smem_desc_sw128(base + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
-                        tc_mma_bf16(acc + 64, smem_desc_sw128(base + kGgTileBytes + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint64_t bx = smem_desc_sw128(xb + ks * 32, 16, 1024);
+                            tc_mma_bf16(acc, smem_desc_sw128(base + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
+                            tc_mma_bf16(acc + 64, smem_desc_sw128(base + kGgTileBytes + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
+                        }
+                        tc_commit(smem_u32(mempty + s));
+                        tc_commit(smem_u32(xempty + xs));
                     }
-                    tc_commit(smem_u32(mempty + s));
-                    tc_commit(smem_u32(xempty + xs));
+                    __syncwarp();
                 }
-                if (ok) tc_commit(smem_u32(acc1_full + b));
+                if (ok && elect_one()) tc_commit(smem_u32(acc1_full + b));
+                __syncwarp();
             };
             auto mma_phase2 = [&](int i) {
-                ok = gg_wait(smem_u32(act_full), i & 1, ab);
+                const uint32_t idesc2 = gg_idesc_n(true, true, gg_pad_tokens(a.units[blockIdx.x + i * gridDim.x].ntok));
+                wait_all(act_full, i & 1);
                 if (!ok) return;
                 tc_fence_after();
                 const uint32_t act_addr = smem_u32(act);
                 for (int dt = 0; dt < n_dt && ok; ++dt, ++t, ++nd) {
                     const uint32_t s = t % kQgOperandStages, b = nd & 1;
-                    ok = gg_wait(smem_u32(mfull + s), (t / kQgOperandStages) & 1, ab);
-                    if (ok && nd >= 2) ok = gg_wait(smem_u32(acc2_empty + b), ((nd >> 1) - 1) & 1, ab);
+                    wait_all(mfull + s, (t / kQgOperandStages) & 1);
+                    if (nd >= 2) wait_all(acc2_empty + b, ((nd >> 1) - 1) & 1);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t base = smem_u32(mst + s * kQgOperandBytes);
+                    if (elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint64_t da = smem_desc_sw128(base + ks * 2048, kGgTileBytes, 1024);
-                        const uint64_t db = smem_desc_sw128(act_addr + ks * 2048, kGgActBytes, 1024);
-                        tc_mma_bf16(tmem + 256 + 64 * b, da, db, idesc2, ks != 0);
+                        for (int ks = 0; ks < 8; ++ks) {
+                            const uint64_t da = smem_desc_sw128(base + ks * 2048, kGgTileBytes, 1024);
+                            const uint64_t db = smem_desc_sw128(act_addr + ks * 2048, kGgActBytes, 1024);
+                            tc_mma_bf16(tmem + 256 + 64 * b, da, db, idesc2, ks != 0);
+                        }
+                        tc_commit(smem_u32(mempty + s));
+                        tc_commit(smem_u32(acc2_full + b));
                     }
-                    tc_commit(smem_u32(mempty + s));
-                    tc_commit(smem_u32(acc2_full + b));
+                    __syncwarp();
                 }
-                if (ok) tc_commit(smem_u32(act_empty));
+                if (ok && elect_one()) tc_commit(smem_u32(act_empty));
+                __syncwarp();
             };
             if (my_units > 0) mma_phase1(0);
             for (int i = 0; i < my_units && ok; ++i) {
@@ -250,52 +247,105 @@ ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_co
                 if (ok) mma_phase2(i);
             }
         }
-    } else if (warp >= 6) {
-        // ---------------- de-quantisation warps: two threads per weight row, one per operand tile ----------------
-        const int dq = warp - 6;
-        const int r = (dq & 3) * 32 + lane;          // row of the 128-row tile
-        const int tile = dq >> 2;                    // phase 1: 0 = gate, 1 = up; phase 2: 0 = d 0..63, 1 = d 64..127 of the d-tile
-        const uint32_t sw = uint32_t(r & 7);         // 128-byte swizzle of the bf16 operand rows
-        const uint32_t sq = uint32_t((r >> 1) & 3);  // 64-byte swizzle of the packed rows
-        uint32_t t = 0, np = 0;                      // operand items written, packed stages consumed
+    } else if (warp == 14) {
+        // ---------------- TMA producer of the token rows: the two K-blocks of every phase-1 super-item ----------------
+        // (its own warp, so that a wait for a token-row stage never holds back the weight stream)
+        uint32_t nx = 0;
         bool ok = true;
-        uint4 sc = make_uint4(0, 0, 0, 0);           // this row's 8 scales for the current pair of super-items
+        for (QgSeq q(my_units, p1_supers, p2_supers); !q.done && ok; q.next()) {
+            if (!q.phase1) continue;
+            const GgUnit un = a.units[blockIdx.x + q.unit() * gridDim.x];
+            for (int j = 0; j < 2 && ok; ++j, ++nx) {
+                const uint32_t xs = nx % kQgTokenStages;
+                if (nx >= uint32_t(kQgTokenStages))
+                    ok = __all_sync(0xffffffffu, gg_wait(smem_u32(xempty + xs), ((nx / kQgTokenStages) - 1) & 1, ab));
+                if (!ok) break;
+                const uint32_t fx = smem_u32(xfull + xs);
+                if (elect_one()) {
+                    mbar_arrive_expect_tx(fx, kGgXBytes);
+                    tma_load_2d(smem_u32(xst + xs * kGgXBytes), &xmap, (q.idx * 2 + j) * kGgKBlock, un.row0, fx);
+                }
+                __syncwarp();
+            }
+        }
+    } else if (warp >= 6) {
+        // ---------------- de-quantisation warps: four groups of two warps, each expanding every fourth item ----------------
+        // A group owns operand stage g and walks the same item sequence as everybody else, so up to
+        // four items are being expanded at a time and one group's waits and fences overlap the
+        // arithmetic of the others. A thread covers rows gt and gt + 64 of both tiles of its item.
+        const int dq = warp - 6;
+        const int grp = dq / kQgGroupWarps;
+        const int gt = (dq % kQgGroupWarps) * 32 + lane;     // 0..63
+        const uint32_t sw = uint32_t(gt & 7);                // 128-byte swizzle of the bf16 operand rows
+        const uint32_t sq = uint32_t((gt >> 1) & 3);         // 64-byte swizzle of the packed rows
+        uint32_t t = 0, np = 0;                              // items seen, packed stages consumed
+        bool ok = true;
+        uint4 sc[2][2];                                      // [tile][row half]: 8 scales per row for the current pair of super-items
+#pragma unroll
+        for (int i = 0; i < 4; ++i) sc[i >> 1][i & 1] = make_uint4(0, 0, 0, 0);
         for (QgSeq q(my_units, p1_supers, p2_supers); !q.done && ok; q.next(), ++np) {
             const uint32_t ps = np % kQgPackedStages;
             ok = __all_sync(0xffffffffu, gg_wait(smem_u32(qfull + ps), (np / kQgPackedStages) & 1, ab));
             if (!ok) break;
             const unsigned char* qb = qst + ps * kQgPackedBytes;
-            const unsigned char* nrow = qb + (q.phase1 ? tile * kQgHalfBytes : 0) + r * 64;    // this row's 64 bytes of nibbles
-            if ((q.idx & 1) == 0)
-                sc = *reinterpret_cast<const uint4*>(qb + kQgNibBytes + (q.phase1 ? tile * kQgScaleBytes : 0) + r * 16);
-            const int items = q.phase1 ? 2 : 1;
-            for (int j = 0; j < items && ok; ++j, ++t) {
-                // phase 1: K-block j of the super-item = packed chunks 2j, 2j+1 of the row;
-                // phase 2: the d-tile, this thread's half = packed chunks 2*tile, 2*tile+1.
-                // A packed chunk (16 bytes, 32 weights) has one scale: number 4 * (idx & 1) + chunk of `sc`.
-                const int c0 = q.phase1 ? 2 * j : 2 * tile;
-                const uint4 n0 = *reinterpret_cast<const uint4*>(nrow + ((uint32_t(c0) ^ sq) << 4));
-                const uint4 n1 = *reinterpret_cast<const uint4*>(nrow + ((uint32_t(c0 + 1) ^ sq) << 4));
-                const int g = 4 * (q.idx & 1) + c0;
-                const __nv_bfloat162 s0 = scale_at(sc, g), s1 = scale_at(sc, g + 1);
-                const uint32_t ms = t % kQgOperandStages;
-                if (t >= uint32_t(kQgOperandStages))
-                    ok = __all_sync(0xffffffffu, gg_wait(smem_u32(mempty + ms), ((t / kQgOperandStages) - 1) & 1, ab));
-                if (!ok) break;
-                unsigned char* row = mst + ms * kQgOperandBytes + tile * kGgTileBytes + r * 128;
-                const uint32_t w0[4] = {n0.x, n0.y, n0.z, n0.w}, w1[4] = {n1.x, n1.y, n1.z, n1.w};
+            if ((q.idx & 1) == 0) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    *reinterpret_cast<uint4*>(row + ((uint32_t(c) ^ sw) << 4)) = dequant_chunk(w0[c], s0);
-                    *reinterpret_cast<uint4*>(row + ((uint32_t(c + 4) ^ sw) << 4)) = dequant_chunk(w1[c], s1);
-                }
-                fence_proxy_async();          // generic-proxy writes -> visible to the MMA's async reads
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(mfull + ms));
+                for (int tile = 0; tile < 2; ++tile)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        sc[tile][h] = *reinterpret_cast<const uint4*>(qb + kQgNibBytes + (q.phase1 ? tile * kQgScaleBytes : 0) +
+                                                                      (gt + 64 * h) * 16);
             }
-            if (!ok) break;
+            // This group's item of the super-item, if it has one (a super-item is one or two items, a group
+            // takes every fourth): its nibbles go to registers and the packed stage is handed back at
+            // once, so the weight stream is never held up by a group that waits for an operand stage.
+            const int items = q.phase1 ? 2 : 1;
+            const int j = int((uint32_t(grp) - t) % kQgGroups);          // t + j = grp (mod 4)
+            const bool mine = j < items;
+            const uint32_t tm = t + uint32_t(j);
+            t += uint32_t(items);
+            // phase 1: K-block j of the super-item = packed chunks 2j, 2j+1 of the row (tile = gate / up plane);
+            // phase 2: the d-tile, tile = its half = packed chunks 2*tile, 2*tile+1.
+            uint4 nib[2][2][2];                                           // [tile][row half][chunk]
+            if (mine) {
+#pragma unroll
+                for (int tile = 0; tile < 2; ++tile) {
+                    const int c0 = q.phase1 ? 2 * j : 2 * tile;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const unsigned char* nrow = qb + (q.phase1 ? tile * kQgHalfBytes : 0) + (gt + 64 * h) * 64;
+                        nib[tile][h][0] = *reinterpret_cast<const uint4*>(nrow + ((uint32_t(c0) ^ sq) << 4));
+                        nib[tile][h][1] = *reinterpret_cast<const uint4*>(nrow + ((uint32_t(c0 + 1) ^ sq) << 4));
+                    }
+                }
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(qempty + ps));
+            if (!mine) continue;
+            const uint32_t ms = uint32_t(grp);                           // = tm % kQgOperandStages
+            if (tm >= uint32_t(kQgOperandStages))
+                ok = __all_sync(0xffffffffu, gg_wait(smem_u32(mempty + ms), ((tm / kQgOperandStages) - 1) & 1, ab));
+            if (!ok) break;
+#pragma unroll
+            for (int tile = 0; tile < 2; ++tile) {
+                // A packed chunk (16 bytes, 32 weights) has one scale: number 4 * (idx & 1) + chunk of the row's vector.
+                const int g = 4 * (q.idx & 1) + (q.phase1 ? 2 * j : 2 * tile);
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const __nv_bfloat162 s0 = scale_at(sc[tile][h], g), s1 = scale_at(sc[tile][h], g + 1);
+                    unsigned char* row = mst + ms * kQgOperandBytes + tile * kGgTileBytes + (gt + 64 * h) * 128;
+                    const uint4 n0 = nib[tile][h][0], n1 = nib[tile][h][1];
+                    const uint32_t w0[4] = {n0.x, n0.y, n0.z, n0.w}, w1[4] = {n1.x, n1.y, n1.z, n1.w};
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        *reinterpret_cast<uint4*>(row + ((uint32_t(c) ^ sw) << 4)) = dequant_chunk(w0[c], s0);
+                        *reinterpret_cast<uint4*>(row + ((uint32_t(c + 4) ^ sw) << 4)) = dequant_chunk(w1[c], s1);
+                    }
+                }
+            }
+            fence_proxy_async();          // generic-proxy writes -> visible to the MMA's async reads
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(mfull + ms));
         }
     } else {
         // ---------------- epilogue warps (as in the bf16 kernel) ----------------
@@ -317,8 +367,10 @@ ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_co
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
+            const int n_pad = int(gg_pad_tokens(un.ntok));      // columns the MMAs of this unit wrote
 #pragma unroll
             for (int c = 0; c < kGgTokens / 16; ++c) {
+                if (c * 16 >= n_pad) break;
                 float g[16], up[16];
                 tmem_ld16(tmem + lane_addr + 128 * b1 + c * 16, g);
                 tmem_ld16(tmem + lane_addr + 128 * b1 + 64 + c * 16, up);

@@ -65,6 +65,21 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     }
 }
 
+// One lane of a converged warp (elect.sync). Code that a whole warp walks in uniform control flow,
+// with only the issuing instructions under this predicate, lets the compiler keep warp-uniform
+// operands (addresses, descriptors) in uniform registers.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n"
+        " .reg .pred p;\n"
+        " elect.sync _|p, 0xffffffff;\n"
+        " selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(pred));
+    return pred != 0;
+}
+
 // Programmatic dependent launch. A kernel launched with the programmatic-serialisation attribute
 // may begin before the preceding kernel of its stream has finished; grid_dep_wait() returns once
 // that kernel has completed and its writes are visible (at once in an ordinary launch).
