@@ -133,6 +133,14 @@ __device__ __forceinline__ uint32_t gg_idesc_n(bool a_mn_major, bool b_mn_major,
 }
 __device__ __forceinline__ uint32_t gg_pad_tokens(int ntok) { return uint32_t(max(16, (ntok + 15) & ~15)); }
 
+// Token-row tensor maps with boxes of 16, 32 and 64 rows: a unit with few tokens brings only the
+// rows its MMAs read. gg_token_box() picks the map, gg_token_rows() is the row count of its box.
+struct GgTokenMaps {
+    CUtensorMap m[3];
+};
+__device__ __forceinline__ int gg_token_box(int ntok) { return ntok <= 16 ? 0 : ntok <= 32 ? 1 : 2; }
+__device__ __forceinline__ uint32_t gg_token_rows(int box) { return 16u << box; }
+
 struct GgAbort {
     volatile int* flag;     // shared: set by the first wait that gives up
     int* status;
@@ -156,7 +164,7 @@ __device__ __forceinline__ bool gg_wait(uint32_t bar, uint32_t parity, const GgA
 }
 
 __global__ void __launch_bounds__(kGgThreads, 1)
-ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_constant__ CUtensorMap xmap, const GgArgs a) {
+ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_constant__ GgTokenMaps xmaps, const GgArgs a) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     // 1024-byte alignment is what the 128-byte swizzle atoms need
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -219,6 +227,9 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
             bool ok = true;
             auto load_phase1 = [&](int i) {
                 const GgUnit un = a.units[blockIdx.x + i * gridDim.x];
+                const int xbox = gg_token_box(un.ntok);
+                const CUtensorMap* xmap = &xmaps.m[xbox];
+                const uint32_t x_bytes = gg_token_rows(xbox) * 128;
                 for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
                     const uint32_t s = it % kGgStages;
                     if (it >= kGgStages) ok = __all_sync(0xffffffffu, gg_wait(smem_u32(empty + s), ((it / kGgStages) - 1) & 1, ab));
@@ -226,10 +237,10 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
                     const uint32_t base = smem_u32(stages + s * kGgStageBytes);
                     const uint32_t fb = smem_u32(full + s);
                     if (elect_one()) {
-                        mbar_arrive_expect_tx(fb, kGgStageBytes);
+                        mbar_arrive_expect_tx(fb, 2 * kGgTileBytes + x_bytes);
                         tma_load_4d(base, &wmap, kb * kGgKBlock, 0, un.jt * kGgTileRows, un.slot, fb);                 // gate rows
                         tma_load_4d(base + kGgTileBytes, &wmap, kb * kGgKBlock, 1, un.jt * kGgTileRows, un.slot, fb);  // up rows
-                        tma_load_2d(base + 2 * kGgTileBytes, &xmap, kb * kGgKBlock, un.row0, fb);                      // token rows
+                        tma_load_2d(base + 2 * kGgTileBytes, xmap, kb * kGgKBlock, un.row0, fb);                      // token rows
                     }
                     __syncwarp();
                 }

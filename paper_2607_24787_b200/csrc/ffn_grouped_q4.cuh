@@ -87,7 +87,7 @@ struct QgSeq {
 
 __global__ void __launch_bounds__(kQgThreads, 1)
 ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_constant__ CUtensorMap sc16,
-                      const __grid_constant__ CUtensorMap xmap, const GgArgs a) {
+                      const __grid_constant__ GgTokenMaps xmaps, const GgArgs a) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned char* mst = smem;                                               // operand stages
@@ -255,6 +255,7 @@ ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_co
         for (QgSeq q(my_units, p1_supers, p2_supers); !q.done && ok; q.next()) {
             if (!q.phase1) continue;
             const GgUnit un = a.units[blockIdx.x + q.unit() * gridDim.x];
+            const int xbox = gg_token_box(un.ntok);
             for (int j = 0; j < 2 && ok; ++j, ++nx) {
                 const uint32_t xs = nx % kQgTokenStages;
                 if (nx >= uint32_t(kQgTokenStages))
@@ -262,8 +263,8 @@ ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_co
                 if (!ok) break;
                 const uint32_t fx = smem_u32(xfull + xs);
                 if (elect_one()) {
-                    mbar_arrive_expect_tx(fx, kGgXBytes);
-                    tma_load_2d(smem_u32(xst + xs * kGgXBytes), &xmap, (q.idx * 2 + j) * kGgKBlock, un.row0, fx);
+                    mbar_arrive_expect_tx(fx, gg_token_rows(xbox) * 128);
+                    tma_load_2d(smem_u32(xst + xs * kGgXBytes), &xmaps.m[xbox], (q.idx * 2 + j) * kGgKBlock, un.row0, fx);
                 }
                 __syncwarp();
             }

@@ -66,7 +66,8 @@ struct spm_ctx {
     bool tc_ok = false;
     int batched_path = 0;                 // 0: tensor cores when possible, 1: always the per-token GEMV
     int rows_cap = 0, n_jt = 0, max_units = 0;
-    CUtensorMap wmap{}, xmap{};
+    CUtensorMap wmap{};
+    GgTokenMaps xmaps{};
     CUtensorMap qmapn{}, qmapsc{};            // 4-bit blobs: nibble box of 128 bytes, scale box of 16 bytes
     __nv_bfloat16* tc_xs = nullptr;
     float *tc_wrow = nullptr, *tc_partial = nullptr;
@@ -660,9 +661,9 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
     GgArgs a{reinterpret_cast<const GgUnit*>(dd), n_units, nullptr, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status};
     if (m.dtype == SPM_DTYPE_Q4)
         ffn_grouped_q4_kernel<<<std::min(c->num_sms, n_units), kQgThreads, ffn_grouped_q4_smem(), c->compute>>>(
-            c->qmapn, c->qmapsc, c->xmap, a);
+            c->qmapn, c->qmapsc, c->xmaps, a);
     else
-        ffn_grouped_kernel<<<std::min(c->num_sms, n_units), kGgThreads, ffn_grouped_smem(), c->compute>>>(c->wmap, c->xmap, a);
+        ffn_grouped_kernel<<<std::min(c->num_sms, n_units), kGgThreads, ffn_grouped_smem(), c->compute>>>(c->wmap, c->xmaps, a);
     CU(c, cudaGetLastError());
     if (t && last) CU(c, cudaEventRecord(t->ffn_end[layer], c->compute));
     if (ring >= 0 && last) { CU(c, cudaEventRecord(c->ring_end[ring], c->compute)); c->ring_used[ring] = 1; }
@@ -1051,9 +1052,9 @@ int enqueue_host_free_layers(spm_ctx* c, int nb, float* h_out, int slot, bool pr
             GgArgs ga{units, 0, c->tc_counts, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status};
             if (m.dtype == SPM_DTYPE_Q4)
                 CU(c, launch_k(ffn_grouped_q4_kernel, dim3(c->num_sms), dim3(kQgThreads), ffn_grouped_q4_smem(), c->compute, true,
-                               c->qmapn, c->qmapsc, c->xmap, ga));
+                               c->qmapn, c->qmapsc, c->xmaps, ga));
             else
-                CU(c, launch_k(ffn_grouped_kernel, dim3(c->num_sms), dim3(kGgThreads), ffn_grouped_smem(), c->compute, true, c->wmap, c->xmap, ga));
+                CU(c, launch_k(ffn_grouped_kernel, dim3(c->num_sms), dim3(kGgThreads), ffn_grouped_smem(), c->compute, true, c->wmap, c->xmaps, ga));
             CU(c, launch_k(gg_combine_kernel, dim3((m.hidden / 4 + 127) / 128, nb), dim3(128), 0, c->compute, true,
                            (const float*)c->tc_partial, (const int32_t*)rowmap, K, c->n_jt, c->rows_cap, m.hidden, h_out));
             c->kernel_launches += 5;
@@ -1297,7 +1298,10 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
         const bool maps_ok = cfg->dtype == SPM_DTYPE_Q4
             ? make_q4_maps(&c->qmapn, &c->qmapsc, c->pools, cfg->hidden, cfg->inter, uint64_t(L) * c->S)
             : make_weight_map(&c->wmap, c->pools, cfg->hidden, cfg->inter, uint64_t(L) * c->S);
-        if (!maps_ok || !make_token_map(&c->xmap, c->tc_xs, cfg->hidden, uint64_t(lay.rows_cap + kGgTokens))) {
+        bool xmaps_ok = true;
+        for (int b = 0; b < 3; ++b)
+            xmaps_ok = xmaps_ok && make_token_map(&c->xmaps.m[b], c->tc_xs, cfg->hidden, uint64_t(lay.rows_cap + kGgTokens), 16u << b);
+        if (!maps_ok || !xmaps_ok) {
             c->err = "cuTensorMapEncodeTiled failed";
             return bail(SPM_ERR_CUDA);
         }

@@ -55,13 +55,13 @@ inline bool make_weight_map(CUtensorMap* map, const void* base, int D, int I, ui
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// bf16 token rows [rows][D]; a box is 64 elements x 64 rows, 128-byte swizzle.
-inline bool make_token_map(CUtensorMap* map, const void* base, int D, uint64_t rows) {
+// bf16 token rows [rows][D]; a box is 64 elements x `box_rows` rows, 128-byte swizzle.
+inline bool make_token_map(CUtensorMap* map, const void* base, int D, uint64_t rows, uint32_t box_rows) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {cuuint64_t(D), rows};
     const cuuint64_t strides[1] = {cuuint64_t(D) * 2};
-    const cuuint32_t box[2] = {64, 64};
+    const cuuint32_t box[2] = {64, box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
