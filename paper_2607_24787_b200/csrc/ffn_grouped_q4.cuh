@@ -2,22 +2,24 @@
 // packed 4-bit blobs (groups of 32 weights + one fp16 scale, see ffn_gemv_q4.cuh).
 //
 // The tensor cores take bf16 operands, so a fourth role is added between the TMA producer and the
-// MMA issuer: eight de-quantisation warps (two threads per weight row of the 128-row tile, one per
-// 16 KB operand tile) turn each packed tile into the bf16 tile the MMA expects, written with the
-// 128-byte swizzle a TMA load of bf16 data would have produced, so descriptors, accumulators,
-// epilogues and the work order are those of the bf16 kernel. The conversion stays in packed bf16
-// arithmetic: a nibble q is OR-ed into the mantissa of 128.0 (exact 128 + q), 136 is subtracted
-// (exact q - 8) and the result is multiplied by the group's scale rounded to bf16:
-// weight = bf16_rn(bf16_rn(scale) * (q - 8)), two instructions per pair of weights.
+// MMA issuer: eight de-quantisation warps turn each packed tile into the bf16 tile the MMA expects,
+// written with the 128-byte swizzle a TMA load of bf16 data would have produced, so descriptors,
+// accumulators, epilogues and the work order are those of the bf16 kernel. The warps form four
+// groups of two; group g expands every fourth item into operand stage g, so four items are in
+// flight and one group's waits and fences overlap the arithmetic of the others. The conversion
+// stays in packed bf16 arithmetic: a nibble q is OR-ed into the mantissa of 128.0 (exact 128 + q),
+// 136 is subtracted (exact q - 8) and the result is multiplied by the group's scale rounded to
+// bf16: weight = bf16_rn(bf16_rn(scale) * (q - 8)), two instructions per pair of weights.
 //
 // Three rings. Packed stages (TMA -> de-quantisation) hold 64 bytes of nibbles per row, i.e. two
 // K-blocks of gate and up rows (phase 1) or one d-tile of the W_down column tile (phase 2), and
-// every second one also the 16 bytes of scales per row that cover it and its successor. Most of
-// the shared memory goes to this ring: a 4-bit tile is a quarter of its bf16 image, so the bytes
-// in flight towards HBM, not the operand stages, decide the streaming rate. Operand stages
-// (de-quantisation -> MMA) hold the two bf16 tiles of one item (one K-block of 64, or one d-tile
-// of 128). Token-row stages (TMA -> MMA) hold the bf16 token rows of one K-block. Every wait is
-// bounded and shares the abort flag of the CTA; no multicast.
+// every second one also the 16 bytes of scales per row that cover it and its successor; a group
+// copies the nibbles of its item to registers and hands the stage back at once, so the producer
+// (warp 0) runs ahead as far as the ring allows. Operand stages (de-quantisation -> MMA) hold the
+// two bf16 tiles of one item (one K-block of 64, or one d-tile of 128). Token-row stages
+// (TMA -> MMA) hold the bf16 token rows of one K-block and have their own producer (warp 14), so
+// that a wait for a token stage never holds back the weight stream. Every wait is bounded and
+// shares the abort flag of the CTA; no multicast.
 #pragma once
 
 #include "ffn_gemv_q4.cuh"
