@@ -122,3 +122,49 @@ def test_free_running_events_match_policy_oracle(setup):
     assert ev == ref.events
     if cfg.slots < cfg.n_experts and nb * cfg.top_k > cfg.slots:
         assert m.stats()["waves"] > 0
+
+
+WIDTH_CASES = {
+    "bf16": synth.get_config("qwen3", n_layers=1, hidden=512, n_experts=8, inter=256, top_k=3, slots=8, budget=1),
+    "q4": synth.get_config("qwen3_q4", n_layers=1, hidden=512, n_experts=8, inter=256, top_k=3, slots=8, budget=1),
+}
+
+
+@pytest.mark.parametrize("name", list(WIDTH_CASES))
+def test_every_tokens_per_expert_width(name):
+    """The grouped kernel issues its MMAs with N = the unit's tokens rounded up to 16 and fetches
+    16, 32 or 64 token rows: experts with 64, 47, 33, 17, 16, 14 and 1 tokens in one launch, each
+    token's output against the oracle's dense definition."""
+    from paper_2607_24787_b200.build import build
+    from paper_2607_24787_b200.synth_model import build_from_synth
+    build()
+    nb = 64
+    cfg = WIDTH_CASES[name].replace(batch=nb)
+    m = build_from_synth(cfg)
+    try:
+        wts = SynthWeights(cfg)
+        ids = np.zeros((nb, 3), dtype=np.int32)                     # expert 0: all 64 tokens
+        ids[:, 1] = np.where(np.arange(nb) < 47, 1, 2)              # expert 1: 47 tokens, expert 2: 17
+        third = np.full(nb, 6, dtype=np.int32)                      # expert 6: 14 tokens
+        third[:33] = 3                                              # expert 3: 33
+        third[33:49] = 4                                            # expert 4: 16
+        third[49] = 5                                               # expert 5: 1
+        ids[:, 2] = third
+        counts = np.bincount(ids.reshape(-1), minlength=8)
+        assert sorted(counts.tolist(), reverse=True)[:7] == [64, 47, 33, 17, 16, 14, 1]
+        rng = np.random.default_rng(11)
+        x = rng.standard_normal((nb, cfg.hidden)).astype(np.float32)
+        w = rng.uniform(0.1, 1.0, size=(nb, 3)).astype(np.float32)
+        w /= w.sum(axis=1, keepdims=True)
+        xd, wd = dev(x), dev(w)
+        hd = torch.zeros(nb, cfg.hidden, device="cuda")
+        m.moe_ffn(0, xd, ids, wd, hd)
+        m.synchronize()
+        got = hd.cpu().numpy().astype(np.float64)
+        experts = lambda e: wts.expert(0, e)
+        for t in range(nb):
+            want = M.moe_ffn(x[t].astype(np.float64), ids[t], w[t].astype(np.float64), experts)
+            assert M.rel_linf(got[t], want) < TOL_BF16, (name, t)
+        assert m.stats()["ffn_launches"] == 1
+    finally:
+        m.close()
