@@ -733,7 +733,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="reduced layer count (profiler captures only)")
     ap.add_argument("--slots", type=int, default=0, help="override slots per layer")
     ap.add_argument("--arm-steps", type=int, default=128)
-    ap.add_argument("--cpu-steps", type=int, default=2)
+    ap.add_argument("--cpu-steps", type=int, default=6)
     ap.add_argument("--sweep", action="store_true", help="budget x slots sweep (prints one JSON object with all cells)")
     ap.add_argument("--sweep-budgets", default="1,2,4,8")
     ap.add_argument("--sweep-slots", default="8,16,32")

@@ -2,24 +2,27 @@
 // packed 4-bit blobs (groups of 32 weights + one fp16 scale, see ffn_gemv_q4.cuh).
 //
 // The tensor cores take bf16 operands, so a fourth role is added between the TMA producer and the
-// MMA issuer: eight de-quantisation warps turn each packed tile into the bf16 tile the MMA expects,
-// written with the 128-byte swizzle a TMA load of bf16 data would have produced, so descriptors,
-// accumulators, epilogues and the work order are those of the bf16 kernel. The warps form four
-// groups of two; group g expands every fourth item into operand stage g, so four items are in
-// flight and one group's waits and fences overlap the arithmetic of the others. The conversion
-// stays in packed bf16 arithmetic: a nibble q is OR-ed into the mantissa of 128.0 (exact 128 + q),
-// 136 is subtracted (exact q - 8) and the result is multiplied by the group's scale rounded to
-// bf16: weight = bf16_rn(bf16_rn(scale) * (q - 8)), two instructions per pair of weights.
+// MMA issuer: eight de-quantisation warps in two groups of four (one warp per TMEM lane quarter);
+// a group expands every second item, so two items are in flight and one group's waits overlap the
+// other's arithmetic. The conversion stays in packed bf16 arithmetic: a nibble q is OR-ed into the
+// mantissa of 128.0 (exact 128 + q), 136 is subtracted (exact q - 8) and the result is multiplied
+// by the group's scale rounded to bf16: weight = bf16_rn(bf16_rn(scale) * (q - 8)), two
+// instructions per pair of weights.
+//   First GEMM (gate and up tiles, K-major): the expanded weights never touch shared memory. Row
+// r of a 128-row tile is TMEM lane r; a thread writes its row's 64 weights of both tiles as 2 x 32
+// columns with tcgen05.st, and tcgen05.mma takes the A operand from tensor memory (two stages of
+// 64 columns behind the accumulators). Second GEMM (W_down's column tile, consumed M-major: the
+// rows of the packed tile run along the contraction): the tile is written to a shared-memory
+// stage with the 128-byte swizzle a TMA load of bf16 data would have produced.
 //
-// Three rings. Packed stages (TMA -> de-quantisation) hold 64 bytes of nibbles per row, i.e. two
+// Rings. Packed stages (TMA -> de-quantisation) hold 64 bytes of nibbles per row, i.e. two
 // K-blocks of gate and up rows (phase 1) or one d-tile of the W_down column tile (phase 2), and
 // every second one also the 16 bytes of scales per row that cover it and its successor; a group
 // copies the nibbles of its item to registers and hands the stage back at once, so the producer
-// (warp 0) runs ahead as far as the ring allows. Operand stages (de-quantisation -> MMA) hold the
-// two bf16 tiles of one item (one K-block of 64, or one d-tile of 128). Token-row stages
-// (TMA -> MMA) hold the bf16 token rows of one K-block and have their own producer (warp 14), so
-// that a wait for a token stage never holds back the weight stream. Every wait is bounded and
-// shares the abort flag of the CTA; no multicast.
+// (warp 0) runs ahead as far as the ring allows. Token-row stages (TMA -> MMA) hold the bf16
+// token rows of one K-block and have their own producer (warp 14), so that a wait for a token
+// stage never holds back the weight stream. Every wait is bounded and shares the abort flag of
+// the CTA; no multicast.
 #pragma once
 
 #include "ffn_gemv_q4.cuh"
@@ -29,10 +32,12 @@ namespace spm {
 
 constexpr int kQgThreads = 480;          // warp 0 TMA (packed weights), 1 MMA + TMEM, 2-5 epilogue, 6-13 de-quantisation, 14 TMA (token rows)
 constexpr int kQgDequantWarps = 8;
-constexpr int kQgGroups = 4;             // de-quantisation groups of two warps; group g expands the items with t % 4 == g
+constexpr int kQgGroups = 2;             // de-quantisation groups of four warps (one per TMEM lane quarter); group g expands every second item
 constexpr int kQgGroupWarps = kQgDequantWarps / kQgGroups;
-constexpr int kQgOperandStages = 4;      // 2 x 16 KB bf16 tiles each
-constexpr int kQgPackedStages = 3;
+constexpr int kQgOperandStages = 2;      // shared-memory operand stages of the second GEMM, 2 x 16 KB bf16 tiles each
+constexpr int kQgTmemStages = 2;         // tensor-memory operand stages of the first GEMM, 2 x 32 columns each
+constexpr uint32_t kQgTmemA = 384;       // first column of those stages (the accumulators end at 383)
+constexpr int kQgPackedStages = 6;
 constexpr int kQgTokenStages = 2;        // 8 KB each
 constexpr uint32_t kQgOperandBytes = 2 * kGgTileBytes;
 constexpr uint32_t kQgHalfBytes = 8192;  // [128 rows][64 B] of nibbles
@@ -57,6 +62,29 @@ __device__ __forceinline__ uint4 dequant_chunk(uint32_t w, __nv_bfloat162 scale2
         r[p] = *reinterpret_cast<const uint32_t*>(&v);
     }
     return make_uint4(r[0], r[1], r[2], r[3]);
+}
+
+// 32 consecutive 32-bit columns of this thread's TMEM lane (the mirror of tmem_ld16)
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]),
+          "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]),
+          "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// D[tmem] (+)= A[tmem] * B[smem desc]: the A operand (128 rows = lanes, 16 bf16 = 8 columns) comes from tensor memory
+__device__ __forceinline__ void tc_mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t"
+        "}\n"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
 __device__ __forceinline__ int qg_unpermute(int m) { return (m & ~7) | ((m & 7) >> 1) | ((m & 1) << 2); }
@@ -103,7 +131,9 @@ ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_co
     uint64_t* xempty = xfull + kQgTokenStages;       // [token]    MMA -> TMA
     uint64_t* mfull = xempty + kQgTokenStages;       // [operand]  de-quantisation -> MMA
     uint64_t* mempty = mfull + kQgOperandStages;     // [operand]  MMA -> de-quantisation
-    uint64_t* acc1_full = mempty + kQgOperandStages; // [2]
+    uint64_t* tfull = mempty + kQgOperandStages;     // [tmem]     de-quantisation -> MMA (first GEMM)
+    uint64_t* tempty = tfull + kQgTmemStages;        // [tmem]     MMA -> de-quantisation
+    uint64_t* acc1_full = tempty + kQgTmemStages;    // [2]
     uint64_t* acc1_empty = acc1_full + 2;            // [2]
     uint64_t* act_full = acc1_empty + 2;
     uint64_t* act_empty = act_full + 1;
@@ -124,6 +154,7 @@ ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_co
         for (int s = 0; s < kQgPackedStages; ++s) { mbar_init(smem_u32(qfull + s), 1); mbar_init(smem_u32(qempty + s), kQgDequantWarps); }
         for (int s = 0; s < kQgTokenStages; ++s) { mbar_init(smem_u32(xfull + s), 1); mbar_init(smem_u32(xempty + s), 1); }
         for (int s = 0; s < kQgOperandStages; ++s) { mbar_init(smem_u32(mfull + s), kQgGroupWarps); mbar_init(smem_u32(mempty + s), 1); }
+        for (int s = 0; s < kQgTmemStages; ++s) { mbar_init(smem_u32(tfull + s), kQgGroupWarps); mbar_init(smem_u32(tempty + s), 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(acc1_full + b), 1);
             mbar_init(smem_u32(acc1_empty + b), 4);
@@ -185,7 +216,7 @@ ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_co
         // ---------------- MMA issuer (as in the bf16 kernel; operands and token rows on separate rings) ----------------
         // The whole warp walks the loop in uniform control flow and one elected lane issues.
         {
-            uint32_t t = 0, nx = 0, nd = 0;     // operand items, token-row stages, d-tiles consumed so far
+            uint32_t t1 = 0, t2 = 0, nx = 0, nd = 0;     // items of the first / second GEMM, token-row stages, d-tiles consumed so far
             bool ok = true;
             auto wait_all = [&](uint64_t* bar, uint32_t parity) { ok = __all_sync(0xffffffffu, ok && gg_wait(smem_u32(bar), parity, ab)); };
             auto mma_phase1 = [&](int i) {
@@ -193,21 +224,21 @@ ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_co
                 const uint32_t idesc1 = gg_idesc_n(false, false, gg_pad_tokens(a.units[blockIdx.x + i * gridDim.x].ntok));
                 if (i >= 2) wait_all(acc1_empty + b, (m - 1) & 1);
                 const uint32_t acc = tmem + 128 * b;
-                for (int kb = 0; kb < n_kb && ok; ++kb, ++t, ++nx) {
-                    const uint32_t s = t % kQgOperandStages, xs = nx % kQgTokenStages;
-                    wait_all(mfull + s, (t / kQgOperandStages) & 1);
+                for (int kb = 0; kb < n_kb && ok; ++kb, ++t1, ++nx) {
+                    const uint32_t s = t1 % kQgTmemStages, xs = nx % kQgTokenStages;
+                    wait_all(tfull + s, (t1 / kQgTmemStages) & 1);
                     wait_all(xfull + xs, (nx / kQgTokenStages) & 1);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t base = smem_u32(mst + s * kQgOperandBytes), xb = smem_u32(xst + xs * kGgXBytes);
+                    const uint32_t at = tmem + kQgTmemA + 64 * s, xb = smem_u32(xst + xs * kGgXBytes);
                     if (elect_one()) {
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks) {
                             const uint64_t bx = smem_desc_sw128(xb + ks * 32, 16, 1024);
-                            tc_mma_bf16(acc, smem_desc_sw128(base + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
-                            tc_mma_bf16(acc + 64, smem_desc_sw128(base + kGgTileBytes + ks * 32, 16, 1024), bx, idesc1, (kb | ks) != 0);
+                            tc_mma_bf16_ts(acc, at + ks * 8, bx, idesc1, (kb | ks) != 0);
+                            tc_mma_bf16_ts(acc + 64, at + 32 + ks * 8, bx, idesc1, (kb | ks) != 0);
                         }
-                        tc_commit(smem_u32(mempty + s));
+                        tc_commit(smem_u32(tempty + s));
                         tc_commit(smem_u32(xempty + xs));
                     }
                     __syncwarp();
@@ -221,9 +252,9 @@ ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_co
                 if (!ok) return;
                 tc_fence_after();
                 const uint32_t act_addr = smem_u32(act);
-                for (int dt = 0; dt < n_dt && ok; ++dt, ++t, ++nd) {
-                    const uint32_t s = t % kQgOperandStages, b = nd & 1;
-                    wait_all(mfull + s, (t / kQgOperandStages) & 1);
+                for (int dt = 0; dt < n_dt && ok; ++dt, ++t2, ++nd) {
+                    const uint32_t s = t2 % kQgOperandStages, b = nd & 1;
+                    wait_all(mfull + s, (t2 / kQgOperandStages) & 1);
                     if (nd >= 2) wait_all(acc2_empty + b, ((nd >> 1) - 1) & 1);
                     if (!ok) break;
                     tc_fence_after();
@@ -272,72 +303,94 @@ ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_co
             }
         }
     } else if (warp >= 6) {
-        // ---------------- de-quantisation warps: four groups of two warps, each expanding every fourth item ----------------
-        // A group owns operand stage g and walks the same item sequence as everybody else, so up to
-        // four items are being expanded at a time and one group's waits and fences overlap the
-        // arithmetic of the others. A thread covers rows gt and gt + 64 of both tiles of its item.
+        // ---------------- de-quantisation warps: two groups of four warps, each expanding every second item ----------------
+        // First GEMM: the expanded weights go straight to tensor memory (tcgen05.st) and the MMA
+        // takes its A operand from there: row r of the tile is TMEM lane r, so the four warps of a
+        // group are those whose warp number mod 4 covers the four lane quarters, and a thread
+        // expands its row of both tiles (gate, up): 2 x 64 weights = 2 x 32 columns. Second GEMM:
+        // W_down's tile is consumed M-major (rows of the packed tile run along the contraction),
+        // so it goes to a swizzled shared-memory stage as a TMA load of bf16 data would have put it.
         const int dq = warp - 6;
         const int grp = dq / kQgGroupWarps;
-        const int gt = (dq % kQgGroupWarps) * 32 + lane;     // 0..63
-        const uint32_t sw = uint32_t(gt & 7);                // 128-byte swizzle of the bf16 operand rows
-        const uint32_t sq = uint32_t((gt >> 1) & 3);         // 64-byte swizzle of the packed rows
-        uint32_t t = 0, np = 0;                              // items seen, packed stages consumed
+        const int r = (warp & 3) * 32 + lane;                // row of the 128-row tile = TMEM lane
+        const uint32_t lane_addr = uint32_t((warp & 3) * 32) << 16;
+        const uint32_t sw = uint32_t(r & 7);                 // 128-byte swizzle of the bf16 operand rows
+        const uint32_t sq = uint32_t((r >> 1) & 3);          // 64-byte swizzle of the packed rows
+        uint32_t t1 = 0, t2 = 0, np = 0;                     // items seen of the first / second GEMM, packed stages consumed
         bool ok = true;
-        uint4 sc[2][2];                                      // [tile][row half]: 8 scales per row for the current pair of super-items
-#pragma unroll
-        for (int i = 0; i < 4; ++i) sc[i >> 1][i & 1] = make_uint4(0, 0, 0, 0);
+        uint4 sc[2];                                         // [tile]: 8 scales of row r for the current pair of super-items
+        sc[0] = sc[1] = make_uint4(0, 0, 0, 0);
         for (QgSeq q(my_units, p1_supers, p2_supers); !q.done && ok; q.next(), ++np) {
             const uint32_t ps = np % kQgPackedStages;
             ok = __all_sync(0xffffffffu, gg_wait(smem_u32(qfull + ps), (np / kQgPackedStages) & 1, ab));
             if (!ok) break;
             const unsigned char* qb = qst + ps * kQgPackedBytes;
             if ((q.idx & 1) == 0) {
-#pragma unroll
-                for (int tile = 0; tile < 2; ++tile)
-#pragma unroll
-                    for (int h = 0; h < 2; ++h)
-                        sc[tile][h] = *reinterpret_cast<const uint4*>(qb + kQgNibBytes + (q.phase1 ? tile * kQgScaleBytes : 0) +
-                                                                      (gt + 64 * h) * 16);
+                sc[0] = *reinterpret_cast<const uint4*>(qb + kQgNibBytes + r * 16);
+                if (q.phase1) sc[1] = *reinterpret_cast<const uint4*>(qb + kQgNibBytes + kQgScaleBytes + r * 16);
             }
-            // This group's item of the super-item, if it has one (a super-item is one or two items, a group
-            // takes every fourth): its nibbles go to registers and the packed stage is handed back at
-            // once, so the weight stream is never held up by a group that waits for an operand stage.
-            const int items = q.phase1 ? 2 : 1;
-            const int j = int((uint32_t(grp) - t) % kQgGroups);          // t + j = grp (mod 4)
-            const bool mine = j < items;
-            const uint32_t tm = t + uint32_t(j);
-            t += uint32_t(items);
-            // phase 1: K-block j of the super-item = packed chunks 2j, 2j+1 of the row (tile = gate / up plane);
-            // phase 2: the d-tile, tile = its half = packed chunks 2*tile, 2*tile+1.
-            uint4 nib[2][2][2];                                           // [tile][row half][chunk]
-            if (mine) {
+            // A packed chunk (16 bytes, 32 weights) has one scale: number 4 * (idx & 1) + chunk of the row's vector.
+            const int g0 = 4 * (q.idx & 1);
+            if (q.phase1) {
+                // two items (K-blocks 2*idx and 2*idx + 1), one per group; t1 is even here, so item j has stage j
+                const int j = grp;
+                const uint32_t tm = t1 + uint32_t(j);
+                t1 += 2;
+                uint4 nib[2][2];                              // [tile][chunk]: packed chunks 2j, 2j+1 of the row
 #pragma unroll
                 for (int tile = 0; tile < 2; ++tile) {
-                    const int c0 = q.phase1 ? 2 * j : 2 * tile;
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const unsigned char* nrow = qb + (q.phase1 ? tile * kQgHalfBytes : 0) + (gt + 64 * h) * 64;
-                        nib[tile][h][0] = *reinterpret_cast<const uint4*>(nrow + ((uint32_t(c0) ^ sq) << 4));
-                        nib[tile][h][1] = *reinterpret_cast<const uint4*>(nrow + ((uint32_t(c0 + 1) ^ sq) << 4));
-                    }
+                    const unsigned char* nrow = qb + tile * kQgHalfBytes + r * 64;
+                    nib[tile][0] = *reinterpret_cast<const uint4*>(nrow + ((uint32_t(2 * j) ^ sq) << 4));
+                    nib[tile][1] = *reinterpret_cast<const uint4*>(nrow + ((uint32_t(2 * j + 1) ^ sq) << 4));
                 }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(qempty + ps));
-            if (!mine) continue;
-            const uint32_t ms = uint32_t(grp);                           // = tm % kQgOperandStages
-            if (tm >= uint32_t(kQgOperandStages))
-                ok = __all_sync(0xffffffffu, gg_wait(smem_u32(mempty + ms), ((tm / kQgOperandStages) - 1) & 1, ab));
-            if (!ok) break;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(qempty + ps));       // nibbles are in registers: hand the stage back
+                const uint32_t s = tm % kQgTmemStages;
+                if (tm >= uint32_t(kQgTmemStages))
+                    ok = __all_sync(0xffffffffu, gg_wait(smem_u32(tempty + s), ((tm / kQgTmemStages) - 1) & 1, ab));
+                if (!ok) break;
+                tc_fence_after();
 #pragma unroll
-            for (int tile = 0; tile < 2; ++tile) {
-                // A packed chunk (16 bytes, 32 weights) has one scale: number 4 * (idx & 1) + chunk of the row's vector.
-                const int g = 4 * (q.idx & 1) + (q.phase1 ? 2 * j : 2 * tile);
+                for (int tile = 0; tile < 2; ++tile) {
+                    const __nv_bfloat162 s0 = scale_at(sc[tile], g0 + 2 * j), s1 = scale_at(sc[tile], g0 + 2 * j + 1);
+                    const uint4 n0 = nib[tile][0], n1 = nib[tile][1];
+                    const uint32_t w0[4] = {n0.x, n0.y, n0.z, n0.w}, w1[4] = {n1.x, n1.y, n1.z, n1.w};
+                    uint32_t cols[32];                        // 64 weights of the row, two per column
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const __nv_bfloat162 s0 = scale_at(sc[tile][h], g), s1 = scale_at(sc[tile][h], g + 1);
-                    unsigned char* row = mst + ms * kQgOperandBytes + tile * kGgTileBytes + (gt + 64 * h) * 128;
-                    const uint4 n0 = nib[tile][h][0], n1 = nib[tile][h][1];
+                    for (int c = 0; c < 4; ++c) {
+                        const uint4 v0 = dequant_chunk(w0[c], s0), v1 = dequant_chunk(w1[c], s1);
+                        cols[4 * c] = v0.x; cols[4 * c + 1] = v0.y; cols[4 * c + 2] = v0.z; cols[4 * c + 3] = v0.w;
+                        cols[16 + 4 * c] = v1.x; cols[16 + 4 * c + 1] = v1.y; cols[16 + 4 * c + 2] = v1.z; cols[16 + 4 * c + 3] = v1.w;
+                    }
+                    tmem_st32(tmem + lane_addr + kQgTmemA + 64 * s + 32 * tile, cols);
+                }
+                tmem_st_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(tfull + s));
+            } else {
+                // one item (a d-tile of the W_down column tile), groups alternate
+                const uint32_t tm = t2;
+                t2 += 1;
+                const bool mine = int(tm % kQgGroups) == grp;
+                uint4 nib[4];                                 // the row's four packed chunks = 128 d-values
+                if (mine) {
+                    const unsigned char* nrow = qb + r * 64;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) nib[c] = *reinterpret_cast<const uint4*>(nrow + ((uint32_t(c) ^ sq) << 4));
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(qempty + ps));
+                if (!mine) continue;
+                const uint32_t ms = tm % kQgOperandStages;
+                if (tm >= uint32_t(kQgOperandStages))
+                    ok = __all_sync(0xffffffffu, gg_wait(smem_u32(mempty + ms), ((tm / kQgOperandStages) - 1) & 1, ab));
+                if (!ok) break;
+#pragma unroll
+                for (int tile = 0; tile < 2; ++tile) {        // d 0..63 and d 64..127 of the d-tile
+                    const __nv_bfloat162 s0 = scale_at(sc[0], g0 + 2 * tile), s1 = scale_at(sc[0], g0 + 2 * tile + 1);
+                    unsigned char* row = mst + ms * kQgOperandBytes + tile * kGgTileBytes + r * 128;
+                    const uint4 n0 = nib[2 * tile], n1 = nib[2 * tile + 1];
                     const uint32_t w0[4] = {n0.x, n0.y, n0.z, n0.w}, w1[4] = {n1.x, n1.y, n1.z, n1.w};
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
@@ -345,10 +398,10 @@ ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_co
                         *reinterpret_cast<uint4*>(row + ((uint32_t(c + 4) ^ sw) << 4)) = dequant_chunk(w1[c], s1);
                     }
                 }
+                fence_proxy_async();          // generic-proxy writes -> visible to the MMA's async reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(mfull + ms));
             }
-            fence_proxy_async();          // generic-proxy writes -> visible to the MMA's async reads
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(mfull + ms));
         }
     } else {
         // ---------------- epilogue warps (as in the bf16 kernel) ----------------
