@@ -69,7 +69,9 @@ def decision_logits(z: np.ndarray) -> np.ndarray:
     """Logits in the precision the Top-K decision is taken in.
 
     The kernels take the decision on fp32 logits, so the oracle rounds its fp64
-    logits to fp32 before ranking them.
+    logits to fp32 before ranking them: values that differ only below fp32
+    resolution tie, and ties go to the lower id (pinned by
+    test_route_decides_in_fp32).
     """
     return np.asarray(z, F64).astype(np.float32)
 

@@ -8,8 +8,9 @@ What the paper fixes (Section 3.3, "Window-Aware Prefetch Budgeting"):
   * the remaining experts are ranked by predicted priority s_e and the first
     M_max are selected: P = Top_{M_max}({s_e : e not in A ∪ U});
   * they are transferred in descending priority and m = |P| <= M_max;
-  * a required expert that is not available is loaded on demand, so routing and
-    outputs never depend on the prediction.
+  * whatever the router asks for and the cache lacks at execution time is fetched
+    then (the on-demand fallback), which is why a wrong prediction can cost time
+    but can never change routing or outputs.
 The paper does not say how the accelerator-side cache is organised. The reading
 taken here: S slots per layer, least-recently-used eviction driven by one global
 tick, ties broken by the lower expert id, empty slots taken lowest index first,

@@ -128,6 +128,45 @@ def test_route_weights():
 
 
 # ---------------------------------------------------------------- SwiGLU expert
+def test_route_decides_in_fp32():
+    """The Top-K decision is taken on logits rounded to fp32 (the precision the kernels decide in):
+    logits that differ only below fp32 resolution tie, and ties go to the lower id; logits that
+    differ above it do not tie."""
+    # 1e-12 apart at the K boundary, the HIGHER id slightly larger in fp64: fp32 rounding makes them
+    # equal, so the lower id must win. Ranking the fp64 values would return the higher id instead.
+    z = np.array([1.0, 1.0 + 1e-12, -3.0])
+    assert np.float32(z[0]) == np.float32(z[1]) and z[1] > z[0]
+    ids, w = M.route(z, 1, renormalize=True)
+    assert list(ids) == [0] and w[0] == pytest.approx(1.0)
+    z = np.array([2.0, 1.0, 1.0 + 1e-12, 0.0])
+    ids, _ = M.route(z, 2, renormalize=False)
+    assert list(ids) == [0, 1]
+    # the weights still come from the fp64 softmax, not from rounded values
+    _, w = M.route(np.array([1.0, 1.0 + 1e-12, -3.0]), 2, renormalize=False)
+    assert w[1] > w[0]
+    # 1e-3 apart: far above fp32 resolution at this magnitude, so no tie and the larger logit wins
+    z = np.array([1.0, 1.001, -3.0])
+    ids, _ = M.route(z, 1, renormalize=True)
+    assert list(ids) == [1]
+    z = np.array([2.0, 1.0, 1.001, 0.0])
+    ids, _ = M.route(z, 2, renormalize=False)
+    assert list(ids) == [0, 2]
+    # decision_logits itself: fp32 values, nearest rounding, same shape
+    d = M.decision_logits(np.array([1.0 + 1e-12, 1.0 + 2.0 ** -24 + 2.0 ** -40, 0.1]))
+    assert d.dtype == np.float32
+    assert d[0] == np.float32(1.0) and d[1] == np.float32(1.0 + 2.0 ** -23) and d[2] == np.float32(0.1)
+
+
+def test_batch_demand_union():
+    """T_batch is the union of the tokens' Top-K sets: duplicates counted once, ascending ids."""
+    assert M.batch_demand([[5, 1], [1, 9], [9, 5]]) == [1, 5, 9]
+    assert M.batch_demand([np.array([7, 3, 3])]) == [3, 7]
+    assert M.batch_demand([]) == []
+    ids = [rng.permutation(32)[:4] for _ in range(6)]
+    want = sorted(set(int(e) for row in ids for e in row))
+    assert M.batch_demand(ids) == want and all(isinstance(e, int) for e in want)
+
+
 def test_swiglu_hand_example():
     # D = 2, I = 1: g = 1, u = 2, silu(1) = 1/(1+e^-1); y = W_down * (silu(g) * u)
     y = M.swiglu_expert([[1.0, 0.0]], [[0.0, 1.0]], [[1.0], [-1.0]], [1.0, 2.0])
