@@ -371,8 +371,16 @@ def run_ours(args):
                 "achieved_in_kernel_window": b2b["gb_s_in_kernel_window"],
                 "frac_in_kernel_window": (b2b["gb_s_in_kernel_window"] or 0) / peak,
                 "frac_of_nominal_8TBs": b2b["gb_s"] / NOMINAL_HBM_GBS,
-                "region": f"{b2b['launches']} spm_moe_ffn launches back to back on the compute stream, all experts resident "
-                          f"(pools of all layers cycled, nothing served from L2), CUDA event pair per launch"}
+                "region": (f"{b2b['launches']} launches of the kernel alone back to back on the compute stream (spm_time_ffn_kernel), "
+                           "all experts resident, pools of all layers cycled (nothing served from L2), one CUDA event pair "
+                           "around all of them, launched as a decode step launches it (programmatic dependent launch); "
+                           "us_per_launch = span / launches") if cfg.batch == 1 else
+                          (f"{b2b['launches']} spm_moe_ffn launches back to back on the compute stream, all experts resident "
+                           "(pools of all layers cycled, nothing served from L2), CUDA event pair per launch"),
+                "us_per_launch_serialized": b2b.get("serialized_us"),
+                "frac_serialized": (b2b["algorithmic_bytes_per_launch"] / (b2b["serialized_us"] * 1e-6) / 1e9 / peak) if b2b.get("serialized_us") else None,
+                "us_per_launch_event_pair_each": b2b["event_pair_each_us"],
+                "frac_event_pair_each": b2b["algorithmic_bytes_per_launch"] / (b2b["event_pair_each_us"] * 1e-6) / 1e9 / peak}
             # The headline is the kernel timed by itself (burst peak as denominator). Inside the main arm every
             # launch follows a wait for PCIe copies and overlaps the next prefetch copy; an event pair there
             # measures mostly launch latency behind the busy link (the in-kernel window stays the same), so
@@ -525,13 +533,28 @@ def ffn_back_to_back(cfg, full, algo_bytes, peak, launches=480):
     e1.record(full.compute)
     full.synchronize()
     per_call = e0.elapsed_time(e1) * 1e3 / launches
+    out = {"launches": launches, "kernel": ffn_kernel_name(cfg),
+           "algorithmic_bytes_per_launch": mean_bytes, "event_pair_each_us": per_kernel,
+           "kernel_window_us": window if window > 0 else None, "call_us_incl_combine": per_call,
+           "misses": st["misses"]}
+    if nb == 1:
+        # the kernel alone, no combine in between: one event pair around all launches. `chained`: launched as a
+        # decode step launches it (programmatic dependent launch: a launch fetches its first weight rows while its
+        # predecessor drains); `serialized`: plain launches, each starts after the one before it has ended.
+        ids1 = np.stack([i[0] for i in ids]).astype(np.int32)
+        full.time_ffn_kernel(0, x[0], ids1[:32], w[0], chained=True)          # warm-up
+        chained = [full.time_ffn_kernel(0, x[0], ids1, w[0], chained=True) for _ in range(3)]
+        serial = [full.time_ffn_kernel(0, x[0], ids1, w[0], chained=False) for _ in range(3)]
+        out["chained_us"] = statistics.median(c[0] for c in chained)
+        out["chained_window_us"] = statistics.median(c[1] for c in chained)
+        out["serialized_us"] = statistics.median(c[0] for c in serial)
+        out["serialized_window_us"] = statistics.median(c[1] for c in serial)
+        per_kernel = out["chained_us"]
+    out["kernel_us"] = per_kernel
     ach = mean_bytes / (per_kernel * 1e-6) / 1e9
-    return {"launches": launches, "kernel": ffn_kernel_name(cfg),
-            "algorithmic_bytes_per_launch": mean_bytes, "kernel_us": per_kernel,
-            "kernel_window_us": window if window > 0 else None, "call_us_incl_combine": per_call, "gb_s": ach,
-            "frac_of_measured_peak": ach / peak,
-            "gb_s_in_kernel_window": mean_bytes / (window * 1e-6) / 1e9 if window > 0 else None,
-            "misses": st["misses"]}
+    out.update(gb_s=ach, frac_of_measured_peak=ach / peak,
+               gb_s_in_kernel_window=mean_bytes / (window * 1e-6) / 1e9 if window > 0 else None)
+    return out
 
 
 def run_sweep(args):

@@ -190,22 +190,31 @@ int spm_adapter_predict(spm_ctx* ctx, int layer, const float* x_norm, int nb,
 int spm_budget_select(spm_ctx* ctx, int target_layer, const int32_t* order, int n_ranked,
                       int budget, int protect_all, int32_t* out_ids, int* out_count);
 
-/* Issue host->HBM copies of experts `ids` (host, descending priority) of `target_layer` on the
- * copy stream into least-recently-used slots of that layer's pool; one CUDA event per slot.
+/* Asynchronous transfer of the selected experts (Section 3.3: the candidates of P are moved in
+ * descending order of predicted priority while computation goes on). Issues host->HBM copies of
+ * experts `ids` (host, descending priority) of `target_layer` on the copy stream into
+ * least-recently-used slots of that layer's pool, in the order given; the copies of one call form
+ * a batch with one CUDA event, recorded after its last copy, which later launches wait on.
  * Experts that already have a slot are skipped. Stops when no unprotected slot is left.
  * *out_issued (may be NULL) = number of copies enqueued. Asynchronous. */
 int spm_prefetch_async(spm_ctx* ctx, int target_layer, const int32_t* ids, int count,
                        int* out_issued);
 
-/* Routed + shared SwiGLU experts of `layer` for nb tokens, slot-indexed (no gather):
+/* Expert computation of `layer` with the on-demand fallback (Section 3.1, second equation: the
+ * batch demand T_batch; Section 3.3, last paragraph: whatever the router asks for and the cache
+ * lacks is loaded at execution time, so outputs never depend on the prediction).
+ * Routed + shared SwiGLU experts for nb tokens, slot-indexed (no gather):
  * resolves the batch demand against the slot table, loads misses on demand, makes the compute
- * stream wait for exactly the slots it reads, and enqueues h_inout += sum_k w_k FFN_{ids_k}(x).
+ * stream wait for exactly the copy batches whose slots it reads, and enqueues
+ * h_inout += sum_k w_k FFN_{ids_k}(x).
  * x_norm dev [nb][D], ids HOST [nb][K], w dev [nb][K], h_inout dev [nb][D]. Asynchronous.
  * When more distinct experts are needed than there are slots the work is split in waves. */
 int spm_moe_ffn(spm_ctx* ctx, int layer, const float* x_norm, const int32_t* ids,
                 const float* w, int nb, float* h_inout);
 
-/* One decode step through all L layers under the context's policy: h_in dev [nb][D] ->
+/* One decode step through all L layers under the context's policy (Sections 3.1 - 3.3 in the order
+ * of the paper's pipeline figure: route layer l, load what is missing, predict and prefetch for
+ * layer l+1 while layer l's experts compute): h_in dev [nb][D] ->
  * h_out dev [nb][D] (may alias h_in). Equivalent to, per layer: spm_router_topk,
  * spm_adapter_predict, spm_moe_ffn, spm_budget_select + spm_prefetch_async for layer+1,
  * with router and adapter fused in one kernel. The last layer's work is left in flight. */
@@ -275,6 +284,18 @@ int spm_set_graph_replay(spm_ctx* ctx, int on);
 int spm_set_attention_stub_us(spm_ctx* ctx, int us);
 /* Host deadline of the routing-kernel handshake, in milliseconds (default 5000). */
 int spm_set_deadline_ms(spm_ctx* ctx, int ms);
+/* Limit of every wait inside the expert kernels (for a weight copy to land in shared memory, for an
+ * arrival counter with spm_set_device_wait, for a pipeline barrier of the grouped kernels), in
+ * microseconds; 0 restores the default of 2 s. A wait that runs out sets a status bit, the kernel
+ * winds down (no copy left in flight, tensor memory released) and returns; the next
+ * spm_synchronize / spm_get_stats reports SPM_ERR_TIMEOUT once and the context stays usable
+ * (spm_cache_reset brings slot table and arrival counters back to a known state). */
+int spm_set_device_wait_limit_us(spm_ctx* ctx, int us);
+/* Host-side fault injection for tests of that time-out: with spm_set_device_wait on, the next
+ * `count` arrival-counter updates are not enqueued (the bytes still land; the counter never says
+ * so), so the kernel that waits for that batch gives up after the limit. Nothing on the GPU
+ * faults or hangs. Cleared by spm_cache_reset. */
+int spm_test_withhold_arrivals(spm_ctx* ctx, int count);
 
 /* Profile the overlap window (Section 3.3): window_us = median device time of the expert FFN of
  * one layer at max_batch tokens with every needed expert resident (kernel(s) + combine, the same
@@ -288,6 +309,21 @@ int spm_profile_window(spm_ctx* ctx, double* window_us, double* t_xfer_us, int* 
  * it) `reps` >= 1 times on the compute stream; *gb_s is the best repetition by CUDA event pair.
  * The pool contents are not modified. Waits for the compute stream. */
 int spm_measure_read_bandwidth(spm_ctx* ctx, size_t bytes, int reps, double* gb_s);
+/* Device time of the batch-1 expert-FFN kernel by itself (measurement aid; the hidden row is not
+ * updated and no combine kernel runs). Enqueues `launches` launches of the slot-indexed GEMV kernel
+ * back to back on the compute stream, launch i on layer (first_layer + i) % L with the K experts
+ * ids[i*K .. i*K+K) (HOST) plus the layer's shared experts, x_norm dev [D], w dev [K], between one
+ * pair of CUDA events, and waits. Every expert named must already hold a slot
+ * (SPM_ERR_NOT_RESIDENT otherwise: nothing is loaded here).
+ * chained = 1: launched as in a decode step, with the programmatic-serialisation attribute, so a
+ * launch fetches its first weight rows while its predecessor drains; 0: plain launches, each
+ * starts after the one before it has ended.
+ * *us_per_launch = event span / launches. *window_us (may be NULL) = mean in-kernel window
+ * (dependency resolved or first CTA started -> last CTA done, %globaltimer) of the first 12288
+ * launches. The partial-row workspace and the in-kernel clock ring are overwritten. */
+int spm_time_ffn_kernel(spm_ctx* ctx, int first_layer, const float* x_norm, const int32_t* ids,
+                        const float* w, int launches, int chained, double* us_per_launch,
+                        double* window_us);
 
 int spm_cache_reset(spm_ctx* ctx);                         /* cold cache, step counter, stats, events */
 /* Checkpoint / resume of the expert cache (Section 3.3's availability state; integers only, no

@@ -93,6 +93,9 @@ _SIG = {
     "spm_set_copy_delay_us": [_P, C.c_int],
     "spm_profile_window": [_P, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int)],
     "spm_measure_read_bandwidth": [_P, C.c_size_t, C.c_int, C.POINTER(C.c_double)],
+    "spm_time_ffn_kernel": [_P, C.c_int, _P, _P, _P, C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double)],
+    "spm_set_device_wait_limit_us": [_P, C.c_int],
+    "spm_test_withhold_arrivals": [_P, C.c_int],
     "spm_cache_reset": [_P],
     "spm_reset_stats": [_P],
     "spm_get_stats": [_P, C.POINTER(Stats)],
@@ -313,6 +316,23 @@ def spm_measure_read_bandwidth(ctx, nbytes, reps=5) -> float:
     g = C.c_double()
     _check(load().spm_measure_read_bandwidth(ctx, nbytes, reps, C.byref(g)), ctx)
     return g.value
+
+
+def spm_time_ffn_kernel(ctx, first_layer, x_norm, ids: np.ndarray, w, chained=True):
+    """(us per launch by one event pair around all launches, mean in-kernel window in us)."""
+    ids = np.ascontiguousarray(ids, np.int32)
+    us, win = C.c_double(), C.c_double()
+    _check(load().spm_time_ffn_kernel(ctx, first_layer, _ptr(x_norm), _ptr(ids), _ptr(w), ids.shape[0], int(chained),
+                                      C.byref(us), C.byref(win)), ctx)
+    return us.value, win.value
+
+
+def spm_set_device_wait_limit_us(ctx, us):
+    _check(load().spm_set_device_wait_limit_us(ctx, us), ctx)
+
+
+def spm_test_withhold_arrivals(ctx, count):
+    _check(load().spm_test_withhold_arrivals(ctx, count), ctx)
 
 
 def spm_cache_reset(ctx):

@@ -16,6 +16,16 @@
 // registers, are summed across warps in a fixed order through shared memory, and each CTA
 // writes one partial row; ffn_reduce_kernel adds the partials in CTA order (deterministic, so
 // outputs are bitwise reproducible for a given launch geometry).
+//
+// Arithmetic of a row: the 24 shared-memory reads of a lane are issued ahead of the math that
+// consumes them; products run as packed fp32 pairs (fma.rn.f32x2: even / odd elements of a 16-byte
+// vector accumulate side by side, two pair accumulators per dot product), silu uses the fast
+// exponential and division (relative error about 1e-6, far inside the parity tolerance).
+//
+// Launched with the programmatic-serialisation attribute and `early` set (slot numbers known to
+// the host), a CTA starts its first weight copies before griddepcontrol.wait, i.e. while the
+// preceding kernel of the stream is still running: weights never depend on that kernel, only the
+// router input and the routing weights do, and those are read after the wait.
 #pragma once
 
 #include "ptx.cuh"
@@ -25,7 +35,7 @@ namespace spm {
 
 constexpr int kFfnMaxWarps = 9;                    // 9 * 32 threads * 216 registers fit one SM
 constexpr int kFfnMaxThreads = kFfnMaxWarps * 32;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s: give up, set status, return
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // default limit of every device-side wait (2 s): give up, set status, return
 
 // kernel status bits (device int, read by the host)
 constexpr int kStatusCopyTimeout = 1;
@@ -48,10 +58,13 @@ struct FfnArgs {
     short watch[SPM_MAX_TOPK];      //   (the counter of the slot that leads the batch of copies entry k's slot was filled by)
     unsigned long long blob_bytes;
     int I, K, n_slots, n_shared;
+    unsigned long long wait_limit_ns;   // every wait in the kernel gives up after this long (0: the 2 s default)
+    int early;                      // 1: start the first weight copies before the launch dependency resolves (needs slot numbers in `code`)
     unsigned char count[MAXNB];                     // expert entries of token t in this launch
     short code[MAXNB * SPM_MAX_TOPK];               // >= 0: slot number; < 0: shared expert -1-s
     unsigned char kidx[MAXNB * SPM_MAX_TOPK];       // column of w[t][.]; 255: weight 1
 
+    __device__ __forceinline__ unsigned long long limit() const { return wait_limit_ns ? wait_limit_ns : kWaitLimitNs; }
     __device__ __forceinline__ int entries(int tok) const { return dev_code ? K + n_shared : int(count[tok]); }
     // slot code of entry `ent`; kBadCode when the device-side table names no slot
     __device__ __forceinline__ int code_of(int tok, int ent) const {
@@ -66,21 +79,52 @@ struct FfnArgs {
     }
 };
 
+// packed fp32 pairs (one 64-bit register pair) for fma.rn.f32x2
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ uint64_t pack2u(uint32_t lo, uint32_t hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+// 16 bytes of weights -> fp32 pairs {element 2i, element 2i + 1}
+__device__ __forceinline__ void unpack16p(const uint4& v, uint64_t (&f)[4]) {   // bf16: 8 values
+    f[0] = pack2u(v.x << 16, v.x & 0xffff0000u); f[1] = pack2u(v.y << 16, v.y & 0xffff0000u);
+    f[2] = pack2u(v.z << 16, v.z & 0xffff0000u); f[3] = pack2u(v.w << 16, v.w & 0xffff0000u);
+}
+__device__ __forceinline__ void unpack16p(const uint4& v, uint64_t (&f)[2]) {   // fp32: 4 values
+    f[0] = pack2u(v.x, v.y); f[1] = pack2u(v.z, v.w);
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
 template <typename WT, int NSEG, int MAXNB>
 __global__ void __launch_bounds__(kFfnMaxThreads, 1)
 ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
     constexpr int VEC = 16 / int(sizeof(WT));
     constexpr int D = NSEG * 32 * VEC;
     constexpr uint32_t ROWB = 3u * D * sizeof(WT);
+    constexpr uint32_t PART = D * sizeof(WT);      // bytes of one matrix's part of a blob row
 
     extern __shared__ __align__(128) unsigned char smem[];
-#ifdef SPM_FFN_TIMESTAMPS
-    const unsigned long long ts_start = global_timer_ns();
-    unsigned long long ts_first = 0, ts_loop = 0;
-#endif
     grid_dep_launch();
     const unsigned long long t_entry = (a.clock && threadIdx.x == 0) ? global_timer_ns() : 0ull;
     const int wi = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const unsigned long long wait_limit = a.limit();
     const int nw = blockDim.x >> 5;      // warps per CTA, chosen by the host to balance rows per warp
     const int tok = blockIdx.y;
     const int G = gridDim.x, c = blockIdx.x;
@@ -101,10 +145,12 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
         fence_barrier_init();
     }
     __syncwarp();
-    // everything above is independent of the preceding kernel; routing results are read below
-    grid_dep_wait();
+    // Everything above is independent of the preceding kernel. Routing results are read below; with
+    // `early` the first weight copies go out before the dependency wait (weights never depend on it).
+    const bool early = a.early && !a.dev_code;
+    if (!early) grid_dep_wait();
     // window start: kernel entry, or the end of the dependency wait when launched ahead of its predecessor's end
-    if (a.clock && threadIdx.x == 0) atomicMin(a.clock, a.dev_code ? global_timer_ns() : t_entry);
+    if (a.clock && threadIdx.x == 0 && !early) atomicMin(a.clock, a.dev_code ? global_timer_ns() : t_entry);
 
     const uint64_t pol = policy_evict_first();
     bool ok = true;
@@ -131,7 +177,7 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
                 asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(f) : "memory");
                 if (int(v - want) >= 0) break;
                 __nanosleep(200);
-                if (global_timer_ns() - t0 > kWaitLimitNs) { atomicOr(a.status, kStatusCopyTimeout); return nullptr; }
+                if (global_timer_ns() - t0 > wait_limit) { atomicOr(a.status, kStatusCopyTimeout); return nullptr; }
             }
             asm volatile("fence.proxy.async;" ::: "memory");   // the weights are read through the async proxy
         }
@@ -151,28 +197,36 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
         return true;
     };
 
-    int n_issued = 0;
-    if (lane == 0) {
-        for (; n_issued < depth && n_issued < my_n; ++n_issued)
-            if (!issue(n_issued)) { ok = false; break; }
-    }
-
-    // router input of this token, laid out like one 16-byte weight vector per lane and segment
+    // router input of this token, laid out like one 16-byte weight vector per lane and segment; its
+    // loads go out ahead of the weight copies so that they do not queue behind them
     float xr[NSEG][VEC];
-    float ya[NSEG][VEC];
-    {
+    uint64_t ya[NSEG][VEC / 2];        // partial y, packed pairs
+    auto load_x = [&]() {
         const float* xt = a.x + size_t(tok) * D;
 #pragma unroll
-        for (int s = 0; s < NSEG; ++s) {
+        for (int s = 0; s < NSEG; ++s)
 #pragma unroll
             for (int v = 0; v < VEC; v += 4) {
                 const float4 t = *reinterpret_cast<const float4*>(xt + s * 32 * VEC + lane * VEC + v);
                 xr[s][v] = t.x; xr[s][v + 1] = t.y; xr[s][v + 2] = t.z; xr[s][v + 3] = t.w;
             }
-#pragma unroll
-            for (int v = 0; v < VEC; ++v) ya[s][v] = 0.f;
-        }
+    };
+    if (!early) load_x();
+    int n_issued = 0;
+    if (lane == 0) {
+        for (; n_issued < depth && n_issued < my_n; ++n_issued)
+            if (!issue(n_issued)) { ok = false; break; }
     }
+    if (early) {
+        grid_dep_wait();
+        if (a.clock && threadIdx.x == 0) atomicMin(a.clock, global_timer_ns());
+        load_x();
+    }
+#pragma unroll
+    for (int s = 0; s < NSEG; ++s)
+#pragma unroll
+        for (int v = 0; v < VEC / 2; ++v) ya[s][v] = 0ull;
+
     ok = __shfl_sync(0xffffffffu, ok, 0);
 
     int cur_ent = -1;
@@ -185,15 +239,12 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
             if (i >= __shfl_sync(0xffffffffu, n_issued, 0)) break;
             const int st = i % depth;
             // warp-uniform outcome: a lane that gave up makes the whole warp give up
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar0 + 8u * st, (i / depth) & 1, kWaitLimitNs))) {
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar0 + 8u * st, (i / depth) & 1, wait_limit))) {
                 if (lane == 0) atomicOr(a.status, kStatusCopyTimeout);
                 ok = false;
                 break;
             }
             done = i + 1;
-#ifdef SPM_FFN_TIMESTAMPS
-            if (i == 0) ts_first = global_timer_ns();
-#endif
             const int r = r_begin + wi + i * nw;
             const int ent = r / I;
             if (ent != cur_ent) {
@@ -201,31 +252,42 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
                 const int kk = a.kidx_of(tok, ent);
                 wk = kk == 255 ? 1.f : a.w[size_t(tok) * a.K + kk];
             }
-            const unsigned char* buf = ring + size_t(st) * ROWB;
-            float pg = 0.f, pu = 0.f;
+            // gate / up rows first (16 reads), then the down row's reads go out ahead of the reductions
+            const uint32_t b32 = ring0 + uint32_t(st) * ROWB + lane * 16;
+            uint4 vg[NSEG], vu[NSEG];
+#pragma unroll
+            for (int s = 0; s < NSEG; ++s) { vg[s] = lds128(b32 + s * 512); vu[s] = lds128(b32 + PART + s * 512); }
+            uint64_t ag[2] = {0ull, 0ull}, au[2] = {0ull, 0ull};
 #pragma unroll
             for (int s = 0; s < NSEG; ++s) {
-                const uint4 vg = *reinterpret_cast<const uint4*>(buf + (s * 32 + lane) * 16);
-                const uint4 vu = *reinterpret_cast<const uint4*>(buf + D * sizeof(WT) + (s * 32 + lane) * 16);
-                float fg[VEC], fu[VEC];
-                unpack16(vg, fg);
-                unpack16(vu, fu);
+                uint64_t fg[VEC / 2], fu[VEC / 2];
+                unpack16p(vg[s], fg);
+                unpack16p(vu[s], fu);
 #pragma unroll
-                for (int v = 0; v < VEC; ++v) {
-                    pg = fmaf(fg[v], xr[s][v], pg);
-                    pu = fmaf(fu[v], xr[s][v], pu);
+                for (int v = 0; v < VEC / 2; ++v) {
+                    const uint64_t xp = pack2(xr[s][2 * v], xr[s][2 * v + 1]);
+                    ag[v & 1] = fma2(fg[v], xp, ag[v & 1]);
+                    au[v & 1] = fma2(fu[v], xp, au[v & 1]);
                 }
             }
+            uint4 vd[NSEG];
+#pragma unroll
+            for (int s = 0; s < NSEG; ++s) vd[s] = lds128(b32 + 2 * PART + s * 512);
+            float a0, a1, a2, a3;
+            unpack2(ag[0], a0, a1); unpack2(ag[1], a2, a3);
+            float pg = (a0 + a1) + (a2 + a3);
+            unpack2(au[0], a0, a1); unpack2(au[1], a2, a3);
+            float pu = (a0 + a1) + (a2 + a3);
             pg = warp_sum(pg);
             pu = warp_sum(pu);
-            const float act = pg / (1.f + expf(-pg)) * pu * wk;
+            const float act = __fdividef(pg, 1.f + __expf(-pg)) * pu * wk;
+            const uint64_t ap = pack2(act, act);
 #pragma unroll
             for (int s = 0; s < NSEG; ++s) {
-                const uint4 vd = *reinterpret_cast<const uint4*>(buf + 2 * D * sizeof(WT) + (s * 32 + lane) * 16);
-                float fd[VEC];
-                unpack16(vd, fd);
+                uint64_t fd[VEC / 2];
+                unpack16p(vd[s], fd);
 #pragma unroll
-                for (int v = 0; v < VEC; ++v) ya[s][v] = fmaf(act, fd[v], ya[s][v]);
+                for (int v = 0; v < VEC / 2; ++v) ya[s][v] = fma2(ap, fd[v], ya[s][v]);
             }
             __syncwarp();   // every lane is done with this buffer before it is refilled
             if (lane == 0 && n_issued < my_n && !halt) {
@@ -238,41 +300,43 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
         // leave no copy in flight into shared memory that is about to be released
         n_issued = __shfl_sync(0xffffffffu, n_issued, 0);
         for (int i = done; i < n_issued; ++i)
-            if (!mbar_wait_bounded(bar0 + 8u * (i % depth), (i / depth) & 1, kWaitLimitNs)) break;
+            if (!mbar_wait_bounded(bar0 + 8u * (i % depth), (i / depth) & 1, wait_limit)) break;
     }
 
-#ifdef SPM_FFN_TIMESTAMPS
-    ts_loop = global_timer_ns();
-#endif
-    // sum the warps' partial y in warp order, one partial row per CTA
+    // Sum the warps' partial y in warp order, one partial row per CTA. Staged as float4s, one per
+    // (segment, quad, lane), so that stores and loads of a warp are contiguous; a thread has the
+    // values of all warps in flight at once and adds them in warp order.
     __syncthreads();
-    float* red = reinterpret_cast<float*>(smem);
+    constexpr int Q = VEC / 4;                  // float4s per lane and segment
+    constexpr int NP = D / 4;                   // float4 positions of a row
+    float4* red4 = reinterpret_cast<float4*>(smem);
 #pragma unroll
     for (int s = 0; s < NSEG; ++s)
 #pragma unroll
-        for (int v = 0; v < VEC; v += 4)
-            *reinterpret_cast<float4*>(red + wi * D + s * 32 * VEC + lane * VEC + v) =
-                make_float4(ya[s][v], ya[s][v + 1], ya[s][v + 2], ya[s][v + 3]);
+        for (int h = 0; h < Q; ++h) {
+            float4 t;
+            unpack2(ya[s][2 * h], t.x, t.y);
+            unpack2(ya[s][2 * h + 1], t.z, t.w);
+            red4[wi * NP + s * (32 * Q) + h * 32 + lane] = t;
+        }
     __syncthreads();
     float* out = a.partial + (size_t(tok) * G + c) * D;
-    for (int d = threadIdx.x; d < D; d += blockDim.x) {
-        float acc = red[d];
-        for (int w2 = 1; w2 < nw; ++w2) acc += red[w2 * D + d];
-        out[d] = acc;
+    for (int p = threadIdx.x; p < NP; p += blockDim.x) {
+        float4 v[kFfnMaxWarps];
+#pragma unroll
+        for (int w2 = 0; w2 < kFfnMaxWarps; ++w2)
+            if (w2 < nw) v[w2] = red4[w2 * NP + p];
+        float4 acc = v[0];
+#pragma unroll
+        for (int w2 = 1; w2 < kFfnMaxWarps; ++w2)
+            if (w2 < nw) { acc.x += v[w2].x; acc.y += v[w2].y; acc.z += v[w2].z; acc.w += v[w2].w; }
+        const int s = p / (32 * Q), h = (p / 32) % Q, ln = p % 32;
+        *reinterpret_cast<float4*>(out + s * 32 * VEC + ln * VEC + 4 * h) = acc;
     }
     if (a.clock) {
         __syncthreads();
         if (threadIdx.x == 0) atomicMax(a.clock + 1, global_timer_ns());
     }
-#ifdef SPM_FFN_TIMESTAMPS
-    // profiling aid: per-warp phase times and the SM id, appended behind the partial rows
-    if (lane == 0) {
-        unsigned long long* ts = reinterpret_cast<unsigned long long*>(a.partial + size_t(gridDim.y) * G * D) + (size_t(c) * nw + wi) * 5;
-        unsigned smid;
-        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-        ts[0] = ts_start; ts[1] = ts_first; ts[2] = ts_loop; ts[3] = global_timer_ns(); ts[4] = smid;
-    }
-#endif
 }
 
 // h_out[t][d] = h_in[t][d] + sum over CTAs (in CTA order) of partial[t][c][d].

@@ -123,7 +123,7 @@ ffn_gemv_q4_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth, co
         for (int i = 0; i < my_n; ++i) {
             if (i >= __shfl_sync(0xffffffffu, n_issued, 0)) break;
             const int st = i % depth;
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar0 + 8u * st, (i / depth) & 1, kWaitLimitNs))) {
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar0 + 8u * st, (i / depth) & 1, a.limit()))) {
                 if (lane == 0) atomicOr(a.status, kStatusCopyTimeout);
                 ok = false;
                 break;
@@ -196,7 +196,7 @@ ffn_gemv_q4_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth, co
     if (!ok) {
         n_issued = __shfl_sync(0xffffffffu, n_issued, 0);
         for (int i = done; i < n_issued; ++i)
-            if (!mbar_wait_bounded(bar0 + 8u * (i % depth), (i / depth) & 1, kWaitLimitNs)) break;
+            if (!mbar_wait_bounded(bar0 + 8u * (i % depth), (i / depth) & 1, a.limit())) break;
     }
 
     // sum the warps' partial y in warp order, one partial row per CTA

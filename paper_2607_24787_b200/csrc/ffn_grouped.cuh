@@ -59,6 +59,7 @@ struct GgArgs {
     int rows_cap;
     int D, I;
     int* status;
+    unsigned long long wait_limit_ns;   // pipeline waits give up after this long (0: the 2 s default)
 };
 
 // ---- tcgen05 / TMA wrappers ---------------------------------------------------
@@ -144,6 +145,7 @@ __device__ __forceinline__ uint32_t gg_token_rows(int box) { return 16u << box; 
 struct GgAbort {
     volatile int* flag;     // shared: set by the first wait that gives up
     int* status;
+    unsigned long long limit_ns;
 };
 
 // bounded wait that also leaves when another role of the CTA has given up
@@ -155,7 +157,7 @@ __device__ __forceinline__ bool gg_wait(uint32_t bar, uint32_t parity, const GgA
         for (int i = 0; i < 32; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*ab.flag) return false;
-        if (global_timer_ns() - t0 > 2000000000ull) {
+        if (global_timer_ns() - t0 > ab.limit_ns) {
             *ab.flag = 1;
             atomicOr(ab.status, kStatusGroupedTimeout);
             return false;
@@ -188,7 +190,7 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
     const int D = a.D;
     const int n_kb = D / kGgKBlock;            // phase-1 stages per unit
     const int n_dt = D / kGgTileRows;          // phase-2 stages per unit
-    GgAbort ab{abort_flag, a.status};
+    GgAbort ab{abort_flag, a.status, a.wait_limit_ns ? a.wait_limit_ns : kWaitLimitNs};
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kGgStages; ++s) { mbar_init(smem_u32(full + s), 1); mbar_init(smem_u32(empty + s), 1); }

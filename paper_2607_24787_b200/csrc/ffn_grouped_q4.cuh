@@ -148,7 +148,7 @@ ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_co
     const int D = a.D;
     const int n_kb = D / kGgKBlock;
     const int n_dt = D / kGgTileRows;
-    GgAbort ab{abort_flag, a.status};
+    GgAbort ab{abort_flag, a.status, a.wait_limit_ns ? a.wait_limit_ns : kWaitLimitNs};
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kQgPackedStages; ++s) { mbar_init(smem_u32(qfull + s), 1); mbar_init(smem_u32(qempty + s), kQgDequantWarps); }

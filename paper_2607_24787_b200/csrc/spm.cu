@@ -109,6 +109,8 @@ struct spm_ctx {
     int stub_us = 0;                          // attention stand-in before each layer's router
     int copy_delay_us = 0;                    // emulated slower storage tier: extra wait after every expert copy
     bool device_wait = false;                 // batch-1 FFN launched at once, waits for its copies on the device
+    unsigned long long wait_limit_ns = 0;     // limit of every device-side wait in the expert kernels (0: their 2 s default)
+    int withhold_arrivals = 0;                // test hook: this many arrival-counter bumps are skipped (a wait then runs out)
     unsigned* ws_slot_gen = nullptr;          // [L][S] arrival counters, bumped by the copy stream
     std::vector<uint32_t> slot_gen_host;      // arrival counter of a slot as a batch leader: batches it has led so far
     std::vector<uint32_t> slot_want;          // counter value of its batch leader at which a slot's latest copy has landed
@@ -533,7 +535,9 @@ int issue_copy(spm_ctx* c, int layer, int e, int slot, size_t lead, bool last_of
             // stream-ordered bump of the lead slot's arrival counter, for launches that wait on the device
             StreamWriteValue32Fn wr = stream_write32_fn();
             if (!wr) return fail(c, SPM_ERR_CUDA, "cuStreamWriteValue32 is not available");
-            if (wr(reinterpret_cast<CUstream>(c->copy), reinterpret_cast<CUdeviceptr>(c->ws_slot_gen + lead), c->slot_gen_host[lead] + 1, 0) != CUDA_SUCCESS)
+            if (c->withhold_arrivals > 0) {
+                --c->withhold_arrivals;        // host-side fault injection: the bytes land, the counter never says so
+            } else if (wr(reinterpret_cast<CUstream>(c->copy), reinterpret_cast<CUdeviceptr>(c->ws_slot_gen + lead), c->slot_gen_host[lead] + 1, 0) != CUDA_SUCCESS)
                 return fail(c, SPM_ERR_CUDA, "cuStreamWriteValue32 failed");
         }
         ++c->slot_gen_host[lead];        // every slot of the batch was given this value as its target below
@@ -658,7 +662,7 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
     CU(c, cudaGetLastError());
     if (t && first) CU(c, cudaEventRecord(t->ffn_start[layer], c->compute));
     if (ring >= 0 && first) CU(c, cudaEventRecord(c->ring_start[ring], c->compute));
-    GgArgs a{reinterpret_cast<const GgUnit*>(dd), n_units, nullptr, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status};
+    GgArgs a{reinterpret_cast<const GgUnit*>(dd), n_units, nullptr, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status, c->wait_limit_ns};
     if (m.dtype == SPM_DTYPE_Q4)
         ffn_grouped_q4_kernel<<<std::min(c->num_sms, n_units), kQgThreads, ffn_grouped_q4_smem(), c->compute>>>(
             c->qmapn, c->qmapsc, c->xmaps, a);
@@ -762,6 +766,8 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
             a.status = c->ws_status;
             a.clock = clock_slot;
             a.ready = dev_wait ? c->ws_slot_gen + size_t(layer) * c->S : nullptr;
+            a.wait_limit_ns = c->wait_limit_ns;
+            a.early = 1;               // slot numbers are launch arguments: the first weight copies need not wait for the preceding kernel
             a.blob_bytes = c->blob;
             a.I = m.inter; a.K = K; a.n_slots = c->S; a.n_shared = m.n_shared;
             for (int tk = 0; tk < nb; ++tk) {
@@ -795,11 +801,11 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
             if (nb == 1) {
                 FfnArgs<1> a{};
                 fill(a);
-                CU(c, launch_gemv<1>(c, a, G, nb));
+                CU(c, launch_gemv<1>(c, a, G, nb, true));
             } else {
                 FfnArgs<SPM_MAX_BATCH> a{};
                 fill(a);
-                CU(c, launch_gemv<SPM_MAX_BATCH>(c, a, G, nb));
+                CU(c, launch_gemv<SPM_MAX_BATCH>(c, a, G, nb, true));
             }
             if (t && last) CU(c, cudaEventRecord(t->ffn_end[layer], c->compute));
             if (ring >= 0 && last) { CU(c, cudaEventRecord(c->ring_end[ring], c->compute)); c->ring_used[ring] = 1; }
@@ -809,9 +815,8 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
             } else {
                 unsigned long long* reduce_clock = nullptr;
                 if (int rc = take_clock(c, kClkReduce, &reduce_clock)) return rc;
-                ffn_reduce_kernel<<<dim3((m.hidden + kReduceCols - 1) / kReduceCols, nb), kReduceCols * kReduceGroups, 0, c->compute>>>(
-                    c->ws_partial, h_inout, h_inout, G, m.hidden, reduce_clock);
-                CU(c, cudaGetLastError());
+                CU(c, launch_k(ffn_reduce_kernel, dim3((m.hidden + kReduceCols - 1) / kReduceCols, nb), dim3(kReduceCols * kReduceGroups), 0,
+                               c->compute, true, (const float*)c->ws_partial, (const float*)h_inout, h_inout, G, m.hidden, reduce_clock));
                 c->kernel_launches += 2;
             }
             c->ffn_launches++;
@@ -1032,6 +1037,7 @@ int enqueue_host_free_layers(spm_ctx* c, int nb, float* h_out, int slot, bool pr
             a.status = c->ws_status;
             a.clock = clock_slot;
             a.ready = nullptr;
+            a.wait_limit_ns = c->wait_limit_ns;
             a.dev_code = codes;
             a.blob_bytes = c->blob;
             a.I = m.inter; a.K = K; a.n_slots = c->S; a.n_shared = m.n_shared;
@@ -1049,7 +1055,7 @@ int enqueue_host_free_layers(spm_ctx* c, int nb, float* h_out, int slot, bool pr
             CU(c, launch_k(gg_gather_kernel, dim3(nb * K), dim3(128), 0, c->compute, true, (const float*)c->ws_x, (const float*)c->ws_w,
                            (const GgRow*)rows, 0, (const int*)(c->tc_counts + 1), m.hidden, K, c->tc_xs, c->tc_wrow,
                            m.dtype == SPM_DTYPE_Q4 ? 1 : 0));
-            GgArgs ga{units, 0, c->tc_counts, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status};
+            GgArgs ga{units, 0, c->tc_counts, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status, c->wait_limit_ns};
             if (m.dtype == SPM_DTYPE_Q4)
                 CU(c, launch_k(ffn_grouped_q4_kernel, dim3(c->num_sms), dim3(kQgThreads), ffn_grouped_q4_smem(), c->compute, true,
                                c->qmapn, c->qmapsc, c->xmaps, ga));
@@ -1561,6 +1567,17 @@ int spm_set_deadline_ms(spm_ctx* c, int ms) {
     return SPM_OK;
 }
 
+int spm_set_device_wait_limit_us(spm_ctx* c, int us) {
+    if (!c || us < 0) return SPM_ERR_INVALID_ARG;
+    c->wait_limit_ns = uint64_t(us) * 1000ull;
+    return SPM_OK;
+}
+int spm_test_withhold_arrivals(spm_ctx* c, int count) {
+    if (!c || count < 0) return SPM_ERR_INVALID_ARG;
+    c->withhold_arrivals = count;
+    return SPM_OK;
+}
+
 int spm_synchronize(spm_ctx* c) {
     if (!c) return SPM_ERR_INVALID_ARG;
     if (int rc = flush_trace(c)) return rc;
@@ -1605,6 +1622,11 @@ int spm_cache_reset(spm_ctx* c) {
     if (int rc = arm_clock(c)) return rc;
     c->window_us = c->router_window_us = c->reduce_window_us = c->gap_us = 0;
     std::fill(c->slot_pending.begin(), c->slot_pending.end(), 0);
+    // arrival counters start over (both streams are idle): a counter bump lost to fault injection is forgotten here
+    std::fill(c->slot_gen_host.begin(), c->slot_gen_host.end(), 0u);
+    std::fill(c->slot_want.begin(), c->slot_want.end(), 0u);
+    CU(c, cudaMemset(c->ws_slot_gen, 0, c->slot_gen_host.size() * sizeof(uint32_t)));
+    c->withhold_arrivals = 0;
     std::fill(c->has_plan.begin(), c->has_plan.end(), 0);
     std::fill(c->layer_stall_us.begin(), c->layer_stall_us.end(), 0.0);
     std::fill(c->layer_ffn_us.begin(), c->layer_ffn_us.end(), 0.0);
@@ -1748,6 +1770,78 @@ int spm_measure_read_bandwidth(spm_ctx* c, size_t bytes, int reps, double* gb_s)
     cudaEventDestroy(e1);
     *gb_s = best;
     return SPM_OK;
+}
+
+int spm_time_ffn_kernel(spm_ctx* c, int first_layer, const float* x_norm, const int32_t* ids, const float* w, int launches,
+                        int chained, double* us_per_launch, double* window_us) {
+    if (int rc = check_layer(c, first_layer, 1)) return rc;
+    if (!x_norm || !ids || !w || !us_per_launch || launches < 1) return fail(c, SPM_ERR_INVALID_ARG, "bad argument");
+    if (int rc = flush_trace(c)) return rc;
+    const spm_model_cfg& m = c->cfg;
+    const int K = m.top_k, L = m.n_layers;
+    SlotTable& tb = *c->table;
+    for (int i = 0; i < launches; ++i)
+        for (int k = 0; k < K; ++k) {
+            const int e = ids[size_t(i) * K + k];
+            if (e < 0 || e >= m.n_experts) return fail(c, SPM_ERR_INVALID_ARG, "expert id %d out of range", e);
+            if (tb.slot_of((first_layer + i) % L, e) < 0)
+                return fail(c, SPM_ERR_NOT_RESIDENT, "expert %d of layer %d holds no slot: this probe loads nothing", e, (first_layer + i) % L);
+        }
+    CU(c, cudaStreamSynchronize(c->copy));          // every transfer issued so far has landed
+    std::fill(c->slot_pending.begin(), c->slot_pending.end(), 0);
+    const bool clocks = window_us != nullptr;
+    if (clocks) { CU(c, cudaStreamSynchronize(c->compute)); if (int rc = arm_clock(c)) return rc; }
+    const int G = ffn_grid_for(c, 1);
+    cudaEvent_t e0, e1;
+    CU(c, cudaEventCreate(&e0));
+    CU(c, cudaEventCreate(&e1));
+    int rc = SPM_OK;
+    cudaError_t ce = cudaEventRecord(e0, c->compute);
+    for (int i = 0; i < launches && ce == cudaSuccess; ++i) {
+        const int layer = (first_layer + i) % L;
+        FfnArgs<1> a{};
+        a.pool = slot_ptr(c, layer, 0);
+        a.shared = m.n_shared ? static_cast<const unsigned char*>(c->buf.shared_experts) + size_t(layer) * m.n_shared * c->blob : nullptr;
+        a.x = x_norm;
+        a.w = w;
+        a.partial = c->ws_partial;
+        a.status = c->ws_status;
+        a.clock = clocks && i < kClockSlots ? c->ws_clock + 2 * size_t(i) : nullptr;
+        a.wait_limit_ns = c->wait_limit_ns;
+        a.early = chained ? 1 : 0;
+        a.blob_bytes = c->blob;
+        a.I = m.inter; a.K = K; a.n_slots = c->S; a.n_shared = m.n_shared;
+        int cnt = 0;
+        for (int k = 0; k < K; ++k) {
+            a.code[cnt] = short(tb.slot_of(layer, ids[size_t(i) * K + k]));
+            a.kidx[cnt++] = (unsigned char)k;
+        }
+        for (int sh = 0; sh < m.n_shared; ++sh) { a.code[cnt] = short(-1 - sh); a.kidx[cnt++] = 255; }
+        a.count[0] = (unsigned char)cnt;
+        ce = launch_gemv<1>(c, a, G, 1, chained != 0);
+    }
+    if (ce == cudaSuccess) ce = cudaEventRecord(e1, c->compute);
+    if (ce == cudaSuccess) ce = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    if (ce == cudaSuccess) ce = cudaEventElapsedTime(&ms, e0, e1);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (ce != cudaSuccess) return fail(c, SPM_ERR_CUDA, "expert kernel probe: %s", cudaGetErrorString(ce));
+    c->kernel_launches += launches;
+    *us_per_launch = double(ms) * 1e3 / launches;
+    if (clocks) {
+        const int n = std::min(launches, kClockSlots);
+        std::vector<unsigned long long> h(size_t(n) * 2);
+        CU(c, cudaMemcpy(h.data(), c->ws_clock, h.size() * 8, cudaMemcpyDeviceToHost));
+        double sum = 0;
+        int got = 0;
+        for (int i = 0; i < n; ++i)
+            if (h[2 * i + 1] > h[2 * i]) { sum += double(h[2 * i + 1] - h[2 * i]) * 1e-3; ++got; }
+        *window_us = got ? sum / got : 0.0;
+        rc = arm_clock(c);
+    }
+    if (rc) return rc;
+    return check_status(c);
 }
 
 int spm_get_stats(spm_ctx* c, spm_stats* out) {

@@ -158,6 +158,9 @@ class OffloadedMoE:
     def set_copy_delay_us(self, us): B.spm_set_copy_delay_us(self.ctx, us)
     def profile_window(self): return B.spm_profile_window(self.ctx)
     def measure_read_bandwidth(self, nbytes, reps=5): return B.spm_measure_read_bandwidth(self.ctx, nbytes, reps)
+    def time_ffn_kernel(self, first_layer, x_norm, ids, w, chained=True): return B.spm_time_ffn_kernel(self.ctx, first_layer, x_norm, ids, w, chained)
+    def set_device_wait_limit_us(self, us): B.spm_set_device_wait_limit_us(self.ctx, us)
+    def test_withhold_arrivals(self, count): B.spm_test_withhold_arrivals(self.ctx, count)
     def cache_reset(self): B.spm_cache_reset(self.ctx)
     def check_invariants(self, with_device=True): B.spm_check_invariants(self.ctx, with_device)
     def cache_export(self): return B.spm_cache_export(self.ctx)
