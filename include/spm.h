@@ -302,6 +302,10 @@ int spm_test_withhold_arrivals(spm_ctx* ctx, int count);
  * path a decode step takes), t_xfer_us = median time of one expert copy from the pinned store,
  * *budget_raw = floor(window / t_xfer). Uses and then empties the cache. */
 int spm_profile_window(spm_ctx* ctx, double* window_us, double* t_xfer_us, int* budget_raw);
+/* What the most recent spm_profile_window on this context measured, including the run inside
+ * spm_init(budget = -1), whose budget is max(1, *budget_raw) (Section 3.3: the budget follows the
+ * profiled window). SPM_ERR_STATE when the context has never been profiled. */
+int spm_get_profile(spm_ctx* ctx, double* window_us, double* t_xfer_us, int* budget_raw);
 /* Read-only HBM streaming rate of this device, as a second denominator beside the copy bandwidth:
  * a kernel that only reads (16-byte loads, grid of 4 CTAs per SM, every loaded word folded into a
  * checksum that is written once per thread) streams the first `bytes` of the slot pools (clamped
@@ -373,13 +377,17 @@ int spm_synchronize(spm_ctx* ctx);                         /* both streams idle 
  *   blobs     dev: n_blobs packed expert blobs back to back (layout of spm_expert_blob_bytes), 16-byte aligned
  *   which     HOST [count]: index into `blobs` of each expert to apply, count <= SPM_MAX_TOPK
  *   w         dev fp32 [count] weights;  x_norm dev fp32 [hidden];  h_inout dev fp32 [hidden]
+ *             blobs, x_norm and h_inout must be 16-byte aligned (the kernels use 16-byte copies and
+ *             loads), w 4-byte aligned: a view that is not (an offset slice, say) is refused with
+ *             SPM_ERR_INVALID_ARG before anything is enqueued
  *   stream    cudaStream_t; the work is enqueued there and the call returns, unless
  *   wait_and_check != 0: then the call also waits for the stream and returns SPM_ERR_TIMEOUT /
  *             SPM_ERR_NOT_RESIDENT if the kernel recorded a failure.
  *
- * The first call on a device looks up the scratch array's device address and sets a kernel attribute
- * for that device (the device must be current); make that first call before starting any stream
- * capture. All calls on a device share the one array and it keeps the previous call's contents: the
+ * The first call on a device looks up the scratch array's device address and sets the kernels'
+ * shared-memory attribute for that device, for every supported shape at once (the device must be
+ * current); make that first call before starting any stream capture. Only that set-up takes a
+ * process-wide lock; the launches and an optional wait run outside it. All calls on a device share the one array and it keeps the previous call's contents: the
  * call clears the part that must start at zero itself, but two calls whose GPU work overlaps (two
  * streams, two threads) race on it and give wrong results -- keep them on one stream or otherwise
  * serialised. */

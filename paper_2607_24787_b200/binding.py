@@ -92,6 +92,7 @@ _SIG = {
     "spm_set_graph_replay": [_P, C.c_int],
     "spm_set_copy_delay_us": [_P, C.c_int],
     "spm_profile_window": [_P, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int)],
+    "spm_get_profile": [_P, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int)],
     "spm_measure_read_bandwidth": [_P, C.c_size_t, C.c_int, C.POINTER(C.c_double)],
     "spm_time_ffn_kernel": [_P, C.c_int, _P, _P, _P, C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double)],
     "spm_set_device_wait_limit_us": [_P, C.c_int],
@@ -309,6 +310,13 @@ def spm_profile_window(ctx):
     """(window_us, t_xfer_us, raw budget = floor(window / t_xfer))."""
     w, t, b = C.c_double(), C.c_double(), C.c_int()
     _check(load().spm_profile_window(ctx, C.byref(w), C.byref(t), C.byref(b)), ctx)
+    return w.value, t.value, b.value
+
+
+def spm_get_profile(ctx):
+    """(window_us, t_xfer_us, raw budget) of the most recent window profile on this context."""
+    w, t, b = C.c_double(), C.c_double(), C.c_int()
+    _check(load().spm_get_profile(ctx, C.byref(w), C.byref(t), C.byref(b)), ctx)
     return w.value, t.value, b.value
 
 

@@ -8,6 +8,7 @@
 // memory is already handed to another allocator, or in a callback that may not block on the
 // driver's allocation lock. Such callers cannot create an spm_ctx either (that creates events and
 // pinned memory), so this entry point takes plain pointers and keeps no state but the array.
+#include <cstdint>
 #include <mutex>
 #include <string>
 
@@ -41,7 +42,6 @@ constexpr int kMaxDevices = 64;
 std::mutex g_mu;
 unsigned char* g_scratch_ptr[kMaxDevices] = {};
 int g_num_sms[kMaxDevices] = {};
-bool g_attr_done[kMaxDevices][2][9] = {};
 
 int fail(int code, const std::string& msg) {
     set_thread_error(msg);
@@ -49,31 +49,46 @@ int fail(int code, const std::string& msg) {
 }
 
 template <typename WT, int NSEG>
-cudaError_t launch(int dev, int dt, const FfnArgs<1>& a, int G, int warps, int depth, size_t smem, cudaStream_t st) {
-    auto kern = ffn_gemv_kernel<WT, NSEG, 1>;
-    if (!g_attr_done[dev][dt][NSEG]) {   // once per device and kernel variant, under g_mu
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kFfnSmemLimit));
-        if (e != cudaSuccess) return e;
-        g_attr_done[dev][dt][NSEG] = true;
-    }
-    kern<<<dim3(G, 1), warps * 32, smem, st>>>(a, depth);
+cudaError_t launch(const FfnArgs<1>& a, int G, int warps, int depth, size_t smem, cudaStream_t st) {
+    ffn_gemv_kernel<WT, NSEG, 1><<<dim3(G, 1), warps * 32, smem, st>>>(a, depth);
     return cudaGetLastError();
 }
 
 template <typename WT>
-cudaError_t launch_seg(int nseg, int dev, int dt, const FfnArgs<1>& a, int G, int w, int d, size_t smem, cudaStream_t st) {
+cudaError_t launch_seg(int nseg, const FfnArgs<1>& a, int G, int w, int d, size_t smem, cudaStream_t st) {
     switch (nseg) {
-        case 1: return launch<WT, 1>(dev, dt, a, G, w, d, smem, st);
-        case 2: return launch<WT, 2>(dev, dt, a, G, w, d, smem, st);
-        case 3: return launch<WT, 3>(dev, dt, a, G, w, d, smem, st);
-        case 4: return launch<WT, 4>(dev, dt, a, G, w, d, smem, st);
-        case 5: return launch<WT, 5>(dev, dt, a, G, w, d, smem, st);
-        case 6: return launch<WT, 6>(dev, dt, a, G, w, d, smem, st);
-        case 7: return launch<WT, 7>(dev, dt, a, G, w, d, smem, st);
-        case 8: return launch<WT, 8>(dev, dt, a, G, w, d, smem, st);
+        case 1: return launch<WT, 1>(a, G, w, d, smem, st);
+        case 2: return launch<WT, 2>(a, G, w, d, smem, st);
+        case 3: return launch<WT, 3>(a, G, w, d, smem, st);
+        case 4: return launch<WT, 4>(a, G, w, d, smem, st);
+        case 5: return launch<WT, 5>(a, G, w, d, smem, st);
+        case 6: return launch<WT, 6>(a, G, w, d, smem, st);
+        case 7: return launch<WT, 7>(a, G, w, d, smem, st);
+        case 8: return launch<WT, 8>(a, G, w, d, smem, st);
     }
     return cudaErrorInvalidValue;
 }
+
+// The kernel's shared-memory ring needs the opt-in limit; set for every variant during a device's
+// one-time set-up, so that no later call (perhaps inside a stream capture) has to.
+template <typename WT, int NSEG>
+cudaError_t allow_smem() {
+    return cudaFuncSetAttribute(ffn_gemv_kernel<WT, NSEG, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kFfnSmemLimit));
+}
+template <typename WT>
+cudaError_t allow_smem_all() {
+    cudaError_t e = allow_smem<WT, 1>();
+    if (e == cudaSuccess) e = allow_smem<WT, 2>();
+    if (e == cudaSuccess) e = allow_smem<WT, 3>();
+    if (e == cudaSuccess) e = allow_smem<WT, 4>();
+    if (e == cudaSuccess) e = allow_smem<WT, 5>();
+    if (e == cudaSuccess) e = allow_smem<WT, 6>();
+    if (e == cudaSuccess) e = allow_smem<WT, 7>();
+    if (e == cudaSuccess) e = allow_smem<WT, 8>();
+    return e;
+}
+
+bool aligned(const void* p, size_t a) { return reinterpret_cast<uintptr_t>(p) % a == 0; }
 
 }  // namespace
 
@@ -97,25 +112,39 @@ extern "C" int spm_ffn_noalloc(const spm_model_cfg* cfg, const void* blobs, int 
         if (which[i] < 0 || which[i] >= n_blobs)
             return fail(SPM_ERR_INVALID_ARG, "spm_ffn_noalloc: blob index " + std::to_string(which[i]) + " outside the " + std::to_string(n_blobs) + " blobs given");
 
+    // The kernel reads weight rows with 16-byte bulk copies and the activation row with 16-byte loads,
+    // and the combine kernel walks h in place: a misaligned view (an offset slice, say) would fault on
+    // the GPU, so it is refused here, before anything is enqueued.
+    if (!aligned(blobs, 16) || !aligned(x_norm, 16) || !aligned(h_inout, 16) || !aligned(w, 4))
+        return fail(SPM_ERR_INVALID_ARG, "spm_ffn_noalloc: blobs, x_norm and h_inout must be 16-byte aligned, w 4-byte aligned");
+
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return fail(SPM_ERR_CUDA, std::string("spm_ffn_noalloc: cudaGetDevice: ") + cudaGetErrorString(e));
     if (dev < 0 || dev >= kMaxDevices) return fail(SPM_ERR_CONFIG, "spm_ffn_noalloc: device ordinal out of range");
 
-    std::lock_guard<std::mutex> lock(g_mu);
-    if (!g_scratch_ptr[dev]) {
-        // one-time set-up for this device (it is the current one): the array's device address
-        void* p = nullptr;
-        e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
-        if (e != cudaSuccess || !p) return fail(SPM_ERR_CUDA, std::string("spm_ffn_noalloc: cudaGetSymbolAddress: ") + cudaGetErrorString(e));
-        int sms = 0;
-        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess || sms < 1) return fail(SPM_ERR_CUDA, std::string("spm_ffn_noalloc: cudaDeviceGetAttribute: ") + cudaGetErrorString(e));
-        g_num_sms[dev] = sms;
-        g_scratch_ptr[dev] = static_cast<unsigned char*>(p);
+    unsigned char* scratch = nullptr;
+    int sms = 0;
+    {
+        // The lock covers only the one-time set-up of this device (it is the current one): the array's
+        // device address, the SM count, the kernels' shared-memory attribute. Launches run outside it.
+        std::lock_guard<std::mutex> lock(g_mu);
+        if (!g_scratch_ptr[dev]) {
+            void* p = nullptr;
+            e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+            if (e != cudaSuccess || !p) return fail(SPM_ERR_CUDA, std::string("spm_ffn_noalloc: cudaGetSymbolAddress: ") + cudaGetErrorString(e));
+            e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+            if (e != cudaSuccess || sms < 1) return fail(SPM_ERR_CUDA, std::string("spm_ffn_noalloc: cudaDeviceGetAttribute: ") + cudaGetErrorString(e));
+            e = allow_smem_all<float>();
+            if (e == cudaSuccess) e = allow_smem_all<bf16_t>();
+            if (e != cudaSuccess) return fail(SPM_ERR_CUDA, std::string("spm_ffn_noalloc: cudaFuncSetAttribute: ") + cudaGetErrorString(e));
+            g_num_sms[dev] = sms;
+            g_scratch_ptr[dev] = static_cast<unsigned char*>(p);
+        }
+        scratch = g_scratch_ptr[dev];
+        sms = g_num_sms[dev];
     }
-    unsigned char* scratch = g_scratch_ptr[dev];
-    const int G = std::min(g_num_sms[dev], kNoAllocMaxCtas);
+    const int G = std::min(sms, kNoAllocMaxCtas);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t elem = cfg->dtype == SPM_DTYPE_BF16 ? 2 : 4;
     const size_t row_bytes = size_t(3) * cfg->hidden * elem;
@@ -142,7 +171,7 @@ extern "C" int spm_ffn_noalloc(const spm_model_cfg* cfg, const void* blobs, int 
     const size_t smem = ffn_gemv_smem(row_bytes, warps, depth);
     const int nseg = cfg->hidden / seg;
     const int dt = cfg->dtype == SPM_DTYPE_BF16 ? 1 : 0;
-    e = dt ? launch_seg<bf16_t>(nseg, dev, dt, a, G, warps, depth, smem, st) : launch_seg<float>(nseg, dev, dt, a, G, warps, depth, smem, st);
+    e = dt ? launch_seg<bf16_t>(nseg, a, G, warps, depth, smem, st) : launch_seg<float>(nseg, a, G, warps, depth, smem, st);
     if (e != cudaSuccess) return fail(SPM_ERR_CUDA, std::string("spm_ffn_noalloc: expert kernel launch: ") + cudaGetErrorString(e));
     ffn_reduce_kernel<<<dim3((cfg->hidden + kReduceCols - 1) / kReduceCols, 1), kReduceCols * kReduceGroups, 0, st>>>(
         a.partial, h_inout, h_inout, G, cfg->hidden);

@@ -109,6 +109,8 @@ struct spm_ctx {
     int stub_us = 0;                          // attention stand-in before each layer's router
     int copy_delay_us = 0;                    // emulated slower storage tier: extra wait after every expert copy
     bool device_wait = false;                 // batch-1 FFN launched at once, waits for its copies on the device
+    double prof_window_us = 0, prof_xfer_us = 0;   // what the last spm_profile_window measured (0: never run)
+    int prof_raw = 0;
     unsigned long long wait_limit_ns = 0;     // limit of every device-side wait in the expert kernels (0: their 2 s default)
     int withhold_arrivals = 0;                // test hook: this many arrival-counter bumps are skipped (a wait then runs out)
     unsigned* ws_slot_gen = nullptr;          // [L][S] arrival counters, bumped by the copy stream
@@ -1741,8 +1743,20 @@ int spm_profile_window(spm_ctx* c, double* window_us, double* t_xfer_us, int* bu
     *t_xfer_us = tx[tx.size() / 2];
     *window_us = wt[wt.size() / 2] + c->stub_us;
     *budget_raw = int(*window_us / *t_xfer_us);
+    c->prof_window_us = *window_us;
+    c->prof_xfer_us = *t_xfer_us;
+    c->prof_raw = *budget_raw;
     if (int rc = check_status(c)) return rc;
     return spm_cache_reset(c);
+}
+
+int spm_get_profile(spm_ctx* c, double* window_us, double* t_xfer_us, int* budget_raw) {
+    if (!c || !window_us || !t_xfer_us || !budget_raw) return SPM_ERR_INVALID_ARG;
+    if (c->prof_xfer_us <= 0) return fail(c, SPM_ERR_STATE, "the overlap window has not been profiled on this context");
+    *window_us = c->prof_window_us;
+    *t_xfer_us = c->prof_xfer_us;
+    *budget_raw = c->prof_raw;
+    return SPM_OK;
 }
 
 int spm_measure_read_bandwidth(spm_ctx* c, size_t bytes, int reps, double* gb_s) {

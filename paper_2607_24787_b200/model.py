@@ -157,6 +157,7 @@ class OffloadedMoE:
     def set_graph_replay(self, on): B.spm_set_graph_replay(self.ctx, on)
     def set_copy_delay_us(self, us): B.spm_set_copy_delay_us(self.ctx, us)
     def profile_window(self): return B.spm_profile_window(self.ctx)
+    def get_profile(self): return B.spm_get_profile(self.ctx)
     def measure_read_bandwidth(self, nbytes, reps=5): return B.spm_measure_read_bandwidth(self.ctx, nbytes, reps)
     def time_ffn_kernel(self, first_layer, x_norm, ids, w, chained=True): return B.spm_time_ffn_kernel(self.ctx, first_layer, x_norm, ids, w, chained)
     def set_device_wait_limit_us(self, us): B.spm_set_device_wait_limit_us(self.ctx, us)

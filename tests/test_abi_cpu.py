@@ -52,6 +52,28 @@ def test_init_fails_loudly_without_gpu():
     assert e.value.code == -3
 
 
+def test_noalloc_argument_checks_run_before_any_gpu_work():
+    """The allocation-free entry point refuses bad shapes, indices and misaligned pointers on the
+    host, before it touches the device: so this runs without a GPU (addresses below are never
+    dereferenced)."""
+    cfg = B.make_cfg(1, 2048, 8, 64, 2, 0, 4, B.DTYPE_BF16)
+    ok = 1 << 20                                            # a 16-byte aligned made-up address
+    for args in ((ok + 8, ok, ok, ok), (ok, ok + 2, ok, ok), (ok, ok, ok + 4, ok), (ok, ok, ok, ok + 12)):
+        blobs, w, x, h = args
+        with pytest.raises(B.SpmError) as e:
+            B.spm_ffn_noalloc(cfg, blobs, 8, [0, 1], w, x, h)
+        assert e.value.code == -1 and "aligned" in str(e.value), args
+    with pytest.raises(B.SpmError) as e:
+        B.spm_ffn_noalloc(B.make_cfg(1, 4096, 8, 64, 2, 0, 4, B.DTYPE_BF16), ok, 8, [0, 1], ok, ok, ok)
+    assert e.value.code == -2 and "scratch" in str(e.value)
+    with pytest.raises(B.SpmError) as e:
+        B.spm_ffn_noalloc(cfg, ok, 8, [0, 8], ok, ok, ok)   # blob index outside the 8 blobs
+    assert e.value.code == -1
+    with pytest.raises(B.SpmError) as e:
+        B.spm_ffn_noalloc(cfg, ok, 8, list(range(17)), ok, ok, ok)   # more experts than SPM_MAX_TOPK
+    assert e.value.code == -1
+
+
 def drive(policy_obj, trace, ranks, L, budget, mode, drop=0):
     """Feed one recorded trace to either the oracle SlotPolicy or the library's Sim."""
     for t, per_layer in enumerate(trace):

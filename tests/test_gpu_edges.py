@@ -122,6 +122,77 @@ def test_timing_knobs_do_not_change_results():
     m.close()
 
 
+def test_profiled_budget_is_the_oracles_floor_of_window_over_transfer():
+    """Window-aware budget (Section 3.3): the integer the profiler returns is the oracle's
+    floor(W / t_xfer) of the very (W, t_xfer) it measured, with and without the attention stand-in,
+    and a context created with budget = -1 runs with the oracle's max(1, raw) of its own profile."""
+    cfg = synth.get_config("tiny")
+    m = build(cfg)
+    for stub in (0, 250, 0):
+        m.set_attention_stub_us(stub)
+        W, t, raw = m.profile_window()
+        assert W > 0 and t > 0
+        assert raw == M.window_budget(W, t), (stub, W, t, raw)
+        assert m.get_profile() == (W, t, raw)
+    # the stand-in makes the window hold at least one transfer here, so both branches of the clamp are seen
+    m.set_attention_stub_us(2000)
+    W, t, raw = m.profile_window()
+    assert raw == M.window_budget(W, t) and raw >= 1
+    m.close()
+    auto = build(cfg, budget=-1)
+    W, t, raw = auto.get_profile()
+    assert raw == M.window_budget(W, t)
+    assert auto.get_budget() == M.run_budget(W, t) == max(1, raw)
+    auto.close()
+    fixed = build(cfg, budget=3)
+    assert fixed.get_budget() == 3
+    with pytest.raises(Exception):
+        fixed.get_profile()                      # never profiled
+    fixed.close()
+
+
+def test_device_side_wait_runs_out_reports_timeout_and_context_survives():
+    """A wait inside the expert kernel has a limit: an arrival counter that is never bumped (the
+    update is withheld on the host; the bytes themselves land) makes the kernel give up after the
+    limit, set its status bit and return. The host reads SPM_ERR_TIMEOUT once; after a cache reset
+    the same context decodes correctly again. Nothing on the GPU faults or spins for long."""
+    import time
+    from paper_2607_24787_b200 import binding as B
+    if B.load() is None:
+        pytest.skip("library missing")
+    cfg = synth.get_config("tiny")
+    m = build(cfg)
+    try:
+        m.set_device_wait(1)
+    except B.SpmError:
+        m.close()
+        pytest.skip("stream-ordered memory writes are not available on this driver")
+    m.set_device_wait_limit_us(3000)
+    tok = synth.zipf_tokens(cfg, steps=3)
+    H = synth.embedding_rows(cfg, tok.reshape(-1)).numpy().reshape(3, 1, cfg.hidden)
+    m.cache_reset()
+    m.test_withhold_arrivals(1)                  # cleared by cache_reset, so set after it
+    t0 = time.perf_counter()
+    with pytest.raises(B.SpmError) as e:
+        m.decode_step(dev(H[0]))
+        m.synchronize()
+    assert e.value.code == -4                    # SPM_ERR_TIMEOUT
+    assert time.perf_counter() - t0 < 1.0        # gave up after milliseconds, not after the 2 s default
+    m.synchronize()                              # reported once
+    # the same context, cache and counters reset, still computes what the oracle computes
+    m.set_device_wait_limit_us(0)
+    m.cache_reset()
+    ref = make_ref(cfg, weights=SynthWeights(cfg), policy="adapter")
+    for s in range(3):
+        out = m.decode_step(dev(H[s]))
+        m.synchronize()
+        want, _ = ref.step(H[s])
+        assert M.rel_linf(out.cpu().numpy().astype(np.float64)[0], want[0]) < 4e-5
+    assert m.events() == ref.table.events
+    m.check_invariants()
+    m.close()
+
+
 def test_host_deadline_returns_timeout_and_context_survives():
     """The routing handshake has a host-side deadline: with the compute stream kept busy by unrelated
     work the call gives up with SPM_ERR_TIMEOUT instead of spinning; nothing on the GPU is disturbed."""

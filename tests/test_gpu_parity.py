@@ -172,6 +172,52 @@ def fragile(recs, K, budget):
     return flags
 
 
+def oracle_cache_words(tbl):
+    """The oracle's slot tables in the word layout of spm_cache_export / spm_cache_import:
+    tick, step, then (expert, tick, origin, used) per slot, layer-major."""
+    words = [tbl.tick, tbl.step]
+    for p in tbl.pools:
+        for sl in range(tbl.S):
+            words += [p.slot_expert[sl], p.slot_tick[sl], p.slot_origin[sl], p.slot_used[sl]]
+    return np.asarray(words, np.int64)
+
+
+def free_run_lockstep(cfg, m, wts, H, steps, policy, budget, hint):
+    """Free-running parity, step by step (level P3): outputs within tolerance and the step's cache
+    events bit-exact, except where the oracle's own decisions of that step sit on a near-tie at or
+    before the layer where the logs part. There either answer is valid, so the divergence is
+    counted, the GPU's cache is re-seeded from the oracle's state after that step, and the run goes
+    on. Returns (oracle, records, divergences, flagged decisions)."""
+    ref = make_ref(cfg, weights=wts, policy=policy, budget=budget)
+    m.cache_reset()
+    m.set_policy(policy)
+    m.set_budget(budget)
+    if policy == "hint_trace":
+        m.set_hint_trace(hint)
+    recs, divergences, n_ref_ev, n_gpu_ev = [], 0, 0, 0
+    for s in range(steps):
+        want, r = ref.step(H[s:s + 1], hint=None if hint is None else hint[s])
+        recs.append(r)
+        ref_ev = ref.table.events[n_ref_ev:]
+        n_ref_ev = len(ref.table.events)
+        out = host(m.decode_step(dev(H[s:s + 1])), m)
+        all_ev = m.events()
+        gpu_ev = all_ev[n_gpu_ev:]
+        n_gpu_ev = len(all_ev)
+        if gpu_ev == ref_ev:
+            assert M.rel_linf(out, want) < 4 * TOL[cfg.dtype], s      # error accumulates over L layers
+            continue
+        first = next((i for i, (x, y) in enumerate(zip(gpu_ev, ref_ev)) if x != y), min(len(gpu_ev), len(ref_ev)))
+        l_bad = (ref_ev[first] if first < len(ref_ev) else gpu_ev[first])[1]
+        flagged_here = [l for (fs, l) in fragile([r], cfg.top_k, budget) if l <= l_bad]
+        assert flagged_here, ("events differ without a near-tie in the oracle", s, first, gpu_ev[first:first + 2], ref_ev[first:first + 2])
+        divergences += 1
+        m.cache_import(oracle_cache_words(ref.table))     # clears the GPU's log and counters
+        ref.prev_rank = [[] for _ in range(cfg.n_layers)]  # ... and its memory of the preceding step (Naive Prefetch): same on both sides
+        n_gpu_ev = 0
+    return ref, recs, divergences, fragile(recs, cfg.top_k, budget)
+
+
 @pytest.mark.parametrize("policy", ["adapter", "on_demand", "pred0", "hint_trace", "naive"])
 def test_decode_step_free_running(setup, policy):
     cfg, m, wts, H = setup
@@ -179,23 +225,11 @@ def test_decode_step_free_running(setup, policy):
     budget = cfg.budget if cfg.budget >= 0 else 2
     _, base_out, base_recs = run_ref(cfg, wts, H, steps, slots=cfg.n_experts, policy=P.ON_DEMAND, budget=budget)
     hint = ref_decode.true_demand_trace(base_recs)
-    ref, out_r, recs = run_ref(cfg, wts, H, steps, policy=policy, budget=budget, hint=hint)
-    m.cache_reset()
-    m.set_policy(policy)
-    m.set_budget(budget)
-    if policy == "hint_trace":
-        m.set_hint_trace(hint)
-    out = run_gpu(m, H, steps)
-    for s in range(steps):
-        assert M.rel_linf(out[s], out_r[s]) < 4 * TOL[cfg.dtype], s      # error accumulates over L layers
-    ev = m.events()
-    if ev != ref.table.events:
-        # only acceptable when the oracle itself sits on a near-tie somewhere before the divergence
-        first = next(i for i, (a, b) in enumerate(zip(ev, ref.table.events)) if a != b)
-        s_bad, l_bad = ref.table.events[first][0], ref.table.events[first][1]
-        fl = fragile(recs, cfg.top_k, budget)
-        assert any(fs < s_bad or (fs == s_bad and fl_ <= l_bad) for fs, fl_ in fl), (first, ev[first], ref.table.events[first])
-        pytest.xfail("near-tie in the oracle's own decisions")
+    ref, recs, divergences, flagged = free_run_lockstep(cfg, m, wts, H, steps, policy, budget, hint)
+    assert divergences <= len(flagged)
+    if divergences:
+        return          # the counters below were restarted by the re-seed; decisions were checked step by step
+    assert m.events() == ref.table.events
     st = m.stats()
     for k in ("hits", "hits_prefetched", "misses", "evictions", "wasted", "prefetch_issued", "touches", "planned"):
         assert st[k] == getattr(ref.table.stats, k), k
@@ -209,6 +243,27 @@ def test_decode_step_free_running(setup, policy):
             assert abs(st["recall_at"][j] / st["recall_count"] - rj) < 1e-9, Mj
     rdy = np.mean([recs[s][l].ready for s in range(steps) for l in range(1, cfg.n_layers)])
     assert abs(st["ready_sum"] / st["ready_count"] - rdy) < 1e-9
+
+
+def test_reseeding_the_gpu_cache_from_the_oracle_keeps_parity(setup):
+    """The recovery step of the lock-step protocol itself: half-way through a run the GPU's slot
+    tables are overwritten with the ORACLE's state (not its own export); the rest of the run must
+    give the oracle's events and outputs."""
+    cfg, m, wts, H = setup
+    steps, half, budget = 8, 4, 2
+    ref = make_ref(cfg, weights=wts, policy="adapter", budget=budget)
+    m.cache_reset(); m.set_policy("adapter"); m.set_budget(budget)
+    for s in range(half):
+        ref.step(H[s:s + 1])
+    n_ref_ev = len(ref.table.events)
+    m.cache_import(oracle_cache_words(ref.table))          # a cold GPU cache takes over the oracle's warm one
+    for s in range(half, steps):
+        want, _ = ref.step(H[s:s + 1])
+        out = host(m.decode_step(dev(H[s:s + 1])), m)
+        assert M.rel_linf(out, want) < 4 * TOL[cfg.dtype], s
+    assert m.events() == ref.table.events[n_ref_ev:]
+    assert [list(m.slot_table(l)) for l in range(cfg.n_layers)] == [list(ref.table.pools[l].slot_expert) for l in range(cfg.n_layers)]
+    m.check_invariants()
 
 
 def test_router_preserving_bitwise_on_gpu(setup):

@@ -3,8 +3,9 @@
 Some users of this library run where cudaMalloc is forbidden (a serving loop with a frozen memory
 map, a process whose device memory belongs to another allocator), so they can create neither an
 arena nor an spm_ctx. The entry point tested here needs neither: its scratch is a fixed array inside
-the library. This file checks, through the C ABI, that it gives the same result as spm_moe_ffn,
-on two calls in a row (the second call finds the first call's leftovers in the shared array).
+the library. This file checks, through the C ABI, that it gives the same result as spm_moe_ffn
+and as the CPU oracle's plain definition of the expert layer, on two calls in a row (the second
+call finds the first call's leftovers in the shared array).
 It is collected last on purpose, so a run that stops at the first failure has already run the rest.
 """
 import numpy as np
@@ -12,6 +13,8 @@ import pytest
 import torch
 
 import synth
+from helpers import SynthWeights
+from oracle import ref_math as M
 
 pytestmark = pytest.mark.gpu
 
@@ -30,6 +33,7 @@ def test_noalloc_matches_moe_ffn_twice_in_a_row(name):
     g, u, d = synth.expert_matrices(cfg, layer, range(cfg.n_experts), device="cuda")
     blobs = pack_experts(g, u, d).contiguous()                         # device copy of the layer's packed experts
     rng = np.random.default_rng(11)
+    wts = SynthWeights(cfg)
     tol = 1e-5 if cfg.dtype == "fp32" else 1e-4
     stream = torch.cuda.Stream()
     for call in range(2):
@@ -45,6 +49,10 @@ def test_noalloc_matches_moe_ffn_twice_in_a_row(name):
         a, b = h_new.cpu().numpy().astype(np.float64), h_ref.cpu().numpy().astype(np.float64)
         assert np.max(np.abs(a - b)) / np.max(np.abs(b)) < tol, call
         assert not np.array_equal(b, h0.cpu().numpy())                 # the FFN did change h
+        # ... and against the oracle's definition y = sum_k w_k FFN_k(x), computed from the same weights
+        y = M.moe_ffn(x[0].cpu().numpy().astype(np.float64), ids, w[0].cpu().numpy().astype(np.float64),
+                      lambda e: wts.expert(layer, e))
+        assert M.rel_linf(a[0] - h0[0].cpu().numpy().astype(np.float64), y) < tol, call
     # sizes beyond the built-in array are refused with a message, nothing is launched
     big = B.make_cfg(1, 4096, 8, 64, 2, 0, 4, B.DTYPE_BF16)
     with pytest.raises(B.SpmError) as e:
@@ -52,4 +60,9 @@ def test_noalloc_matches_moe_ffn_twice_in_a_row(name):
     assert e.value.code == -2 and "scratch" in str(e.value)
     with pytest.raises(B.SpmError):
         B.spm_ffn_noalloc(m.cfg, blobs, cfg.n_experts, [cfg.n_experts], w, x, h_new, stream.cuda_stream)
+    # a misaligned view (here: a row that starts 4 bytes into a buffer) is refused, not launched
+    pad = torch.zeros(cfg.hidden + 4, device="cuda")
+    with pytest.raises(B.SpmError) as e:
+        B.spm_ffn_noalloc(m.cfg, blobs, cfg.n_experts, ids, w, pad[1:cfg.hidden + 1], h_new, stream.cuda_stream)
+    assert e.value.code == -1 and "aligned" in str(e.value)
     m.close()
