@@ -141,6 +141,7 @@ typedef struct {
     double gap_us;               /* device idle time between consecutive clocked kernels of the compute stream  */
     double recall_at[3];         /* sums like recall_sum for M = max(1, K/2), K, K+2 (the coverage levels of
                                     the paper's model-level table); divide by recall_count                    */
+    uint64_t events_dropped;     /* cache events not stored because the event log was full (spm_set_event_log_limit) */
 } spm_stats;
 
 /* ---- packed expert layout ------------------------------------------------
@@ -282,6 +283,11 @@ int spm_set_graph_replay(spm_ctx* ctx, int on);
  * stream. It widens the overlap window W_l = t_exec(l+1) - t_pred(l) (Section 3.1) toward the
  * paper's regime; spm_profile_window adds it to the window it reports. Outputs are unchanged. */
 int spm_set_attention_stub_us(spm_ctx* ctx, int us);
+/* The cache-event log (spm_get_events) keeps at most `max_events` records between two calls of
+ * spm_reset_stats / spm_cache_reset (default 1,048,576, about 20 MB of host memory; a Qwen3-shaped
+ * step logs 400 - 800 events); events beyond that are only counted, in spm_stats.events_dropped.
+ * 0 switches the log off. Counters and recall statistics do not depend on the log. */
+int spm_set_event_log_limit(spm_ctx* ctx, size_t max_events);
 /* Host deadline of the routing-kernel handshake, in milliseconds (default 5000). */
 int spm_set_deadline_ms(spm_ctx* ctx, int ms);
 /* Limit of every wait inside the expert kernels (for a weight copy to land in shared memory, for an

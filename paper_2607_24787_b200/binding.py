@@ -54,7 +54,7 @@ class Stats(C.Structure):
                 + [("ffn_us", C.c_double), ("ffn_window_us", C.c_double), ("stall_us", C.c_double), ("ready_sum", C.c_double),
                    ("ready_count", C.c_uint64), ("recall_sum", C.c_double), ("recall_count", C.c_uint64),
                    ("host_free_steps", C.c_uint64), ("router_window_us", C.c_double), ("reduce_window_us", C.c_double),
-                   ("gap_us", C.c_double), ("recall_at", C.c_double * 3)])
+                   ("gap_us", C.c_double), ("recall_at", C.c_double * 3), ("events_dropped", C.c_uint64)])
 
     def as_dict(self):
         d = {k: getattr(self, k) for k, _ in self._fields_}
@@ -96,6 +96,7 @@ _SIG = {
     "spm_measure_read_bandwidth": [_P, C.c_size_t, C.c_int, C.POINTER(C.c_double)],
     "spm_time_ffn_kernel": [_P, C.c_int, _P, _P, _P, C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double)],
     "spm_set_device_wait_limit_us": [_P, C.c_int],
+    "spm_set_event_log_limit": [_P, C.c_size_t],
     "spm_test_withhold_arrivals": [_P, C.c_int],
     "spm_cache_reset": [_P],
     "spm_reset_stats": [_P],
@@ -333,6 +334,10 @@ def spm_time_ffn_kernel(ctx, first_layer, x_norm, ids: np.ndarray, w, chained=Tr
     _check(load().spm_time_ffn_kernel(ctx, first_layer, _ptr(x_norm), _ptr(ids), _ptr(w), ids.shape[0], int(chained),
                                       C.byref(us), C.byref(win)), ctx)
     return us.value, win.value
+
+
+def spm_set_event_log_limit(ctx, max_events):
+    _check(load().spm_set_event_log_limit(ctx, max_events), ctx)
 
 
 def spm_set_device_wait_limit_us(ctx, us):

@@ -84,16 +84,8 @@ __device__ __forceinline__ bool elect_one() {
 // may begin before the preceding kernel of its stream has finished; grid_dep_wait() returns once
 // that kernel has completed and its writes are visible (at once in an ordinary launch).
 // grid_dep_launch() lets the next kernel of the stream begin its own preamble early.
-#ifndef SPM_AB_NO_WAIT
 __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-#else
-__device__ __forceinline__ void grid_dep_wait() {}
-#endif
-#ifndef SPM_AB_NO_LAUNCH
 __device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-#else
-__device__ __forceinline__ void grid_dep_launch() {}
-#endif
 
 __device__ __forceinline__ uint64_t policy_evict_first() {
     uint64_t p;

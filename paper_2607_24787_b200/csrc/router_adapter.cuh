@@ -216,13 +216,6 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
     short* smap = reinterpret_cast<short*>(part + a.D);          // [n] slot of each expert (leader)
     __shared__ int s_last;
 
-#ifdef SPM_ROUTER_TIMESTAMPS
-    unsigned long long ts[12] = {};
-    ts[0] = global_timer_ns();
-#define SPM_TS(i) ts[i] = global_timer_ns()
-#else
-#define SPM_TS(i)
-#endif
     const int tok = blockIdx.y;
     const uint32_t cr = cluster_ctarank();
     const bool leader = cr == 0;
@@ -290,7 +283,6 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
 
     // ---- router input: the hidden row (written by the preceding kernels) is normalised ----------
     grid_dep_wait();
-    SPM_TS(8);
     if (a.clock && leader && threadIdx.x == 0) atomicMin(a.clock, global_timer_ns());
     bool cluster_started = false;      // the start-of-kernel cluster barrier has been waited for
     if constexpr (MINB == 1) if (fused) {
@@ -340,9 +332,7 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
             for (uint32_t dst = 0; dst < kRouterCluster; ++dst) dsmem_store(xs + col0 + threadIdx.x, dst, hv1);
         }
         load_rows(row0);                 // L2 hits by now; in flight across the barrier and the normalisation
-        SPM_TS(9);
         cluster_sync_all();              // every CTA holds the whole updated row in xs
-        SPM_TS(10);
     }
     if (a.do_router) {
         const float* ht = fused ? xs : a.h + size_t(tok) * D;
@@ -379,7 +369,6 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
         for (int i = threadIdx.x; i < D; i += kRouterThreads) xs[i] = xt[i];
     }
     __syncthreads();
-    SPM_TS(1);
 
     if (!cluster_started) asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
     while (row0 < rows) {
@@ -416,10 +405,8 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
         row0 += ROWS * STRIDE;
         if (row0 < rows) load_rows(row0);
     }
-    SPM_TS(2);
     cluster_sync_all();
     if (!leader) return;
-    SPM_TS(3);
 
     // ---- tails (leader CTA): router on warps 0-3, adapter on warps 4-7, concurrently ----------
     Mailbox* mb = a.mailbox;
@@ -454,7 +441,6 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
             if (a.codes_out) a.codes_out[tok * a.K + ht] = smap[isel[ht]];
         }
     }
-    SPM_TS(4);
     if (half == 1 && a.do_adapter) {
         for (int e = ht; e < n; e += 128) {
             float acc = 0.f;
@@ -478,7 +464,6 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
             }
         }
     }
-    SPM_TS(5);
 
     // ---- several tokens: the last leader to finish aggregates and ranks -------------------------
     if (a.nb > 1) {
@@ -507,7 +492,6 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
         }
         if (threadIdx.x == 0) a.counters[0] = 0u;
     }
-    SPM_TS(6);
     // final flag for callers that read untagged payload (scores): fence, then the sequence number
     if (a.publish_seq) {
         __threadfence_system();
@@ -515,11 +499,6 @@ router_adapter_kernel(const __grid_constant__ RouterArgs a) {
         if (threadIdx.x == 0 && mb) mb->seq = a.seq;
     }
     if (threadIdx.x == 0 && a.clock) atomicMax(a.clock + 1, global_timer_ns());
-#ifdef SPM_ROUTER_TIMESTAMPS
-    SPM_TS(7);
-    if (threadIdx.x == 0 || threadIdx.x == 128)
-        for (int i = 0; i < 12; ++i) reinterpret_cast<unsigned long long*>(a.pihat)[(threadIdx.x >> 7) * 12 + i] = ts[i];
-#endif
 }
 
 inline size_t router_smem_bytes(int D, int n, int r) {

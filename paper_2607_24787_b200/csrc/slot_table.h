@@ -54,6 +54,7 @@ public:
     int step() const { return step_; }
     void end_step() { ++step_; }
     void set_plain_lru(bool on) { plain_lru_ = on; }
+    void set_event_cap(size_t cap) { event_cap_ = cap; }
     int slot_of(int layer, int e) const { return expert_slot_[size_t(layer) * n_ + e]; }
     int expert_in(int layer, int s) const { return slot_expert_[size_t(layer) * S_ + s]; }
     const std::vector<spm_event>& events() const { return events_; }
@@ -227,7 +228,10 @@ public:
     }
 
 private:
+    // The event log is bounded: once `event_cap_` records are held, further events are counted in
+    // stats().events_dropped instead of being stored (statistics are unaffected).
     void log(int layer, int kind, int expert, int slot) {
+        if (events_.size() >= event_cap_) { ++stats_.events_dropped; return; }
         events_.push_back({step_, layer, kind, expert, slot});
     }
 
@@ -270,6 +274,7 @@ private:
     std::vector<uint64_t> slot_tick_;
     std::vector<uint8_t> slot_origin_, slot_used_, mark_;
     std::vector<spm_event> events_;
+    size_t event_cap_ = size_t(1) << 20;       // records kept between two resets of the accounting
     spm_stats stats_{};
 };
 

@@ -1569,6 +1569,12 @@ int spm_set_deadline_ms(spm_ctx* c, int ms) {
     return SPM_OK;
 }
 
+int spm_set_event_log_limit(spm_ctx* c, size_t max_events) {
+    if (!c) return SPM_ERR_INVALID_ARG;
+    if (int rc = flush_trace(c)) return rc;
+    c->table->set_event_cap(max_events);
+    return SPM_OK;
+}
 int spm_set_device_wait_limit_us(spm_ctx* c, int us) {
     if (!c || us < 0) return SPM_ERR_INVALID_ARG;
     c->wait_limit_ns = uint64_t(us) * 1000ull;

@@ -160,6 +160,7 @@ class OffloadedMoE:
     def get_profile(self): return B.spm_get_profile(self.ctx)
     def measure_read_bandwidth(self, nbytes, reps=5): return B.spm_measure_read_bandwidth(self.ctx, nbytes, reps)
     def time_ffn_kernel(self, first_layer, x_norm, ids, w, chained=True): return B.spm_time_ffn_kernel(self.ctx, first_layer, x_norm, ids, w, chained)
+    def set_event_log_limit(self, n): B.spm_set_event_log_limit(self.ctx, n)
     def set_device_wait_limit_us(self, us): B.spm_set_device_wait_limit_us(self.ctx, us)
     def test_withhold_arrivals(self, count): B.spm_test_withhold_arrivals(self.ctx, count)
     def cache_reset(self): B.spm_cache_reset(self.ctx)

@@ -193,6 +193,28 @@ def test_device_side_wait_runs_out_reports_timeout_and_context_survives():
     m.close()
 
 
+def test_event_log_is_bounded_and_counters_do_not_depend_on_it():
+    cfg = synth.get_config("tiny")
+    tok = synth.zipf_tokens(cfg, steps=6)
+    H = synth.embedding_rows(cfg, tok.reshape(-1)).numpy().reshape(6, 1, cfg.hidden)
+    m = build(cfg)
+    runs = []
+    for cap in (1 << 20, 7, 0):
+        m.set_event_log_limit(cap)
+        m.cache_reset()
+        for s in range(6):
+            m.decode_step(dev(H[s]))
+        m.synchronize()
+        runs.append((m.events(), m.stats()))
+    full, st_full = runs[0]
+    assert st_full["events_dropped"] == 0 and len(full) > 7
+    for (ev, st), cap in zip(runs[1:], (7, 0)):
+        assert ev == full[:cap] and st["events_dropped"] == len(full) - cap
+        for k in ("hits", "misses", "evictions", "prefetch_issued", "wasted", "touches"):
+            assert st[k] == st_full[k], k
+    m.close()
+
+
 def test_host_deadline_returns_timeout_and_context_survives():
     """The routing handshake has a host-side deadline: with the compute stream kept busy by unrelated
     work the call gives up with SPM_ERR_TIMEOUT instead of spinning; nothing on the GPU is disturbed."""
