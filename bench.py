@@ -158,6 +158,19 @@ def affordable_store_layers(cfg, world):
     return int(max(1, min(cfg.n_layers, (0.6 * avail / max(ranks, 1)) // per_layer)))
 
 
+def workload_name(cfg):
+    return (f"{cfg.name}: L{cfg.n_layers} D{cfg.hidden} n{cfg.n_experts} I{cfg.inter} K{cfg.top_k}"
+            f"+{cfg.n_shared}sh r{cfg.adapter_rank} {cfg.dtype} slots{cfg.slots} batch{cfg.batch}")
+
+
+def config_block(cfg, args):
+    """What is run, in words both arms share (measured quantities live under `profile`)."""
+    return {"workload": workload_name(cfg), "policy": "adapter",
+            "budget_rule": "max(1, floor(window / t_xfer)) from the profiled window" if cfg.budget < 0 else f"fixed {cfg.budget}",
+            "attention_stub_us": args.stub_us, "copy_delay_us": args.copy_delay_us, "seed": cfg.seed, "token_ids": "Zipf(1.1)",
+            "l2": "inputs larger than L2: every layer streams its own slot pool, 3.6 GB of weights per step"}
+
+
 def ffn_kernel_name(cfg):
     if cfg.batch > 1 and cfg.n_shared == 0 and cfg.dtype in ("bf16", "q4"):
         return "ffn_grouped_q4_kernel" if cfg.dtype == "q4" else "ffn_grouped_kernel"
@@ -283,13 +296,9 @@ def run_ours(args):
         "value": tokens / (el_max / 1e3), "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": el_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 weights, fp32 accumulate" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": f"{cfg.name}: L{cfg.n_layers} D{cfg.hidden} n{cfg.n_experts} I{cfg.inter} K{cfg.top_k}"
-                               f"+{cfg.n_shared}sh r{cfg.adapter_rank} {cfg.dtype} slots{cfg.slots} batch{cfg.batch}",
-                   "policy": "adapter", "budget": budget, "budget_raw": raw_budget, "window_us": window_us,
-                   "t_xfer_us": t_xfer_us, "attention_stub_us": args.stub_us, "copy_delay_us": args.copy_delay_us,
-                   "host_store_layers": store_layers, "seed": cfg.seed, "token_ids": "Zipf(1.1)",
-                   "l2": "inputs larger than L2: every layer streams its own slot pool, 3.6 GB of weights per step",
-                   "setup_s": setup_s, "wall_ms_per_step": wall_ms / K},
+        "config": config_block(cfg, args),
+        "profile": {"budget": budget, "budget_raw": raw_budget, "window_us": window_us, "t_xfer_us": t_xfer_us,
+                    "host_store_layers": store_layers, "setup_s": setup_s, "wall_ms_per_step": wall_ms / K},
         "clocks": clk,
         "e2e": {"value": tokens / (e2e_max / 1e3), "unit": "tokens/s",
                 "h2d_bytes_per_step": cfg.batch * cfg.hidden * 4 + int(st["h2d_bytes"] / K),
@@ -395,6 +404,22 @@ def run_ours(args):
         except Exception as e:   # noqa: BLE001 (reported, not hidden)
             result["resident"] = {"error": str(e)[:200]}
 
+    if world == 1 and not args.no_arms and not args.no_extra and cfg.name == "qwen3":
+        # what the targets are read from: exposed transfer time of the adapter-guided arm against on-demand loading
+        # at the same slots, with the configuration's random adapters and with an informative stand-in (gate reuse)
+        try:
+            result["targets"] = targets_block(cfg, m, H_dev, W, min(K, args.arm_steps), result, device)
+        except Exception as e:   # noqa: BLE001
+            result["targets"] = {"error": str(e)[:200]}
+    if world == 1 and not args.no_extra and cfg.name == "qwen3":
+        legs = {}
+        for name, fn in (("batched", batched_leg), ("dsvl2", dsvl2_leg)):
+            try:
+                legs[name] = fn(args, m, peak, which, device)
+            except Exception as e:   # noqa: BLE001 (reported, not hidden)
+                legs[name] = {"error": str(e)[:300]}
+        result["configs"] = legs
+
     # second denominator: what a kernel that only reads reaches on this device (the copy figure pays for writes too)
     try:
         ro = m.measure_read_bandwidth(4 << 30)
@@ -407,6 +432,157 @@ def run_ours(args):
     m.close()
     if rank == 0:
         print(json.dumps(result))
+
+
+def targets_block(cfg, m, H_dev, W, n_arm, result, device):
+    """Exposed (non-overlapped) transfer time per layer: adapter arms against on-demand loading, same slots."""
+    from paper_2607_24787_b200.synth_model import build_from_synth
+    od = result["arms"]["on_demand"]
+    out = {"slots": cfg.slots, "steps_per_arm": n_arm,
+           "on_demand": {"stall_us_per_layer": od["stall_us_per_layer"], "tok_s": od["tok_s"]},
+           "adapter_random": {"stall_us_per_layer": result["main_arm"]["stall_us_per_layer"], "tok_s": result["main_arm"]["tok_s"],
+                              "expert_recall_at_budget": result["main_arm"]["expert_recall_at_budget"]},
+           "perfect_knowledge": {"stall_us_per_layer": result["arms"]["perfect_knowledge"]["stall_us_per_layer"],
+                                 "tok_s": result["arms"]["perfect_knowledge"]["tok_s"]}}
+    g = build_from_synth(cfg, budget=result["profile"]["budget"], device=device, store=m.store, adapter="gate_reuse",
+                         store_layers=m.store_layers)
+    g.set_policy("adapter"); g.set_timing(1); g.cache_reset()
+    timed_run(g, H_dev, 0, W, 1); g.reset_stats()
+    el, _, _ = timed_run(g, H_dev, W, n_arm, 1)
+    a = arm_summary(g, cfg, el, n_arm)
+    g.close()
+    out["adapter_gate_reuse"] = {"stall_us_per_layer": a["stall_us_per_layer"], "tok_s": a["tok_s"],
+                                 "expert_recall_at_budget": a["expert_recall_at_budget"], "ready_recall": a["ready_recall"]}
+    out["exposed_below_on_demand"] = {k: out[k]["stall_us_per_layer"] < od["stall_us_per_layer"]
+                                      for k in ("adapter_random", "adapter_gate_reuse", "perfect_knowledge")}
+    return out
+
+
+def leg_offloaded(m, cfg, H_dev, W, K):
+    m.set_policy("adapter"); m.set_timing(1); m.cache_reset()
+    timed_run(m, H_dev, 0, W, 1); m.reset_stats()
+    el, _, _ = timed_run(m, H_dev, W, K, 1)
+    out = arm_summary(m, cfg, el, K)
+    st = m.stats()
+    out["steps"] = K
+    out["gpu_launches"] = int(st["kernel_launches"])
+    return out, st
+
+
+def batched_leg(args, m, peak, which, device):
+    """Batched decode on the Qwen3 shape (64 sequences, 32 slots per layer), on the pinned store the main arm
+    filled: offloaded tokens/s, then the grouped tcgen05 kernel by itself at the size of one wave (the 32 experts a
+    pool holds: 302 MB) and with every expert resident (about 120 distinct experts per launch: 1.1 GB)."""
+    from paper_2607_24787_b200.synth_model import build_from_synth
+    cfg = synth.get_config("batched")
+    W, K = 3, max(2, min(args.steps, args.batched_steps))
+    mb = build_from_synth(cfg, device=device, store=m.store, store_layers=m.store_layers)     # budget -1: profiled
+    window_us, t_xfer_us, raw = mb.get_profile()
+    _, H = hidden_rows(cfg, W + K, stream=0)
+    H_dev = H.to(device)
+    torch.cuda.synchronize()
+    out = {"workload": workload_name(cfg), "profile": {"window_us": window_us, "t_xfer_us": t_xfer_us, "budget_raw": raw,
+                                                        "budget": mb.get_budget()}}
+    off, st = leg_offloaded(mb, cfg, H_dev, W, K)
+    out["offloaded"] = off
+    if st["ffn_us"] > 0:
+        # inside the offloaded run every launch is one wave; its bytes are the experts that wave computes
+        wave_bytes = (st["hits"] + st["misses"]) * cfg.expert_bytes / max(st["ffn_launches"], 1)
+        us = st["ffn_us"] / max(st["ffn_launches"], 1)
+        out["offloaded"]["ffn_wave_in_run"] = {"us_per_launch": us, "algorithmic_bytes_per_launch": wave_bytes,
+                                                "gb_s": wave_bytes / (us * 1e-6) / 1e9, "launches": int(st["ffn_launches"])}
+    # one wave by itself: the first `slots` experts of every layer resident, tokens routed among them (all hits)
+    mb.cache_reset(); mb.set_policy("on_demand")
+    S = cfg.slots
+    for l in range(cfg.n_layers):
+        mb.prefetch_async(l, np.arange(S, dtype=np.int32))
+    mb.synchronize()
+    out["roofline_wave"] = grouped_alone(cfg, mb, S, peak, which, launches=96)
+    mb.close()
+    full = build_from_synth(cfg, slots=cfg.n_experts, budget=0, device=device, store=m.store, store_layers=m.store_layers)
+    full.set_policy("on_demand")
+    for l in range(cfg.n_layers):
+        full.prefetch_async(l, np.arange(cfg.n_experts, dtype=np.int32))
+    full.synchronize()
+    out["roofline"] = grouped_alone(cfg, full, cfg.n_experts, peak, which, launches=96)
+    full.set_timing(0)
+    for _ in range(3):
+        timed_run(full, H_dev, 0, W, 1)
+    el, _, _ = timed_run(full, H_dev, W, K, 1)
+    out["resident_host_free_tok_s"] = K * cfg.batch / (el / 1e3)
+    full.close()
+    return out
+
+
+def grouped_alone(cfg, ctx, n_resident, peak, which, launches):
+    """`launches` spm_moe_ffn calls back to back, every token's K experts drawn among the first `n_resident`
+    (all resident): CUDA event pair around each grouped-kernel launch (gather and combine kernels outside it)."""
+    rng = np.random.default_rng(1)
+    nb = cfg.batch
+    x = torch.randn(nb, cfg.hidden, device=ctx.device)
+    w = torch.full((nb, cfg.top_k), 1.0 / cfg.top_k, device=ctx.device)
+    h = torch.zeros(nb, cfg.hidden, device=ctx.device)
+    ids = [np.stack([np.sort(rng.permutation(n_resident)[:cfg.top_k]) for _ in range(nb)]).astype(np.int32) for _ in range(launches)]
+    mean_bytes = float(np.mean([len(np.unique(i)) * cfg.expert_bytes for i in ids]))
+    torch.cuda.synchronize()
+    ctx.set_timing(1)
+    for i in range(8):
+        ctx.moe_ffn(i % cfg.n_layers, x, ids[i], w, h)
+    ctx.reset_stats()
+    for i in range(launches):
+        ctx.moe_ffn(i % cfg.n_layers, x, ids[i], w, h)
+    ctx.synchronize()
+    st = ctx.stats()
+    us = st["ffn_us"] / max(st["ffn_launches"], 1)
+    ach = mean_bytes / (us * 1e-6) / 1e9
+    return {"bound": "hbm", "kernel": ffn_kernel_name(cfg), "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+            "traffic": None, "peak_source": f"of {which}", "algorithmic_bytes_per_launch": mean_bytes, "us_per_launch": us,
+            "launches": int(st["ffn_launches"]), "misses": int(st["misses"]), "distinct_experts_per_launch": mean_bytes / cfg.expert_bytes,
+            "region": f"{launches} spm_moe_ffn launches back to back, {nb} tokens x top-{cfg.top_k} among {n_resident} resident "
+                      "experts per layer, pools of all layers cycled, CUDA event pair per grouped-kernel launch"}
+
+
+def dsvl2_leg(args, m, peak, which, device):
+    """DeepSeek-VL2-Tiny-shaped decode (12 layers, hidden 1280, 64 experts of intermediate 896, top-6 + 2 shared,
+    8 slots): offloaded tokens/s with its own 5.3 GB pinned store, and the GEMV expert kernel by itself."""
+    from paper_2607_24787_b200.synth_model import build_from_synth
+    cfg = synth.get_config("dsvl2")
+    W, K = 3, max(2, min(args.steps, args.dsvl2_steps))
+    md = build_from_synth(cfg, device=device)
+    window_us, t_xfer_us, raw = md.get_profile()
+    _, H = hidden_rows(cfg, W + K, stream=0)
+    H_dev = H.to(device)
+    torch.cuda.synchronize()
+    out = {"workload": workload_name(cfg), "profile": {"window_us": window_us, "t_xfer_us": t_xfer_us, "budget_raw": raw,
+                                                        "budget": md.get_budget()}}
+    out["offloaded"], _ = leg_offloaded(md, cfg, H_dev, W, K)
+    md.set_policy("on_demand"); md.cache_reset()
+    timed_run(md, H_dev, 0, W, 1); md.reset_stats()
+    el, _, _ = timed_run(md, H_dev, W, K, 1)
+    od = arm_summary(md, cfg, el, K)
+    out["on_demand"] = {"tok_s": od["tok_s"], "stall_us_per_layer": od["stall_us_per_layer"]}
+    full = build_from_synth(cfg, slots=cfg.n_experts, budget=0, device=device, store=md.store)
+    full.set_policy("on_demand")
+    for l in range(cfg.n_layers):
+        full.prefetch_async(l, np.arange(cfg.n_experts, dtype=np.int32))
+    full.synchronize()
+    algo = (cfg.top_k + cfg.n_shared) * cfg.expert_bytes
+    b2b = ffn_back_to_back(cfg, full, algo, peak, launches=240)
+    out["roofline"] = {"bound": "hbm", "kernel": b2b["kernel"], "achieved": b2b["gb_s"], "peak": peak, "unit": "GB/s",
+                       "frac": b2b["frac_of_measured_peak"], "traffic": None, "peak_source": f"of {which}",
+                       "algorithmic_bytes_per_launch": algo, "us_per_launch": b2b["kernel_us"],
+                       "us_per_launch_serialized": b2b.get("serialized_us"), "us_per_launch_event_pair_each": b2b["event_pair_each_us"],
+                       "in_kernel_window_us": b2b.get("chained_window_us"),
+                       "region": "240 launches of the kernel alone back to back (spm_time_ffn_kernel, programmatic dependent "
+                                 "launch), all experts resident, one CUDA event pair around all of them"}
+    full.set_timing(0)
+    for _ in range(3):
+        timed_run(full, H_dev, 0, W, 1)
+    el, _, _ = timed_run(full, H_dev, W, K, 1)
+    out["resident_host_free_tok_s"] = K * cfg.batch / (el / 1e3)
+    full.close()
+    md.close()
+    return out
 
 
 def h2d_probe(m, cfg):
@@ -664,12 +840,34 @@ class LazyWeights:
         return [self.expert(l, self.cfg.n_experts + s) for s in range(self.cfg.n_shared)]
 
 
-def oracle_threads():
+def host_cores():
     try:
-        from threadpoolctl import threadpool_info
-        return max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+        return len(os.sched_getaffinity(0))
     except Exception:
         return os.cpu_count() or 1
+
+
+class blas_threads:
+    """Pins the thread count of every BLAS / OpenMP pool numpy and torch use, for the duration of a block."""
+
+    def __init__(self, n):
+        self.n, self.ctx, self.torch_before = n, None, None
+
+    def __enter__(self):
+        try:
+            from threadpoolctl import threadpool_limits
+            self.ctx = threadpool_limits(limits=self.n)
+            self.ctx.__enter__()
+        except Exception:
+            self.ctx = None
+        self.torch_before = torch.get_num_threads()
+        torch.set_num_threads(self.n)
+        return self
+
+    def __exit__(self, *exc):
+        torch.set_num_threads(self.torch_before)
+        if self.ctx is not None:
+            self.ctx.__exit__(*exc)
 
 
 def make_oracle(cfg, wts, budget, slots=None, policy="adapter"):
@@ -678,31 +876,48 @@ def make_oracle(cfg, wts, budget, slots=None, policy="adapter"):
                       budget, policy=policy, renormalize=bool(cfg.renormalize), rms_eps=cfg.rms_eps, keep_records=False)
 
 
-def cpu_baseline(cfg, H, device, budget, mem_budget=40e9):
-    """The oracle, as it stands, on a bounded sample: a few decode steps of the same token stream.
+def oracle_steps(cfg, H, device, budget, threads, layers=None, mem_budget=40e9):
+    """Times the oracle, as it stands, on the decode steps H[s] with `threads` BLAS threads.
     Weights are generated before the clock starts (an untimed pass of the same step fills the
     provider's cache, which is emptied after the step). The fp64 matrices of one step stay below
     `mem_budget` bytes: a batched step touches nearly every expert of every layer, so there the
-    sample is the first Ls layers and tokens/s is scaled by Ls / n_layers."""
+    sample is the first Ls layers. Returns (seconds per step, list; layers used)."""
     per_layer = min(cfg.n_experts, cfg.batch * cfg.top_k) * 3 * cfg.inter * cfg.hidden * 8
     Ls = int(max(1, min(cfg.n_layers, mem_budget // max(per_layer, 1))))
+    if layers:
+        Ls = min(Ls, layers)
     sub = cfg.replace(n_layers=Ls) if Ls < cfg.n_layers else cfg
     wts = LazyWeights(sub, device if torch.cuda.is_available() else "cpu")
     warm = make_oracle(sub, wts, 0, slots=cfg.n_experts, policy="on_demand")
     ref = make_oracle(sub, wts, budget)
-    dt = 0.0
-    for s in range(H.shape[0]):
-        warm.step(H[s])                      # untimed: fills the weight cache for this step
-        t0 = time.perf_counter()
-        ref.step(H[s])
-        dt += time.perf_counter() - t0
-        wts.cache = {k: v for k, v in wts.cache.items() if k[0] != "e"}   # bound memory
+    times = []
+    with blas_threads(threads):
+        for s in range(H.shape[0]):
+            warm.step(H[s])                      # untimed: fills the weight cache for this step
+            t0 = time.perf_counter()
+            ref.step(H[s])
+            times.append(time.perf_counter() - t0)
+            wts.cache = {k: v for k, v in wts.cache.items() if k[0] != "e"}   # bound memory
+    return times, Ls
+
+
+def cpu_baseline(cfg, H, device, budget, repeats=3):
+    """The oracle on a bounded sample: the same few decode steps `repeats` times with every host core
+    the process may use (thread count pinned and reported), and once single-threaded."""
+    cores = host_cores()
+    runs = []
+    Ls = cfg.n_layers
+    for _ in range(repeats):
+        times, Ls = oracle_steps(cfg, H, device, budget, cores)
+        runs.append(H.shape[0] * cfg.batch * (Ls / cfg.n_layers) / sum(times))
+    one, _ = oracle_steps(cfg, H[:1], device, budget, 1)
     layers = f"all {cfg.n_layers} layers" if Ls == cfg.n_layers else \
         f"the first {Ls} of {cfg.n_layers} layers, tokens/s scaled by {Ls}/{cfg.n_layers}"
-    return {"value": H.shape[0] * cfg.batch * (Ls / cfg.n_layers) / dt, "unit": "tokens/s", "cores": oracle_threads(),
-            "kind": "oracle",
-            "sample": f"{H.shape[0]} decode steps ({layers}) of the bench token stream, "
-                      f"numpy fp64, weights pre-generated; {dt:.2f} s"}
+    return {"value": statistics.median(runs), "unit": "tokens/s", "cores": cores, "kind": "oracle",
+            "repeats": runs, "spread": (max(runs) - min(runs)) / statistics.median(runs),
+            "single_thread": {"value": cfg.batch * (Ls / cfg.n_layers) / sum(one), "cores": 1, "sample": "the first of those steps"},
+            "sample": f"{H.shape[0]} decode steps ({layers}) of the bench token stream, numpy fp64, weights pre-generated, "
+                      f"BLAS pinned to {cores} threads; median of {repeats} repeats"}
 
 
 def run_reference(args):
@@ -715,32 +930,21 @@ def run_reference(args):
     # a step = one decode step over the first Ls layers, Ls sized so the run ends within minutes
     per_layer_s = 0.05
     Ls = int(max(1, min(cfg.n_layers, 150.0 / max((K + W) * per_layer_s * 2, 1e-9))))
-    sub = cfg.replace(n_layers=Ls)
     _, H = hidden_rows(cfg, W + K, stream=0)
     H = H.numpy()
     budget = 1 if cfg.budget < 0 else cfg.budget
-    wts = LazyWeights(sub, dev)
-    warm = make_oracle(sub, wts, 0, slots=cfg.n_experts, policy="on_demand")
-    ref = make_oracle(sub, wts, budget)
-    times = []
-    for s in range(W + K):
-        warm.step(H[s])                      # untimed: fills the weight cache for this step
-        t0 = time.perf_counter()
-        ref.step(H[s])
-        times.append(time.perf_counter() - t0)
-        wts.cache = {k: v for k, v in wts.cache.items() if k[0] != "e"}   # bound memory
+    cores = host_cores()
+    times, Ls = oracle_steps(cfg, H, dev, budget, cores, layers=Ls)
     dt = sum(times[W:])
     tok_s = K * cfg.batch * (Ls / cfg.n_layers) / dt
     sample = (f"each step = one decode step over the first {Ls} of {cfg.n_layers} layers, numpy fp64 oracle, "
-              f"weights pre-generated; tokens/s scaled by {Ls}/{cfg.n_layers}")
+              f"weights pre-generated, BLAS pinned to {cores} threads; tokens/s scaled by {Ls}/{cfg.n_layers}")
     print(json.dumps({
         "impl": "reference", "metric": "decode tokens/s with offloaded experts", "value": tok_s, "unit": "tokens/s",
         "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": dt / K * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{cfg.name}: L{cfg.n_layers} D{cfg.hidden} n{cfg.n_experts} I{cfg.inter} K{cfg.top_k}"
-                               f"+{cfg.n_shared}sh r{cfg.adapter_rank} {cfg.dtype} slots{cfg.slots} batch{cfg.batch}",
-                   "policy": "adapter", "budget": budget},
-        "cpu_baseline": {"value": tok_s, "unit": "tokens/s", "cores": oracle_threads(), "kind": "oracle", "sample": sample},
+        "config": config_block(cfg, args),
+        "cpu_baseline": {"value": tok_s, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": tok_s, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }))
@@ -756,7 +960,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="reduced layer count (profiler captures only)")
     ap.add_argument("--slots", type=int, default=0, help="override slots per layer")
     ap.add_argument("--arm-steps", type=int, default=128)
-    ap.add_argument("--cpu-steps", type=int, default=6)
+    ap.add_argument("--cpu-steps", type=int, default=3)
     ap.add_argument("--sweep", action="store_true", help="budget x slots sweep (prints one JSON object with all cells)")
     ap.add_argument("--sweep-budgets", default="1,2,4,8")
     ap.add_argument("--sweep-slots", default="8,16,32")
@@ -770,6 +974,9 @@ def main():
     ap.add_argument("--no-arms", action="store_true")
     ap.add_argument("--no-resident", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extra", action="store_true", help="skip the batched / DeepSeek-shaped legs and the targets block")
+    ap.add_argument("--batched-steps", type=int, default=8)
+    ap.add_argument("--dsvl2-steps", type=int, default=64)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":

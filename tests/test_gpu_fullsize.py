@@ -138,3 +138,80 @@ def test_fully_resident_host_free_steps_give_the_offloaded_bits(qwen):
             assert np.array_equal(outs[s].cpu().numpy(), offloaded[s]), s
     finally:
         full.close()
+
+
+# ---------------------------------------------------------------- batched configuration (64 sequences, 32 slots)
+@pytest.mark.parametrize("base", ["qwen3", "qwen3_q4"])
+def test_batched_shape_tensor_core_path_teacher_forced(base):
+    """The batched configuration's per-layer shape (hidden 2048, 128 experts of intermediate 768,
+    top-8, 64 sequences, 32 slots per layer -> about 120 distinct experts per layer in waves of 32)
+    through the grouped tcgen05 kernels, two layers deep, teacher-forced: layer 1 gets the oracle's
+    layer-0 output. Expert ids bit-exact off near-ties for all 64 tokens, outputs of all tokens
+    (layer 0) and of 8 sampled tokens (layer 1) within the bf16 tolerance, cache events equal to the
+    policy oracle replayed on the GPU's own demand sets."""
+    from paper_2607_24787_b200.build import build
+    from paper_2607_24787_b200.synth_model import build_from_synth
+    from oracle import ref_policy as P
+    build()
+    nb, tol = 64, 2e-2
+    cfg = synth.get_config(base, n_layers=2, batch=nb, slots=32, budget=1)
+    free_host = int(open("/proc/meminfo").read().split("MemAvailable:")[1].split()[0]) * 1024
+    if free_host < 8 * 2 ** 30 or torch.cuda.mem_get_info()[0] < 8 * 2 ** 30:
+        pytest.skip("not enough memory for two layers of 128 experts")
+    m = build_from_synth(cfg)
+    try:
+        tok = synth.zipf_tokens(synth.get_config("batched"), steps=1)[0]          # the batched configuration's token stream
+        H0 = f64(synth.embedding_rows(cfg, tok))                                    # [64, D]
+        m.set_policy("on_demand")
+        m.cache_reset()
+        h_in = H0
+        for layer in range(2):
+            hd = torch.as_tensor(h_in, dtype=torch.float32).cuda()
+            torch.cuda.synchronize()
+            x, ids, w, logits = m.router_topk(layer, hd, want_logits=True)
+            m.moe_ffn(layer, x, ids, w, hd)
+            m.synchronize()
+            got = f64(hd)
+            # oracle routing of all 64 tokens
+            W_r = f64(synth.router_w(cfg, layer, "cuda"))
+            X = np.stack([M.rmsnorm(h_in[t], np.ones(cfg.hidden), cfg.rms_eps) for t in range(nb)])
+            Z = X @ W_r.T
+            routed = [M.route(Z[t], cfg.top_k, True) for t in range(nb)]
+            tie = [M.near_tie(Z[t], cfg.top_k) for t in range(nb)]
+            assert sum(tie) < 8                       # (a token may repeat in the batch)
+            zg = f64(logits)
+            for t in range(nb):
+                assert list(ids[t]) == list(M.top_k(zg[t].astype(np.float32), cfg.top_k))     # bit-exact given the same logits
+                if not tie[t]:
+                    assert list(ids[t]) == list(routed[t][0]), (layer, t)
+            sample = range(nb) if layer == 0 else (0, 9, 18, 27, 36, 45, 54, 63)
+            # expert by expert (each regenerated once), the oracle's dense definition for the sampled tokens
+            need = sorted({int(e) for t in sample for e in routed[t][0]})
+            Y = {t: np.zeros(cfg.hidden) for t in sample}
+            for e in need:
+                g, u, d = synth.expert_matrices(cfg, layer, [e], "cuda")
+                trip = (f64(g[0]), f64(u[0]), f64(d[0]))
+                for t in sample:
+                    ids_t, w_t = routed[t]
+                    for k in range(cfg.top_k):
+                        if int(ids_t[k]) == e:
+                            Y[t] = Y[t] + M.moe_ffn(X[t], [e], [w_t[k]], lambda _e: trip)
+            for t in sample:
+                if not tie[t]:
+                    assert M.rel_linf(got[t] - h_in[t], Y[t]) < tol, (layer, t)
+            if layer == 0:
+                h_in = np.stack([h_in[t] + Y[t] for t in range(nb)])             # teacher forcing
+        st = m.stats()
+        assert st["waves"] >= 2 and st["ffn_launches"] >= 6                       # ~120 distinct experts through 32 slots
+        ev = m.events()
+        demand = {}
+        for (s, l, kind, e, slot) in ev:
+            if kind in ("HIT", "HIT_PREFETCHED", "MISS"):
+                demand.setdefault(l, []).append(e)
+        ref = P.SlotPolicy(cfg.n_layers, cfg.n_experts, cfg.slots)
+        for l in range(2):
+            ref.demand(l, demand[l])
+        assert ev == ref.events
+        m.check_invariants()
+    finally:
+        m.close()
