@@ -408,6 +408,15 @@ int spm_ffn_noalloc(const spm_model_cfg* cfg, const void* blobs, int n_blobs, co
 int spm_host_alloc(size_t bytes, void** out);
 int spm_host_free(void* p);
 
+/* Host logic of the batched tensor-core kernel's work distribution, exposed for tests (no GPU
+ * needed). A launch has n_units units (expert x 128 intermediate rows); phase 1 of a unit runs on
+ * CTA unit % grid, phase 2 is n_dt pipeline stages (one per 128 output columns) that may be cut
+ * between d-tiles and are taken, chunk by chunk in list order, by whichever CTA is free. Writes the
+ * chunk list: chunks[3 * i] = {unit, dt0, dt1} = d-tiles dt0 .. dt1-1 of that unit; *count = number
+ * of chunks (SPM_ERR_INVALID_ARG when capacity is too small, *count still set). */
+int spm_plan_grouped_chunks(int n_units, int n_dt, int grid, int32_t* chunks, size_t capacity,
+                            size_t* count);
+
 /* ---- host-only slot-table policy (no GPU needed) ------------------------
  * The same slot table the context uses, exposed so the cache policy can be driven and checked
  * on a machine without a GPU. Arrays are host memory.                                        */

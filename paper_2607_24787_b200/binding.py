@@ -110,6 +110,7 @@ _SIG = {
     "spm_host_free": [_P],
     "spm_sim_create": [C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(_P)],
     "spm_sim_destroy": [_P],
+    "spm_plan_grouped_chunks": [C.c_int, C.c_int, C.c_int, _P, C.c_size_t, C.POINTER(C.c_size_t)],
     "spm_sim_demand": [_P, C.c_int, _P, C.c_int, _P, _P, _P, _P, C.POINTER(C.c_int), C.POINTER(C.c_int)],
     "spm_sim_plan": [_P, C.c_int, _P, C.c_int, C.c_int, C.c_int, _P, C.POINTER(C.c_int), _P, C.POINTER(C.c_int)],
     "spm_sim_prefetch": [_P, C.c_int, _P, C.c_int, _P, C.c_int, C.c_int, _P, C.POINTER(C.c_int)],
@@ -417,6 +418,15 @@ def spm_ffn_noalloc(cfg: ModelCfg, blobs, n_blobs, which, w, x_norm, h_inout, st
     which = np.ascontiguousarray(which, np.int32)
     _check(load().spm_ffn_noalloc(C.byref(cfg), _ptr(blobs), n_blobs, _ptr(which), _ptr(w), len(which),
                                   _ptr(x_norm), _ptr(h_inout), stream, int(wait_and_check)))
+
+
+def spm_plan_grouped_chunks(n_units, n_dt, grid):
+    """chunks[count][3] = unit, dt0, dt1 of the grouped tensor-core kernel's phase-2 chunk list."""
+    cap = n_units * n_dt
+    chunks = np.zeros((cap, 3), np.int32)
+    count = C.c_size_t()
+    _check(load().spm_plan_grouped_chunks(n_units, n_dt, grid, _ptr(chunks), cap, C.byref(count)))
+    return chunks[:count.value]
 
 
 def spm_host_alloc(nbytes: int) -> int:

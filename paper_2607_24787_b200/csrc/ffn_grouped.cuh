@@ -16,8 +16,22 @@
 //            accumulator [128 d x 64 tokens] per d-tile, double buffered; the epilogue writes the
 //            rows of real tokens to the partial buffer P[j-tile][token row][d].
 // A combine kernel then adds, per token, its K experts x (I/128) partial rows and the residual in
-// a fixed order. Phase 1 of the next unit is issued before phase 2 of the current one (two G^T/U^T
-// accumulator pairs), so the weight stream does not pause while the epilogue builds A^T.
+// a fixed order.
+//
+// Work is handed out as tasks, so that a launch with few units (a wave of 32 experts is 192 units
+// on 148 SMs) still keeps every SM streaming until the end: a P1 task is phase 1 of one unit, a P2
+// task ("chunk") is phase 2 of one unit for a range of d-tiles. P1 tasks are static: CTA b runs the
+// units b, b + grid, ... first. P2 chunks are then taken from one list in order through an atomic
+// counter, by whichever CTA is free: a chunk's output tiles are its own and are computed by the same
+// sequence of MMAs whoever runs it, so results do not depend on who took what. A^T travels from the
+// CTA that ran P1 to the CTA(s) that run P2 through a 16 KB slot of global memory (L2-resident)
+// guarded by a per-unit arrival counter: the P1 epilogue warps store their rows, fence, and bump the
+// counter; the P2 side's producer warp polls it (bounded), then pulls the slot into shared memory
+// with one bulk copy. Every CTA finishes its P1 tasks before it takes its first chunk, so no CTA
+// ever waits for a counter while its owner waits for it. The host cuts the chunks finer towards the
+// end of the list (gg_plan_chunks) so that all CTAs finish together; without a list a chunk is a
+// whole unit. The producer warp tells the other warps of its CTA what it took through a small queue
+// in shared memory.
 // One warp issues TMA, one thread issues tcgen05.mma, four warps run the epilogues;
 // all of them talk through mbarriers, every wait is bounded and an abort flag lets the whole CTA
 // leave together (freeing its TMEM) if a wait ever gives up. No multicast anywhere.
@@ -27,6 +41,7 @@
 #include <cuda_bf16.h>
 
 #include "ptx.cuh"
+#include "ffn_gemv.cuh"      // kWaitLimitNs, kernel status bits
 #include "../../include/spm.h"
 
 namespace spm {
@@ -50,6 +65,15 @@ struct GgUnit {
     int32_t ntok;      // tokens of this expert (1..64)
 };
 
+// One task of a CTA: phase 1 of `unit` (dt0 < 0), or phase 2 of `unit` for d-tiles dt0 .. dt1-1;
+// unit < 0 ends the list.
+struct GgTask {
+    int32_t unit;
+    int16_t dt0, dt1;
+};
+constexpr int kGgActReady = 4;           // arrivals (one per epilogue warp) that complete a unit's A^T
+constexpr int kGgQueue = 4;              // tasks the producer warp may be ahead of the other warps
+
 struct GgArgs {
     const GgUnit* units;
     int n_units;           // ... or, when n_units_dev is set, read from device memory (plan built on the device)
@@ -60,6 +84,13 @@ struct GgArgs {
     int D, I;
     int* status;
     unsigned long long wait_limit_ns;   // pipeline waits give up after this long (0: the 2 s default)
+    // bf16 kernel only: the list of P2 chunks (null: one chunk per unit), the counter they are taken with,
+    // the A^T slots and their arrival counters
+    const GgTask* chunks;
+    int n_chunks;              // (ignored without a list: the number of units)
+    int* next_chunk;           // zeroed before the launch (by the gather kernel), like act_ready
+    unsigned char* act_g;      // [units][16 KB] A^T of each unit, in the shared-memory operand layout
+    int* act_ready;            // [units]
 };
 
 // ---- tcgen05 / TMA wrappers ---------------------------------------------------
@@ -165,6 +196,23 @@ __device__ __forceinline__ bool gg_wait(uint32_t bar, uint32_t parity, const GgA
     }
 }
 
+// bounded wait for a counter in global memory (another CTA's arrivals) to reach `want`
+__device__ __forceinline__ bool gg_wait_count(const int* p, int want, const GgAbort& ab) {
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+        if (v >= want) return true;
+        if (*ab.flag) return false;
+        if (global_timer_ns() - t0 > ab.limit_ns) {
+            *ab.flag = 1;
+            atomicOr(ab.status, kStatusGroupedTimeout);
+            return false;
+        }
+        __nanosleep(100);
+    }
+}
+
 __global__ void __launch_bounds__(kGgThreads, 1)
 ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_constant__ GgTokenMaps xmaps, const GgArgs a) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -177,13 +225,16 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
     uint64_t* empty = full + kGgStages;       // [stages]  MMA -> TMA
     uint64_t* acc1_full = empty + kGgStages;  // [2] MMA -> epilogue: G^T, U^T of a unit complete
     uint64_t* acc1_empty = acc1_full + 2;     // [2] epilogue -> MMA: that pair drained
-    uint64_t* act_full = acc1_empty + 2;      // epilogue -> MMA: A^T written
-    uint64_t* act_empty = act_full + 1;       // MMA -> epilogue: phase 2 has consumed A^T
+    uint64_t* act_full = acc1_empty + 2;      // TMA -> MMA: A^T of the P2 task's unit has landed in shared memory
+    uint64_t* act_empty = act_full + 1;       // MMA -> TMA: the P2 task has consumed A^T
     uint64_t* acc2_full = act_empty + 1;      // [2] MMA -> epilogue
     uint64_t* acc2_empty = acc2_full + 2;     // [2] epilogue -> MMA
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc2_empty + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     float* wrow_all = reinterpret_cast<float*>(tmem_slot + 4);      // [4 epilogue warps][64]
+    uint64_t* q_full = reinterpret_cast<uint64_t*>(wrow_all + 4 * kGgTokens);   // [kGgQueue] producer -> MMA, epilogue warps
+    uint64_t* q_empty = q_full + kGgQueue;                                      // [kGgQueue] they -> producer
+    GgTask* queue = reinterpret_cast<GgTask*>(q_empty + kGgQueue);              // [kGgQueue]
 
     grid_dep_launch();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -200,7 +251,8 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
             mbar_init(smem_u32(acc2_full + b), 1);
             mbar_init(smem_u32(acc2_empty + b), 4);
         }
-        mbar_init(smem_u32(act_full), 4);
+        mbar_init(smem_u32(act_full), 1);        // the producer's arrival + the bytes of the A^T bulk copy
+        for (int i = 0; i < kGgQueue; ++i) { mbar_init(smem_u32(q_full + i), 1); mbar_init(smem_u32(q_empty + i), 5); }
         mbar_init(smem_u32(act_empty), 1);
         *abort_flag = 0;
         fence_barrier_init();
@@ -213,73 +265,123 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
     // barriers and TMEM are set up; everything below reads what the preceding kernels wrote
     grid_dep_wait();
     const int n_units = a.n_units_dev ? __ldcg(a.n_units_dev) : a.n_units;
+    // P1 tasks of this CTA: the units b, b + grid, ...; P2 chunks: taken from the common list.
     const int my_units = int(blockIdx.x) < n_units ? (n_units - 1 - int(blockIdx.x)) / int(gridDim.x) + 1 : 0;
+    const int n_chunks = a.chunks ? a.n_chunks : n_units;
+    // consumer side of the task queue (MMA warp and epilogue warps): next task, or unit < 0 at the end / after an abort
+    uint32_t n_got = 0;
+    auto next_task = [&]() -> GgTask {
+        const uint32_t qs = n_got % kGgQueue;
+        if (!__all_sync(0xffffffffu, gg_wait(smem_u32(q_full + qs), (n_got / kGgQueue) & 1, ab))) return GgTask{-1, 0, 0};
+        const GgTask tk = queue[qs];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(q_empty + qs));
+        ++n_got;
+        return tk;
+    };
 
-    // Order of work, identical for the producer and the MMA issuer:
-    //   phase1(0), then for i = 0, 1, ...: phase1(i + 1) if it exists, phase2(i).
-    // Phase 1 of the next unit is issued before phase 2 of the current one, so the weight stream
-    // keeps flowing while the epilogue warps turn G^T, U^T of the current unit into A^T.
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         // The producer and the MMA issuer are walked by their whole warp in uniform control flow and
         // one elected lane issues: addresses and descriptors then stay in uniform registers (issued
         // from inside a one-lane branch, each tcgen05.mma cost the issuing thread about 90 cycles).
-        {
-            uint32_t it = 0;      // ring position over all stages
-            bool ok = true;
-            auto load_phase1 = [&](int i) {
-                const GgUnit un = a.units[blockIdx.x + i * gridDim.x];
-                const int xbox = gg_token_box(un.ntok);
-                const CUtensorMap* xmap = &xmaps.m[xbox];
-                const uint32_t x_bytes = gg_token_rows(xbox) * 128;
-                for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
-                    const uint32_t s = it % kGgStages;
-                    if (it >= kGgStages) ok = __all_sync(0xffffffffu, gg_wait(smem_u32(empty + s), ((it / kGgStages) - 1) & 1, ab));
-                    if (!ok) break;
-                    const uint32_t base = smem_u32(stages + s * kGgStageBytes);
-                    const uint32_t fb = smem_u32(full + s);
-                    if (elect_one()) {
-                        mbar_arrive_expect_tx(fb, 2 * kGgTileBytes + x_bytes);
-                        tma_load_4d(base, &wmap, kb * kGgKBlock, 0, un.jt * kGgTileRows, un.slot, fb);                 // gate rows
-                        tma_load_4d(base + kGgTileBytes, &wmap, kb * kGgKBlock, 1, un.jt * kGgTileRows, un.slot, fb);  // up rows
-                        tma_load_2d(base + 2 * kGgTileBytes, xmap, kb * kGgKBlock, un.row0, fb);                      // token rows
-                    }
-                    __syncwarp();
+        uint32_t it = 0;      // ring position over all stages
+        uint32_t n_p2 = 0;    // P2 tasks started
+        uint32_t n_pub = 0;   // tasks published to the other warps
+        bool ok = true;
+        auto stage_free = [&](uint32_t s) {
+            if (it >= kGgStages) ok = __all_sync(0xffffffffu, gg_wait(smem_u32(empty + s), ((it / kGgStages) - 1) & 1, ab));
+        };
+        auto publish = [&](GgTask tk) {
+            const uint32_t qs = n_pub % kGgQueue;
+            if (n_pub >= kGgQueue) ok = __all_sync(0xffffffffu, gg_wait(smem_u32(q_empty + qs), ((n_pub / kGgQueue) - 1) & 1, ab));
+            if (ok && lane == 0) {
+                queue[qs] = tk;
+                mbar_arrive(smem_u32(q_full + qs));       // (release: the entry is visible to whoever sees the arrival)
+            }
+            __syncwarp();
+            ++n_pub;
+        };
+        // ---- P1: gate / up rows of this CTA's own units
+        for (int i = 0; i < my_units && ok; ++i) {
+            const int32_t u = int32_t(blockIdx.x + i * gridDim.x);
+            publish(GgTask{u, -1, -1});
+            if (!ok) break;
+            const GgUnit un = a.units[u];
+            const int xbox = gg_token_box(un.ntok);
+            const CUtensorMap* xmap = &xmaps.m[xbox];
+            const uint32_t x_bytes = gg_token_rows(xbox) * 128;
+            for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
+                const uint32_t s = it % kGgStages;
+                stage_free(s);
+                if (!ok) break;
+                const uint32_t base = smem_u32(stages + s * kGgStageBytes);
+                const uint32_t fb = smem_u32(full + s);
+                if (elect_one()) {
+                    mbar_arrive_expect_tx(fb, 2 * kGgTileBytes + x_bytes);
+                    tma_load_4d(base, &wmap, kb * kGgKBlock, 0, un.jt * kGgTileRows, un.slot, fb);                 // gate rows
+                    tma_load_4d(base + kGgTileBytes, &wmap, kb * kGgKBlock, 1, un.jt * kGgTileRows, un.slot, fb);  // up rows
+                    tma_load_2d(base + 2 * kGgTileBytes, xmap, kb * kGgKBlock, un.row0, fb);                      // token rows
                 }
-            };
-            auto load_phase2 = [&](int i) {
-                const GgUnit un = a.units[blockIdx.x + i * gridDim.x];
-                for (int dt = 0; dt < n_dt && ok; ++dt, ++it) {
-                    const uint32_t s = it % kGgStages;
-                    if (it >= kGgStages) ok = __all_sync(0xffffffffu, gg_wait(smem_u32(empty + s), ((it / kGgStages) - 1) & 1, ab));
-                    if (!ok) break;
-                    const uint32_t base = smem_u32(stages + s * kGgStageBytes);
-                    const uint32_t fb = smem_u32(full + s);
-                    if (elect_one()) {
-                        mbar_arrive_expect_tx(fb, 2 * kGgTileBytes);
-                        tma_load_4d(base, &wmap, dt * kGgTileRows, 2, un.jt * kGgTileRows, un.slot, fb);                      // d 0..63
-                        tma_load_4d(base + kGgTileBytes, &wmap, dt * kGgTileRows + 64, 2, un.jt * kGgTileRows, un.slot, fb); // d 64..127
-                    }
-                    __syncwarp();
-                }
-            };
-            if (my_units > 0) load_phase1(0);
-            for (int i = 0; i < my_units && ok; ++i) {
-                if (i + 1 < my_units) load_phase1(i + 1);
-                if (ok) load_phase2(i);
+                __syncwarp();
             }
         }
+        // ---- P2: W_down tiles, chunk by chunk from the common list
+        while (ok) {
+            int idx = 0;
+            if (lane == 0) idx = atomicAdd(a.next_chunk, 1);
+            idx = __shfl_sync(0xffffffffu, idx, 0);
+            if (idx >= n_chunks) break;
+            const GgTask tk = a.chunks ? a.chunks[idx] : GgTask{idx, 0, int16_t(n_dt)};
+            publish(tk);
+            if (!ok) break;
+            const GgUnit un = a.units[tk.unit];
+            // The first ring-full of tiles is issued before A^T is fetched: those stage slots are freed by
+            // MMAs of earlier tasks only, so the weight stream does not pause while this warp waits for the
+            // preceding chunk's MMAs and for the unit's arrival counter.
+            auto load_w = [&](int dt) {
+                const uint32_t s = it % kGgStages;
+                stage_free(s);
+                if (!ok) return;
+                const uint32_t base = smem_u32(stages + s * kGgStageBytes);
+                const uint32_t fb = smem_u32(full + s);
+                if (elect_one()) {
+                    mbar_arrive_expect_tx(fb, 2 * kGgTileBytes);
+                    tma_load_4d(base, &wmap, dt * kGgTileRows, 2, un.jt * kGgTileRows, un.slot, fb);                      // d 0..63
+                    tma_load_4d(base + kGgTileBytes, &wmap, dt * kGgTileRows + 64, 2, un.jt * kGgTileRows, un.slot, fb); // d 64..127
+                }
+                __syncwarp();
+                ++it;
+            };
+            int dt = tk.dt0;
+            for (int pre = 0; pre < kGgStages && dt < tk.dt1 && ok; ++pre, ++dt) load_w(dt);
+            if (ok && n_p2 > 0) ok = __all_sync(0xffffffffu, gg_wait(smem_u32(act_empty), (n_p2 - 1) & 1, ab));
+            if (ok) ok = __all_sync(0xffffffffu, gg_wait_count(a.act_ready + tk.unit, kGgActReady, ab));
+            if (!ok) break;
+            if (elect_one()) {
+                asm volatile("fence.proxy.async;" ::: "memory");     // A^T was written with ordinary stores, is read by a bulk copy
+                mbar_arrive_expect_tx(smem_u32(act_full), kGgActBytes);
+                bulk_g2s_plain(smem_u32(act), a.act_g + size_t(tk.unit) * kGgActBytes, kGgActBytes, smem_u32(act_full));
+            }
+            __syncwarp();
+            ++n_p2;
+            for (; dt < tk.dt1 && ok; ++dt) load_w(dt);
+        }
+        if (ok) publish(GgTask{-1, 0, 0});
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        {
-            uint32_t it = 0, nd = 0;     // stage counter, d-tile counter
-            bool ok = true;
-            auto wait_all = [&](uint64_t* bar, uint32_t parity) { ok = __all_sync(0xffffffffu, ok && gg_wait(smem_u32(bar), parity, ab)); };
-            auto mma_phase1 = [&](int i) {
-                const uint32_t b = i & 1, m = uint32_t(i) >> 1;
+        uint32_t it = 0, nd = 0, n_p1 = 0, n_p2 = 0;     // stage, d-tile, P1 and P2 counters
+        bool ok = true;
+        auto wait_all = [&](uint64_t* bar, uint32_t parity) { ok = __all_sync(0xffffffffu, ok && gg_wait(smem_u32(bar), parity, ab)); };
+        while (ok) {
+            const GgTask tk = next_task();
+            if (tk.unit < 0) break;
+            const uint32_t n_pad = gg_pad_tokens(a.units[tk.unit].ntok);
+            if (tk.dt0 < 0) {
+                const uint32_t b = n_p1 & 1, m = n_p1 >> 1;
                 // weights K-major, tokens K-major; N = the unit's tokens rounded up to 16
-                const uint32_t idesc1 = gg_idesc_n(false, false, gg_pad_tokens(a.units[blockIdx.x + i * gridDim.x].ntok));
-                if (i >= 2) wait_all(acc1_empty + b, (m - 1) & 1);   // pair drained two units ago
+                const uint32_t idesc1 = gg_idesc_n(false, false, n_pad);
+                if (n_p1 >= 2) wait_all(acc1_empty + b, (m - 1) & 1);   // pair drained two P1 tasks ago
                 const uint32_t acc = tmem + 128 * b;
                 for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
                     const uint32_t s = it % kGgStages;
@@ -300,41 +402,37 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
                 }
                 if (ok && elect_one()) tc_commit(smem_u32(acc1_full + b));
                 __syncwarp();
-            };
-            auto mma_phase2 = [&](int i) {
-                // W_down column tile M-major, A^T N-major
-                const uint32_t idesc2 = gg_idesc_n(true, true, gg_pad_tokens(a.units[blockIdx.x + i * gridDim.x].ntok));
-                wait_all(act_full, i & 1);
-                if (!ok) return;
-                tc_fence_after();
-                const uint32_t act_addr = smem_u32(act);
-                for (int dt = 0; dt < n_dt && ok; ++dt, ++it, ++nd) {
-                    const uint32_t s = it % kGgStages, b = nd & 1;
-                    wait_all(full + s, (it / kGgStages) & 1);
-                    if (nd >= 2) wait_all(acc2_empty + b, ((nd >> 1) - 1) & 1);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t base = smem_u32(stages + s * kGgStageBytes);
-                    if (elect_one()) {
-#pragma unroll
-                        for (int ks = 0; ks < 8; ++ks) {      // K = 16 rows j per step, 2048 bytes of each operand
-                            const uint64_t da = smem_desc_sw128(base + ks * 2048, kGgTileBytes, 1024);
-                            const uint64_t db = smem_desc_sw128(act_addr + ks * 2048, kGgActBytes, 1024);
-                            tc_mma_bf16(tmem + 256 + 64 * b, da, db, idesc2, ks != 0);
-                        }
-                        tc_commit(smem_u32(empty + s));
-                        tc_commit(smem_u32(acc2_full + b));
-                    }
-                    __syncwarp();
-                }
-                if (ok && elect_one()) tc_commit(smem_u32(act_empty));
-                __syncwarp();
-            };
-            if (my_units > 0) mma_phase1(0);
-            for (int i = 0; i < my_units && ok; ++i) {
-                if (i + 1 < my_units) mma_phase1(i + 1);
-                if (ok) mma_phase2(i);
+                ++n_p1;
+                continue;
             }
+            // W_down column tile M-major, A^T N-major
+            const uint32_t idesc2 = gg_idesc_n(true, true, n_pad);
+            wait_all(act_full, n_p2 & 1);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t act_addr = smem_u32(act);
+            for (int dt = tk.dt0; dt < tk.dt1 && ok; ++dt, ++it, ++nd) {
+                const uint32_t s = it % kGgStages, b = nd & 1;
+                wait_all(full + s, (it / kGgStages) & 1);
+                if (nd >= 2) wait_all(acc2_empty + b, ((nd >> 1) - 1) & 1);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t base = smem_u32(stages + s * kGgStageBytes);
+                if (elect_one()) {
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {      // K = 16 rows j per step, 2048 bytes of each operand
+                        const uint64_t da = smem_desc_sw128(base + ks * 2048, kGgTileBytes, 1024);
+                        const uint64_t db = smem_desc_sw128(act_addr + ks * 2048, kGgActBytes, 1024);
+                        tc_mma_bf16(tmem + 256 + 64 * b, da, db, idesc2, ks != 0);
+                    }
+                    tc_commit(smem_u32(empty + s));
+                    tc_commit(smem_u32(acc2_full + b));
+                }
+                __syncwarp();
+            }
+            if (ok && elect_one()) tc_commit(smem_u32(act_empty));
+            __syncwarp();
+            ++n_p2;
         }
     } else {
         // ---------------- epilogue warps (TMEM lane quarter = warp % 4) ----------------
@@ -342,50 +440,56 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
         const int row = q * 32 + lane;                  // accumulator row handled by this thread
         const uint32_t lane_addr = uint32_t(q * 32) << 16;
         float* wrow_s = wrow_all + q * kGgTokens;       // this warp's copy: no cross-warp barrier needed
-        uint32_t nd = 0;
+        uint32_t nd = 0, n_p1 = 0;
         bool ok = true;
-        for (int i = 0; i < my_units && ok; ++i) {
-            const GgUnit un = a.units[blockIdx.x + i * gridDim.x];
-            const uint32_t b1 = i & 1;
-            // routing weights of this expert's token rows (0 beyond the real tokens)
-            __syncwarp();
+        while (ok) {
+            const GgTask tk = next_task();
+            if (tk.unit < 0) break;
+            const GgUnit un = a.units[tk.unit];
+            if (tk.dt0 < 0) {
+                const uint32_t b1 = n_p1 & 1;
+                // routing weights of this expert's token rows (0 beyond the real tokens)
+                __syncwarp();
 #pragma unroll
-            for (int t = lane; t < kGgTokens; t += 32) wrow_s[t] = t < un.ntok ? a.wrow[un.row0 + t] : 0.f;
-            __syncwarp();
-
-            ok = gg_wait(smem_u32(acc1_full + b1), (uint32_t(i) >> 1) & 1, ab);
-            if (ok && i > 0) ok = gg_wait(smem_u32(act_empty), (i - 1) & 1, ab);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            // A^T[j = row][t] = silu(G) * U * w_t, bf16, 16-byte chunks swizzled by (row % 8)
-            const int n_pad = int(gg_pad_tokens(un.ntok));      // columns the MMAs of this unit wrote
+                for (int t = lane; t < kGgTokens; t += 32) wrow_s[t] = t < un.ntok ? a.wrow[un.row0 + t] : 0.f;
+                __syncwarp();
+                ok = __all_sync(0xffffffffu, gg_wait(smem_u32(acc1_full + b1), (n_p1 >> 1) & 1, ab));
+                if (!ok) break;
+                tc_fence_after();
+                // A^T[j = row][t] = silu(G) * U * w_t, bf16, 16-byte chunks swizzled by (row % 8): the layout
+                // the second GEMM's B operand has in shared memory, stored to the unit's slot in global memory
+                const int n_pad = int(gg_pad_tokens(un.ntok));      // columns the MMAs of this unit wrote
+                unsigned char* rowp = a.act_g + size_t(tk.unit) * kGgActBytes + row * 128;
 #pragma unroll
-            for (int c = 0; c < kGgTokens / 16; ++c) {
-                if (c * 16 >= n_pad) break;
-                float g[16], up[16];
-                tmem_ld16(tmem + lane_addr + 128 * b1 + c * 16, g);
-                tmem_ld16(tmem + lane_addr + 128 * b1 + 64 + c * 16, up);
-                uint32_t packed[8];
+                for (int c = 0; c < kGgTokens / 16; ++c) {
+                    if (c * 16 >= n_pad) break;
+                    float g[16], up[16];
+                    tmem_ld16(tmem + lane_addr + 128 * b1 + c * 16, g);
+                    tmem_ld16(tmem + lane_addr + 128 * b1 + 64 + c * 16, up);
+                    uint32_t packed[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const float a0 = g[2 * e] / (1.f + expf(-g[2 * e])) * up[2 * e] * wrow_s[c * 16 + 2 * e];
-                    const float a1 = g[2 * e + 1] / (1.f + expf(-g[2 * e + 1])) * up[2 * e + 1] * wrow_s[c * 16 + 2 * e + 1];
-                    const __nv_bfloat162 p = __floats2bfloat162_rn(a0, a1);
-                    packed[e] = *reinterpret_cast<const uint32_t*>(&p);
+                    for (int k2 = 0; k2 < 8; ++k2) {
+                        const float a0 = g[2 * k2] / (1.f + expf(-g[2 * k2])) * up[2 * k2] * wrow_s[c * 16 + 2 * k2];
+                        const float a1 = g[2 * k2 + 1] / (1.f + expf(-g[2 * k2 + 1])) * up[2 * k2 + 1] * wrow_s[c * 16 + 2 * k2 + 1];
+                        const __nv_bfloat162 p = __floats2bfloat162_rn(a0, a1);
+                        packed[k2] = *reinterpret_cast<const uint32_t*>(&p);
+                    }
+                    *reinterpret_cast<uint4*>(rowp + (((2 * c) ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                    *reinterpret_cast<uint4*>(rowp + (((2 * c + 1) ^ (row & 7)) << 4)) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
                 }
-                unsigned char* rowp = act + row * 128;
-                *reinterpret_cast<uint4*>(rowp + (((2 * c) ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-                *reinterpret_cast<uint4*>(rowp + (((2 * c + 1) ^ (row & 7)) << 4)) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+                tc_fence_before();
+                __syncwarp();                   // the warp's 32 rows are written ...
+                if (lane == 0) {
+                    mbar_arrive(smem_u32(acc1_empty + b1));
+                    __threadfence();            // ... and made visible device-wide before the arrival is counted
+                    asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(a.act_ready + tk.unit) : "memory");
+                }
+                ++n_p1;
+                continue;
             }
-            fence_proxy_async();            // generic-proxy writes of A^T -> visible to the MMA's async reads
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) { mbar_arrive(smem_u32(acc1_empty + b1)); mbar_arrive(smem_u32(act_full)); }
-
-            // phase 2: one [128 d x 64 tokens] accumulator per d-tile; store the real tokens' rows
+            // phase 2: one [128 d x tokens] accumulator per d-tile; store the real tokens' rows
             float* prow = a.partial + (size_t(un.jt) * a.rows_cap + un.row0) * D;
-            for (int dt = 0; dt < n_dt && ok; ++dt, ++nd) {
+            for (int dt = tk.dt0; dt < tk.dt1 && ok; ++dt, ++nd) {
                 const uint32_t b = nd & 1;
                 ok = __all_sync(0xffffffffu, gg_wait(smem_u32(acc2_full + b), (nd >> 1) & 1, ab));
                 if (!ok) break;
@@ -394,8 +498,8 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
                     float y[16];
                     tmem_ld16(tmem + lane_addr + 256 + 64 * b + c * 16, y);
 #pragma unroll
-                    for (int e = 0; e < 16; ++e)
-                        if (c * 16 + e < un.ntok) prow[size_t(c * 16 + e) * D + dt * kGgTileRows + row] = y[e];
+                    for (int k2 = 0; k2 < 16; ++k2)
+                        if (c * 16 + k2 < un.ntok) prow[size_t(c * 16 + k2) * D + dt * kGgTileRows + row] = y[k2];
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -411,7 +515,8 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
 }
 
 inline size_t ffn_grouped_smem() {
-    return 1024 + size_t(kGgStages) * kGgStageBytes + kGgActBytes + 256 + 4 * kGgTokens * sizeof(float) + 64;
+    return 1024 + size_t(kGgStages) * kGgStageBytes + kGgActBytes + 256 + 4 * kGgTokens * sizeof(float) + 64 +
+           2 * kGgQueue * sizeof(uint64_t) + kGgQueue * sizeof(GgTask);
 }
 
 // Sorted token rows of one wave: Xs[row][:] = bf16(x[token][:]), wrow[row] = w[token][k].
@@ -419,9 +524,11 @@ struct GgRow { int32_t token, k; };
 
 static __global__ void gg_gather_kernel(const float* __restrict__ x, const float* __restrict__ w, const GgRow* __restrict__ rows,
                                         int n_rows, const int* n_rows_dev, int D, int K, __nv_bfloat16* __restrict__ xs,
-                                        float* __restrict__ wrow, int perm8) {
+                                        float* __restrict__ wrow, int perm8, int* act_ready = nullptr, int n_ready = 0) {
     grid_dep_launch();
     grid_dep_wait();
+    // the grouped kernel that follows counts arrivals per unit from zero
+    if (blockIdx.x == 0) for (int i = threadIdx.x; i < n_ready; i += blockDim.x) act_ready[i] = 0;
     if (n_rows_dev) n_rows = __ldcg(n_rows_dev);
     const int r = blockIdx.x;
     if (r >= n_rows) return;

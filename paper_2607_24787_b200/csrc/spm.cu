@@ -22,6 +22,7 @@
 #include "ffn_grouped_q4.cuh"
 #include "router_adapter.cuh"
 #include "tma_maps.h"
+#include "gg_plan.h"
 #include "slot_table.h"
 
 using namespace spm;
@@ -74,7 +75,10 @@ struct spm_ctx {
     unsigned char* tc_desc_dev = nullptr;     // kDescRing wave descriptors
     unsigned char* tc_desc_host = nullptr;    // pinned staging, same layout
     int* tc_counts = nullptr;                 // {units, rows} of a wave planned on the device
-    size_t tc_desc_bytes = 0, tc_off_rows = 0, tc_off_rowmap = 0;
+    size_t tc_desc_bytes = 0, tc_off_rows = 0, tc_off_rowmap = 0, tc_off_chunks = 0, tc_chunk_cap = 0;
+    unsigned char* tc_act = nullptr;          // [max_units][16 KB] A^T slots of the bf16 grouped kernel
+    int* tc_ready = nullptr;                  // [1 + max_units] chunk counter, then the slots' arrival counters
+    std::vector<GgTaskHost> plan_chunks;
     std::vector<cudaEvent_t> tc_desc_ev;
     std::vector<uint8_t> tc_desc_ev_valid;
     size_t tc_desc_pos = 0;
@@ -201,6 +205,7 @@ constexpr int kMaxCtasBatch1 = 296;
 constexpr int kClockSlots = 12288;    // in-kernel {start, end} pairs between two harvests
 constexpr int kDescRing = 8;          // wave descriptors in flight for the batched tensor-core path
 constexpr int kTraceRing = 8;         // host-free steps whose bookkeeping may be outstanding
+static_assert(sizeof(GgTask) == sizeof(GgTaskHost), "host plan and device task share one layout");
 
 // The grouped tcgen05 kernels handle bf16 or 4-bit weights, more than one sequence per step, no
 // shared experts, and intermediate / hidden sizes that tile by 128.
@@ -225,8 +230,8 @@ struct Carve {
 
 struct Layout {
     size_t pools, slot_gen, x, logits, pihat, w, scores, partial, h, ids, order, clock, slot_map, codes, counters, status, total;
-    size_t tc_xs, tc_wrow, tc_partial, tc_desc, tc_counts;       // batched tensor-core path only
-    size_t desc_bytes, off_rows, off_rowmap;
+    size_t tc_xs, tc_wrow, tc_partial, tc_desc, tc_counts, tc_act, tc_ready;       // batched tensor-core path only
+    size_t desc_bytes, off_rows, off_rowmap, off_chunks, chunk_cap;
     int rows_cap, n_jt, max_units;
     bool tc;
 };
@@ -256,12 +261,17 @@ Layout layout_of(const spm_model_cfg* m, int S) {
         l.max_units = std::min(S, m->n_experts) * l.n_jt;
         l.off_rows = align_up(size_t(l.max_units) * sizeof(GgUnit), 256);
         l.off_rowmap = l.off_rows + align_up(size_t(l.rows_cap) * sizeof(GgRow), 256);
-        l.desc_bytes = l.off_rowmap + align_up(size_t(m->max_batch) * SPM_MAX_TOPK * 4, 256);
+        // phase-2 chunk list of the bf16 kernel: at most one chunk per kGgMinChunk d-tiles, at least one per unit
+        l.off_chunks = l.off_rowmap + align_up(size_t(m->max_batch) * SPM_MAX_TOPK * 4, 256);
+        l.chunk_cap = size_t(l.max_units) * size_t(std::max(1, (m->hidden / kGgTileRows + kGgMinChunk - 1) / kGgMinChunk));
+        l.desc_bytes = l.off_chunks + align_up(l.chunk_cap * sizeof(GgTask), 256);
         l.tc_xs = c.take(size_t(l.rows_cap + kGgTokens) * D * 2);
         l.tc_wrow = c.take(size_t(l.rows_cap) * 4);
         l.tc_partial = c.take(size_t(l.n_jt) * l.rows_cap * D * 4);
         l.tc_desc = c.take(size_t(kDescRing) * l.desc_bytes);
         l.tc_counts = c.take(2 * sizeof(int));
+        l.tc_act = c.take(size_t(l.max_units) * kGgActBytes);
+        l.tc_ready = c.take(size_t(l.max_units + 1) * sizeof(int));
     }
     l.counters = c.take(256);
     l.status = c.take(4);
@@ -656,26 +666,40 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
             rows[r] = GgRow{tk, k};
         }
     if (n_units == 0) return SPM_OK;
+    const bool q4 = m.dtype == SPM_DTYPE_Q4;
+    if (!q4) {
+        // bf16 kernel: phase-2 chunks, finer towards the end, so that every SM streams until the launch ends
+        gg_plan_chunks(n_units, m.hidden / kGgTileRows, c->num_sms, c->plan_chunks);
+        if (c->plan_chunks.size() > c->tc_chunk_cap) return fail(c, SPM_ERR_STATE, "grouped-kernel chunk list exceeds its buffer");
+        std::memcpy(hd + c->tc_off_chunks, c->plan_chunks.data(), c->plan_chunks.size() * sizeof(GgTaskHost));
+    }
     CU(c, cudaMemcpyAsync(dd, hd, c->tc_desc_bytes, cudaMemcpyHostToDevice, c->compute));
     CU(c, cudaEventRecord(c->tc_desc_ev[d], c->compute));
     c->tc_desc_ev_valid[d] = 1;
-    gg_gather_kernel<<<n_rows, 128, 0, c->compute>>>(x_norm, w, reinterpret_cast<const GgRow*>(dd + c->tc_off_rows), n_rows,
-                                                     nullptr, m.hidden, K, c->tc_xs, c->tc_wrow, m.dtype == SPM_DTYPE_Q4 ? 1 : 0);
-    CU(c, cudaGetLastError());
+    // (all three kernels of a wave are launched so that their preambles may overlap their predecessor's tail)
+    CU(c, launch_k(gg_gather_kernel, dim3(n_rows), dim3(128), 0, c->compute, true, x_norm, w,
+                   reinterpret_cast<const GgRow*>(dd + c->tc_off_rows), n_rows, (const int*)nullptr, m.hidden, K, c->tc_xs, c->tc_wrow,
+                   q4 ? 1 : 0, q4 ? (int*)nullptr : c->tc_ready, q4 ? 0 : n_units + 1));
     if (t && first) CU(c, cudaEventRecord(t->ffn_start[layer], c->compute));
     if (ring >= 0 && first) CU(c, cudaEventRecord(c->ring_start[ring], c->compute));
-    GgArgs a{reinterpret_cast<const GgUnit*>(dd), n_units, nullptr, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status, c->wait_limit_ns};
-    if (m.dtype == SPM_DTYPE_Q4)
-        ffn_grouped_q4_kernel<<<std::min(c->num_sms, n_units), kQgThreads, ffn_grouped_q4_smem(), c->compute>>>(
-            c->qmapn, c->qmapsc, c->xmaps, a);
-    else
-        ffn_grouped_kernel<<<std::min(c->num_sms, n_units), kGgThreads, ffn_grouped_smem(), c->compute>>>(c->wmap, c->xmaps, a);
-    CU(c, cudaGetLastError());
+    GgArgs a{reinterpret_cast<const GgUnit*>(dd), n_units, nullptr, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status, c->wait_limit_ns,
+             nullptr, 0, nullptr, nullptr, nullptr};
+    if (q4) {
+        CU(c, launch_k(ffn_grouped_q4_kernel, dim3(std::min(c->num_sms, n_units)), dim3(kQgThreads), ffn_grouped_q4_smem(), c->compute, true,
+                       c->qmapn, c->qmapsc, c->xmaps, a));
+    } else {
+        a.chunks = reinterpret_cast<const GgTask*>(dd + c->tc_off_chunks);
+        a.n_chunks = int(c->plan_chunks.size());
+        a.next_chunk = c->tc_ready;
+        a.act_ready = c->tc_ready + 1;
+        a.act_g = c->tc_act;
+        // every SM takes part: CTAs without a unit of their own still run phase-2 chunks
+        CU(c, launch_k(ffn_grouped_kernel, dim3(c->num_sms), dim3(kGgThreads), ffn_grouped_smem(), c->compute, true, c->wmap, c->xmaps, a));
+    }
     if (t && last) CU(c, cudaEventRecord(t->ffn_end[layer], c->compute));
     if (ring >= 0 && last) { CU(c, cudaEventRecord(c->ring_end[ring], c->compute)); c->ring_used[ring] = 1; }
-    gg_combine_kernel<<<dim3((m.hidden / 4 + 127) / 128, nb), 128, 0, c->compute>>>(
-        c->tc_partial, reinterpret_cast<const int32_t*>(dd + c->tc_off_rowmap), K, c->n_jt, c->rows_cap, m.hidden, h_inout);
-    CU(c, cudaGetLastError());
+    CU(c, launch_k(gg_combine_kernel, dim3((m.hidden / 4 + 127) / 128, nb), dim3(128), 0, c->compute, true,
+                   (const float*)c->tc_partial, reinterpret_cast<const int32_t*>(dd + c->tc_off_rowmap), K, c->n_jt, c->rows_cap, m.hidden, h_inout));
     c->kernel_launches += 3;
     c->ffn_launches++;
     c->tc_launches++;
@@ -1056,8 +1080,11 @@ int enqueue_host_free_layers(spm_ctx* c, int nb, float* h_out, int slot, bool pr
                            units, rows, rowmap, c->tc_counts, c->ws_status));
             CU(c, launch_k(gg_gather_kernel, dim3(nb * K), dim3(128), 0, c->compute, true, (const float*)c->ws_x, (const float*)c->ws_w,
                            (const GgRow*)rows, 0, (const int*)(c->tc_counts + 1), m.hidden, K, c->tc_xs, c->tc_wrow,
-                           m.dtype == SPM_DTYPE_Q4 ? 1 : 0));
-            GgArgs ga{units, 0, c->tc_counts, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status, c->wait_limit_ns};
+                           m.dtype == SPM_DTYPE_Q4 ? 1 : 0, m.dtype == SPM_DTYPE_Q4 ? (int*)nullptr : c->tc_ready,
+                           m.dtype == SPM_DTYPE_Q4 ? 0 : c->max_units + 1));
+            // (no chunk list here: the plan is built on the device, a chunk is a whole unit)
+            GgArgs ga{units, 0, c->tc_counts, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status, c->wait_limit_ns,
+                      nullptr, 0, c->tc_ready, c->tc_act, c->tc_ready + 1};
             if (m.dtype == SPM_DTYPE_Q4)
                 CU(c, launch_k(ffn_grouped_q4_kernel, dim3(c->num_sms), dim3(kQgThreads), ffn_grouped_q4_smem(), c->compute, true,
                                c->qmapn, c->qmapsc, c->xmaps, ga));
@@ -1298,6 +1325,9 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
         c->tc_desc_dev = base + lay.tc_desc;
         c->tc_counts = reinterpret_cast<int*>(base + lay.tc_counts);
         c->tc_desc_bytes = lay.desc_bytes; c->tc_off_rows = lay.off_rows; c->tc_off_rowmap = lay.off_rowmap;
+        c->tc_off_chunks = lay.off_chunks; c->tc_chunk_cap = lay.chunk_cap;
+        c->tc_act = base + lay.tc_act;
+        c->tc_ready = reinterpret_cast<int*>(base + lay.tc_ready);
         if (!cu(cudaMemsetAsync(c->tc_xs, 0, size_t(lay.rows_cap + kGgTokens) * cfg->hidden * 2, c->compute), "cudaMemsetAsync")) return bail(SPM_ERR_CUDA);
         if (!cu(cudaHostAlloc(reinterpret_cast<void**>(&c->tc_desc_host), size_t(kDescRing) * lay.desc_bytes, cudaHostAllocDefault), "cudaHostAlloc(descriptors)")) return bail(SPM_ERR_CUDA);
         c->tc_desc_ev.resize(kDescRing);
@@ -1947,6 +1977,20 @@ int spm_sim_create(int n_layers, int n_experts, int slots, int plain_lru, spm_si
     return SPM_OK;
 }
 int spm_sim_destroy(spm_sim* s) { delete s; return SPM_OK; }
+
+int spm_plan_grouped_chunks(int n_units, int n_dt, int grid, int32_t* chunks, size_t capacity, size_t* count) {
+    if (n_units < 1 || n_dt < 1 || n_dt > 32767 || grid < 1 || !chunks || !count) return SPM_ERR_INVALID_ARG;
+    std::vector<GgTaskHost> list;
+    gg_plan_chunks(n_units, n_dt, grid, list);
+    *count = list.size();
+    if (list.size() > capacity) return SPM_ERR_INVALID_ARG;
+    for (size_t i = 0; i < list.size(); ++i) {
+        chunks[3 * i] = list[i].unit;
+        chunks[3 * i + 1] = list[i].dt0;
+        chunks[3 * i + 2] = list[i].dt1;
+    }
+    return SPM_OK;
+}
 
 static bool sim_ids_ok(spm_sim* s, int layer, const int32_t* ids, int count) {
     if (!s || layer < 0 || layer >= s->table.layers() || count < 0 || (count > 0 && !ids)) return false;

@@ -52,6 +52,36 @@ def test_init_fails_loudly_without_gpu():
     assert e.value.code == -3
 
 
+@pytest.mark.parametrize("n_units,n_dt,grid", [(192, 16, 148), (6, 2, 148), (755, 16, 148), (148, 16, 148), (48, 10, 148),
+                                              (1, 4, 7), (300, 3, 16), (40, 1, 148)])
+def test_grouped_kernel_chunk_plan(n_units, n_dt, grid):
+    """Phase-2 chunk list of the batched tensor-core kernel: every (unit, d-tile) exactly once, in
+    unit order (the units whose phase 1 ends first come first), chunk sizes shrinking towards the
+    end of the list but never below the minimum while a unit has that many d-tiles left, so that
+    the CTAs that take them in order run out of work together."""
+    ch = B.spm_plan_grouped_chunks(n_units, n_dt, grid)
+    seen = np.zeros((n_units, n_dt), int)
+    for u, dt0, dt1 in ch:
+        assert 0 <= dt0 < dt1 <= n_dt
+        seen[u, dt0:dt1] += 1
+    assert np.all(seen == 1)
+    order = [(int(u), int(d0)) for u, d0, _ in ch]
+    assert order == sorted(order)
+    sizes = np.array([int(d1 - d0) for _, d0, d1 in ch])
+    min_chunk = min(4, n_dt)
+    assert sizes.min() >= min_chunk and sizes.max() <= n_dt
+    total = n_units * n_dt
+    # guided: no chunk is larger than its fair share of what was left when it was cut (or the minimum, or a unit's rest)
+    left = total
+    for (u, d0, d1), sz in zip(ch, sizes):
+        fair = -(-left // (2 * grid))
+        assert sz <= max(fair, min_chunk) + min_chunk - 1, (u, d0, d1, left)
+        left -= sz
+    # the tail is fine-grained: the last grid chunks are all near the minimum size (when there is that much work)
+    if total >= 8 * grid * min_chunk and n_dt >= 2 * min_chunk:
+        assert np.all(sizes[-grid:] <= 2 * min_chunk - 1)
+
+
 def test_noalloc_argument_checks_run_before_any_gpu_work():
     """The allocation-free entry point refuses bad shapes, indices and misaligned pointers on the
     host, before it touches the device: so this runs without a GPU (addresses below are never
