@@ -130,8 +130,10 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
     const int G = gridDim.x, c = blockIdx.x;
     const int I = a.I;
     const int R = a.entries(tok) * I;
-    const int r_begin = int((long long)R * c / G);
-    const int r_end = int((long long)R * (c + 1) / G);
+    // even split: CTA c takes q rows, the first R % G CTAs one more (one 32-bit division)
+    const int q_rows = R / G, rem_rows = R - q_rows * G;
+    const int r_begin = q_rows * c + min(c, rem_rows);
+    const int r_end = r_begin + q_rows + (c < rem_rows ? 1 : 0);
     const int span = r_end - r_begin - wi;
     const int my_n = span > 0 ? (span + nw - 1) / nw : 0;
 

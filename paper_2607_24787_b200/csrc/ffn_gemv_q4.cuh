@@ -51,8 +51,10 @@ ffn_gemv_q4_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth, co
     const uint32_t RB = uint32_t(D / 2 + D / 16);     // bytes of one packed row
     const uint32_t ROWB = 3u * RB;
     const int R = a.entries(tok) * I;
-    const int r_begin = int((long long)R * c / G);
-    const int r_end = int((long long)R * (c + 1) / G);
+    // even split: CTA c takes q rows, the first R % G CTAs one more (one 32-bit division)
+    const int q_rows = R / G, rem_rows = R - q_rows * G;
+    const int r_begin = q_rows * c + min(c, rem_rows);
+    const int r_end = r_begin + q_rows + (c < rem_rows ? 1 : 0);
     const int span = r_end - r_begin - wi;
     const int my_n = span > 0 ? (span + nw - 1) / nw : 0;
 
