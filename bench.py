@@ -39,10 +39,10 @@ import torch
 
 import synth
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one ffn_gemv_kernel launch, from the ncu capture
-# summarised in profiles/ffn_gemv_kernel_qwen3.md (taken on the 4-layer reduction of the workload;
-# a launch reads the same 8 expert blobs whatever the layer count)
-NCU_DRAM_BYTES_PER_LAUNCH = {"qwen3": 77.2e6}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from one ncu capture of a reduced
+# case of the same workload (4 layers; a launch reads the same expert blobs whatever the layer count): 75.54 MB read +
+# 1.0 - 1.7 MB written for the GEMV kernel, 306.7 + 8.7 MB for one 32-expert wave of the grouped kernel.
+NCU_DRAM_BYTES_PER_LAUNCH = {"qwen3": 76.9e6, "batched_wave": 315.4e6}
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
@@ -536,7 +536,8 @@ def grouped_alone(cfg, ctx, n_resident, peak, which, launches):
     us = st["ffn_us"] / max(st["ffn_launches"], 1)
     ach = mean_bytes / (us * 1e-6) / 1e9
     return {"bound": "hbm", "kernel": ffn_kernel_name(cfg), "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
-            "traffic": None, "peak_source": f"of {which}", "algorithmic_bytes_per_launch": mean_bytes, "us_per_launch": us,
+            "traffic": NCU_DRAM_BYTES_PER_LAUNCH["batched_wave"] if (cfg.name == "batched" and n_resident == cfg.slots) else None,
+            "peak_source": f"of {which}", "algorithmic_bytes_per_launch": mean_bytes, "us_per_launch": us,
             "launches": int(st["ffn_launches"]), "misses": int(st["misses"]), "distinct_experts_per_launch": mean_bytes / cfg.expert_bytes,
             "region": f"{launches} spm_moe_ffn launches back to back, {nb} tokens x top-{cfg.top_k} among {n_resident} resident "
                       "experts per layer, pools of all layers cycled, CUDA event pair per grouped-kernel launch"}
@@ -909,6 +910,7 @@ def cpu_baseline(cfg, H, device, budget, repeats=3):
     thread(s) (the headline: reproducible), and once with every host core the process may use."""
     runs = []
     Ls = cfg.n_layers
+    oracle_steps(cfg, H[:1], device, budget, ORACLE_THREADS)          # untimed: first-touch of the allocator and the libraries
     for _ in range(repeats):
         times, Ls = oracle_steps(cfg, H, device, budget, ORACLE_THREADS)
         runs.append(H.shape[0] * cfg.batch * (Ls / cfg.n_layers) / sum(times))

@@ -250,7 +250,7 @@ int spm_set_drop_modulo(spm_ctx* ctx, int modulo);
  * copy is followed on the copy stream by a wait of `us` microseconds (0 = off, at most 100000)
  * before the slot counts as loaded. Outputs are unchanged. */
 int spm_set_copy_delay_us(spm_ctx* ctx, int us);
-/* Device-side wait for batch-1 expert FFNs (default off). Off: the compute stream waits on the
+/* Device-side wait for batch-1 expert FFNs (default off; bf16, fp32 and 4-bit experts). Off: the compute stream waits on the
  * event of the batch of copies that fills the slots a launch reads, then the kernel starts. On: the
  * kernel is launched at once and its warps wait (bounded, SPM_ERR_TIMEOUT on expiry) on an arrival
  * counter that the copy stream bumps after the last copy of that batch has landed, so rows of

@@ -79,6 +79,22 @@ struct FfnArgs {
     }
 };
 
+// Device-side wait for a batch of expert copies: the copy stream bumps the batch leader's counter
+// after the batch's bytes have landed. Bounded: false when the limit ran out (the caller records
+// the status and winds the launch down).
+__device__ __forceinline__ bool ffn_wait_arrival(const unsigned* counter, unsigned want, unsigned long long limit_ns) {
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+        unsigned v;
+        asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+        if (int(v - want) >= 0) break;
+        __nanosleep(200);
+        if (global_timer_ns() - t0 > limit_ns) return false;
+    }
+    asm volatile("fence.proxy.async;" ::: "memory");   // the weights are read through the async proxy
+    return true;
+}
+
 // packed fp32 pairs (one 64-bit register pair) for fma.rn.f32x2
 __device__ __forceinline__ uint64_t pack2(float lo, float hi) {
     uint64_t r;
@@ -168,20 +184,9 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
             return a.shared + size_t(-1 - code) * a.blob_bytes;
         }
         if (code >= a.n_slots) { atomicOr(a.status, kStatusBadSlot); return nullptr; }
-        if (a.ready) {
-            // Device-side wait: the copy stream bumps the slot's counter after the expert's bytes
-            // have landed. Bounded; on timeout the status word is set and the launch winds down.
-            const unsigned* f = a.ready + a.watch[ent];
-            const unsigned want = a.want[ent];
-            const unsigned long long t0 = global_timer_ns();
-            for (;;) {
-                unsigned v;
-                asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(f) : "memory");
-                if (int(v - want) >= 0) break;
-                __nanosleep(200);
-                if (global_timer_ns() - t0 > wait_limit) { atomicOr(a.status, kStatusCopyTimeout); return nullptr; }
-            }
-            asm volatile("fence.proxy.async;" ::: "memory");   // the weights are read through the async proxy
+        if (a.ready && !ffn_wait_arrival(a.ready + a.watch[ent], a.want[ent], wait_limit)) {
+            atomicOr(a.status, kStatusCopyTimeout);
+            return nullptr;
         }
         return a.pool + size_t(code) * a.blob_bytes;
     };

@@ -86,6 +86,11 @@ ffn_gemv_q4_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth, co
             return a.shared + size_t(-1 - code) * a.blob_bytes;
         }
         if (code >= a.n_slots) { atomicOr(a.status, kStatusBadSlot); return nullptr; }
+        // device-side wait for the batch of copies that fills this slot (see ffn_gemv_kernel)
+        if (a.ready && !ffn_wait_arrival(a.ready + a.watch[ent], a.want[ent], a.limit())) {
+            atomicOr(a.status, kStatusCopyTimeout);
+            return nullptr;
+        }
         return a.pool + size_t(code) * a.blob_bytes;
     };
     auto issue = [&](int i) {

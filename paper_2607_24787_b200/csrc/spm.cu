@@ -741,7 +741,7 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
     }
 
     const int G = ffn_grid_for(c, nb);
-    const bool dev_wait = c->device_wait && nb == 1 && m.dtype != SPM_DTYPE_Q4 && stream_write32_fn() != nullptr;
+    const bool dev_wait = c->device_wait && nb == 1 && stream_write32_fn() != nullptr;
     std::vector<int16_t>& slot_of_expert = c->wave_slot;   // experts computed in the current wave
     for (int wave = 0; wave < n_waves; ++wave) {
         slot_of_expert.assign(m.n_experts, -1);
