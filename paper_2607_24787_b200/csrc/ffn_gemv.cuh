@@ -394,19 +394,31 @@ inline size_t ffn_gemv_smem(size_t row_bytes, int warps, int depth) {
     return size_t(warps) * depth * row_bytes + size_t(warps) * depth * 8;
 }
 
-// Launch shape for `rows_per_cta` rows of `row_bytes`: the warp count that leaves the fewest rows
-// on the busiest warp (the kernel ends when that warp does), then the most bytes in flight.
+// Launch shape for `rows_per_cta` rows of `row_bytes`. A ring of at least three rows per warp comes first:
+// with two, the slot of a row is blocked while that row is being computed, and the first row of a launch
+// is slow to compute (cold instruction fetch), so the copy stream ran dry once per launch (Qwen3 shape,
+// plain launches: 9 warps x 2 rows 17.5 us, 6 warps x 3 rows 16.5 us; same bytes in flight). Among such
+// shapes the most warps win. Rows too large for that fall back to the warp count that leaves the fewest
+// rows on the busiest warp (the kernel ends when that warp does), then the most bytes in flight.
 inline void ffn_gemv_shape(size_t row_bytes, int rows_per_cta, int* warps, int* depth) {
-    int best_w = 0, best_d = 0, best_cost = 1 << 30;
-    size_t best_flight = 0;
+    int best_w = 0, best_d = 0;
     for (int w = 4; w <= kFfnMaxWarps; ++w) {
         int d = int((kFfnSmemLimit - 1024) / (size_t(w) * row_bytes));
         if (d > 4) d = 4;
-        if (d < 2 && !(w == 4 && d == 1)) continue;      // want double buffering; 4 warps x 1 is the last resort
-        const int cost = (rows_per_cta + w - 1) / w;
-        const size_t flight = size_t(w) * d * row_bytes;
-        if (cost < best_cost || (cost == best_cost && flight > best_flight)) {
-            best_w = w; best_d = d; best_cost = cost; best_flight = flight;
+        if (d >= 3 && (w > best_w || (w == best_w && d > best_d))) { best_w = w; best_d = d; }
+    }
+    if (best_w == 0) {
+        int best_cost = 1 << 30;
+        size_t best_flight = 0;
+        for (int w = 4; w <= kFfnMaxWarps; ++w) {
+            int d = int((kFfnSmemLimit - 1024) / (size_t(w) * row_bytes));
+            if (d > 4) d = 4;
+            if (d < 2 && !(w == 4 && d == 1)) continue;      // want double buffering; 4 warps x 1 is the last resort
+            const int cost = (rows_per_cta + w - 1) / w;
+            const size_t flight = size_t(w) * d * row_bytes;
+            if (cost < best_cost || (cost == best_cost && flight > best_flight)) {
+                best_w = w; best_d = d; best_cost = cost; best_flight = flight;
+            }
         }
     }
     *warps = best_w;
