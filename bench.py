@@ -428,7 +428,10 @@ def run_ours(args):
     except Exception as e:   # noqa: BLE001 (pools smaller than 256 MiB: nothing to measure)
         result["roofline"]["read_only_stream_gb_s"] = None
     if world == 1 and rank == 0 and not args.no_cpu_baseline:
-        result["cpu_baseline"] = cpu_baseline(cfg, H[W:W + args.cpu_steps].numpy(), device, budget)
+        try:
+            result["cpu_baseline"] = cpu_baseline(args, cfg, budget)
+        except Exception as e:   # noqa: BLE001 (reported, not hidden)
+            result["cpu_baseline"] = {"error": str(e)[:300]}
     m.close()
     if rank == 0:
         print(json.dumps(result))
@@ -905,25 +908,35 @@ def oracle_steps(cfg, H, device, budget, threads, layers=None, mem_budget=40e9):
 ORACLE_THREADS = 1      # the oracle's numpy calls are small matrix-vector products: more BLAS threads make it slower and erratic
 
 
-def cpu_baseline(cfg, H, device, budget, repeats=3):
-    """The oracle on a bounded sample: the same few decode steps `repeats` times on ORACLE_THREADS pinned
-    thread(s) (the headline: reproducible), and once with every host core the process may use."""
-    runs = []
-    Ls = cfg.n_layers
-    oracle_steps(cfg, H[:1], device, budget, ORACLE_THREADS)          # untimed: first-touch of the allocator and the libraries
-    for _ in range(repeats):
-        times, Ls = oracle_steps(cfg, H, device, budget, ORACLE_THREADS)
-        runs.append(H.shape[0] * cfg.batch * (Ls / cfg.n_layers) / sum(times))
+def cpu_baseline(args, cfg, budget):
+    """The oracle on a bounded sample, timed in a process of its own: `bench.py --impl reference` on the first decode
+    steps of the bench's token stream, on ORACLE_THREADS pinned thread(s) (the headline: reproducible), and once with
+    every host core the process may use. A fresh process, because the same code measured 0.5 and 0.9 tokens/s on the
+    same box depending on what the calling process had allocated before; this way the figure is the one the reference
+    arm gives."""
+    def run(steps, threads):
+        cmd = [sys.executable, os.path.abspath(__file__), "--impl", "reference", "--config", args.config, "--steps", str(steps),
+               "--warmup", "3", "--oracle-threads", str(threads), "--oracle-budget", str(budget)]
+        if args.layers:
+            cmd += ["--layers", str(args.layers)]
+        if args.slots:
+            cmd += ["--slots", str(args.slots)]
+        env = dict(os.environ)
+        for k in ("RANK", "LOCAL_RANK", "WORLD_SIZE"):
+            env.pop(k, None)
+        out = subprocess.run(cmd, capture_output=True, text=True, timeout=1200, env=env)
+        lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+        if out.returncode != 0 or not lines:
+            raise RuntimeError("reference arm failed: " + out.stderr[-300:])
+        return json.loads(lines[-1])
+    one = run(max(2, args.cpu_steps), ORACLE_THREADS)
     cores = host_cores()
-    wide, _ = oracle_steps(cfg, H[:2], device, budget, cores)
-    layers = f"all {cfg.n_layers} layers" if Ls == cfg.n_layers else \
-        f"the first {Ls} of {cfg.n_layers} layers, tokens/s scaled by {Ls}/{cfg.n_layers}"
-    return {"value": statistics.median(runs), "unit": "tokens/s", "cores": ORACLE_THREADS, "kind": "oracle",
-            "repeats": runs, "spread": (max(runs) - min(runs)) / statistics.median(runs),
-            "all_host_cores": {"value": len(wide) * cfg.batch * (Ls / cfg.n_layers) / sum(wide), "cores": cores,
-                               "sample": "the first two of those steps, BLAS pinned to every core of the affinity mask"},
-            "sample": f"{H.shape[0]} decode steps ({layers}) of the bench token stream, numpy fp64, weights pre-generated, "
-                      f"BLAS pinned to {ORACLE_THREADS} thread(s); median of {repeats} repeats"}
+    wide = run(2, cores)
+    per_step = one["step_tok_s"]
+    return {"value": one["value"], "unit": "tokens/s", "cores": ORACLE_THREADS, "kind": "oracle",
+            "per_step": per_step, "spread": (max(per_step) - min(per_step)) / one["value"],
+            "all_host_cores": {"value": wide["value"], "cores": cores, "sample": wide["cpu_baseline"]["sample"]},
+            "sample": one["cpu_baseline"]["sample"] + f"; {len(per_step)} steps after 3 warm-up steps, in a process of its own"}
 
 
 def run_reference(args):
@@ -938,8 +951,8 @@ def run_reference(args):
     Ls = int(max(1, min(cfg.n_layers, 150.0 / max((K + W) * per_layer_s * 2, 1e-9))))
     _, H = hidden_rows(cfg, W + K, stream=0)
     H = H.numpy()
-    budget = 1 if cfg.budget < 0 else cfg.budget
-    cores = ORACLE_THREADS
+    budget = args.oracle_budget if args.oracle_budget >= 0 else (1 if cfg.budget < 0 else cfg.budget)
+    cores = args.oracle_threads if args.oracle_threads > 0 else ORACLE_THREADS
     times, Ls = oracle_steps(cfg, H, dev, budget, cores, layers=Ls)
     dt = sum(times[W:])
     tok_s = K * cfg.batch * (Ls / cfg.n_layers) / dt
@@ -952,7 +965,7 @@ def run_reference(args):
         "config": config_block(cfg, args),
         "cpu_baseline": {"value": tok_s, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": tok_s, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-        "gpu_launches": 0,
+        "gpu_launches": 0, "step_tok_s": [cfg.batch * (Ls / cfg.n_layers) / t for t in times[W:]],
     }))
 
 
@@ -980,6 +993,8 @@ def main():
     ap.add_argument("--no-arms", action="store_true")
     ap.add_argument("--no-resident", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--oracle-threads", type=int, default=0, help="reference arm: BLAS threads (default: one)")
+    ap.add_argument("--oracle-budget", type=int, default=-1, help="reference arm: prefetch budget (default: the configuration's, 1 if profiled)")
     ap.add_argument("--no-extra", action="store_true", help="skip the batched / DeepSeek-shaped legs and the targets block")
     ap.add_argument("--batched-steps", type=int, default=8)
     ap.add_argument("--dsvl2-steps", type=int, default=64)

@@ -102,7 +102,7 @@ def bench_tables(d):
                  "in-kernel window us"], rows))
     r = d["roofline"]
     print(f"\n(peak {fmt(r['peak'], 0)} GB/s {r.get('peak_source', '')}; read-only streaming rate of the device {fmt(r.get('read_only_stream_gb_s'), 0)} GB/s; "
-          f"ncu DRAM traffic per launch {fmt((r.get('traffic') or 0) / 1e6, 1)} MB.)")
+          + (f"ncu DRAM traffic per launch {fmt(r['traffic'] / 1e6, 1)} MB.)" if r.get("traffic") else "no ncu traffic figure for this workload.)"))
     res = d.get("resident")
     if res and "error" not in res:
         hf = res.get("host_free_on_demand", {})
@@ -120,7 +120,7 @@ def bench_tables(d):
               f"{fmt(leg.get('resident_host_free_tok_s'), 0)} tok/s; W = {fmt(leg['profile']['window_us'], 1)} us, t_xfer = {fmt(leg['profile']['t_xfer_us'], 1)} us.")
     c = d.get("cpu_baseline")
     if c:
-        print(f"\nCPU oracle: {fmt(c['value'], 3)} tok/s on {c['cores']} thread(s) (repeats {[round(x, 3) for x in c.get('repeats', [])]}); "
+        print(f"\nCPU oracle: {fmt(c['value'], 3)} tok/s on {c['cores']} thread(s) (per step {[round(x, 3) for x in c.get('per_step', c.get('repeats', []))]}); "
               f"{fmt(c.get('all_host_cores', {}).get('value'), 3)} tok/s with {c.get('all_host_cores', {}).get('cores')} threads. {c['sample']}.")
     print()
 
