@@ -40,8 +40,8 @@ import torch
 import synth
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from one ncu capture of a reduced
-# case of the same workload (4 layers; a launch reads the same expert blobs whatever the layer count): 75.54 MB read +
-# 1.0 - 1.7 MB written for the GEMV kernel, 306.7 + 8.7 MB for one 32-expert wave of the grouped kernel.
+# case of the same workload (4 layers; a launch reads the same expert blobs whatever the layer count): 75.53 MB read +
+# 0.8 - 1.2 MB written for the GEMV kernel, 306.7 + 8.7 MB for one 32-expert wave of the grouped kernel.
 NCU_DRAM_BYTES_PER_LAUNCH = {"qwen3": 76.6e6, "batched_wave": 315.4e6}
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
