@@ -22,6 +22,7 @@ the data path; value = all ranks' tokens / max-over-ranks time.
 from __future__ import annotations
 
 import argparse
+import copy
 import json
 import os
 import statistics
@@ -882,8 +883,9 @@ def make_oracle(cfg, wts, budget, slots=None, policy="adapter"):
 
 def oracle_steps(cfg, H, device, budget, threads, layers=None, mem_budget=40e9):
     """Times the oracle, as it stands, on the decode steps H[s] with `threads` BLAS threads.
-    Weights are generated before the clock starts (an untimed pass of the same step fills the
-    provider's cache, which is emptied after the step). The fp64 matrices of one step stay below
+    Weights are generated before the clock starts: an untimed pass of the same step from a copy of
+    the decoder's cache state asks the provider for exactly the experts the timed step will ask for
+    (demanded and prefetched), and the provider's cache is emptied after the step. The fp64 matrices of one step stay below
     `mem_budget` bytes: a batched step touches nearly every expert of every layer, so there the
     sample is the first Ls layers. Returns (seconds per step, list; layers used)."""
     per_layer = min(cfg.n_experts, cfg.batch * cfg.top_k) * 3 * cfg.inter * cfg.hidden * 8
@@ -892,12 +894,16 @@ def oracle_steps(cfg, H, device, budget, threads, layers=None, mem_budget=40e9):
         Ls = min(Ls, layers)
     sub = cfg.replace(n_layers=Ls) if Ls < cfg.n_layers else cfg
     wts = LazyWeights(sub, device if torch.cuda.is_available() else "cpu")
-    warm = make_oracle(sub, wts, 0, slots=cfg.n_experts, policy="on_demand")
     ref = make_oracle(sub, wts, budget)
     times = []
     with blas_threads(threads):
         for s in range(H.shape[0]):
-            warm.step(H[s])                      # untimed: fills the weight cache for this step
+            dry = copy.copy(ref)                 # same slot-table state, same weights: untimed, fills the weight cache for this step
+            dry.table = copy.deepcopy(ref.table)
+            dry.storage = [dict(d) for d in ref.storage]
+            dry.prev_rank = [list(r) for r in ref.prev_rank]
+            dry.step(H[s])
+            del dry
             t0 = time.perf_counter()
             ref.step(H[s])
             times.append(time.perf_counter() - t0)
@@ -911,9 +917,7 @@ ORACLE_THREADS = 1      # the oracle's numpy calls are small matrix-vector produ
 def cpu_baseline(args, cfg, budget):
     """The oracle on a bounded sample, timed in a process of its own: `bench.py --impl reference` on the first decode
     steps of the bench's token stream, on ORACLE_THREADS pinned thread(s) (the headline: reproducible), and once with
-    every host core the process may use. A fresh process, because the same code measured 0.5 and 0.9 tokens/s on the
-    same box depending on what the calling process had allocated before; this way the figure is the one the reference
-    arm gives."""
+    every host core the process may use. A process of its own, so that the figure is the one the reference arm gives."""
     def run(steps, threads):
         cmd = [sys.executable, os.path.abspath(__file__), "--impl", "reference", "--config", args.config, "--steps", str(steps),
                "--warmup", "3", "--oracle-threads", str(threads), "--oracle-budget", str(budget)]
