@@ -539,7 +539,9 @@ def grouped_alone(cfg, ctx, n_resident, peak, which, launches):
     st = ctx.stats()
     us = st["ffn_us"] / max(st["ffn_launches"], 1)
     ach = mean_bytes / (us * 1e-6) / 1e9
+    win = st["ffn_window_us"] / max(st["ffn_launches"], 1)      # in-kernel clock: first CTA past its dependency wait -> last CTA end
     return {"bound": "hbm", "kernel": ffn_kernel_name(cfg), "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+            "in_kernel_window_us": win, "frac_in_kernel_window": mean_bytes / (win * 1e-6) / 1e9 / peak if win > 0 else None,
             "traffic": NCU_DRAM_BYTES_PER_LAUNCH["batched_wave"] if (cfg.name == "batched" and n_resident == cfg.slots) else None,
             "peak_source": f"of {which}", "algorithmic_bytes_per_launch": mean_bytes, "us_per_launch": us,
             "launches": int(st["ffn_launches"]), "misses": int(st["misses"]), "distinct_experts_per_launch": mean_bytes / cfg.expert_bytes,

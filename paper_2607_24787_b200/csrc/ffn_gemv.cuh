@@ -310,29 +310,33 @@ ffn_gemv_kernel(const __grid_constant__ FfnArgs<MAXNB> a, const int depth) {
             if (!mbar_wait_bounded(bar0 + 8u * (i % depth), (i / depth) & 1, wait_limit)) break;
     }
 
-    // Sum the warps' partial y in warp order, one partial row per CTA. Staged as float4s, one per
-    // (segment, quad, lane), so that stores and loads of a warp are contiguous; a thread has the
-    // values of all warps in flight at once and adds them in warp order.
-    __syncthreads();
+    // Sum the warps' partial y in warp order, one partial row per CTA. A warp stages its values in
+    // its own ring (all its copies have landed and been read), so it need not wait for the others
+    // first: as float4s, one per (segment, quad, lane), so that stores and loads of a warp are
+    // contiguous; a thread has the values of all warps in flight at once and adds them in warp order.
     constexpr int Q = VEC / 4;                  // float4s per lane and segment
     constexpr int NP = D / 4;                   // float4 positions of a row
-    float4* red4 = reinterpret_cast<float4*>(smem);
+    static_assert(ROWB >= NP * sizeof(float4), "a ring row holds a warp's partial y");
+    {
+        float4* mine = reinterpret_cast<float4*>(ring);
 #pragma unroll
-    for (int s = 0; s < NSEG; ++s)
+        for (int s = 0; s < NSEG; ++s)
 #pragma unroll
-        for (int h = 0; h < Q; ++h) {
-            float4 t;
-            unpack2(ya[s][2 * h], t.x, t.y);
-            unpack2(ya[s][2 * h + 1], t.z, t.w);
-            red4[wi * NP + s * (32 * Q) + h * 32 + lane] = t;
-        }
+            for (int h = 0; h < Q; ++h) {
+                float4 t;
+                unpack2(ya[s][2 * h], t.x, t.y);
+                unpack2(ya[s][2 * h + 1], t.z, t.w);
+                mine[s * (32 * Q) + h * 32 + lane] = t;
+            }
+    }
     __syncthreads();
+    const size_t ring_stride = size_t(depth) * ROWB;
     float* out = a.partial + (size_t(tok) * G + c) * D;
     for (int p = threadIdx.x; p < NP; p += blockDim.x) {
         float4 v[kFfnMaxWarps];
 #pragma unroll
         for (int w2 = 0; w2 < kFfnMaxWarps; ++w2)
-            if (w2 < nw) v[w2] = red4[w2 * NP + p];
+            if (w2 < nw) v[w2] = reinterpret_cast<const float4*>(smem + w2 * ring_stride)[p];
         float4 acc = v[0];
 #pragma unroll
         for (int w2 = 1; w2 < kFfnMaxWarps; ++w2)

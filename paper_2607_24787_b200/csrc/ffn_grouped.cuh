@@ -91,6 +91,7 @@ struct GgArgs {
     int* next_chunk;           // zeroed before the launch (by the gather kernel), like act_ready
     unsigned char* act_g;      // [units][16 KB] A^T of each unit, in the shared-memory operand layout
     int* act_ready;            // [units]
+    unsigned long long* clock; // optional {earliest CTA past its dependency wait, latest CTA end} in ns (globaltimer)
 };
 
 // ---- tcgen05 / TMA wrappers ---------------------------------------------------
@@ -264,6 +265,7 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
     const uint32_t tmem = *tmem_slot;
     // barriers and TMEM are set up; everything below reads what the preceding kernels wrote
     grid_dep_wait();
+    if (a.clock && threadIdx.x == 0) atomicMin(a.clock, global_timer_ns());
     const int n_units = a.n_units_dev ? __ldcg(a.n_units_dev) : a.n_units;
     // P1 tasks of this CTA: the units b, b + grid, ...; P2 chunks: taken from the common list.
     const int my_units = int(blockIdx.x) < n_units ? (n_units - 1 - int(blockIdx.x)) / int(gridDim.x) + 1 : 0;
@@ -512,6 +514,7 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, kGgTmemCols);
+    if (a.clock && threadIdx.x == 0) atomicMax(a.clock + 1, global_timer_ns());
 }
 
 inline size_t ffn_grouped_smem() {

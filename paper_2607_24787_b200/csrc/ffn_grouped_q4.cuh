@@ -172,6 +172,7 @@ ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_co
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
     grid_dep_wait();
+    if (a.clock && threadIdx.x == 0) atomicMin(a.clock, global_timer_ns());
     const int n_units = a.n_units_dev ? __ldcg(a.n_units_dev) : a.n_units;
     const int my_units = int(blockIdx.x) < n_units ? (n_units - 1 - int(blockIdx.x)) / int(gridDim.x) + 1 : 0;
     const int sc_x0 = D / 2;                         // byte offset of the scales inside a packed row
@@ -471,6 +472,7 @@ ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_co
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, kGgTmemCols);
+    if (a.clock && threadIdx.x == 0) atomicMax(a.clock + 1, global_timer_ns());
 }
 
 inline size_t ffn_grouped_q4_smem() {

@@ -683,7 +683,8 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
     if (t && first) CU(c, cudaEventRecord(t->ffn_start[layer], c->compute));
     if (ring >= 0 && first) CU(c, cudaEventRecord(c->ring_start[ring], c->compute));
     GgArgs a{reinterpret_cast<const GgUnit*>(dd), n_units, nullptr, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status, c->wait_limit_ns,
-             nullptr, 0, nullptr, nullptr, nullptr};
+             nullptr, 0, nullptr, nullptr, nullptr, nullptr};
+    if (int rc = take_clock(c, kClkFfn, &a.clock)) return rc;
     if (q4) {
         CU(c, launch_k(ffn_grouped_q4_kernel, dim3(std::min(c->num_sms, n_units)), dim3(kQgThreads), ffn_grouped_q4_smem(), c->compute, true,
                        c->qmapn, c->qmapsc, c->xmaps, a));
@@ -1053,7 +1054,7 @@ int enqueue_host_free_layers(spm_ctx* c, int nb, float* h_out, int slot, bool pr
                           fold ? c->ws_partial : nullptr, G};
         if (int rc = launch_router(c, l, h_out, nullptr, nb, c->ws_x, nullptr, true, predict && l <= L - 2, &route, false)) return rc;
         unsigned long long* clock_slot = nullptr;
-        if (!use_tc) if (int rc = take_clock(c, kClkFfn, &clock_slot)) return rc;
+        if (int rc = take_clock(c, kClkFfn, &clock_slot)) return rc;
         auto fill = [&](auto& a) {
             a.pool = slot_ptr(c, l, 0);
             a.shared = m.n_shared ? static_cast<const unsigned char*>(c->buf.shared_experts) + size_t(l) * m.n_shared * c->blob : nullptr;
@@ -1084,7 +1085,7 @@ int enqueue_host_free_layers(spm_ctx* c, int nb, float* h_out, int slot, bool pr
                            m.dtype == SPM_DTYPE_Q4 ? 0 : c->max_units + 1));
             // (no chunk list here: the plan is built on the device, a chunk is a whole unit)
             GgArgs ga{units, 0, c->tc_counts, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status, c->wait_limit_ns,
-                      nullptr, 0, c->tc_ready, c->tc_act, c->tc_ready + 1};
+                      nullptr, 0, c->tc_ready, c->tc_act, c->tc_ready + 1, clock_slot};
             if (m.dtype == SPM_DTYPE_Q4)
                 CU(c, launch_k(ffn_grouped_q4_kernel, dim3(c->num_sms), dim3(kQgThreads), ffn_grouped_q4_smem(), c->compute, true,
                                c->qmapn, c->qmapsc, c->xmaps, ga));
