@@ -495,6 +495,16 @@ def batched_leg(args, m, peak, which, device):
         us = st["ffn_us"] / max(st["ffn_launches"], 1)
         out["offloaded"]["ffn_wave_in_run"] = {"us_per_launch": us, "algorithmic_bytes_per_launch": wave_bytes,
                                                 "gb_s": wave_bytes / (us * 1e-6) / 1e9, "launches": int(st["ffn_launches"])}
+    # the same steps with the grouped kernel's producer warp waiting for the copies itself (per unit) instead of the
+    # host ordering each launch behind the copy events
+    try:
+        mb.set_device_wait(1)
+        dw, _ = leg_offloaded(mb, cfg, H_dev, W, K)
+        out["offloaded_device_wait"] = {k: dw[k] for k in ("tok_s", "stall_us_per_layer", "router_done_to_ffn_done_us_per_layer",
+                                                          "late_arrivals", "h2d_gb_s_avg")}
+    except Exception as e:   # noqa: BLE001 (no stream-ordered memory writes on this driver)
+        out["offloaded_device_wait"] = {"error": str(e)[:200]}
+    mb.set_device_wait(0)
     # one wave by itself: the first `slots` experts of every layer resident, tokens routed among them (all hits)
     mb.cache_reset(); mb.set_policy("on_demand")
     S = cfg.slots

@@ -250,9 +250,11 @@ int spm_set_drop_modulo(spm_ctx* ctx, int modulo);
  * copy is followed on the copy stream by a wait of `us` microseconds (0 = off, at most 100000)
  * before the slot counts as loaded. Outputs are unchanged. */
 int spm_set_copy_delay_us(spm_ctx* ctx, int us);
-/* Device-side wait for batch-1 expert FFNs (default off; bf16, fp32 and 4-bit experts). Off: the compute stream waits on the
- * event of the batch of copies that fills the slots a launch reads, then the kernel starts. On: the
- * kernel is launched at once and its warps wait (bounded, SPM_ERR_TIMEOUT on expiry) on an arrival
+/* Device-side wait for the expert FFNs (default off): the batch-1 kernels (bf16, fp32 and 4-bit
+ * experts) and the grouped tensor-core kernels of batched decode (bf16 and 4-bit experts). Off: the
+ * compute stream waits on the event of the batch of copies that fills the slots a launch reads,
+ * then the kernel starts. On: the kernel is launched at once and its warps (batch 1) or the producer
+ * warp of each unit (grouped kernels) wait, bounded, SPM_ERR_TIMEOUT on expiry, on an arrival
  * counter that the copy stream bumps after the last copy of that batch has landed, so rows of
  * resident experts are streamed while missing ones are still in flight and no launch latency
  * follows the last copy. Outputs are bit-identical either way. With it on, the timed FFN duration

@@ -71,6 +71,12 @@ struct GgTask {
     int32_t unit;
     int16_t dt0, dt1;
 };
+// Optional device-side wait of a unit: its expert's copy has landed once ready[watch] has reached `want`
+// (the arrival counter of the slot that leads the batch of copies); watch < 0: nothing to wait for.
+struct GgWait {
+    int32_t watch;
+    uint32_t want;
+};
 constexpr int kGgActReady = 4;           // arrivals (one per epilogue warp) that complete a unit's A^T
 constexpr int kGgQueue = 4;              // tasks the producer warp may be ahead of the other warps
 
@@ -92,6 +98,9 @@ struct GgArgs {
     unsigned char* act_g;      // [units][16 KB] A^T of each unit, in the shared-memory operand layout
     int* act_ready;            // [units]
     unsigned long long* clock; // optional {earliest CTA past its dependency wait, latest CTA end} in ns (globaltimer)
+    // optional device-side waiting: per unit, what its expert's copy is awaited by; the arrival counters of all slots
+    const GgWait* unit_wait;
+    const unsigned* ready;
 };
 
 // ---- tcgen05 / TMA wrappers ---------------------------------------------------
@@ -195,6 +204,26 @@ __device__ __forceinline__ bool gg_wait(uint32_t bar, uint32_t parity, const GgA
             return false;
         }
     }
+}
+
+// bounded wait for the copy stream's arrival counter of a batch of expert copies (written from outside the GPU's
+// kernels, hence system scope); the weights are then read through the async proxy
+__device__ __forceinline__ bool gg_wait_arrival(const unsigned* p, unsigned want, const GgAbort& ab) {
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+        unsigned v;
+        asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+        if (int(v - want) >= 0) break;
+        if (*ab.flag) return false;
+        if (global_timer_ns() - t0 > ab.limit_ns) {
+            *ab.flag = 1;
+            atomicOr(ab.status, kStatusCopyTimeout);
+            return false;
+        }
+        __nanosleep(200);
+    }
+    asm volatile("fence.proxy.async;" ::: "memory");
+    return true;
 }
 
 // bounded wait for a counter in global memory (another CTA's arrivals) to reach `want`
@@ -310,6 +339,11 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
             publish(GgTask{u, -1, -1});
             if (!ok) break;
             const GgUnit un = a.units[u];
+            if (a.unit_wait) {       // the expert's copy may still be on its way: wait for it here, not on the host
+                const GgWait uw = a.unit_wait[u];
+                if (uw.watch >= 0) ok = __all_sync(0xffffffffu, gg_wait_arrival(a.ready + uw.watch, uw.want, ab));
+                if (!ok) break;
+            }
             const int xbox = gg_token_box(un.ntok);
             const CUtensorMap* xmap = &xmaps.m[xbox];
             const uint32_t x_bytes = gg_token_rows(xbox) * 128;
@@ -338,6 +372,11 @@ ffn_grouped_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_consta
             publish(tk);
             if (!ok) break;
             const GgUnit un = a.units[tk.unit];
+            if (a.unit_wait) {       // the tiles below are requested before the unit's A^T (and with it its expert's arrival) is known
+                const GgWait uw = a.unit_wait[tk.unit];
+                if (uw.watch >= 0) ok = __all_sync(0xffffffffu, gg_wait_arrival(a.ready + uw.watch, uw.want, ab));
+                if (!ok) break;
+            }
             // The first ring-full of tiles is issued before A^T is fetched: those stage slots are freed by
             // MMAs of earlier tasks only, so the weight stream does not pause while this warp waits for the
             // preceding chunk's MMAs and for the unit's arrival counter.

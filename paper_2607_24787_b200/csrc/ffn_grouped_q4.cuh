@@ -185,7 +185,13 @@ ffn_grouped_q4_kernel(const __grid_constant__ CUtensorMap nib64, const __grid_co
             uint32_t np = 0;              // packed stages issued so far
             bool ok = true;
             auto load_packed = [&](const QgSeq& q) {
-                const GgUnit un = a.units[blockIdx.x + q.unit() * gridDim.x];
+                const int32_t u = int32_t(blockIdx.x + q.unit() * gridDim.x);
+                const GgUnit un = a.units[u];
+                if (a.unit_wait && q.phase1 && q.idx == 0) {     // first item of a unit: its expert's copy may still be on its way
+                    const GgWait uw = a.unit_wait[u];
+                    if (uw.watch >= 0) ok = __all_sync(0xffffffffu, gg_wait_arrival(a.ready + uw.watch, uw.want, ab));
+                    if (!ok) return;
+                }
                 const uint32_t ps = np % kQgPackedStages;
                 if (np >= uint32_t(kQgPackedStages))
                     ok = __all_sync(0xffffffffu, gg_wait(smem_u32(qempty + ps), ((np / kQgPackedStages) - 1) & 1, ab));

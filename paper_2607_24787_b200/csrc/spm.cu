@@ -75,7 +75,7 @@ struct spm_ctx {
     unsigned char* tc_desc_dev = nullptr;     // kDescRing wave descriptors
     unsigned char* tc_desc_host = nullptr;    // pinned staging, same layout
     int* tc_counts = nullptr;                 // {units, rows} of a wave planned on the device
-    size_t tc_desc_bytes = 0, tc_off_rows = 0, tc_off_rowmap = 0, tc_off_chunks = 0, tc_chunk_cap = 0;
+    size_t tc_desc_bytes = 0, tc_off_rows = 0, tc_off_rowmap = 0, tc_off_chunks = 0, tc_chunk_cap = 0, tc_off_wait = 0;
     unsigned char* tc_act = nullptr;          // [max_units][16 KB] A^T slots of the bf16 grouped kernel
     int* tc_ready = nullptr;                  // [1 + max_units] chunk counter, then the slots' arrival counters
     std::vector<GgTaskHost> plan_chunks;
@@ -231,7 +231,7 @@ struct Carve {
 struct Layout {
     size_t pools, slot_gen, x, logits, pihat, w, scores, partial, h, ids, order, clock, slot_map, codes, counters, status, total;
     size_t tc_xs, tc_wrow, tc_partial, tc_desc, tc_counts, tc_act, tc_ready;       // batched tensor-core path only
-    size_t desc_bytes, off_rows, off_rowmap, off_chunks, chunk_cap;
+    size_t desc_bytes, off_rows, off_rowmap, off_chunks, chunk_cap, off_wait;
     int rows_cap, n_jt, max_units;
     bool tc;
 };
@@ -264,7 +264,8 @@ Layout layout_of(const spm_model_cfg* m, int S) {
         // phase-2 chunk list of the bf16 kernel: at most one chunk per kGgMinChunk d-tiles, at least one per unit
         l.off_chunks = l.off_rowmap + align_up(size_t(m->max_batch) * SPM_MAX_TOPK * 4, 256);
         l.chunk_cap = size_t(l.max_units) * size_t(std::max(1, (m->hidden / kGgTileRows + kGgMinChunk - 1) / kGgMinChunk));
-        l.desc_bytes = l.off_chunks + align_up(l.chunk_cap * sizeof(GgTask), 256);
+        l.off_wait = l.off_chunks + align_up(l.chunk_cap * sizeof(GgTask), 256);      // per unit: what its expert's copy is awaited by
+        l.desc_bytes = l.off_wait + align_up(size_t(l.max_units) * sizeof(GgWait), 256);
         l.tc_xs = c.take(size_t(l.rows_cap + kGgTokens) * D * 2);
         l.tc_wrow = c.take(size_t(l.rows_cap) * 4);
         l.tc_partial = c.take(size_t(l.n_jt) * l.rows_cap * D * 4);
@@ -632,7 +633,7 @@ void harvest_ring(spm_ctx* c, size_t i) {
 // expert, upload the wave descriptor, then gather -> grouped tcgen05 FFN -> combine.
 int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, const float* w, int nb,
                         float* h_inout, const std::vector<int16_t>& slot_of_expert, bool first, bool last,
-                        Timing* t, int ring) {
+                        Timing* t, int ring, bool dev_wait) {
     const spm_model_cfg& m = c->cfg;
     const int K = m.top_k;
     const size_t d = c->tc_desc_pos++ % kDescRing;
@@ -642,6 +643,7 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
     GgUnit* units = reinterpret_cast<GgUnit*>(hd);
     GgRow* rows = reinterpret_cast<GgRow*>(hd + c->tc_off_rows);
     int32_t* rowmap = reinterpret_cast<int32_t*>(hd + c->tc_off_rowmap);
+    GgWait* waits = reinterpret_cast<GgWait*>(hd + c->tc_off_wait);
     std::fill(rowmap, rowmap + size_t(nb) * SPM_MAX_TOPK, -1);
     // counting sort of the wave's (token, k) pairs by expert: rows of an expert keep token-major order
     int n_rows = 0, n_units = 0;
@@ -653,8 +655,14 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
         const int cnt = row_of[e + 1];
         row_of[e + 1] = row_of[e] + cnt;
         if (cnt == 0) continue;
-        for (int jt = 0; jt < c->n_jt; ++jt)
+        // with device-side waiting a slot whose copy had not landed when the host looked stays pending: the
+        // producer warp of its units waits for the batch's arrival counter
+        const size_t ks = size_t(layer) * c->S + slot_of_expert[e];
+        const GgWait uw = (dev_wait && c->slot_pending[ks]) ? GgWait{int32_t(c->slot_dep[ks]), c->slot_want[ks]} : GgWait{-1, 0u};
+        for (int jt = 0; jt < c->n_jt; ++jt) {
+            waits[n_units] = uw;
             units[n_units++] = GgUnit{layer * c->S + slot_of_expert[e], jt, row_of[e], cnt};
+        }
     }
     n_rows = row_of[m.n_experts];
     for (int tk = 0; tk < nb; ++tk)
@@ -683,8 +691,12 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
     if (t && first) CU(c, cudaEventRecord(t->ffn_start[layer], c->compute));
     if (ring >= 0 && first) CU(c, cudaEventRecord(c->ring_start[ring], c->compute));
     GgArgs a{reinterpret_cast<const GgUnit*>(dd), n_units, nullptr, c->tc_wrow, c->tc_partial, c->rows_cap, m.hidden, m.inter, c->ws_status, c->wait_limit_ns,
-             nullptr, 0, nullptr, nullptr, nullptr, nullptr};
+             nullptr, 0, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     if (int rc = take_clock(c, kClkFfn, &a.clock)) return rc;
+    if (dev_wait) {
+        a.unit_wait = reinterpret_cast<const GgWait*>(dd + c->tc_off_wait);
+        a.ready = c->ws_slot_gen;
+    }
     if (q4) {
         CU(c, launch_k(ffn_grouped_q4_kernel, dim3(std::min(c->num_sms, n_units)), dim3(kQgThreads), ffn_grouped_q4_smem(), c->compute, true,
                        c->qmapn, c->qmapsc, c->xmaps, a));
@@ -742,7 +754,9 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
     }
 
     const int G = ffn_grid_for(c, nb);
-    const bool dev_wait = c->device_wait && nb == 1 && stream_write32_fn() != nullptr;
+    const bool use_tc = nb > 1 && c->tc_ok && c->batched_path == 0;
+    // kernels that can wait for a copy themselves: the batch-1 GEMV kernels and the grouped tensor-core kernels
+    const bool dev_wait = c->device_wait && (nb == 1 || use_tc) && stream_write32_fn() != nullptr;
     std::vector<int16_t>& slot_of_expert = c->wave_slot;   // experts computed in the current wave
     for (int wave = 0; wave < n_waves; ++wave) {
         slot_of_expert.assign(m.n_experts, -1);
@@ -781,7 +795,6 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
         }
 
         const bool first = wave == 0, last = wave == n_waves - 1;
-        const bool use_tc = nb > 1 && c->tc_ok && c->batched_path == 0;
         unsigned long long* clock_slot = nullptr;
         if (!use_tc) if (int rc = take_clock(c, kClkFfn, &clock_slot)) return rc;
         auto fill = [&](auto& a) {
@@ -821,7 +834,7 @@ int run_ffn(spm_ctx* c, int layer, const float* x_norm, const int32_t* ids, cons
             }
         };
         if (use_tc) {
-            if (int rc = launch_grouped_wave(c, layer, x_norm, ids, w, nb, h_inout, slot_of_expert, first, last, t, ring)) return rc;
+            if (int rc = launch_grouped_wave(c, layer, x_norm, ids, w, nb, h_inout, slot_of_expert, first, last, t, ring, dev_wait)) return rc;
         } else {
             if (t && first) CU(c, cudaEventRecord(t->ffn_start[layer], c->compute));
             if (ring >= 0 && first) CU(c, cudaEventRecord(c->ring_start[ring], c->compute));
@@ -1326,7 +1339,7 @@ int spm_init(const spm_model_cfg* cfg, int slots_per_layer, int budget, const sp
         c->tc_desc_dev = base + lay.tc_desc;
         c->tc_counts = reinterpret_cast<int*>(base + lay.tc_counts);
         c->tc_desc_bytes = lay.desc_bytes; c->tc_off_rows = lay.off_rows; c->tc_off_rowmap = lay.off_rowmap;
-        c->tc_off_chunks = lay.off_chunks; c->tc_chunk_cap = lay.chunk_cap;
+        c->tc_off_chunks = lay.off_chunks; c->tc_chunk_cap = lay.chunk_cap; c->tc_off_wait = lay.off_wait;
         c->tc_act = base + lay.tc_act;
         c->tc_ready = reinterpret_cast<int*>(base + lay.tc_ready);
         if (!cu(cudaMemsetAsync(c->tc_xs, 0, size_t(lay.rows_cap + kGgTokens) * cfg->hidden * 2, c->compute), "cudaMemsetAsync")) return bail(SPM_ERR_CUDA);

@@ -124,6 +124,78 @@ def test_free_running_events_match_policy_oracle(setup):
         assert m.stats()["waves"] > 0
 
 
+def test_device_side_wait_in_the_producer_warp_is_bit_identical(setup):
+    """The grouped kernels' producer warp can wait for a unit's expert copy itself (per unit, on the
+    batch's arrival counter) instead of the host ordering the launch behind the copy events: same
+    outputs, same cache events, and some launches really had copies in flight."""
+    from paper_2607_24787_b200 import binding as B
+    cfg, nb, m, wts, H = setup
+    runs = {}
+    for on in (0, 1):
+        m.cache_reset(); m.set_policy("adapter"); m.set_budget(2)
+        try:
+            m.set_device_wait(on)
+        except B.SpmError:
+            pytest.skip("stream-ordered memory writes are not available on this driver")
+        outs = []
+        for s in range(H.shape[0]):
+            outs.append(m.decode_step(dev(H[s])))
+        m.synchronize()
+        runs[on] = (np.stack([o.cpu().numpy() for o in outs]), m.events(), m.stats())
+    m.set_device_wait(0)
+    assert np.array_equal(runs[0][0], runs[1][0]) and runs[0][1] == runs[1][1]
+    assert runs[1][2]["misses"] > 0 and runs[1][2]["ffn_launches"] > 0
+    m.check_invariants()
+
+
+@pytest.mark.parametrize("name", ["small_waves", "q4_small_waves"])
+def test_producer_warp_wait_runs_out_and_the_context_survives(name):
+    """An arrival counter that is never bumped (withheld on the host; the bytes land) makes the
+    producer warp's wait run out after the configured limit: the kernel winds down, the host reads
+    SPM_ERR_TIMEOUT once, and after a cache reset the same context computes the same outputs as a
+    context that never waited on the device."""
+    import time
+    from paper_2607_24787_b200 import binding as B
+    from paper_2607_24787_b200.build import build
+    from paper_2607_24787_b200.synth_model import build_from_synth
+    build()
+    cfg, nb = CASES[name]
+    cfg = cfg.replace(batch=nb)
+    tok = synth.zipf_tokens(cfg, steps=2)
+    H = synth.embedding_rows(cfg, tok.reshape(-1)).numpy().reshape(2, nb, cfg.hidden)
+    m = build_from_synth(cfg)
+    try:
+        m.set_policy("on_demand")
+        want = []
+        for s in range(2):
+            want.append(m.decode_step(dev(H[s])))
+        m.synchronize()
+        want = [o.cpu().numpy() for o in want]
+        try:
+            m.set_device_wait(1)
+        except B.SpmError:
+            pytest.skip("stream-ordered memory writes are not available on this driver")
+        m.set_device_wait_limit_us(3000)
+        m.cache_reset()
+        m.test_withhold_arrivals(1)
+        t0 = time.perf_counter()
+        with pytest.raises(B.SpmError) as e:
+            m.decode_step(dev(H[0]))
+            m.synchronize()
+        assert e.value.code == -4                    # SPM_ERR_TIMEOUT
+        assert time.perf_counter() - t0 < 2.0
+        m.synchronize()                              # reported once
+        m.set_device_wait_limit_us(0)
+        m.cache_reset()
+        for s in range(2):
+            out = m.decode_step(dev(H[s]))
+            m.synchronize()
+            assert np.array_equal(out.cpu().numpy(), want[s])
+        m.check_invariants()
+    finally:
+        m.close()
+
+
 WIDTH_CASES = {
     "bf16": synth.get_config("qwen3", n_layers=1, hidden=512, n_experts=8, inter=256, top_k=3, slots=8, budget=1),
     "q4": synth.get_config("qwen3_q4", n_layers=1, hidden=512, n_experts=8, inter=256, top_k=3, slots=8, budget=1),
