@@ -118,6 +118,9 @@ def bench_tables(d):
         print(f"\n`{leg['workload']}`: offloaded {fmt(o['tok_s'], 1)} tok/s (adapter policy, {o['steps']} steps, stall {fmt(o['stall_us_per_layer'], 0)} us per layer, "
               f"{fmt(o['copies_per_token'], 1)} copies per token, H2D {fmt(o['h2d_gb_s_avg'], 1)} GB/s); all resident, host-free "
               f"{fmt(leg.get('resident_host_free_tok_s'), 0)} tok/s; W = {fmt(leg['profile']['window_us'], 1)} us, t_xfer = {fmt(leg['profile']['t_xfer_us'], 1)} us.")
+        dw = leg.get("offloaded_device_wait")
+        if dw and "error" not in dw:
+            print(f"With the kernel's producer warps waiting for the copies themselves: {fmt(dw['tok_s'], 1)} tok/s.")
     c = d.get("cpu_baseline")
     if c:
         print(f"\nCPU oracle: {fmt(c['value'], 3)} tok/s on {c['cores']} thread(s) (per step {[round(x, 3) for x in c.get('per_step', c.get('repeats', []))]}); "
