@@ -383,7 +383,9 @@ def run_ours(args):
                 "frac_of_nominal_8TBs": b2b["gb_s"] / NOMINAL_HBM_GBS,
                 "region": (f"{b2b['launches']} launches of the kernel alone back to back on the compute stream (spm_time_ffn_kernel), "
                            "all experts resident, pools of all layers cycled (nothing served from L2), one CUDA event pair "
-                           "around all of them, launched as a decode step launches it (programmatic dependent launch); "
+                           "around all of them, every launch with the programmatic-serialisation attribute all kernels of a decode step "
+                           "carry: a launch requests its first weight rows while the FFN launch before it drains (inside a decode "
+                           "step its predecessor is the routing kernel, so there us_per_launch_serialized applies); "
                            "us_per_launch = span / launches") if cfg.batch == 1 else
                           (f"{b2b['launches']} spm_moe_ffn launches back to back on the compute stream, all experts resident "
                            "(pools of all layers cycled, nothing served from L2), CUDA event pair per launch"),

@@ -327,7 +327,7 @@ int spm_measure_read_bandwidth(spm_ctx* ctx, size_t bytes, int reps, double* gb_
  * ids[i*K .. i*K+K) (HOST) plus the layer's shared experts, x_norm dev [D], w dev [K], between one
  * pair of CUDA events, and waits. Every expert named must already hold a slot
  * (SPM_ERR_NOT_RESIDENT otherwise: nothing is loaded here).
- * chained = 1: launched as in a decode step, with the programmatic-serialisation attribute, so a
+ * chained = 1: launched with the programmatic-serialisation attribute (as all kernels of a decode step are), so a
  * launch fetches its first weight rows while its predecessor drains; 0: plain launches, each
  * starts after the one before it has ended.
  * *us_per_launch = event span / launches. *window_us (may be NULL) = mean in-kernel window
