@@ -604,34 +604,52 @@ static __global__ void gg_gather_kernel(const float* __restrict__ x, const float
     if (threadIdx.x == 0) wrow[r] = w[size_t(ri.token) * K + ri.k];
 }
 
-// h[t][d] += sum over the token's experts of this wave (in k order) and j-tiles (ascending) of
+// h[t][d] += sum over the token's experts of this wave (in k order) of the sum over j-tiles (ascending) of
 // P[jt][rowmap[t][k]][d]; rowmap < 0 marks experts that belong to another wave.
+// Block = (32 groups of four columns) x (K experts): thread (c, k) has all j-tiles of its expert in flight at
+// once and adds them in j order; the K sums meet in shared memory and are added in k order, so the result does
+// not depend on the launch geometry beyond this fixed tree.
+constexpr int kCombineCols = 32;          // float4 column groups per block
+constexpr int kCombineMaxJt = 16;         // j-tiles a thread keeps in flight (intermediate size <= 2048)
 static __global__ void gg_combine_kernel(const float* __restrict__ partial, const int32_t* __restrict__ rowmap, int K, int n_jt,
                                          int rows_cap, int D, float* h) {
+    __shared__ float4 part[SPM_MAX_TOPK][kCombineCols];
     grid_dep_launch();
     grid_dep_wait();
     const int t = blockIdx.y;
-    const int d = (blockIdx.x * blockDim.x + threadIdx.x) * 4;     // four columns per thread
-    if (d >= D) return;
-    const float4 h_in = *reinterpret_cast<const float4*>(h + size_t(t) * D + d);
+    const int c = threadIdx.x % kCombineCols, k = threadIdx.x / kCombineCols;
+    const int d = (blockIdx.x * kCombineCols + c) * 4;
+    const int r = (k < K && d < D) ? rowmap[t * SPM_MAX_TOPK + k] : -1;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    constexpr int JB = 8;                 // j-tiles fetched together
-    for (int k = 0; k < K; ++k) {
-        const int r = rowmap[t * SPM_MAX_TOPK + k];
-        if (r < 0) continue;
-        for (int j0 = 0; j0 < n_jt; j0 += JB) {
-            float4 v[JB];
+    if (r >= 0) {
+        for (int j0 = 0; j0 < n_jt; j0 += kCombineMaxJt) {
+            float4 v[kCombineMaxJt];
 #pragma unroll
-            for (int j = 0; j < JB; ++j)
+            for (int j = 0; j < kCombineMaxJt; ++j)
                 v[j] = j0 + j < n_jt ? __ldcg(reinterpret_cast<const float4*>(partial + (size_t(j0 + j) * rows_cap + r) * D + d))
                                      : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-            for (int j = 0; j < JB; ++j)
+            for (int j = 0; j < kCombineMaxJt; ++j)
                 if (j0 + j < n_jt) { acc.x += v[j].x; acc.y += v[j].y; acc.z += v[j].z; acc.w += v[j].w; }
         }
     }
-    *reinterpret_cast<float4*>(h + size_t(t) * D + d) = make_float4(h_in.x + acc.x, h_in.y + acc.y, h_in.z + acc.z, h_in.w + acc.w);
+    if (k < K) part[k][c] = acc;
+    __syncthreads();
+    if (k == 0 && d < D) {
+        float4 tot = *reinterpret_cast<const float4*>(h + size_t(t) * D + d);
+        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int kk = 0; kk < K; ++kk) {
+            if (rowmap[t * SPM_MAX_TOPK + kk] < 0) continue;
+            const float4 p = part[kk][c];
+            sum.x += p.x; sum.y += p.y; sum.z += p.z; sum.w += p.w;
+        }
+        tot.x += sum.x; tot.y += sum.y; tot.z += sum.z; tot.w += sum.w;
+        *reinterpret_cast<float4*>(h + size_t(t) * D + d) = tot;
+    }
 }
+// launch geometry of gg_combine_kernel for hidden size D and top-K
+inline dim3 gg_combine_grid(int D, int nb) { return dim3((D / 4 + kCombineCols - 1) / kCombineCols, nb); }
+inline dim3 gg_combine_block(int K) { return dim3(kCombineCols * K); }
 
 // Wave plan built on the device (all experts resident, one wave): the (token, k) pairs sorted by
 // expert id, then token, then k — the order the host-side planner produces — the units of every

@@ -711,7 +711,7 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
     }
     if (t && last) CU(c, cudaEventRecord(t->ffn_end[layer], c->compute));
     if (ring >= 0 && last) { CU(c, cudaEventRecord(c->ring_end[ring], c->compute)); c->ring_used[ring] = 1; }
-    CU(c, launch_k(gg_combine_kernel, dim3((m.hidden / 4 + 127) / 128, nb), dim3(128), 0, c->compute, true,
+    CU(c, launch_k(gg_combine_kernel, gg_combine_grid(m.hidden, nb), gg_combine_block(K), 0, c->compute, true,
                    (const float*)c->tc_partial, reinterpret_cast<const int32_t*>(dd + c->tc_off_rowmap), K, c->n_jt, c->rows_cap, m.hidden, h_inout));
     c->kernel_launches += 3;
     c->ffn_launches++;
@@ -1104,7 +1104,7 @@ int enqueue_host_free_layers(spm_ctx* c, int nb, float* h_out, int slot, bool pr
                                c->qmapn, c->qmapsc, c->xmaps, ga));
             else
                 CU(c, launch_k(ffn_grouped_kernel, dim3(c->num_sms), dim3(kGgThreads), ffn_grouped_smem(), c->compute, true, c->wmap, c->xmaps, ga));
-            CU(c, launch_k(gg_combine_kernel, dim3((m.hidden / 4 + 127) / 128, nb), dim3(128), 0, c->compute, true,
+            CU(c, launch_k(gg_combine_kernel, gg_combine_grid(m.hidden, nb), gg_combine_block(K), 0, c->compute, true,
                            (const float*)c->tc_partial, (const int32_t*)rowmap, K, c->n_jt, c->rows_cap, m.hidden, h_out));
             c->kernel_launches += 5;
             c->ffn_launches++;
