@@ -215,3 +215,47 @@ def test_batched_shape_tensor_core_path_teacher_forced(base):
         m.check_invariants()
     finally:
         m.close()
+
+
+# ---------------------------------------------------------------- DeepSeek-shaped configuration at full size
+def test_deepseek_shape_full_size_free_running_against_the_oracle():
+    """The DeepSeek-VL2-Tiny-shaped configuration as it is benchmarked (12 layers, hidden 1280, 64
+    routed experts of intermediate 896, top-6 plus two always-resident shared experts, 8 slots per
+    layer, adapter policy), free-running and step by step against the whole oracle: outputs within
+    the bf16 tolerance, every cache event and counter bit-exact (near-ties handled by the re-seed
+    protocol of the small-size parity tests). The oracle's matrices are regenerated on demand."""
+    from helpers import SynthWeights
+    from paper_2607_24787_b200.build import build
+    from paper_2607_24787_b200.synth_model import build_from_synth
+    from test_gpu_parity import free_run_lockstep
+    build()
+
+    class OnDemandWeights(SynthWeights):
+        def expert(self, l, e):
+            if (l, e) not in self._cache:
+                g, u, d = synth.expert_matrices(self.cfg, l, [e], "cuda")
+                self._cache[(l, e)] = (f64(g[0]), f64(u[0]), f64(d[0]))
+            return self._cache[(l, e)]
+
+    cfg = synth.get_config("dsvl2")
+    free_host = int(open("/proc/meminfo").read().split("MemAvailable:")[1].split()[0]) * 1024
+    if free_host < 16 * 2 ** 30 or torch.cuda.mem_get_info()[0] < 8 * 2 ** 30:
+        pytest.skip("not enough host or device memory for the 5.3 GB expert store")
+    steps, budget = 5, 2
+    m = build_from_synth(cfg, budget=budget)
+    try:
+        wts = OnDemandWeights(cfg)
+        tok = synth.zipf_tokens(cfg, steps=steps)
+        H = synth.embedding_rows(cfg, tok[:, 0]).numpy()
+        ref, recs, divergences, flagged = free_run_lockstep(cfg, m, wts, H, steps, "adapter", budget, None)
+        assert divergences <= len(flagged)
+        if not divergences:
+            assert m.events() == ref.table.events
+            st = m.stats()
+            for k in ("hits", "hits_prefetched", "misses", "evictions", "wasted", "prefetch_issued", "touches", "planned"):
+                assert st[k] == getattr(ref.table.stats, k), k
+            assert st["misses"] > 0 and st["prefetch_issued"] > 0
+        m.check_invariants()
+    finally:
+        m.close()
+
