@@ -23,6 +23,8 @@ CASES = {
     "small_waves": (synth.get_config("qwen3", n_layers=2, hidden=256, n_experts=24, inter=256, top_k=4, slots=6, budget=2), 17),
     "wide": (synth.get_config("qwen3", n_layers=2, hidden=1280, n_experts=16, inter=384, top_k=3, slots=16, budget=2), 64),
     "one_wave_many_tokens": (synth.get_config("qwen3", n_layers=3, hidden=512, n_experts=8, inter=128, top_k=2, slots=8, budget=1), 64),
+    # the largest top-k the boundary allows minus shared experts: the combine kernel's block is 32 x K threads
+    "many_k": (synth.get_config("qwen3", n_layers=2, hidden=256, n_experts=32, inter=256, top_k=16, slots=32, budget=2), 9),
     # 4-bit experts de-quantised inside the grouped kernel (scales every fourth K-block / second d-tile)
     "q4_small_waves": (synth.get_config("qwen3_q4", n_layers=2, hidden=256, n_experts=24, inter=256, top_k=4, slots=6, budget=2), 17),
     "q4_wide": (synth.get_config("qwen3_q4", n_layers=2, hidden=1280, n_experts=16, inter=384, top_k=3, slots=16, budget=2), 64),
