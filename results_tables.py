@@ -89,6 +89,14 @@ def bench_tables(d):
                  fmt(t["exposed_below_on_demand"].get(k)) if k != "on_demand" else ""]
                 for k, v in t.items() if isinstance(v, dict) and "stall_us_per_layer" in v]
         print(table(["arm", "stall us/layer", "tok/s", "ExpertRecall@M", "below on-demand"], rows))
+    pr = (t or {}).get("paper_regime")
+    if pr and "error" not in pr:
+        print(f"\nWith an attention stand-in of {pr['attention_stub_us']} us per layer (window {fmt(pr['window_us'], 0)} us = "
+              f"{fmt(pr['window_us'] / pr['t_xfer_us'], 2)} transfers, the paper's regime; budget = floor(W / t_xfer) = {pr['budget_raw']}), "
+              f"{pr['steps_per_arm']} steps per arm:\n")
+        rows = [[k, fmt(v["tok_s"]), fmt(v["stall_us_per_layer"], 1), fmt(v.get("ready_recall"), 3), fmt(v.get("expert_recall_at_budget"), 3),
+                 f"{100 * v['gain_over_on_demand']:+.1f} %"] for k, v in pr.items() if isinstance(v, dict) and "tok_s" in v]
+        print(table(["arm", "tok/s", "stall us/layer", "ReadyRecall", "ExpertRecall@M", "against on-demand"], rows))
     print("\nExpert-FFN kernels against the measured HBM copy bandwidth:\n")
     rows = [roofline_row(cfg.split(":")[0], d["roofline"])]
     for name, leg in (d.get("configs") or {}).items():
