@@ -307,3 +307,52 @@ def test_non_finite_hidden_row_is_reported_not_propagated_silently():
     want, _ = ref.step(H[1])
     assert M.rel_linf(out.cpu().numpy().astype(np.float64)[0], want[0]) < 4e-5
     m.close()
+
+
+def test_long_run_with_changing_policies_and_wait_modes_stays_router_preserving():
+    """800 decode steps on one context while the policy, the budget, the way the FFN waits for its copies
+    and the fault injection on prefetch requests change every 40 steps: every step's output equals, bit for
+    bit, the output of a context that holds all experts (Section 3.1: prediction never changes routing or
+    outputs), the slot table's invariants hold throughout, and the counters add up."""
+    from paper_2607_24787_b200 import binding as B
+    cfg = synth.get_config("tiny", n_layers=3, n_experts=12, slots=5, budget=2)
+    steps, span = 800, 40
+    tok = synth.zipf_tokens(cfg, steps=steps)
+    H = synth.embedding_rows(cfg, tok.reshape(-1)).numpy().reshape(steps, 1, cfg.hidden)
+    full = build(cfg, slots=cfg.n_experts, budget=0)
+    full.set_policy("on_demand")
+    want = []
+    for s in range(steps):
+        want.append(full.decode_step(dev(H[s])))
+    full.synchronize()
+    want = [w.cpu().numpy() for w in want]
+    full.close()
+    m = build(cfg)
+    try:
+        can_wait = True
+        try:
+            m.set_device_wait(1); m.set_device_wait(0)
+        except B.SpmError:
+            can_wait = False
+        policies = ["adapter", "on_demand", "naive", "pred0", "adapter"]
+        outs = []
+        for s in range(steps):
+            if s % span == 0:
+                phase = s // span
+                m.synchronize()
+                m.check_invariants()
+                m.set_policy(policies[phase % len(policies)])
+                m.set_budget(phase % 4)
+                m.set_drop_modulo(3 if phase % 3 == 2 else 0)
+                if can_wait:
+                    m.set_device_wait(phase % 2)
+            outs.append(m.decode_step(dev(H[s])))
+        m.synchronize()
+        for s in range(steps):
+            assert np.array_equal(outs[s].cpu().numpy(), want[s]), s
+        st = m.stats()
+        assert st["hits"] + st["misses"] == steps * cfg.n_layers * cfg.top_k
+        assert st["steps"] == steps and st["prefetch_issued"] > 0 and st["dropped"] > 0
+        m.check_invariants()
+    finally:
+        m.close()
