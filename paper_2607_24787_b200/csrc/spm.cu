@@ -76,6 +76,8 @@ struct spm_ctx {
     unsigned char* tc_desc_host = nullptr;    // pinned staging, same layout
     int* tc_counts = nullptr;                 // {units, rows} of a wave planned on the device
     size_t tc_desc_bytes = 0, tc_off_rows = 0, tc_off_rowmap = 0, tc_off_chunks = 0, tc_chunk_cap = 0, tc_off_wait = 0;
+    int wave_row_off = 0;                     // rows of the sorted token arrays taken by the earlier waves of this layer
+    std::vector<int32_t> wave_rowmap;         // [nb][SPM_MAX_TOPK] row of each (token, k) pair over all waves so far
     unsigned char* tc_act = nullptr;          // [max_units][16 KB] A^T slots of the bf16 grouped kernel
     int* tc_ready = nullptr;                  // [1 + max_units] chunk counter, then the slots' arrival counters
     std::vector<GgTaskHost> plan_chunks;
@@ -644,7 +646,15 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
     GgRow* rows = reinterpret_cast<GgRow*>(hd + c->tc_off_rows);
     int32_t* rowmap = reinterpret_cast<int32_t*>(hd + c->tc_off_rowmap);
     GgWait* waits = reinterpret_cast<GgWait*>(hd + c->tc_off_wait);
-    std::fill(rowmap, rowmap + size_t(nb) * SPM_MAX_TOPK, -1);
+    // Every (token, k) pair of the layer gets a row of its own in the sorted token arrays and in the partial
+    // outputs, whatever wave its expert is computed in: the waves append their rows, and one combine after the
+    // last wave adds each token's experts in k order. The sum then does not depend on which experts shared a
+    // wave, i.e. on the cache state: batched outputs are bit-identical with and without offloading.
+    if (first) {
+        c->wave_row_off = 0;
+        c->wave_rowmap.assign(size_t(nb) * SPM_MAX_TOPK, -1);
+    }
+    const int off = c->wave_row_off;
     // counting sort of the wave's (token, k) pairs by expert: rows of an expert keep token-major order
     int n_rows = 0, n_units = 0;
     std::vector<int32_t>& row_of = c->plan_first;       // per expert: pairs in this wave, then the next free row of its run
@@ -661,7 +671,7 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
         const GgWait uw = (dev_wait && c->slot_pending[ks]) ? GgWait{int32_t(c->slot_dep[ks]), c->slot_want[ks]} : GgWait{-1, 0u};
         for (int jt = 0; jt < c->n_jt; ++jt) {
             waits[n_units] = uw;
-            units[n_units++] = GgUnit{layer * c->S + slot_of_expert[e], jt, row_of[e], cnt};
+            units[n_units++] = GgUnit{layer * c->S + slot_of_expert[e], jt, off + row_of[e], cnt};
         }
     }
     n_rows = row_of[m.n_experts];
@@ -670,10 +680,13 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
             const int e = ids[tk * K + k];
             if (slot_of_expert[e] < 0) continue;
             const int r = row_of[e]++;
-            rowmap[tk * SPM_MAX_TOPK + k] = r;
+            c->wave_rowmap[tk * SPM_MAX_TOPK + k] = off + r;
             rows[r] = GgRow{tk, k};
         }
-    if (n_units == 0) return SPM_OK;
+    if (off + n_rows > c->rows_cap) return fail(c, SPM_ERR_STATE, "token rows of a layer exceed the workspace");
+    std::memcpy(rowmap, c->wave_rowmap.data(), size_t(nb) * SPM_MAX_TOPK * sizeof(int32_t));
+    c->wave_row_off = off + n_rows;
+    if (n_units == 0 && !last) return SPM_OK;
     const bool q4 = m.dtype == SPM_DTYPE_Q4;
     if (!q4) {
         // bf16 kernel: phase-2 chunks, finer towards the end, so that every SM streams until the launch ends
@@ -685,8 +698,9 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
     CU(c, cudaEventRecord(c->tc_desc_ev[d], c->compute));
     c->tc_desc_ev_valid[d] = 1;
     // (all three kernels of a wave are launched so that their preambles may overlap their predecessor's tail)
-    CU(c, launch_k(gg_gather_kernel, dim3(n_rows), dim3(128), 0, c->compute, true, x_norm, w,
-                   reinterpret_cast<const GgRow*>(dd + c->tc_off_rows), n_rows, (const int*)nullptr, m.hidden, K, c->tc_xs, c->tc_wrow,
+    CU(c, launch_k(gg_gather_kernel, dim3(std::max(n_rows, 1)), dim3(128), 0, c->compute, true, x_norm, w,
+                   reinterpret_cast<const GgRow*>(dd + c->tc_off_rows), n_rows, (const int*)nullptr, m.hidden, K,
+                   c->tc_xs + size_t(off) * m.hidden, c->tc_wrow + off,
                    q4 ? 1 : 0, q4 ? (int*)nullptr : c->tc_ready, q4 ? 0 : n_units + 1));
     if (t && first) CU(c, cudaEventRecord(t->ffn_start[layer], c->compute));
     if (ring >= 0 && first) CU(c, cudaEventRecord(c->ring_start[ring], c->compute));
@@ -697,7 +711,9 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
         a.unit_wait = reinterpret_cast<const GgWait*>(dd + c->tc_off_wait);
         a.ready = c->ws_slot_gen;
     }
-    if (q4) {
+    if (n_units == 0) {
+        // (nothing to compute in this wave; the combine below still closes the layer)
+    } else if (q4) {
         CU(c, launch_k(ffn_grouped_q4_kernel, dim3(std::min(c->num_sms, n_units)), dim3(kQgThreads), ffn_grouped_q4_smem(), c->compute, true,
                        c->qmapn, c->qmapsc, c->xmaps, a));
     } else {
@@ -711,9 +727,10 @@ int launch_grouped_wave(spm_ctx* c, int layer, const float* x_norm, const int32_
     }
     if (t && last) CU(c, cudaEventRecord(t->ffn_end[layer], c->compute));
     if (ring >= 0 && last) { CU(c, cudaEventRecord(c->ring_end[ring], c->compute)); c->ring_used[ring] = 1; }
-    CU(c, launch_k(gg_combine_kernel, gg_combine_grid(m.hidden, nb), gg_combine_block(K), 0, c->compute, true,
-                   (const float*)c->tc_partial, reinterpret_cast<const int32_t*>(dd + c->tc_off_rowmap), K, c->n_jt, c->rows_cap, m.hidden, h_inout));
-    c->kernel_launches += 3;
+    if (last)
+        CU(c, launch_k(gg_combine_kernel, gg_combine_grid(m.hidden, nb), gg_combine_block(K), 0, c->compute, true,
+                       (const float*)c->tc_partial, reinterpret_cast<const int32_t*>(dd + c->tc_off_rowmap), K, c->n_jt, c->rows_cap, m.hidden, h_inout));
+    c->kernel_launches += last ? 3 : 2;
     c->ffn_launches++;
     c->tc_launches++;
     return SPM_OK;

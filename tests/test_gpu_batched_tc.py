@@ -126,6 +126,33 @@ def test_free_running_events_match_policy_oracle(setup):
         assert m.stats()["waves"] > 0
 
 
+def test_offloaded_waves_give_the_bits_of_a_fully_resident_context(setup):
+    """Router-preserving guarantee for batched decode (Section 3.1, last paragraph; Section 3.3, last
+    paragraph), bit for bit: a (token, expert) pair's partial output does not depend on the wave its
+    expert is computed in, and one combine per layer adds a token's experts in rank order, so a
+    context with fewer slots than experts (waves, on-demand loads, prefetches, evictions) and a
+    context that holds every expert (host-free steps, plan built on the device) agree exactly."""
+    from paper_2607_24787_b200.synth_model import build_from_synth
+    cfg, nb, m, wts, H = setup
+    outs = {}
+    for policy in ("adapter", "on_demand"):
+        m.cache_reset(); m.set_policy(policy); m.set_budget(2)
+        o = [m.decode_step(dev(H[s])) for s in range(H.shape[0])]
+        m.synchronize()
+        outs[policy] = np.stack([x.cpu().numpy() for x in o])
+    assert np.array_equal(outs["adapter"], outs["on_demand"])
+    full = build_from_synth(cfg, slots=cfg.n_experts, budget=0)
+    try:
+        full.set_policy("on_demand")
+        o = [full.decode_step(dev(H[s])) for s in range(H.shape[0])]
+        full.synchronize()
+        got = np.stack([x.cpu().numpy() for x in o])
+        assert full.stats()["misses"] > 0          # the first step loads; later steps run without a host turn
+        assert np.array_equal(got, outs["on_demand"])
+    finally:
+        full.close()
+
+
 def test_device_side_wait_in_the_producer_warp_is_bit_identical(setup):
     """The grouped kernels' producer warp can wait for a unit's expert copy itself (per unit, on the
     batch's arrival counter) instead of the host ordering the launch behind the copy events: same
