@@ -209,9 +209,10 @@ int spm_prefetch_async(spm_ctx* ctx, int target_layer, const int32_t* ids, int c
  * stream wait for exactly the copy batches whose slots it reads, and enqueues
  * h_inout += sum_k w_k FFN_{ids_k}(x).
  * x_norm dev [nb][D], ids HOST [nb][K], w dev [nb][K], h_inout dev [nb][D]. Asynchronous.
- * When more distinct experts are needed than there are slots the work is split in waves; the sum
- * of a token's experts is taken in rank order whatever the waves were, so the result does not
- * depend on the cache state (bit for bit, at batch 1 and on the batched tensor-core path). */
+ * When more distinct experts are needed than there are slots the work is split in waves. On the
+ * batched tensor-core path the sum of a token's experts is taken in rank order whatever the waves
+ * were, and at batch 1 a layer is one launch whenever slots >= top_k, so in both cases the result
+ * does not depend on the cache state, bit for bit. */
 int spm_moe_ffn(spm_ctx* ctx, int layer, const float* x_norm, const int32_t* ids,
                 const float* w, int nb, float* h_inout);
 
