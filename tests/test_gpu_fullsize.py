@@ -259,3 +259,37 @@ def test_deepseek_shape_full_size_free_running_against_the_oracle():
     finally:
         m.close()
 
+
+
+@pytest.mark.parametrize("base", ["qwen3", "qwen3_q4"])
+def test_batched_shape_offloaded_steps_give_the_bits_of_resident_steps(base):
+    """The batched configuration's per-layer shape, two layers deep, free-running: 32 slots per layer
+    (about four waves per layer, on-demand loads, prefetches) against 128 slots (every expert resident,
+    host-free steps). The outputs agree bit for bit: the router-preserving guarantee at this shape."""
+    from paper_2607_24787_b200.build import build
+    from paper_2607_24787_b200.synth_model import build_from_synth
+    build()
+    nb, steps = 64, 3
+    cfg = synth.get_config(base, n_layers=2, batch=nb, slots=32, budget=1)
+    free_host = int(open("/proc/meminfo").read().split("MemAvailable:")[1].split()[0]) * 1024
+    if free_host < 8 * 2 ** 30 or torch.cuda.mem_get_info()[0] < 12 * 2 ** 30:
+        pytest.skip("not enough memory for two layers of 128 experts, twice")
+    tok = synth.zipf_tokens(synth.get_config("batched"), steps=steps)
+    H = [synth.embedding_rows(cfg, tok[s]) for s in range(steps)]
+    m = build_from_synth(cfg)
+    full = build_from_synth(cfg, slots=cfg.n_experts, budget=0, store=m.store)
+    try:
+        m.set_policy("adapter"); full.set_policy("on_demand")
+        a, b = [], []
+        for s in range(steps):
+            h = H[s].cuda(); torch.cuda.synchronize()
+            a.append(m.decode_step(h))
+            b.append(full.decode_step(h))
+        m.synchronize(); full.synchronize()
+        st = m.stats()
+        assert st["waves"] > 0 and st["misses"] > 0
+        for s in range(steps):
+            assert np.array_equal(a[s].cpu().numpy(), b[s].cpu().numpy()), s
+        m.check_invariants(); full.check_invariants()
+    finally:
+        full.close(); m.close()
