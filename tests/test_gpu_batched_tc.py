@@ -212,7 +212,7 @@ def test_producer_warp_wait_runs_out_and_the_context_survives(name):
             m.decode_step(dev(H[0]))
             m.synchronize()
         assert e.value.code == -4                    # SPM_ERR_TIMEOUT
-        assert time.perf_counter() - t0 < 2.0
+        assert time.perf_counter() - t0 < 1.9        # the configured limit applied, not the 2 s default
         m.synchronize()                              # reported once
         m.set_device_wait_limit_us(0)
         m.cache_reset()
