@@ -390,6 +390,9 @@ def run_ours(args):
                           (f"{b2b['launches']} spm_moe_ffn launches back to back on the compute stream, all experts resident "
                            "(pools of all layers cycled, nothing served from L2), CUDA event pair per launch"),
                 "us_per_launch_serialized": b2b.get("serialized_us"),
+                "us_per_launch_graph_plain": b2b.get("graph_plain_us"),
+                "frac_graph_plain": (b2b["algorithmic_bytes_per_launch"] / (b2b["graph_plain_us"] * 1e-6) / 1e9 / peak) if b2b.get("graph_plain_us") else None,
+                "us_per_launch_graph_chained": b2b.get("graph_chained_us"),
                 "frac_serialized": (b2b["algorithmic_bytes_per_launch"] / (b2b["serialized_us"] * 1e-6) / 1e9 / peak) if b2b.get("serialized_us") else None,
                 "us_per_launch_event_pair_each": b2b["event_pair_each_us"],
                 "frac_event_pair_each": b2b["algorithmic_bytes_per_launch"] / (b2b["event_pair_each_us"] * 1e-6) / 1e9 / peak}
@@ -635,7 +638,10 @@ def dsvl2_leg(args, m, peak, which, device):
     out["roofline"] = {"bound": "hbm", "kernel": b2b["kernel"], "achieved": b2b["gb_s"], "peak": peak, "unit": "GB/s",
                        "frac": b2b["frac_of_measured_peak"], "traffic": None, "peak_source": f"of {which}",
                        "algorithmic_bytes_per_launch": algo, "us_per_launch": b2b["kernel_us"],
-                       "us_per_launch_serialized": b2b.get("serialized_us"), "us_per_launch_event_pair_each": b2b["event_pair_each_us"],
+                       "us_per_launch_serialized": b2b.get("serialized_us"),
+                "us_per_launch_graph_plain": b2b.get("graph_plain_us"),
+                "frac_graph_plain": (b2b["algorithmic_bytes_per_launch"] / (b2b["graph_plain_us"] * 1e-6) / 1e9 / peak) if b2b.get("graph_plain_us") else None,
+                "us_per_launch_graph_chained": b2b.get("graph_chained_us"), "us_per_launch_event_pair_each": b2b["event_pair_each_us"],
                        "in_kernel_window_us": b2b.get("chained_window_us"),
                        "region": "240 launches of the kernel alone back to back (spm_time_ffn_kernel, programmatic dependent "
                                  "launch), all experts resident, one CUDA event pair around all of them"}
@@ -789,6 +795,12 @@ def ffn_back_to_back(cfg, full, algo_bytes, peak, launches=480):
         out["chained_window_us"] = statistics.median(c[1] for c in chained)
         out["serialized_us"] = statistics.median(c[0] for c in serial)
         out["serialized_window_us"] = statistics.median(c[1] for c in serial)
+        # the same two launch sequences captured into one CUDA graph and replayed (how a host-free decode step is launched)
+        try:
+            out["graph_plain_us"] = statistics.median(full.time_ffn_kernel(0, x[0], ids1, w[0], chained=2)[0] for _ in range(3))
+            out["graph_chained_us"] = statistics.median(full.time_ffn_kernel(0, x[0], ids1, w[0], chained=3)[0] for _ in range(3))
+        except Exception as e:   # noqa: BLE001 (reported, not hidden)
+            out["graph_error"] = str(e)[:200]
         per_kernel = out["chained_us"]
     out["kernel_us"] = per_kernel
     ach = mean_bytes / (per_kernel * 1e-6) / 1e9

@@ -332,7 +332,9 @@ int spm_measure_read_bandwidth(spm_ctx* ctx, size_t bytes, int reps, double* gb_
  * (SPM_ERR_NOT_RESIDENT otherwise: nothing is loaded here).
  * chained = 1: launched with the programmatic-serialisation attribute (as all kernels of a decode step are), so a
  * launch fetches its first weight rows while its predecessor drains; 0: plain launches, each
- * starts after the one before it has ended.
+ * starts after the one before it has ended; 2 and 3: the same as 0 and 1 with the launches captured
+ * into one CUDA graph and replayed (what a host-free decode step does), which takes the host's
+ * launch path out of the gaps between kernels.
  * *us_per_launch = event span / launches. *window_us (may be NULL) = mean in-kernel window
  * (dependency resolved or first CTA started -> last CTA done, %globaltimer) of the first 12288
  * launches. The partial-row workspace and the in-kernel clock ring are overwritten. */

@@ -1877,7 +1877,21 @@ int spm_time_ffn_kernel(spm_ctx* c, int first_layer, const float* x_norm, const 
     CU(c, cudaEventCreate(&e0));
     CU(c, cudaEventCreate(&e1));
     int rc = SPM_OK;
-    cudaError_t ce = cudaEventRecord(e0, c->compute);
+    const bool pdl = (chained & 1) != 0, graph = chained >= 2;
+    cudaGraph_t gr = nullptr;
+    cudaGraphExec_t ge = nullptr;
+    cudaError_t ce = cudaSuccess;
+    if (graph) {
+        // (kernel attributes are set outside the capture: one ordinary launch of this variant comes first)
+        FfnArgs<1> warm{};
+        warm.pool = slot_ptr(c, first_layer, 0); warm.x = x_norm; warm.w = w; warm.partial = c->ws_partial; warm.status = c->ws_status;
+        warm.blob_bytes = c->blob; warm.I = m.inter; warm.K = K; warm.n_slots = c->S; warm.n_shared = 0; warm.count[0] = 0;
+        ce = launch_gemv<1>(c, warm, G, 1, false);
+        if (ce == cudaSuccess) ce = cudaStreamSynchronize(c->compute);
+        if (ce == cudaSuccess) ce = cudaStreamBeginCapture(c->compute, cudaStreamCaptureModeThreadLocal);
+    } else {
+        ce = cudaEventRecord(e0, c->compute);
+    }
     for (int i = 0; i < launches && ce == cudaSuccess; ++i) {
         const int layer = (first_layer + i) % L;
         FfnArgs<1> a{};
@@ -1889,7 +1903,7 @@ int spm_time_ffn_kernel(spm_ctx* c, int first_layer, const float* x_norm, const 
         a.status = c->ws_status;
         a.clock = clocks && i < kClockSlots ? c->ws_clock + 2 * size_t(i) : nullptr;
         a.wait_limit_ns = c->wait_limit_ns;
-        a.early = chained ? 1 : 0;
+        a.early = pdl ? 1 : 0;
         a.blob_bytes = c->blob;
         a.I = m.inter; a.K = K; a.n_slots = c->S; a.n_shared = m.n_shared;
         int cnt = 0;
@@ -1899,7 +1913,14 @@ int spm_time_ffn_kernel(spm_ctx* c, int first_layer, const float* x_norm, const 
         }
         for (int sh = 0; sh < m.n_shared; ++sh) { a.code[cnt] = short(-1 - sh); a.kidx[cnt++] = 255; }
         a.count[0] = (unsigned char)cnt;
-        ce = launch_gemv<1>(c, a, G, 1, chained != 0);
+        ce = launch_gemv<1>(c, a, G, 1, pdl);
+    }
+    if (graph) {
+        cudaError_t end = cudaStreamEndCapture(c->compute, &gr);       // (always ends the capture, also after a failed launch)
+        if (ce == cudaSuccess) ce = end;
+        if (ce == cudaSuccess) ce = cudaGraphInstantiate(&ge, gr, 0);
+        if (ce == cudaSuccess) ce = cudaEventRecord(e0, c->compute);
+        if (ce == cudaSuccess) ce = cudaGraphLaunch(ge, c->compute);
     }
     if (ce == cudaSuccess) ce = cudaEventRecord(e1, c->compute);
     if (ce == cudaSuccess) ce = cudaEventSynchronize(e1);
@@ -1907,6 +1928,8 @@ int spm_time_ffn_kernel(spm_ctx* c, int first_layer, const float* x_norm, const 
     if (ce == cudaSuccess) ce = cudaEventElapsedTime(&ms, e0, e1);
     cudaEventDestroy(e0);
     cudaEventDestroy(e1);
+    if (ge) cudaGraphExecDestroy(ge);
+    if (gr) cudaGraphDestroy(gr);
     if (ce != cudaSuccess) return fail(c, SPM_ERR_CUDA, "expert kernel probe: %s", cudaGetErrorString(ce));
     c->kernel_launches += launches;
     *us_per_launch = double(ms) * 1e3 / launches;

@@ -58,6 +58,7 @@ def sweep_tables(d):
 def roofline_row(name, r):
     return [name, r.get("kernel", ""), fmt(r.get("algorithmic_bytes_per_launch", 0) / 1e6, 1), fmt(r.get("us_per_launch"), 1),
             fmt(r.get("achieved"), 0), fmt(r.get("frac"), 3), fmt(r.get("us_per_launch_serialized"), 1), fmt(r.get("frac_serialized"), 3),
+            fmt(r.get("us_per_launch_graph_plain"), 1), fmt(r.get("frac_graph_plain"), 3),
             fmt(r.get("us_per_launch_event_pair_each"), 1), fmt(r.get("in_kernel_window_us"), 1)]
 
 
@@ -101,13 +102,13 @@ def bench_tables(d):
     rows = [roofline_row(cfg.split(":")[0], d["roofline"])]
     for name, leg in (d.get("configs") or {}).items():
         if "error" in leg:
-            rows.append([name, "error: " + leg["error"][:60]] + [""] * 8)
+            rows.append([name, "error: " + leg["error"][:60]] + [""] * 10)
             continue
         if "roofline_wave" in leg:
             rows.append(roofline_row(name + " (one wave)", leg["roofline_wave"]))
         rows.append(roofline_row(name + (" (all resident)" if "roofline_wave" in leg else ""), leg["roofline"]))
-    print(table(["workload", "kernel", "MB per launch", "us per launch", "GB/s", "of peak", "us serialized", "of peak", "us event pair each",
-                 "in-kernel window us"], rows))
+    print(table(["workload", "kernel", "MB per launch", "us per launch", "GB/s", "of peak", "us serialized", "of peak",
+                 "us plain, replayed from a CUDA graph", "of peak", "us event pair each", "in-kernel window us"], rows))
     r = d["roofline"]
     print(f"\n(peak {fmt(r['peak'], 0)} GB/s {r.get('peak_source', '')}; read-only streaming rate of the device {fmt(r.get('read_only_stream_gb_s'), 0)} GB/s; "
           + (f"ncu DRAM traffic per launch {fmt(r['traffic'] / 1e6, 1)} MB.)" if r.get("traffic") else "no ncu traffic figure for this workload.)"))
