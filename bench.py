@@ -639,9 +639,11 @@ def dsvl2_leg(args, m, peak, which, device):
                        "frac": b2b["frac_of_measured_peak"], "traffic": None, "peak_source": f"of {which}",
                        "algorithmic_bytes_per_launch": algo, "us_per_launch": b2b["kernel_us"],
                        "us_per_launch_serialized": b2b.get("serialized_us"),
-                "us_per_launch_graph_plain": b2b.get("graph_plain_us"),
-                "frac_graph_plain": (b2b["algorithmic_bytes_per_launch"] / (b2b["graph_plain_us"] * 1e-6) / 1e9 / peak) if b2b.get("graph_plain_us") else None,
-                "us_per_launch_graph_chained": b2b.get("graph_chained_us"), "us_per_launch_event_pair_each": b2b["event_pair_each_us"],
+                       "frac_serialized": (algo / (b2b["serialized_us"] * 1e-6) / 1e9 / peak) if b2b.get("serialized_us") else None,
+                       "us_per_launch_graph_plain": b2b.get("graph_plain_us"),
+                       "frac_graph_plain": (algo / (b2b["graph_plain_us"] * 1e-6) / 1e9 / peak) if b2b.get("graph_plain_us") else None,
+                       "us_per_launch_graph_chained": b2b.get("graph_chained_us"),
+                       "us_per_launch_event_pair_each": b2b["event_pair_each_us"],
                        "in_kernel_window_us": b2b.get("chained_window_us"),
                        "region": "240 launches of the kernel alone back to back (spm_time_ffn_kernel, programmatic dependent "
                                  "launch), all experts resident, one CUDA event pair around all of them"}
