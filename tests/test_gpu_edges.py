@@ -356,3 +356,35 @@ def test_long_run_with_changing_policies_and_wait_modes_stays_router_preserving(
         m.check_invariants()
     finally:
         m.close()
+
+
+def test_ffn_kernel_probe_in_all_launch_modes_leaves_the_context_usable():
+    """`spm_time_ffn_kernel` (the measurement aid behind the bench's roofline): plain and chained launches,
+    each also replayed from a CUDA graph, return positive times and an in-kernel window; an expert without a
+    slot is refused; a decode step afterwards still matches the oracle."""
+    from paper_2607_24787_b200 import binding as B
+    cfg = synth.get_config("tiny", n_layers=2)
+    m = build(cfg, slots=cfg.n_experts, budget=0)
+    try:
+        m.set_policy("on_demand")
+        x = torch.randn(cfg.hidden, device="cuda")
+        w = torch.full((cfg.top_k,), 1.0 / cfg.top_k, device="cuda")
+        ids = np.stack([np.arange(cfg.top_k, dtype=np.int32) + (i % 3) for i in range(24)])
+        with pytest.raises(B.SpmError):
+            m.time_ffn_kernel(0, x, ids, w, chained=0)         # nothing resident yet: the probe loads nothing
+        for l in range(cfg.n_layers):
+            m.prefetch_async(l, np.arange(cfg.n_experts, dtype=np.int32))
+        m.synchronize()
+        for mode in (0, 1, 2, 3):
+            us, win = m.time_ffn_kernel(0, x, ids, w, chained=mode)
+            assert 0.0 < us < 1e4 and 0.0 < win < 1e4, (mode, us, win)
+        tok = synth.zipf_tokens(cfg, steps=2)
+        H = synth.embedding_rows(cfg, tok.reshape(-1)).numpy().reshape(2, 1, cfg.hidden)
+        ref = make_ref(cfg, weights=SynthWeights(cfg), policy="on_demand", slots=cfg.n_experts, budget=0)
+        for s in range(2):
+            out = m.decode_step(dev(H[s]))
+            m.synchronize()
+            want, _ = ref.step(H[s])
+            assert M.rel_linf(out.cpu().numpy().astype(np.float64)[0], want[0]) < 4e-5
+    finally:
+        m.close()
